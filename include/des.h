@@ -1,0 +1,249 @@
+/*
+ * des.h — C ABI of the single-GPU hot path of Distributed Equivalent
+ * Substitution (DES) training (arXiv 1909.04823).
+ *
+ * What the library computes
+ * -------------------------
+ * The weights-rich sparse operators of CTR models, each rewritten as S
+ * per-shard sub-operators M_j over a partition of the weights, an
+ * aggregation (+) over shards and a substitution operator F (Algorithm 1,
+ * Eq. 1).  The S "processes" of the paper are S logical shards resident on
+ * one GPU; the aggregation is an in-device reduction in fixed shard order.
+ *
+ *   LR      M_1 = sum_{j in shard} w_j x_j                (Section 4.1)
+ *   FM      M_1 = sum v_j x_j (k-vector),
+ *           M_2 = sum <v_j x_j, v_j x_j> (scalar),
+ *           F   = 1/2 <(+)M_1,(+)M_1> - 1/2 (+)M_2        (Section 4.2)
+ *   POOL    sum-pooled latent vectors per (sample, field) (Section 4.3,
+ *           embedding layer; same field on the same shard under FIELD)
+ *   DENSE1  V^T W = sum_s V_s^T W_s, the first FC layer split over the
+ *           rows of W by owning shard                      (Section 4.3)
+ *   table   lookup / insert / update on a dynamic hash table of
+ *           uint64 keys and float32 weights               (Section 5)
+ *   backward: the aggregated gradient flows back into each shard's own
+ *           sub-operator, no cross-shard term             (Section 3.2,
+ *           "Back-propagation Phase"); one optimizer application per
+ *           unique key per step, state local to the shard (Section 4.3,
+ *           last paragraph before "Extending to General Models").
+ *
+ * Conventions
+ * -----------
+ * - Every function returns des_status_t; nothing throws, nothing aborts.
+ * - Pointers named d_* (and every pointer inside des_batch_t, des_partials_t,
+ *   des_outputs_t, des_grads_t) are DEVICE pointers owned by the caller; they
+ *   must stay valid until the stream has passed the call.  Pointers named h_*
+ *   are HOST pointers.  The library owns only what des_table_create allocates
+ *   and frees it in des_table_destroy.
+ * - All device work is enqueued on the caller's stream (a cudaStream_t passed
+ *   as void*; NULL = the legacy default stream).  Only des_table_status,
+ *   des_table_size, des_table_export, des_dense1_get/set on host pointers and
+ *   des_step_host synchronise.
+ * - Device-side problems (reserved key, full shard) never fault: the
+ *   offending occurrences get row DES_ROW_NONE, are skipped by every later
+ *   kernel, and a sticky error word is raised that des_table_status returns.
+ * - There is no CPU fallback: without a CUDA device every call that would
+ *   launch returns DES_ERR_CUDA.
+ *
+ * Batch layout (CSR over bags): bag (b, f) = sample b, field f, holds the
+ * occurrences offsets[b*F+f] .. offsets[b*F+f+1]-1 of ids[] / vals[].
+ * An id that appears twice in a bag is two terms of every sum.
+ */
+#ifndef DES_H_
+#define DES_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DES_OK = 0,
+  DES_ERR_INVALID_ARG = 1,   /* bad argument, found on the host before any launch      */
+  DES_ERR_RESERVED_KEY = 2,  /* an id equals DES_KEY_EMPTY (sticky, device-side)        */
+  DES_ERR_CAPACITY = 3,      /* a shard ran out of slots or rows (sticky, device-side)  */
+  DES_ERR_UNSUPPORTED = 4,
+  DES_ERR_CUDA = 5,          /* a CUDA runtime call failed, or no device                */
+  DES_ERR_NOT_FOUND = 6
+} des_status_t;
+
+/* operator kind bitmask */
+enum { DES_OP_LR = 1, DES_OP_FM = 2, DES_OP_POOL = 4, DES_OP_DENSE1 = 8 };
+/* weight placement: HASH = mix64(id) mod S ("any partition policy that
+ * balances", Section 4.2); FIELD = field mod S (Section 5, "Large-scale
+ * Sparse Features"; required for a weight-disjoint row split, Section 4.3). */
+enum { DES_PART_HASH = 0, DES_PART_FIELD = 1 };
+enum { DES_OPT_SGD = 0, DES_OPT_ADAGRAD = 1 };
+
+#define DES_KEY_EMPTY 0xFFFFFFFFFFFFFFFFull /* reserved id                         */
+#define DES_ROW_NONE  0xFFFFFFFFu           /* "no row": missing key / failed insert */
+
+typedef struct des_table des_table_t;
+
+typedef struct {
+  uint32_t num_shards;   /* S, 1..64                                                  */
+  uint32_t num_fields;   /* F >= 1                                                    */
+  uint32_t emb_dim;      /* k, a multiple of 4, 4..64                                 */
+  uint32_t hidden;       /* H of the first dense layer, multiple of 4; 0 = no DENSE1  */
+  uint32_t partition;    /* DES_PART_*                                                */
+  uint32_t optimizer;    /* DES_OPT_*                                                 */
+  uint64_t max_rows;     /* total key capacity over all shards, < 2^32 - 1            */
+  float    max_load;     /* slots per shard = rows of the shard / max_load; (0, 0.9]  */
+  const uint64_t* h_rows_per_shard; /* optional host [S] row capacity per shard; NULL =
+                                       max_rows/S * 1.05 + 1024 each                  */
+  uint64_t seed;         /* seed of the counter-based row initialiser                 */
+  float    init_scale;   /* new latent vectors ~ U[-init_scale, init_scale)           */
+  float    lr, eps, init_acc; /* theta -= lr*G            (SGD)
+                                 a += G*G; theta -= lr*G/(sqrt(a)+eps)   (Adagrad),
+                                 a starts at init_acc                                */
+  int64_t  max_nnz;      /* largest nnz of any batch (sizes the workspace)            */
+  int32_t  max_batch;    /* largest B of any batch                                    */
+  /* optional device allocator (e.g. backed by the caller's caching allocator);
+   * NULL = cudaMalloc / cudaFree.  alloc must return 256-byte aligned memory.   */
+  void* (*alloc)(size_t bytes, void* ctx);
+  void  (*dealloc)(void* ptr, void* ctx);
+  void*  alloc_ctx;
+} des_config_t;
+
+/* One batch.  find_or_insert reads offsets/ids and fills rows, shards, uidx,
+ * uniq_rows, n_uniq; the other calls read them. */
+typedef struct {
+  int32_t         batch;      /* B                                                    */
+  int64_t         nnz;        /* occurrences, < 2^31                                  */
+  const int32_t*  offsets;    /* [B*F+1]                                              */
+  const uint64_t* ids;        /* [nnz]                                                */
+  const float*    vals;       /* [nnz] feature values x_j, or NULL = all 1.0          */
+  uint32_t*       rows;       /* [nnz] shard-local row of each occurrence             */
+  uint8_t*        shards;     /* [nnz] owning shard of each occurrence                */
+  uint32_t*       uidx;       /* [nnz] batch-unique index of the occurrence's key:
+                                 keys numbered 0..U-1 by first occurrence in CSR order */
+  uint32_t*       uniq_rows;  /* [nnz] (first U used) table-global row of unique key u
+                                 = des_table_row_base()[shard] + shard-local row      */
+  uint32_t*       n_uniq;     /* [1]   U                                              */
+} des_batch_t;
+
+/* Per-shard partial results (the paper's intermediate results S_M).
+ * SMALL_STRIDE(k) = k + 4 floats per (shard, sample):
+ *   [0..k)  M_1 of FM   (sum v x)
+ *   [k]     M_1 of LR   (sum w x)
+ *   [k+1]   M_2 of FM   (sum <v x, v x>)
+ *   [k+2], [k+3]  zero padding (keeps rows 16-byte aligned). */
+typedef struct {
+  float* part_small;   /* [S][B][k+4], required for LR / FM                            */
+  float* pooled;       /* [B][F*k] sum-pooled field embeddings, already aggregated over
+                          shards on chip; required for POOL / DENSE1                   */
+  float* part_pooled;  /* optional [S][B][F*k] dense per-shard pooled partials
+                          (parity / inspection at small sizes), or NULL                */
+  float* part_dense;   /* optional [S][B][H] per-shard partial products P_s = V_s W_s,
+                          or NULL (then only Z is produced by des_aggregate)           */
+} des_partials_t;
+
+/* Aggregated results.  out_small has k + 4 floats per sample:
+ *   [0..k) A = (+)M_1 ; [k] R_lr = (+)M_1^lr ; [k+1] fm2 = F ; [k+2] Q = (+)M_2 ;
+ *   [k+3] zero. */
+typedef struct {
+  float* out_small;    /* [B][k+4]                                                     */
+  float* pooled;       /* [B][F*k]; may alias des_partials_t.pooled                    */
+  float* Z;            /* [B][H] = sum_s P_s (DENSE1), fp32                            */
+} des_outputs_t;
+
+/* Upstream gradients of the aggregated results (what the rest of the model
+ * sends back).  Any pointer may be NULL when its operator is not in `ops`. */
+typedef struct {
+  const float* gL;     /* [B]      dLoss/dR_lr                                         */
+  const float* gF;     /* [B]      dLoss/dfm2                                          */
+  const float* gE;     /* [B][F*k] dLoss/dpooled (direct consumers of pooled), or NULL */
+  const float* gZ;     /* [B][H]   dLoss/dZ (DENSE1), or NULL                          */
+  float*       gE_work;/* [B][F*k] scratch, required with DENSE1: receives
+                          gE + gZ * W1^T                                               */
+} des_grads_t;
+
+/* ---- table life cycle (Section 5, "Dynamic Hash Table") ------------------- */
+
+/* Allocates slots, rows, optimizer state and the per-call workspace on the
+ * current device.  *out is NULL on failure. */
+des_status_t des_table_create(const des_config_t* cfg, des_table_t** out);
+des_status_t des_table_destroy(des_table_t* t);
+
+/* lookup + insert (Section 5).  insert != 0: ids not yet in the table are
+ * inserted; a new key gets the next shard-local row, numbered in order of the
+ * key's first occurrence in CSR order within this call, its latent vector is
+ * initialised from a counter-based generator keyed on (seed, id) — so row
+ * contents never depend on insertion order —, its linear weight is 0 and its
+ * optimizer state init_acc.  insert == 0: lookup only; missing ids get
+ * DES_ROW_NONE, and uidx / uniq_rows / n_uniq are not written.
+ * Errors: DES_ERR_INVALID_ARG (nnz > max_nnz, batch > max_batch, NULL
+ * pointers); device-side sticky DES_ERR_RESERVED_KEY / DES_ERR_CAPACITY. */
+des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* batch, int insert, void* stream);
+
+/* Sub-operators M_j of every shard (Eq. of Sections 4.1-4.3), see
+ * des_partials_t.  `batch` must have been through des_find_or_insert. */
+des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_t* batch,
+                                  const des_partials_t* part, void* stream);
+
+/* Aggregation (+) over shards in the fixed order s = 0..S-1 (Eq. 1) and the
+ * substitution operator F (Algorithm 1, R = F(f_1..f_m)): out_small from
+ * part_small; Z from pooled and W1 (K loop in shard order) or, when
+ * part->part_dense is given, P_s materialised first and Z = sum_s P_s. */
+des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* batch,
+                           const des_partials_t* part, const des_outputs_t* out, void* stream);
+
+/* Mirror of the forward (Section 3.2): per-occurrence gradients
+ *   g_w(j) = x_j gL[b],  g_v(j) = x_j ( gF[b] (A[b] - v_j x_j) + gE[b][f] ),
+ * summed per unique key, then one SGD / Adagrad application per key with the
+ * state kept in the shard.  With DENSE1: gE_work = gE + gZ W1^T (each shard's
+ * own column block), gW1 = pooled^T gZ, and the same optimizer on W1.
+ * `out` supplies A (out_small) and pooled. */
+des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t* batch,
+                                 const des_outputs_t* out, const des_grads_t* grads, void* stream);
+
+/* ---- first dense layer weights W1 [F*k][H], fp32 master (Section 4.3) ----- */
+des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream);
+des_status_t des_dense1_get(des_table_t* t, float* d_W1, void* stream);
+
+/* ---- inspection (synchronising) ------------------------------------------ */
+
+/* Synchronises the device and returns the sticky device-side error, if any. */
+des_status_t des_table_status(des_table_t* t);
+/* Number of keys per shard, host array [S]. */
+des_status_t des_table_size(des_table_t* t, uint64_t* h_rows_per_shard);
+/* First table-global row of each shard and the grand total, host array [S+1]. */
+des_status_t des_table_row_base(des_table_t* t, uint64_t* h_row_base);
+/* Dumps up to `cap` keys (device arrays, any order): key, shard, shard-local
+ * row, latent vector [k], linear weight and their optimizer state.  *h_n_out =
+ * number of keys in the table (may exceed cap; then only cap are written). */
+des_status_t des_table_export(des_table_t* t, uint64_t* d_keys, uint8_t* d_shards, uint32_t* d_rows,
+                              float* d_emb, float* d_lin, float* d_acc_emb, float* d_acc_lin,
+                              uint64_t cap, uint64_t* h_n_out);
+/* Copies the rows (latent vector, linear weight, optimizer state) of the n
+ * table-global rows d_global_rows[] into dense device arrays; any output
+ * pointer may be NULL. */
+des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                 float* d_emb, float* d_lin, float* d_acc_emb, float* d_acc_lin,
+                                 void* stream);
+
+/* ---- whole step from host buffers ---------------------------------------- */
+
+/* One full step — find_or_insert, forward partials, aggregate, backward
+ * update — on a batch that lives in HOST memory (pinned for full speed):
+ * offsets/ids/vals are copied to device staging owned by the table, the step
+ * runs on `stream`, out_small [B][k+4] is copied back to h_out_small and the
+ * call returns after synchronising.  Upstream gradients stay device resident
+ * (they come from the rest of the model, which lives on the GPU).  d_pooled
+ * [B][F*k] is device scratch/output for POOL.  Requires max_nnz/max_batch
+ * workspace like the other calls. */
+des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
+                           const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                           const des_grads_t* d_grads, float* d_pooled, float* d_Z,
+                           float* h_out_small, void* stream);
+
+/* Number of kernel launches the library has issued for this table so far. */
+uint64_t des_table_launch_count(des_table_t* t);
+
+const char* des_status_string(des_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DES_H_ */

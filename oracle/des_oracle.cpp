@@ -1,0 +1,481 @@
+// CPU oracle of the DES sparse step (arXiv 1909.04823).
+//
+// TEST INFRASTRUCTURE ONLY: a plain, slow, sequential implementation that the
+// tests, the smoke check and the benchmark's cpu_baseline leg compare the CUDA
+// path against.  The product never calls it; it shares no code, header, table
+// or constant generator with the CUDA sources.
+//
+// What it computes, and from which passage:
+//   * the ORIGINAL (unsubstituted) operators F — LR's W^T X (Section 4.1), FM's
+//     order-2 sum in both its O(n^2) pair form and its linear form (Eq. 5),
+//     the embedding layer's per-field pooling and the first FC layer V^T W
+//     (Eq. 6) — looked up by key with no notion of shards;
+//   * the DES form — per-shard sub-operators M_j (Eqs. 2, 7, and
+//     M_1(V_i,W_i) = V_i^T W_i of Section 4.3), aggregation (+) in shard order
+//     (Eq. 1), and the substitution operator F (Eqs. 3, 8, 10; Algorithm 1);
+//   * the backward rule of Section 3.2 ("Back-propagation Phase"): the
+//     gradient of the aggregate flows unchanged into each shard's own
+//     sub-operator; one optimizer application per unique key on the summed
+//     gradient, state local to the shard (Section 4.3, closing paragraph);
+//   * the dynamic hash table's lookup / insert / update (Section 5).
+// Where the paper is silent (which hash, how a new weight is initialised, how
+// rows are numbered, Adagrad's exact form) it follows the readings listed in
+// the design notes; each is marked "reading" below.
+//
+// Arithmetic: weights and optimizer state are float32 (the paper's storage
+// type, Section 4.1); every sum is accumulated in double and rounded once.
+//
+// Pins (tests/, marked not-gpu): Philox known-answer vectors; mix64 inverse;
+// FM pair form == linear form; DES form == original for any S and both
+// partitions; S = 1 == any S; gradients == central finite differences;
+// dedup/Adagrad special cases; row-split GEMM == one dense matmul; canonical
+// row numbering vs a dictionary walk.  The hash/shard rule itself is fixed by
+// no passage: "parity unpinned" beyond bijectivity and balance.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <unordered_map>
+#include <vector>
+
+namespace {
+
+const uint32_t ROW_NONE = 0xFFFFFFFFu;
+enum { OP_LR = 1, OP_FM = 2, OP_POOL = 4, OP_DENSE1 = 8 };
+enum { PART_HASH = 0, PART_FIELD = 1 };
+enum { OPT_SGD = 0, OPT_ADAGRAD = 1 };
+
+// reading: the table's 64-bit mixer (splitmix64 finaliser steps)
+uint64_t mix64(uint64_t z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27; z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64
+// multiplies with the key bumped by the Weyl constants each round.
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int r = 0; r < 10; ++r) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    uint32_t n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// reading: component c of a new key's latent vector is
+//   ((r >> 8) * 2^-23 - 1) * init_scale,   r = word (c mod 4) of
+//   Philox4x32-10(counter = (c/4, 0, seed_lo, seed_hi), key = (id_lo, id_hi)).
+// Everything before the final multiply is exact in float32.
+float init_value(uint64_t seed, uint64_t id, uint32_t c, float init_scale) {
+  uint32_t ctr[4] = {c / 4u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t key[2] = {(uint32_t)id, (uint32_t)(id >> 32)};
+  uint32_t r[4];
+  philox4x32_10(ctr, key, r);
+  float u = (float)(r[c % 4u] >> 8);          // 24 bits, exact
+  float x = u * (1.0f / 8388608.0f);          // * 2^-23, exact, in [0, 2)
+  float y = x - 1.0f;                          // exact, in [-1, 1)
+  volatile float z = y * init_scale;           // one rounding (no contraction)
+  return z;
+}
+
+float bf16_round(float x) {                    // round-to-nearest-even to bfloat16
+  uint32_t u; std::memcpy(&u, &x, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return x;
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;
+  u &= 0xFFFF0000u;
+  float y; std::memcpy(&y, &u, 4);
+  return y;
+}
+
+struct Shard {
+  std::unordered_map<uint64_t, uint32_t> map;   // key -> shard-local row
+  std::vector<uint64_t> keys;                   // row -> key
+  std::vector<float> emb, lin, acc_emb, acc_lin;
+};
+
+struct Table {
+  uint32_t S, F, k, H, partition, optimizer;
+  uint64_t seed; float init_scale, lr, eps, init_acc;
+  std::vector<Shard> sh;
+  std::vector<float> W1, accW1;                 // [F*k][H]
+  uint32_t shard_of(uint64_t id, uint32_t field) const {
+    return partition == PART_HASH ? (uint32_t)(mix64(id) % S) : field % S;
+  }
+  uint32_t insert(uint32_t s, uint64_t id) {
+    Shard& h = sh[s];
+    uint32_t row = (uint32_t)h.keys.size();
+    h.map.emplace(id, row);
+    h.keys.push_back(id);
+    for (uint32_t c = 0; c < k; ++c) h.emb.push_back(init_value(seed, id, c, init_scale));
+    h.lin.push_back(0.0f);
+    for (uint32_t c = 0; c < k; ++c) h.acc_emb.push_back(init_acc);
+    h.acc_lin.push_back(init_acc);
+    return row;
+  }
+};
+
+inline void apply_opt(const Table& t, float& theta, float& acc, double Gd) {
+  float G = (float)Gd;                          // summed gradient, rounded once
+  if (t.optimizer == OPT_SGD) {
+    theta = (float)((double)theta - (double)t.lr * (double)G);
+  } else {                                      // reading: eps outside the root
+    float a = (float)((double)acc + (double)G * (double)G);
+    acc = a;
+    theta = (float)((double)theta - (double)t.lr * (double)G / (std::sqrt((double)a) + (double)t.eps));
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+uint64_t orc_mix64(uint64_t x) { return mix64(x); }
+void orc_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) { philox4x32_10(ctr, key, out); }
+float orc_init_value(uint64_t seed, uint64_t id, uint32_t c, float scale) { return init_value(seed, id, c, scale); }
+float orc_bf16_round(float x) { return bf16_round(x); }
+
+void orc_shard_of_many(const uint64_t* ids, int64_t n, uint32_t S, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = (uint8_t)(mix64(ids[i]) % S);
+}
+
+// Communication-saving ratios of Section 4 (R_lr, R_fm(2), R_dnn) from the
+// byte sizes of what DES exchanges (the per-shard partials above: B, B*k + B
+// and B*H float32 values) against the mesh strategy's keys + weights for U
+// unique features (uint64 keys, float32 weights, k-vectors; S_W = bytes of the
+// first FC layer's weights).
+void orc_comm_saving(int64_t B, int64_t U, int64_t k, int64_t H, double S_W, double* out3) {
+  double S_key = 8.0 * U, S_w = 4.0 * U, S_V = 4.0 * k * U;
+  double S_M1_lr = 4.0 * B, S_M1_fm = 4.0 * B * k, S_M2_fm = 4.0 * B, S_M1_dnn = 4.0 * B * H;
+  out3[0] = 1.0 - 2.0 * S_M1_lr / (S_key + S_w);
+  out3[1] = 1.0 - 2.0 * (S_M1_fm + S_M2_fm) / (S_key + S_V);
+  out3[2] = 1.0 - 2.0 * S_M1_dnn / (S_key + S_V + S_W);
+}
+
+void* orc_create(uint32_t S, uint32_t F, uint32_t k, uint32_t H, uint32_t partition, uint32_t optimizer,
+                 uint64_t seed, float init_scale, float lr, float eps, float init_acc) {
+  Table* t = new Table();
+  t->S = S; t->F = F; t->k = k; t->H = H; t->partition = partition; t->optimizer = optimizer;
+  t->seed = seed; t->init_scale = init_scale; t->lr = lr; t->eps = eps; t->init_acc = init_acc;
+  t->sh.resize(S);
+  if (H) { t->W1.assign((size_t)F * k * H, 0.0f); t->accW1.assign((size_t)F * k * H, init_acc); }
+  return t;
+}
+void orc_destroy(void* p) { delete (Table*)p; }
+
+void orc_dense1_set(void* p, const float* W1) { Table* t = (Table*)p; std::memcpy(t->W1.data(), W1, t->W1.size() * 4); }
+void orc_dense1_get(void* p, float* W1, float* acc) {
+  Table* t = (Table*)p;
+  if (W1) std::memcpy(W1, t->W1.data(), t->W1.size() * 4);
+  if (acc) std::memcpy(acc, t->accW1.data(), t->accW1.size() * 4);
+}
+
+void orc_size(void* p, uint64_t* per_shard) {
+  Table* t = (Table*)p;
+  for (uint32_t s = 0; s < t->S; ++s) per_shard[s] = t->sh[s].keys.size();
+}
+
+// lookup + insert (Section 5).  Rows are numbered per shard in order of first
+// occurrence in CSR order (reading); batch-unique indices likewise over the
+// whole batch.  Outputs: rows[nnz], shards[nnz], uidx[nnz], and for each
+// unique key u its (shard, row) in uniq_shard/uniq_row; returns U.
+int64_t orc_find_or_insert(void* p, const int32_t* offsets, const uint64_t* ids, int32_t B, int insert,
+                           uint32_t* rows, uint8_t* shards, uint32_t* uidx,
+                           uint8_t* uniq_shard, uint32_t* uniq_row) {
+  Table* t = (Table*)p;
+  std::unordered_map<uint64_t, uint32_t> seen;   // (shard<<32 | row) -> u
+  int64_t U = 0;
+  for (int64_t bag = 0; bag < (int64_t)B * t->F; ++bag) {
+    uint32_t f = (uint32_t)(bag % t->F);
+    for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
+      uint64_t id = ids[j];
+      uint32_t s = t->shard_of(id, f);
+      shards[j] = (uint8_t)s;
+      auto it = t->sh[s].map.find(id);
+      uint32_t row;
+      if (it != t->sh[s].map.end()) row = it->second;
+      else if (insert) row = t->insert(s, id);
+      else row = ROW_NONE;
+      rows[j] = row;
+      if (row == ROW_NONE) { if (uidx) uidx[j] = ROW_NONE; continue; }
+      uint64_t gk = ((uint64_t)s << 32) | row;
+      auto iu = seen.find(gk);
+      uint32_t u;
+      if (iu == seen.end()) {
+        u = (uint32_t)U++;
+        seen.emplace(gk, u);
+        if (uniq_shard) uniq_shard[u] = (uint8_t)s;
+        if (uniq_row) uniq_row[u] = row;
+      } else u = iu->second;
+      if (uidx) uidx[j] = u;
+    }
+  }
+  return U;
+}
+
+// The ORIGINAL operators, per sample, over all of the sample's occurrences
+// regardless of shard.  Outputs (double): lr0[B] = W^T X (Section 4.1);
+// A0[B][k] = sum v x, Q0[B] = sum <vx,vx>, fm2[B] linear form (Eq. 5, last
+// line); pooled0[B][F*k] (embedding layer, Section 4.3); Z0[B][H] = V^T W
+// (Eq. 6) on bfloat16-rounded operands (reading), accumulated in double.
+void orc_forward_original(void* p, uint32_t ops, const int32_t* offsets, const uint64_t* ids,
+                          const float* vals, int32_t B, double* lr0, double* A0, double* Q0,
+                          double* fm2, double* pooled0, double* Z0) {
+  Table* t = (Table*)p;
+  const uint32_t F = t->F, k = t->k, H = t->H;
+  std::vector<double> A(k), pool((size_t)F * k);
+  for (int32_t b = 0; b < B; ++b) {
+    double lr = 0, Q = 0;
+    std::fill(A.begin(), A.end(), 0.0);
+    std::fill(pool.begin(), pool.end(), 0.0);
+    for (uint32_t f = 0; f < F; ++f) {
+      int64_t bag = (int64_t)b * F + f;
+      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
+        uint32_t s = t->shard_of(ids[j], f);
+        auto it = t->sh[s].map.find(ids[j]);
+        if (it == t->sh[s].map.end()) continue;            // unknown key: no weight
+        const Shard& h = t->sh[s];
+        uint32_t row = it->second;
+        double x = vals ? (double)vals[j] : 1.0;
+        lr += (double)h.lin[row] * x;
+        for (uint32_t c = 0; c < k; ++c) {
+          double vx = (double)h.emb[(size_t)row * k + c] * x;
+          A[c] += vx; Q += vx * vx; pool[(size_t)f * k + c] += vx;
+        }
+      }
+    }
+    if (lr0) lr0[b] = lr;
+    double AA = 0;
+    for (uint32_t c = 0; c < k; ++c) { if (A0) A0[(size_t)b * k + c] = A[c]; AA += A[c] * A[c]; }
+    if (Q0) Q0[b] = Q;
+    if (fm2) fm2[b] = 0.5 * AA - 0.5 * Q;
+    if (pooled0) for (size_t i = 0; i < (size_t)F * k; ++i) pooled0[(size_t)b * F * k + i] = pool[i];
+    if ((ops & OP_DENSE1) && Z0) {
+      for (uint32_t h2 = 0; h2 < H; ++h2) {
+        double z = 0;
+        for (size_t i = 0; i < (size_t)F * k; ++i)
+          z += (double)bf16_round((float)pool[i]) * (double)bf16_round(t->W1[i * H + h2]);
+        Z0[(size_t)b * H + h2] = z;
+      }
+    }
+  }
+}
+
+// FM order-2 in its defining pair form, sum_{i<i'} <v_i, v_i'> x_i x_i'
+// (Eq. 5, first line): O(n^2 k), tiny inputs only.
+void orc_fm_pairs(void* p, const int32_t* offsets, const uint64_t* ids, const float* vals,
+                  int32_t B, double* fm_pairs) {
+  Table* t = (Table*)p;
+  const uint32_t F = t->F, k = t->k;
+  for (int32_t b = 0; b < B; ++b) {
+    std::vector<const float*> v; std::vector<double> x;
+    for (uint32_t f = 0; f < F; ++f) {
+      int64_t bag = (int64_t)b * F + f;
+      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
+        uint32_t s = t->shard_of(ids[j], f);
+        auto it = t->sh[s].map.find(ids[j]);
+        if (it == t->sh[s].map.end()) continue;
+        v.push_back(&t->sh[s].emb[(size_t)it->second * k]);
+        x.push_back(vals ? (double)vals[j] : 1.0);
+      }
+    }
+    double acc = 0;
+    for (size_t i = 0; i < v.size(); ++i)
+      for (size_t i2 = i + 1; i2 < v.size(); ++i2) {
+        double dot = 0;
+        for (uint32_t c = 0; c < k; ++c) dot += (double)v[i][c] * (double)v[i2][c];
+        acc += dot * x[i] * x[i2];
+      }
+    fm_pairs[b] = acc;
+  }
+}
+
+// Sub-operators of every shard (Eqs. 2 and 7; pooled per-field partials;
+// M_1(V_s, W_s) = V_s^T W_s).  Shard s only ever touches the keys it owns and
+// finds them through the (shard, row) pair that find_or_insert returned.
+//   part_small[S][B][k+2] = (M1_fm[0..k), M1_lr, M2_fm)
+//   part_pooled[S][B][F*k]  (optional)
+//   part_dense[S][B][H]     (optional; needs part_pooled semantics internally)
+void orc_forward_partials(void* p, uint32_t ops, const int32_t* offsets, const float* vals,
+                          const uint32_t* rows, const uint8_t* shards, int32_t B,
+                          double* part_small, double* part_pooled, double* part_dense) {
+  Table* t = (Table*)p;
+  const uint32_t S = t->S, F = t->F, k = t->k, H = t->H;
+  const size_t FK = (size_t)F * k;
+  std::vector<double> pool(FK);
+  for (uint32_t s = 0; s < S; ++s) {
+    const Shard& h = t->sh[s];
+    for (int32_t b = 0; b < B; ++b) {
+      double* ps = part_small ? part_small + ((size_t)s * B + b) * (k + 2) : nullptr;
+      if (ps) for (uint32_t c = 0; c < k + 2; ++c) ps[c] = 0;
+      std::fill(pool.begin(), pool.end(), 0.0);
+      for (uint32_t f = 0; f < F; ++f) {
+        int64_t bag = (int64_t)b * F + f;
+        for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
+          if (shards[j] != s || rows[j] == ROW_NONE) continue;
+          uint32_t row = rows[j];
+          double x = vals ? (double)vals[j] : 1.0;
+          if (ps) ps[k] += (double)h.lin[row] * x;
+          for (uint32_t c = 0; c < k; ++c) {
+            double vx = (double)h.emb[(size_t)row * k + c] * x;
+            if (ps) { ps[c] += vx; ps[k + 1] += vx * vx; }
+            pool[(size_t)f * k + c] += vx;
+          }
+        }
+      }
+      if (part_pooled) std::memcpy(part_pooled + ((size_t)s * B + b) * FK, pool.data(), FK * 8);
+      if ((ops & OP_DENSE1) && part_dense) {
+        for (uint32_t h2 = 0; h2 < H; ++h2) {
+          double z = 0;
+          for (size_t i = 0; i < FK; ++i)
+            if (pool[i] != 0.0) z += (double)bf16_round((float)pool[i]) * (double)bf16_round(t->W1[i * H + h2]);
+          part_dense[((size_t)s * B + b) * H + h2] = z;
+        }
+      }
+    }
+  }
+}
+
+// Aggregation over shards s = 0..S-1 (Eq. 1) and substitution operator F
+// (Eqs. 3 without sigma/bias, 8, 10).  out_small[B][k+3] = (A[0..k), R_lr, fm2, Q).
+void orc_aggregate(void* p, int32_t B, const double* part_small, const double* part_pooled,
+                   const double* part_dense, double* out_small, double* pooled, double* Z) {
+  Table* t = (Table*)p;
+  const uint32_t S = t->S, F = t->F, k = t->k, H = t->H;
+  const size_t FK = (size_t)F * k;
+  for (int32_t b = 0; b < B; ++b) {
+    if (part_small && out_small) {
+      double* o = out_small + (size_t)b * (k + 3);
+      for (uint32_t c = 0; c < k + 3; ++c) o[c] = 0;
+      double Q = 0;
+      for (uint32_t s = 0; s < S; ++s) {
+        const double* ps = part_small + ((size_t)s * B + b) * (k + 2);
+        for (uint32_t c = 0; c < k; ++c) o[c] += ps[c];
+        o[k] += ps[k]; Q += ps[k + 1];
+      }
+      double AA = 0;
+      for (uint32_t c = 0; c < k; ++c) AA += o[c] * o[c];
+      o[k + 1] = 0.5 * AA - 0.5 * Q; o[k + 2] = Q;
+    }
+    if (part_pooled && pooled)
+      for (size_t i = 0; i < FK; ++i) {
+        double a = 0;
+        for (uint32_t s = 0; s < S; ++s) a += part_pooled[((size_t)s * B + b) * FK + i];
+        pooled[(size_t)b * FK + i] = a;
+      }
+    if (part_dense && Z)
+      for (uint32_t h2 = 0; h2 < H; ++h2) {
+        double a = 0;
+        for (uint32_t s = 0; s < S; ++s) a += part_dense[((size_t)s * B + b) * H + h2];
+        Z[(size_t)b * H + h2] = a;
+      }
+  }
+}
+
+// Backward + update.  Per occurrence j of bag (b, f), owned by shard s:
+//   g_w(j) = x_j gL[b]                                   (d/dw of Eq. 3's sum)
+//   g_v(j) = x_j ( gF[b] (A[b] - v_j x_j) + gE[b][f] )   (d/dv of Eq. 8 + pooling)
+// evaluated with the PRE-update weights; with DENSE1, gE += gZ bf16(W1)^T first
+// (each shard only needs its own column block: no cross-shard term, Section
+// 3.2) and gW1 = bf16(pooled)^T gZ.  Then one optimizer application per unique
+// key on the summed gradient.  A is the aggregated (+)M_1 the caller got from
+// the forward (float32).  Optional outputs: Gw[U], Gv[U][k] (the summed
+// gradients, rounded to float32), gE_total[B][F*k].
+void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const float* vals,
+                         const uint32_t* rows, const uint8_t* shards, const uint32_t* uidx,
+                         int32_t B, int64_t U, const float* A, const float* pooled,
+                         const float* gL, const float* gF, const float* gE, const float* gZ,
+                         float* Gw_out, float* Gv_out, float* gE_total_out) {
+  Table* t = (Table*)p;
+  const uint32_t F = t->F, k = t->k, H = t->H;
+  const size_t FK = (size_t)F * k;
+  std::vector<float> gEt;
+  const bool use_pool = (ops & (OP_POOL | OP_DENSE1)) != 0;
+  if (use_pool) {
+    gEt.assign((size_t)B * FK, 0.0f);
+    for (size_t i = 0; i < (size_t)B * FK; ++i) {
+      double a = ((ops & OP_POOL) && gE) ? (double)gE[i] : 0.0;
+      if ((ops & OP_DENSE1) && gZ) {
+        size_t b = i / FK, col = i % FK;
+        for (uint32_t h2 = 0; h2 < H; ++h2)
+          a += (double)gZ[b * H + h2] * (double)bf16_round(t->W1[col * H + h2]);
+      }
+      gEt[i] = (float)a;
+    }
+    if (gE_total_out) std::memcpy(gE_total_out, gEt.data(), gEt.size() * 4);
+  }
+  std::vector<double> Gw((size_t)U, 0.0), Gv((size_t)U * k, 0.0);
+  std::vector<uint8_t> us((size_t)U); std::vector<uint32_t> ur((size_t)U);
+  for (int32_t b = 0; b < B; ++b)
+    for (uint32_t f = 0; f < F; ++f) {
+      int64_t bag = (int64_t)b * F + f;
+      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
+        if (rows[j] == ROW_NONE) continue;
+        uint32_t u = uidx[j], s = shards[j], row = rows[j];
+        us[u] = (uint8_t)s; ur[u] = row;
+        const Shard& h = t->sh[s];
+        double x = vals ? (double)vals[j] : 1.0;
+        if (ops & OP_LR) Gw[u] += x * (double)gL[b];
+        for (uint32_t c = 0; c < k; ++c) {
+          double g = 0;
+          if (ops & OP_FM) g += (double)gF[b] * ((double)A[(size_t)b * k + c] - (double)h.emb[(size_t)row * k + c] * x);
+          if (use_pool) g += (double)gEt[(size_t)b * FK + (size_t)f * k + c];
+          Gv[(size_t)u * k + c] += x * g;
+        }
+      }
+    }
+  for (int64_t u = 0; u < U; ++u) {
+    Shard& h = t->sh[us[u]];
+    uint32_t row = ur[u];
+    if (ops & OP_LR) apply_opt(*t, h.lin[row], h.acc_lin[row], Gw[u]);
+    if (ops & (OP_FM | OP_POOL | OP_DENSE1))
+      for (uint32_t c = 0; c < k; ++c)
+        apply_opt(*t, h.emb[(size_t)row * k + c], h.acc_emb[(size_t)row * k + c], Gv[(size_t)u * k + c]);
+    if (Gw_out) Gw_out[u] = (float)Gw[u];
+    if (Gv_out) for (uint32_t c = 0; c < k; ++c) Gv_out[(size_t)u * k + c] = (float)Gv[(size_t)u * k + c];
+  }
+  if ((ops & OP_DENSE1) && gZ && pooled) {
+    for (size_t i = 0; i < FK; ++i)
+      for (uint32_t h2 = 0; h2 < H; ++h2) {
+        double g = 0;
+        for (int32_t b = 0; b < B; ++b)
+          g += (double)bf16_round(pooled[(size_t)b * FK + i]) * (double)gZ[(size_t)b * H + h2];
+        apply_opt(*t, t->W1[i * H + h2], t->accW1[i * H + h2], g);
+      }
+  }
+}
+
+// Row contents by (shard, row).  Any output may be NULL.
+void orc_read_rows(void* p, int64_t n, const uint8_t* shard, const uint32_t* row,
+                   uint64_t* keys, float* emb, float* lin, float* acc_emb, float* acc_lin) {
+  Table* t = (Table*)p;
+  const uint32_t k = t->k;
+  for (int64_t i = 0; i < n; ++i) {
+    const Shard& h = t->sh[shard[i]];
+    uint32_t r = row[i];
+    if (keys) keys[i] = h.keys[r];
+    if (emb) std::memcpy(emb + (size_t)i * k, &h.emb[(size_t)r * k], k * 4);
+    if (lin) lin[i] = h.lin[r];
+    if (acc_emb) std::memcpy(acc_emb + (size_t)i * k, &h.acc_emb[(size_t)r * k], k * 4);
+    if (acc_lin) acc_lin[i] = h.acc_lin[r];
+  }
+}
+
+// Test hook: add delta to one stored weight (col < k: latent component,
+// col == k: linear weight).  Used by the finite-difference pins.
+void orc_poke(void* p, uint32_t shard, uint32_t row, uint32_t col, float value, int set) {
+  Table* t = (Table*)p;
+  Shard& h = t->sh[shard];
+  float& w = (col < t->k) ? h.emb[(size_t)row * t->k + col] : h.lin[row];
+  w = set ? value : w + value;
+}
+
+}  // extern "C"

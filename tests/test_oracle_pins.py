@@ -1,0 +1,325 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix
+(no GPU): known-answer vectors, closed forms, invariants, brute force."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import Oracle
+from paper_1909_04823_b200 import synth
+from paper_1909_04823_b200.synth import (OP_DENSE1, OP_FM, OP_LR, OP_POOL, OPT_ADAGRAD, OPT_SGD,
+                                          PART_FIELD, PART_HASH)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+ALL_OPS = OP_LR | OP_FM | OP_POOL
+
+
+def tiny(S=4, partition=PART_HASH, optimizer=OPT_SGD, k=8, F=6, B=24, H=0, ops=ALL_OPS, seed=11,
+         vocab=60, with_vals=False, len_b=4):
+    w = synth.Workload("tiny", B, F, k, S, partition, optimizer, ops, hidden=H, zipf_s=1.1, vocab=vocab,
+                       shared_vocab=(partition == PART_HASH), len_law="uniform", len_a=0, len_b=len_b,
+                       seed=seed, init_scale=0.5)
+    st = synth.Stream(w, with_vals=with_vals)
+    return w, st.next_batch()
+
+
+# --------------------------------------------------------------------------- RNG / hash
+def test_philox_known_answers():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 3
+    for r in rows:
+        v = [int(x, 16) for x in r]
+        assert oracle.philox4x32_10(v[0:4], v[4:6]) == v[6:10]
+
+
+def test_mix64_is_a_bijection():
+    # each step of the mixer is invertible; undo them here independently
+    M = (1 << 64) - 1
+    inv1 = pow(0xBF58476D1CE4E5B9, -1, 1 << 64)
+    inv2 = pow(0x94D049BB133111EB, -1, 1 << 64)
+
+    def unxorshift(y, s):
+        x = y
+        for _ in range(64 // s + 1):
+            x = y ^ (x >> s)
+        return x
+
+    rng = np.random.default_rng(0)
+    xs = [0, 1, M, 0x0123456789ABCDEF] + [int(v) for v in rng.integers(0, 2 ** 63, 2000)]
+    for x in xs:
+        z = oracle.mix64(x)
+        z = unxorshift(z, 31); z = (z * inv2) & M
+        z = unxorshift(z, 27); z = (z * inv1) & M
+        z = unxorshift(z, 30)
+        assert z == x
+
+
+def test_shard_balance_hash():
+    ids = synth.fmix64(np.arange(200_000, dtype=np.uint64))
+    for S in (3, 7, 64):
+        h = np.bincount(oracle.shard_of_many(ids, S), minlength=S)
+        mean = ids.size / S
+        assert np.all(np.abs(h - mean) < 6 * np.sqrt(mean))
+
+
+def test_init_is_exact_uniform_and_order_free():
+    # closed form: (r>>8) * 2^-23 - 1 times the scale, one rounding
+    seed, key = 0x1234567811223344, 0xDEADBEEFCAFEF00D
+    for c in range(12):
+        r = oracle.philox4x32_10([c // 4, 0, seed & 0xFFFFFFFF, seed >> 32], [key & 0xFFFFFFFF, key >> 32])[c % 4]
+        want = np.float32(np.float64(r >> 8) * 2.0 ** -23 - 1.0) * np.float32(0.37)
+        assert oracle.init_value(seed, key, c, 0.37) == np.float32(want)
+    vals = np.array([oracle.init_value(5, i, i % 8, 1.0) for i in range(20000)])
+    assert vals.min() >= -1.0 and vals.max() < 1.0
+    assert abs(vals.mean()) < 0.02 and abs(vals.var() - 1 / 3) < 0.02
+    # row contents depend on the key only, not on insertion order
+    w, b = tiny()
+    o1, o2 = Oracle.for_workload(w), Oracle.for_workload(w)
+    f1 = o1.find_or_insert(b)
+    rev = synth.Batch(b.batch, b.fields, b.offsets, b.ids.copy(), None)
+    perm = np.random.default_rng(1).permutation(b.nnz)
+    rev.ids = b.ids[perm]
+    f2 = o2.find_or_insert(rev)
+    r1 = o1.read_rows(f1["shards"], f1["rows"])
+    r2 = o2.read_rows(f2["shards"], f2["rows"])
+    d1 = {int(k): e.tobytes() for k, e in zip(r1["keys"], r1["emb"])}
+    d2 = {int(k): e.tobytes() for k, e in zip(r2["keys"], r2["emb"])}
+    assert d1 == d2 and len(d1) == len(np.unique(b.ids))
+
+
+def test_bf16_round_matches_torch():
+    x = torch.randn(5000, dtype=torch.float32) * 3
+    x = torch.cat([x, torch.tensor([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38])])
+    want = x.to(torch.bfloat16).to(torch.float32).numpy()
+    got = np.array([oracle.bf16_round(float(v)) for v in x.numpy()], dtype=np.float32)
+    assert np.array_equal(want.view(np.uint32), got.view(np.uint32))
+
+
+# --------------------------------------------------------------------------- table
+@pytest.mark.parametrize("partition", [PART_HASH, PART_FIELD])
+def test_row_numbering_first_occurrence_order(partition):
+    w, b = tiny(S=3, partition=partition, B=40)
+    o = Oracle.for_workload(w)
+    fi = o.find_or_insert(b)
+    # dictionary walk in CSR order
+    nxt = [0] * w.shards
+    seen, useen = {}, {}
+    for bag in range(b.batch * b.fields):
+        f = bag % b.fields
+        for j in range(b.offsets[bag], b.offsets[bag + 1]):
+            key = int(b.ids[j])
+            s = int(fi["shards"][j])
+            if partition == PART_FIELD:
+                assert s == f % w.shards
+            else:
+                assert s == oracle.mix64(key) % w.shards
+            if (s, key) not in seen:
+                seen[(s, key)] = nxt[s]; nxt[s] += 1
+                useen[(s, key)] = len(useen)
+            assert fi["rows"][j] == seen[(s, key)]
+            assert fi["uidx"][j] == useen[(s, key)]
+    assert list(o.size()) == nxt and fi["U"] == len(useen)
+    # lookup-only: known keys found, unknown ones get ROW_NONE, nothing inserted
+    b2 = synth.Batch(b.batch, b.fields, b.offsets, b.ids.copy(), None)
+    b2.ids[::5] = b2.ids[::5] ^ np.uint64(1 << 50)
+    f2 = o.find_or_insert(b2, insert=False)
+    assert list(o.size()) == nxt
+    miss = f2["rows"] == oracle.ROW_NONE
+    known = {(s, k) for (s, k) in seen}
+    for j in range(b.nnz):
+        assert miss[j] == ((int(f2["shards"][j]), int(b2.ids[j])) not in known)
+    # second insert call continues the numbering
+    f3 = o.find_or_insert(b2)
+    assert np.array_equal(f3["rows"][~miss], f2["rows"][~miss])
+    assert int(o.size().sum()) == len(seen) + len({(int(s), int(k)) for s, k in zip(f2["shards"][miss], b2.ids[miss])})
+
+
+# --------------------------------------------------------------------------- forward
+def test_fm_linear_form_equals_pair_form():
+    # Eq. 5: the O(nk) form equals the defining sum over pairs, duplicates included
+    w, b = tiny(with_vals=True, F=5, B=16, vocab=12)
+    o = Oracle.for_workload(w)
+    o.find_or_insert(b)
+    orig = o.forward_original(ALL_OPS, b)
+    pairs = o.fm_pairs(b)
+    assert np.max(np.abs(pairs)) > 1e-3
+    np.testing.assert_allclose(orig["fm2"], pairs, rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("partition", [PART_HASH, PART_FIELD])
+@pytest.mark.parametrize("S", [1, 2, 3, 4, 7, 64])
+def test_des_form_equals_original_operator(S, partition):
+    # Algorithm 1: F({(+) M_j}) == F_original, any S, both placements
+    w, b = tiny(S=S, partition=partition, with_vals=True, H=12, ops=ALL_OPS | OP_DENSE1)
+    o = Oracle.for_workload(w)
+    o.dense1_set(synth.dense1_weights(w))
+    fi = o.find_or_insert(b)
+    orig = o.forward_original(w.ops, b)
+    part = o.forward_partials(w.ops, b, fi, want_pooled=True, want_dense=True)
+    agg = o.aggregate(b.batch, part)
+    np.testing.assert_allclose(agg["lr"], orig["lr"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(agg["A"], orig["A"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(agg["Q"], orig["Q"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(agg["fm2"], orig["fm2"], rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(agg["pooled"], orig["pooled"], rtol=1e-12, atol=1e-14)
+    # under FIELD the row split is exact (each bag lives in one shard); under HASH
+    # the bf16 rounding of per-shard pooled partials differs from rounding the sum
+    tol = 1e-12 if partition == PART_FIELD or S == 1 else 2e-2
+    np.testing.assert_allclose(agg["Z"], orig["Z"], rtol=tol, atol=tol * np.abs(orig["Z"]).max())
+    if partition == PART_FIELD:
+        # a bag is owned by exactly one shard
+        pp = part["part_pooled"].reshape(S, b.batch, w.fields, w.emb_dim)
+        for f in range(w.fields):
+            others = [s for s in range(S) if s != f % S]
+            assert not np.any(pp[others, :, f, :])
+
+
+def test_any_S_gives_the_S1_result():
+    res = []
+    for S in (1, 2, 3, 4, 7, 64):
+        w, b = tiny(S=S, with_vals=True)
+        o = Oracle.for_workload(w)
+        fi = o.find_or_insert(b)
+        agg = o.aggregate(b.batch, o.forward_partials(w.ops, b, fi))
+        rows = o.read_rows(fi["shards"], fi["rows"])
+        res.append((agg["out_small"], agg["pooled"], rows["keys"], rows["emb"]))
+    for r in res[1:]:
+        np.testing.assert_allclose(r[0], res[0][0], rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(r[1], res[0][1], rtol=1e-11, atol=1e-13)
+        assert np.array_equal(r[2], res[0][2]) and np.array_equal(r[3], res[0][3])
+
+
+def test_row_split_gemm_is_one_dense_matmul():
+    # Eq. 9: [V_1^T .. V_N^T] [W_1; ..; W_N] == V^T W on the same rounded operands
+    w, b = tiny(S=4, partition=PART_FIELD, H=20, ops=OP_POOL | OP_DENSE1, k=4, F=7)
+    o = Oracle.for_workload(w)
+    W1 = synth.dense1_weights(w)
+    o.dense1_set(W1)
+    fi = o.find_or_insert(b)
+    part = o.forward_partials(w.ops, b, fi, want_pooled=True, want_dense=True)
+    agg = o.aggregate(b.batch, part)
+    bf = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    want = bf(agg["pooled"]) @ bf(W1)
+    np.testing.assert_allclose(agg["Z"], want, rtol=1e-12, atol=1e-14)
+    # each shard's partial uses only its own row block of W1
+    FK = w.fields * w.emb_dim
+    for s in range(w.shards):
+        mask = np.zeros(FK, bool)
+        for f in range(w.fields):
+            if f % w.shards == s:
+                mask[f * w.emb_dim:(f + 1) * w.emb_dim] = True
+        want_s = bf(agg["pooled"])[:, mask] @ bf(W1)[mask]
+        np.testing.assert_allclose(part["part_dense"][s], want_s, rtol=1e-12, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- backward
+def _functional(o, w, b, fi, g):
+    """L = <gL,R_lr> + <gF,fm2> + <gE,pooled> + <gZ,Z> on the oracle's own forward."""
+    orig = o.forward_original(w.ops, b)
+    L = 0.0
+    if w.ops & OP_LR:
+        L += float(np.dot(g["gL"].astype(np.float64), orig["lr"]))
+    if w.ops & OP_FM:
+        L += float(np.dot(g["gF"].astype(np.float64), orig["fm2"]))
+    if w.ops & OP_POOL:
+        L += float(np.sum(g["gE"].astype(np.float64) * orig["pooled"]))
+    return L
+
+
+@pytest.mark.parametrize("partition", [PART_HASH, PART_FIELD])
+def test_gradients_match_central_differences(partition):
+    # Section 3.2: the aggregate's gradient, sent back to each shard's own
+    # sub-operator, is the gradient of the unsubstituted model.
+    w, b = tiny(S=3, partition=partition, with_vals=True, B=10, F=4, vocab=15)
+    g = synth.upstream_grads(w, b.batch, 0)
+    o = Oracle.for_workload(w)                      # SGD: theta_new = theta - lr * G
+    fi = o.find_or_insert(b)
+    agg = o.aggregate(b.batch, o.forward_partials(w.ops, b, fi))
+    # finite differences first (table still unchanged)
+    us, ur = fi["uniq_shard"], fi["uniq_row"]
+    fd = np.zeros((fi["U"], w.emb_dim + 1))
+    h = 1e-3
+    for u in range(fi["U"]):
+        for c in range(w.emb_dim + 1):
+            o.poke(us[u], ur[u], c, h); Lp = _functional(o, w, b, fi, g)
+            o.poke(us[u], ur[u], c, -2 * h); Lm = _functional(o, w, b, fi, g)
+            o.poke(us[u], ur[u], c, h)
+            fd[u, c] = (Lp - Lm) / (2 * h)
+    before = o.read_rows(us, ur)
+    res = o.backward_update(w.ops, b, fi, agg["A"], agg["pooled"], g["gL"], g["gF"], g["gE"])
+    after = o.read_rows(us, ur)
+    assert np.abs(fd).max() > 0.1
+    np.testing.assert_allclose(res["Gv"], fd[:, :w.emb_dim], rtol=2e-3, atol=2e-4)
+    np.testing.assert_allclose(res["Gw"], fd[:, w.emb_dim], rtol=2e-3, atol=2e-4)
+    # and the SGD step applied exactly that gradient, once per key
+    np.testing.assert_allclose(before["emb"] - after["emb"], w.lr * res["Gv"], rtol=1e-4, atol=1e-7)
+    np.testing.assert_allclose(before["lin"] - after["lin"], w.lr * res["Gw"], rtol=1e-4, atol=1e-7)
+
+
+def test_dense1_backward_matches_dense_algebra():
+    w, b = tiny(S=4, partition=PART_FIELD, H=10, ops=OP_LR | OP_POOL | OP_DENSE1, k=4, F=5, B=12)
+    o = Oracle.for_workload(w)
+    W1 = synth.dense1_weights(w)
+    o.dense1_set(W1)
+    fi = o.find_or_insert(b)
+    agg = o.aggregate(b.batch, o.forward_partials(w.ops, b, fi, True, True))
+    g = synth.upstream_grads(w, b.batch, 0)
+    pooled32 = agg["pooled"].astype(np.float32)
+    res = o.backward_update(w.ops, b, fi, agg["A"], pooled32, g["gL"], None, g["gE"], g["gZ"])
+    bf = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    want_gE = g["gE"].astype(np.float64) + g["gZ"].astype(np.float64) @ bf(W1).T
+    np.testing.assert_allclose(res["gE_total"], want_gE, rtol=1e-6, atol=1e-6)
+    W1n, _ = o.dense1_get()
+    gW = bf(pooled32).T @ g["gZ"].astype(np.float64)
+    np.testing.assert_allclose(W1.astype(np.float64) - W1n, w.lr * gW, rtol=1e-4, atol=1e-7)
+
+
+def test_dedup_special_cases():
+    k, F = 4, 1
+    mk = lambda opt: Oracle(2, F, k, 0, PART_HASH, opt, seed=3, init_scale=0.5, lr=0.1, eps=1e-8)
+    n = 5
+    key = np.uint64(777)
+    # n copies of one key, one per sample  ==  one update with G = sum of the n terms
+    bn = synth.Batch(n, F, np.arange(n + 1, dtype=np.int32), np.full(n, key, np.uint64), None)
+    b1 = synth.Batch(1, F, np.arange(2, dtype=np.int32), np.full(1, key, np.uint64), None)
+    gE = np.random.default_rng(0).standard_normal((n, k)).astype(np.float32)
+    for opt in (OPT_SGD, OPT_ADAGRAD):
+        oa, ob = mk(opt), mk(opt)
+        fa = oa.find_or_insert(bn); fb = ob.find_or_insert(b1)
+        assert fa["U"] == 1
+        oa.backward_update(OP_POOL, bn, fa, np.zeros((n, k)), None, None, None, gE)
+        ob.backward_update(OP_POOL, b1, fb, np.zeros((1, k)), None, None, None, gE.sum(0, keepdims=True))
+        ra = oa.read_rows(fa["uniq_shard"], fa["uniq_row"]); rb = ob.read_rows(fb["uniq_shard"], fb["uniq_row"])
+        np.testing.assert_allclose(ra["emb"], rb["emb"], rtol=1e-6, atol=1e-7)
+        np.testing.assert_allclose(ra["acc_emb"], rb["acc_emb"], rtol=1e-6, atol=1e-7)
+    # Adagrad from a = 0: a' = G^2 (the square of the SUM), step = lr * G / (|G| + eps)
+    o = mk(OPT_ADAGRAD)
+    f = o.find_or_insert(bn)
+    before = o.read_rows(f["uniq_shard"], f["uniq_row"])
+    o.backward_update(OP_POOL, bn, f, np.zeros((n, k)), None, None, None, gE)
+    after = o.read_rows(f["uniq_shard"], f["uniq_row"])
+    G = gE.astype(np.float64).sum(0)
+    np.testing.assert_allclose(after["acc_emb"][0], G * G, rtol=1e-6)
+    np.testing.assert_allclose(before["emb"][0] - after["emb"][0], 0.1 * np.sign(G), rtol=1e-5, atol=1e-7)
+    # all-unique batch: dedup changes nothing (each key sees its own single term)
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    bu = synth.Batch(n, F, np.arange(n + 1, dtype=np.int32), keys, None)
+    o = mk(OPT_ADAGRAD)
+    f = o.find_or_insert(bu)
+    assert f["U"] == n
+    before = o.read_rows(f["uniq_shard"], f["uniq_row"])
+    o.backward_update(OP_POOL, bu, f, np.zeros((n, k)), None, None, None, gE)
+    after = o.read_rows(f["uniq_shard"], f["uniq_row"])
+    np.testing.assert_allclose(before["emb"] - after["emb"], 0.1 * np.sign(gE), rtol=1e-5, atol=1e-7)
+
+
+def test_paper_table2_comm_saving():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_table2_comm_saving.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 5
+    for r in rows:
+        B, U = int(r[0]), int(r[1])
+        got = 100.0 * oracle.comm_saving(B, U, 8, 256, 4800 * 256 * 4)
+        for gv, want in zip(got, r[2:5]):
+            assert f"{gv:.3f}" == want
