@@ -99,6 +99,8 @@ typedef struct {
                                  a starts at init_acc                                */
   int64_t  max_nnz;      /* largest nnz of any batch (sizes the workspace)            */
   int32_t  max_batch;    /* largest B of any batch                                    */
+  int64_t  max_uniq;     /* largest number of distinct keys in one batch (sizes the
+                            gradient buffer: max_uniq*(k+4)*4 bytes); 0 = max_nnz     */
   /* optional device allocator (e.g. backed by the caller's caching allocator);
    * NULL = cudaMalloc / cudaFree.  alloc must return 256-byte aligned memory.   */
   void* (*alloc)(size_t bytes, void* ctx);
@@ -222,6 +224,13 @@ des_status_t des_table_export(des_table_t* t, uint64_t* d_keys, uint8_t* d_shard
 des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
                                  float* d_emb, float* d_lin, float* d_acc_emb, float* d_acc_lin,
                                  void* stream);
+
+/* Inverse of des_table_read_rows (restore from a checkpoint, re-seeding rows):
+ * overwrites the rows of the n table-global rows d_global_rows[] from dense
+ * device arrays; NULL inputs leave that part untouched.  Rows must exist. */
+des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                  const float* d_emb, const float* d_lin, const float* d_acc_emb,
+                                  const float* d_acc_lin, void* stream);
 
 /* ---- whole step from host buffers ---------------------------------------- */
 

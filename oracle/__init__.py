@@ -150,11 +150,13 @@ class Oracle:
         lr0 = np.zeros(B); A0 = np.zeros((B, k)); Q0 = np.zeros(B); fm2 = np.zeros(B)
         pooled0 = np.zeros((B, F * k))
         Z0 = np.zeros((B, H)) if H else None
+        Sabs = np.zeros((B, k + 1))
         self.L.orc_forward_original(self.h, C.c_uint32(ops), _p(batch.offsets, C.c_int32),
                                     _p(batch.ids, C.c_uint64), _p(batch.vals, C.c_float), C.c_int32(B),
                                     _p(lr0, C.c_double), _p(A0, C.c_double), _p(Q0, C.c_double),
-                                    _p(fm2, C.c_double), _p(pooled0, C.c_double), _p(Z0, C.c_double))
-        return dict(lr=lr0, A=A0, Q=Q0, fm2=fm2, pooled=pooled0, Z=Z0)
+                                    _p(fm2, C.c_double), _p(pooled0, C.c_double), _p(Z0, C.c_double),
+                                    _p(Sabs, C.c_double))
+        return dict(lr=lr0, A=A0, Q=Q0, fm2=fm2, pooled=pooled0, Z=Z0, Sabs=Sabs)
 
     def fm_pairs(self, batch):
         out = np.zeros(batch.batch)
@@ -195,13 +197,15 @@ class Oracle:
         Gw = np.zeros(U, dtype=np.float32)
         Gv = np.zeros((U, k), dtype=np.float32)
         gEt = np.zeros((B, F * k), dtype=np.float32)
+        Sw = np.zeros(U); Sv = np.zeros((U, k))
         self.L.orc_backward_update(self.h, C.c_uint32(ops), _p(batch.offsets, C.c_int32),
                                    _p(batch.vals, C.c_float), _p(fi["rows"], C.c_uint32),
                                    _p(fi["shards"], C.c_uint8), _p(fi["uidx"], C.c_uint32),
                                    C.c_int32(B), C.c_int64(U), _p(A, C.c_float), _p(pooled, C.c_float),
                                    _p(gL, C.c_float), _p(gF, C.c_float), _p(gE, C.c_float), _p(gZ, C.c_float),
-                                   _p(Gw, C.c_float), _p(Gv, C.c_float), _p(gEt, C.c_float))
-        return dict(Gw=Gw, Gv=Gv, gE_total=gEt)
+                                   _p(Gw, C.c_float), _p(Gv, C.c_float), _p(gEt, C.c_float),
+                                   _p(Sw, C.c_double), _p(Sv, C.c_double))
+        return dict(Gw=Gw, Gv=Gv, gE_total=gEt, Sw=Sw, Sv=Sv)
 
     def read_rows(self, shard, row):
         shard = np.ascontiguousarray(shard, dtype=np.uint8)

@@ -226,9 +226,11 @@ int64_t orc_find_or_insert(void* p, const int32_t* offsets, const uint64_t* ids,
 // A0[B][k] = sum v x, Q0[B] = sum <vx,vx>, fm2[B] linear form (Eq. 5, last
 // line); pooled0[B][F*k] (embedding layer, Section 4.3); Z0[B][H] = V^T W
 // (Eq. 6) on bfloat16-rounded operands (reading), accumulated in double.
+// Sabs[B][k+1] (optional): sums of the absolute values of the terms of A0 and
+// lr0, the scale of a float32 summation error when the terms cancel.
 void orc_forward_original(void* p, uint32_t ops, const int32_t* offsets, const uint64_t* ids,
                           const float* vals, int32_t B, double* lr0, double* A0, double* Q0,
-                          double* fm2, double* pooled0, double* Z0) {
+                          double* fm2, double* pooled0, double* Z0, double* Sabs) {
   Table* t = (Table*)p;
   const uint32_t F = t->F, k = t->k, H = t->H;
   std::vector<double> A(k), pool((size_t)F * k);
@@ -246,9 +248,11 @@ void orc_forward_original(void* p, uint32_t ops, const int32_t* offsets, const u
         uint32_t row = it->second;
         double x = vals ? (double)vals[j] : 1.0;
         lr += (double)h.lin[row] * x;
+        if (Sabs) Sabs[(size_t)b * (k + 1) + k] += std::fabs((double)h.lin[row] * x);
         for (uint32_t c = 0; c < k; ++c) {
           double vx = (double)h.emb[(size_t)row * k + c] * x;
           A[c] += vx; Q += vx * vx; pool[(size_t)f * k + c] += vx;
+          if (Sabs) Sabs[(size_t)b * (k + 1) + c] += std::fabs(vx);
         }
       }
     }
@@ -388,12 +392,14 @@ void orc_aggregate(void* p, int32_t B, const double* part_small, const double* p
 // 3.2) and gW1 = bf16(pooled)^T gZ.  Then one optimizer application per unique
 // key on the summed gradient.  A is the aggregated (+)M_1 the caller got from
 // the forward (float32).  Optional outputs: Gw[U], Gv[U][k] (the summed
-// gradients, rounded to float32), gE_total[B][F*k].
+// gradients, rounded to float32), gE_total[B][F*k], and Sw[U], Sv[U][k]: the sums
+// of the ABSOLUTE values of the same per-occurrence terms (the scale against
+// which a float32 summation error is measured when the terms cancel).
 void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const float* vals,
                          const uint32_t* rows, const uint8_t* shards, const uint32_t* uidx,
                          int32_t B, int64_t U, const float* A, const float* pooled,
                          const float* gL, const float* gF, const float* gE, const float* gZ,
-                         float* Gw_out, float* Gv_out, float* gE_total_out) {
+                         float* Gw_out, float* Gv_out, float* gE_total_out, double* Sw_out, double* Sv_out) {
   Table* t = (Table*)p;
   const uint32_t F = t->F, k = t->k, H = t->H;
   const size_t FK = (size_t)F * k;
@@ -413,6 +419,7 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
     if (gE_total_out) std::memcpy(gE_total_out, gEt.data(), gEt.size() * 4);
   }
   std::vector<double> Gw((size_t)U, 0.0), Gv((size_t)U * k, 0.0);
+  std::vector<double> Sw((size_t)U, 0.0), Sv((size_t)U * k, 0.0);
   std::vector<uint8_t> us((size_t)U); std::vector<uint32_t> ur((size_t)U);
   for (int32_t b = 0; b < B; ++b)
     for (uint32_t f = 0; f < F; ++f) {
@@ -423,12 +430,13 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
         us[u] = (uint8_t)s; ur[u] = row;
         const Shard& h = t->sh[s];
         double x = vals ? (double)vals[j] : 1.0;
-        if (ops & OP_LR) Gw[u] += x * (double)gL[b];
+        if (ops & OP_LR) { Gw[u] += x * (double)gL[b]; Sw[u] += std::fabs(x * (double)gL[b]); }
         for (uint32_t c = 0; c < k; ++c) {
           double g = 0;
           if (ops & OP_FM) g += (double)gF[b] * ((double)A[(size_t)b * k + c] - (double)h.emb[(size_t)row * k + c] * x);
           if (use_pool) g += (double)gEt[(size_t)b * FK + (size_t)f * k + c];
           Gv[(size_t)u * k + c] += x * g;
+          Sv[(size_t)u * k + c] += std::fabs(x * g);
         }
       }
     }
@@ -439,6 +447,8 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
     if (ops & (OP_FM | OP_POOL | OP_DENSE1))
       for (uint32_t c = 0; c < k; ++c)
         apply_opt(*t, h.emb[(size_t)row * k + c], h.acc_emb[(size_t)row * k + c], Gv[(size_t)u * k + c]);
+    if (Sw_out) Sw_out[u] = Sw[u];
+    if (Sv_out) for (uint32_t c = 0; c < k; ++c) Sv_out[(size_t)u * k + c] = Sv[(size_t)u * k + c];
     if (Gw_out) Gw_out[u] = (float)Gw[u];
     if (Gv_out) for (uint32_t c = 0; c < k; ++c) Gv_out[(size_t)u * k + c] = (float)Gv[(size_t)u * k + c];
   }

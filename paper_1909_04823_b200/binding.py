@@ -1,0 +1,293 @@
+"""Thin ctypes binding of libdes.so — argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; torch is used for
+device memory and streams.  If the library cannot be loaded this module raises:
+there is no CPU fallback."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OP_LR, OP_FM, OP_POOL, OP_DENSE1 = 1, 2, 4, 8
+PART_HASH, PART_FIELD = 0, 1
+OPT_SGD, OPT_ADAGRAD = 0, 1
+ROW_NONE = 0xFFFFFFFF
+KEY_EMPTY = 0xFFFFFFFFFFFFFFFF
+
+STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "DES_ERR_CAPACITY",
+          4: "DES_ERR_UNSUPPORTED", 5: "DES_ERR_CUDA", 6: "DES_ERR_NOT_FOUND"}
+
+EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
+           "des_aggregate", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_table_status",
+           "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
+           "des_step_host", "des_table_launch_count", "des_status_string"]
+
+
+class DesError(RuntimeError):
+    def __init__(self, code, where):
+        super().__init__(f"{where}: {STATUS.get(code, code)}")
+        self.code = code
+
+
+class des_config_t(C.Structure):
+    _fields_ = [("num_shards", C.c_uint32), ("num_fields", C.c_uint32), ("emb_dim", C.c_uint32),
+                ("hidden", C.c_uint32), ("partition", C.c_uint32), ("optimizer", C.c_uint32),
+                ("max_rows", C.c_uint64), ("max_load", C.c_float),
+                ("h_rows_per_shard", C.POINTER(C.c_uint64)),
+                ("seed", C.c_uint64), ("init_scale", C.c_float),
+                ("lr", C.c_float), ("eps", C.c_float), ("init_acc", C.c_float),
+                ("max_nnz", C.c_int64), ("max_batch", C.c_int32), ("max_uniq", C.c_int64),
+                ("alloc", C.c_void_p), ("dealloc", C.c_void_p), ("alloc_ctx", C.c_void_p)]
+
+
+class des_batch_t(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("nnz", C.c_int64), ("offsets", C.c_void_p), ("ids", C.c_void_p),
+                ("vals", C.c_void_p), ("rows", C.c_void_p), ("shards", C.c_void_p), ("uidx", C.c_void_p),
+                ("uniq_rows", C.c_void_p), ("n_uniq", C.c_void_p)]
+
+
+class des_partials_t(C.Structure):
+    _fields_ = [("part_small", C.c_void_p), ("pooled", C.c_void_p), ("part_pooled", C.c_void_p),
+                ("part_dense", C.c_void_p)]
+
+
+class des_outputs_t(C.Structure):
+    _fields_ = [("out_small", C.c_void_p), ("pooled", C.c_void_p), ("Z", C.c_void_p)]
+
+
+class des_grads_t(C.Structure):
+    _fields_ = [("gL", C.c_void_p), ("gF", C.c_void_p), ("gE", C.c_void_p), ("gZ", C.c_void_p),
+                ("gE_work", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load():
+    """Loads (building first if the sources are newer) the CUDA library."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        for name in EXPORTS:
+            getattr(L, name)  # fail loudly on a missing symbol
+        L.des_table_create.argtypes = [C.POINTER(des_config_t), C.POINTER(C.c_void_p)]
+        L.des_table_destroy.argtypes = [C.c_void_p]
+        L.des_find_or_insert.argtypes = [C.c_void_p, C.POINTER(des_batch_t), C.c_int, C.c_void_p]
+        L.des_forward_partials.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
+                                           C.POINTER(des_partials_t), C.c_void_p]
+        L.des_aggregate.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
+                                    C.POINTER(des_outputs_t), C.c_void_p]
+        L.des_backward_update.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
+                                          C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
+        L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_dense1_get.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_table_status.argtypes = [C.c_void_p]
+        L.des_table_size.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+        L.des_table_row_base.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+        L.des_table_export.argtypes = [C.c_void_p] + [C.c_void_p] * 7 + [C.c_uint64, C.POINTER(C.c_uint64)]
+        L.des_table_read_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
+        L.des_table_write_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
+        L.des_step_host.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                    C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_void_p]
+        L.des_table_launch_count.argtypes = [C.c_void_p]
+        L.des_table_launch_count.restype = C.c_uint64
+        L.des_status_string.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class DeviceBatch:
+    """Device-resident batch plus the index arrays find_or_insert fills."""
+
+    def __init__(self, offsets, ids, vals, batch, device="cuda"):
+        as_dev = lambda a, dt: a.to(device=device, dtype=dt) if isinstance(a, torch.Tensor) else \
+            torch.from_numpy(a).to(device=device, dtype=dt)
+        self.batch = int(batch)
+        self.offsets = as_dev(offsets, torch.int32).contiguous()
+        if isinstance(ids, torch.Tensor):
+            self.ids = ids.to(device).contiguous()
+        else:
+            self.ids = torch.from_numpy(ids.view("int64")).to(device).contiguous()
+        self.vals = None if vals is None else as_dev(vals, torch.float32).contiguous()
+        self.nnz = int(self.ids.numel())
+        n = max(self.nnz, 1)
+        self.rows = torch.empty(n, dtype=torch.int32, device=device)      # uint32 payload
+        self.shards = torch.empty(n, dtype=torch.uint8, device=device)
+        self.uidx = torch.empty(n, dtype=torch.int32, device=device)
+        self.uniq_rows = torch.empty(n, dtype=torch.int32, device=device)
+        self.n_uniq = torch.zeros(1, dtype=torch.int32, device=device)
+
+    @classmethod
+    def from_synth(cls, b, device="cuda"):
+        return cls(b.offsets, b.ids, b.vals, b.batch, device)
+
+    def c(self) -> des_batch_t:
+        return des_batch_t(self.batch, self.nnz, _ptr(self.offsets), _ptr(self.ids), _ptr(self.vals),
+                           _ptr(self.rows), _ptr(self.shards), _ptr(self.uidx), _ptr(self.uniq_rows),
+                           _ptr(self.n_uniq))
+
+
+class Table:
+    """Owner of one des_table_t.  Methods have the names of the C entry points
+    and only marshal arguments."""
+
+    def __init__(self, num_shards, num_fields, emb_dim, hidden=0, partition=PART_HASH, optimizer=OPT_SGD,
+                 max_rows=1 << 20, max_load=0.5, rows_per_shard=None, seed=0, init_scale=0.01, lr=0.01,
+                 eps=1e-8, init_acc=0.0, max_nnz=1 << 20, max_batch=1 << 16, max_uniq=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_1909_04823_b200 needs a CUDA device; there is no CPU path")
+        self.L = load()
+        self.S, self.F, self.k, self.H = num_shards, num_fields, emb_dim, hidden
+        self.stride = emb_dim + 4
+        cfg = des_config_t()
+        cfg.num_shards, cfg.num_fields, cfg.emb_dim, cfg.hidden = num_shards, num_fields, emb_dim, hidden
+        cfg.partition, cfg.optimizer = partition, optimizer
+        cfg.max_rows, cfg.max_load = int(max_rows), max_load
+        self._rps = None
+        if rows_per_shard is not None:
+            self._rps = (C.c_uint64 * num_shards)(*[int(v) for v in rows_per_shard])
+            cfg.h_rows_per_shard = C.cast(self._rps, C.POINTER(C.c_uint64))
+        cfg.seed, cfg.init_scale, cfg.lr, cfg.eps, cfg.init_acc = int(seed), init_scale, lr, eps, init_acc
+        cfg.max_nnz, cfg.max_batch, cfg.max_uniq = int(max_nnz), int(max_batch), int(max_uniq)
+        self.h = C.c_void_p()
+        self._check(self.L.des_table_create(C.byref(cfg), C.byref(self.h)), "des_table_create")
+
+    @classmethod
+    def for_workload(cls, w, max_rows, max_nnz, max_batch=None, rows_per_shard=None, max_uniq=0, max_load=0.5):
+        return cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, max_rows=max_rows,
+                   max_load=max_load, rows_per_shard=rows_per_shard, seed=w.seed, init_scale=w.init_scale,
+                   lr=w.lr, eps=w.eps, init_acc=w.init_acc, max_nnz=max_nnz,
+                   max_batch=max_batch or w.batch, max_uniq=max_uniq)
+
+    def _check(self, code, where):
+        if code != 0:
+            raise DesError(code, where)
+
+    def close(self):
+        if getattr(self, "h", None) and self.h.value:
+            self.L.des_table_destroy(self.h)
+            self.h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the five calls of the path -------------------------------------------
+    def find_or_insert(self, batch: DeviceBatch, insert: bool = True):
+        cb = batch.c()
+        self._check(self.L.des_find_or_insert(self.h, C.byref(cb), 1 if insert else 0, _stream()),
+                    "des_find_or_insert")
+
+    def forward_partials(self, ops, batch, part_small=None, pooled=None, part_pooled=None, part_dense=None):
+        cb = batch.c()
+        p = des_partials_t(_ptr(part_small), _ptr(pooled), _ptr(part_pooled), _ptr(part_dense))
+        self._check(self.L.des_forward_partials(self.h, ops, C.byref(cb), C.byref(p), _stream()),
+                    "des_forward_partials")
+
+    def aggregate(self, ops, batch, part_small=None, pooled=None, part_pooled=None, part_dense=None,
+                  out_small=None, out_pooled=None, Z=None):
+        cb = batch.c()
+        p = des_partials_t(_ptr(part_small), _ptr(pooled), _ptr(part_pooled), _ptr(part_dense))
+        o = des_outputs_t(_ptr(out_small), _ptr(out_pooled if out_pooled is not None else pooled), _ptr(Z))
+        self._check(self.L.des_aggregate(self.h, ops, C.byref(cb), C.byref(p), C.byref(o), _stream()),
+                    "des_aggregate")
+
+    def backward_update(self, ops, batch, out_small=None, pooled=None, Z=None, gL=None, gF=None, gE=None,
+                        gZ=None, gE_work=None):
+        cb = batch.c()
+        o = des_outputs_t(_ptr(out_small), _ptr(pooled), _ptr(Z))
+        g = des_grads_t(_ptr(gL), _ptr(gF), _ptr(gE), _ptr(gZ), _ptr(gE_work))
+        self._check(self.L.des_backward_update(self.h, ops, C.byref(cb), C.byref(o), C.byref(g), _stream()),
+                    "des_backward_update")
+
+    def step_host(self, ops, batch_size, nnz, h_offsets, h_ids, h_vals, h_out_small, d_pooled=None, d_Z=None,
+                  gL=None, gF=None, gE=None, gZ=None, gE_work=None):
+        g = des_grads_t(_ptr(gL), _ptr(gF), _ptr(gE), _ptr(gZ), _ptr(gE_work))
+        self._check(self.L.des_step_host(self.h, ops, batch_size, nnz, _ptr(h_offsets), _ptr(h_ids),
+                                         _ptr(h_vals), C.byref(g), _ptr(d_pooled), _ptr(d_Z),
+                                         _ptr(h_out_small), _stream()), "des_step_host")
+
+    # -- first dense layer ----------------------------------------------------------
+    def dense1_set(self, W1: torch.Tensor):
+        assert W1.is_cuda and W1.dtype == torch.float32 and W1.shape == (self.F * self.k, self.H)
+        self._check(self.L.des_dense1_set(self.h, _ptr(W1.contiguous()), _stream()), "des_dense1_set")
+        torch.cuda.current_stream().synchronize()
+
+    def dense1_get(self) -> torch.Tensor:
+        W1 = torch.empty((self.F * self.k, self.H), dtype=torch.float32, device="cuda")
+        self._check(self.L.des_dense1_get(self.h, _ptr(W1), _stream()), "des_dense1_get")
+        return W1
+
+    # -- inspection -------------------------------------------------------------------
+    def status(self) -> int:
+        return int(self.L.des_table_status(self.h))
+
+    def check_status(self):
+        self._check(self.status(), "des_table_status")
+
+    def size(self):
+        out = (C.c_uint64 * self.S)()
+        self._check(self.L.des_table_size(self.h, out), "des_table_size")
+        return [int(v) for v in out]
+
+    def row_base(self):
+        out = (C.c_uint64 * (self.S + 1))()
+        self._check(self.L.des_table_row_base(self.h, out), "des_table_row_base")
+        return [int(v) for v in out]
+
+    def launch_count(self) -> int:
+        return int(self.L.des_table_launch_count(self.h))
+
+    def export(self, cap: int):
+        dev = "cuda"
+        keys = torch.empty(cap, dtype=torch.int64, device=dev)
+        shards = torch.empty(cap, dtype=torch.uint8, device=dev)
+        rows = torch.empty(cap, dtype=torch.int32, device=dev)
+        emb = torch.empty((cap, self.k), dtype=torch.float32, device=dev)
+        lin = torch.empty(cap, dtype=torch.float32, device=dev)
+        ae = torch.empty((cap, self.k), dtype=torch.float32, device=dev)
+        al = torch.empty(cap, dtype=torch.float32, device=dev)
+        n = C.c_uint64(0)
+        torch.cuda.synchronize()
+        self._check(self.L.des_table_export(self.h, _ptr(keys), _ptr(shards), _ptr(rows), _ptr(emb), _ptr(lin),
+                                            _ptr(ae), _ptr(al), cap, C.byref(n)), "des_table_export")
+        m = min(int(n.value), cap)
+        return dict(n=int(n.value), keys=keys[:m], shards=shards[:m], rows=rows[:m], emb=emb[:m], lin=lin[:m],
+                    acc_emb=ae[:m], acc_lin=al[:m])
+
+    def read_rows(self, global_rows: torch.Tensor):
+        n = int(global_rows.numel())
+        dev = "cuda"
+        emb = torch.empty((n, self.k), dtype=torch.float32, device=dev)
+        lin = torch.empty(n, dtype=torch.float32, device=dev)
+        ae = torch.empty((n, self.k), dtype=torch.float32, device=dev)
+        al = torch.empty(n, dtype=torch.float32, device=dev)
+        self._check(self.L.des_table_read_rows(self.h, _ptr(global_rows), n, _ptr(emb), _ptr(lin), _ptr(ae),
+                                               _ptr(al), _stream()), "des_table_read_rows")
+        return dict(emb=emb, lin=lin, acc_emb=ae, acc_lin=al)
+
+    def write_rows(self, global_rows: torch.Tensor, emb=None, lin=None, acc_emb=None, acc_lin=None):
+        n = int(global_rows.numel())
+        self._check(self.L.des_table_write_rows(self.h, _ptr(global_rows), n, _ptr(emb), _ptr(lin), _ptr(acc_emb),
+                                                _ptr(acc_lin), _stream()), "des_table_write_rows")

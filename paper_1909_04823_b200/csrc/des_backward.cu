@@ -1,0 +1,326 @@
+// Backward of the DES sparse operators and the table update (Section 3.2,
+// "Back-propagation Phase"; Section 5, `update`).
+//
+// The aggregation hands every shard the same upstream gradient, so each
+// occurrence j of bag (b, f) contributes, to its own key only,
+//   g_w(j) = x_j gL[b]
+//   g_v(j) = x_j ( gF[b] (A[b] - v_j x_j) + gE[b][f] )
+// Summed over a key's occurrences (v is the same row for all of them):
+//   G_v = sum_j x_j c_bag(j)  -  v * sum_j x_j^2 gF[b_j],   c_bag = gF[b] A[b] + gE[b][f]
+// so the kernel walks the batch in BAG order — c_bag is formed once per bag
+// from rows that stream through exactly once — and scatter-adds x_j c_bag into
+// the gradient row of the key's batch-unique index (dedup by the index that
+// find_or_insert assigned).  A second kernel visits every unique key once:
+// it finishes G_v with the key's own row, applies SGD / Adagrad to weights and
+// state in place, and clears the gradient row for the next step.
+//
+// Hot keys.  CTR ids are Zipf distributed: a handful of keys own most of a
+// batch's occurrences.  Millions of float atomics on one gradient row would
+// serialise in L2 and, summed one after the other in fp32, lose the 1e-5
+// accuracy the step must keep.  So before the scatter, occurrences are counted
+// per unique key on a sample of the batch; a key whose estimated count reaches
+// HOT_MIN gets R = count / CHAIN private replica rows, every occurrence is sent
+// to replica hash(j) mod R, and after the scatter the replicas of a key are
+// summed in double into its gradient row.  No accumulator ever takes more than
+// a few hundred float additions, and no address is shared by more than that
+// many atomics.
+#include "des_internal.cuh"
+
+#define HOT_MIN 512u      // estimated occurrences from which a key is treated as hot
+#define HOT_CHAIN 256u    // target number of additions per replica row
+
+__device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
+  return x;
+}
+
+// hinfo[u] += 1 for a 1 / 2^shift sample of the occurrences.
+__global__ void __launch_bounds__(256) sample_count_kernel(const uint32_t* __restrict__ uidx, int nnz, int shift,
+                                                           long long max_uniq, uint32_t* hinfo) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const long long j = ((long long)i << shift) + (shift ? (hash_u32((uint32_t)i) & ((1u << shift) - 1u)) : 0u);
+  if (j >= nnz) return;
+  const uint32_t u = __ldg(uidx + j);
+  if (u != DES_ROW_NONE && (long long)u < max_uniq) atomicAdd(hinfo + u, 1u);
+}
+
+// Turns the sampled counts into the hot list: hinfo[u] becomes the key's hot
+// index, or DES_ROW_NONE for a cold key.  ctr[0] = hot keys, ctr[1] = replica rows.
+__global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const uint32_t* __restrict__ n_uniq,
+                                                         long long max_uniq, int shift, uint32_t* hot_base,
+                                                         uint32_t* hot_R, uint32_t* hot_u, uint32_t* ctr,
+                                                         uint32_t h_max, uint32_t rep_max) {
+  long long U = *n_uniq;
+  if (U > max_uniq) U = max_uniq;
+  for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (long long)gridDim.x * blockDim.x) {
+    const uint32_t est = hinfo[u] << shift;
+    uint32_t h = DES_ROW_NONE;
+    if (est >= HOT_MIN) {
+      const uint32_t R = (est + HOT_CHAIN - 1) / HOT_CHAIN;
+      const uint32_t hh = atomicAdd(&ctr[0], 1u);
+      if (hh < h_max) {
+        const uint32_t base = atomicAdd(&ctr[1], R);
+        if (base + R <= rep_max) { hot_base[hh] = base; hot_R[hh] = R; hot_u[hh] = (uint32_t)u; h = hh; }
+        else hot_R[hh] = 0;
+      }
+    }
+    hinfo[u] = h;
+  }
+}
+
+// dest[j] = gradient row of occurrence j: the key's own row, or one of its replicas.
+__global__ void __launch_bounds__(256) make_dest_kernel(const uint32_t* __restrict__ uidx, int nnz,
+                                                        const uint32_t* __restrict__ hinfo,
+                                                        const uint32_t* __restrict__ hot_base,
+                                                        const uint32_t* __restrict__ hot_R, long long max_uniq,
+                                                        uint32_t* __restrict__ dest) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= nnz) return;
+  const uint32_t u = __ldg(uidx + j);
+  uint32_t d = DES_ROW_NONE;
+  if (u != DES_ROW_NONE && (long long)u < max_uniq) {
+    const uint32_t h = __ldg(hinfo + u);
+    d = (h == DES_ROW_NONE) ? u : (uint32_t)max_uniq + __ldg(hot_base + h) + hash_u32((uint32_t)j) % __ldg(hot_R + h);
+  }
+  dest[j] = d;
+}
+
+// One block per hot key: sum its replica rows in double (fixed order inside a
+// thread, tree across threads), add into the key's gradient row, clear the replicas.
+__global__ void __launch_bounds__(256) hot_reduce_kernel(const uint32_t* __restrict__ ctr, uint32_t h_max,
+                                                         const uint32_t* __restrict__ hot_base,
+                                                         const uint32_t* __restrict__ hot_R,
+                                                         const uint32_t* __restrict__ hot_u, long long max_uniq,
+                                                         int k, float* Gbuf) {
+  __shared__ double red[256];
+  const int stride = k + 4;
+  uint32_t nh = ctr[0];
+  if (nh > h_max) nh = h_max;
+  for (uint32_t h = blockIdx.x; h < nh; h += gridDim.x) {
+    const uint32_t R = hot_R[h];
+    if (R == 0) continue;
+    float* rep = Gbuf + ((size_t)max_uniq + hot_base[h]) * stride;
+    float* dst = Gbuf + (size_t)hot_u[h] * stride;
+    // thread t handles column t % stride of rows t / stride, t / stride + rows_par, ...
+    const int rows_par = 256 / stride;                       // stride <= 68
+    const int c = threadIdx.x % stride, r0 = threadIdx.x / stride;
+    double a = 0.0;
+    if (r0 < rows_par)
+      for (uint32_t r = r0; r < R; r += rows_par) { a += (double)rep[(size_t)r * stride + c]; rep[(size_t)r * stride + c] = 0.f; }
+    red[threadIdx.x] = a;
+    __syncthreads();
+    if (threadIdx.x < stride) {
+      double t = 0.0;
+      for (int q = 0; q < rows_par; ++q) t += red[q * stride + threadIdx.x];
+      dst[threadIdx.x] += (float)t;
+    }
+    __syncthreads();
+  }
+}
+
+template <int G>
+__global__ void __launch_bounds__(256) grad_scatter_kernel(
+    const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ dest,
+    long long nbags, int F, int k, uint32_t ops, const float* __restrict__ out_small,
+    const float* __restrict__ gL, const float* __restrict__ gF, const float* __restrict__ gE, float* Gbuf) {
+  const int K4 = k >> 2, stride = k + 4;
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long bag = t / G;
+  const int c4 = (int)(t % G);
+  if (bag >= nbags) return;
+  const int lo = __ldg(offsets + bag), hi = __ldg(offsets + bag + 1);
+  if (lo == hi) return;
+  const bool col = c4 < K4;
+  if (!col && c4 != 0) return;
+  const long long b = bag / F;
+  const float gf = (ops & DES_OP_FM) ? __ldg(gF + b) : 0.f;
+  const float gl = (ops & DES_OP_LR) ? __ldg(gL + b) : 0.f;
+  float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col) {
+    if (ops & DES_OP_FM) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(out_small + b * stride) + c4);
+      c = make_float4(gf * a.x, gf * a.y, gf * a.z, gf * a.w);
+    }
+    if (gE) {
+      const float4 e = __ldg(reinterpret_cast<const float4*>(gE + bag * k) + c4);
+      c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
+    }
+  }
+  for (int j = lo; j < hi; ++j) {
+    const uint32_t u = __ldg(dest + j);
+    if (u == DES_ROW_NONE) continue;
+    const float x = vals ? __ldg(vals + j) : 1.f;
+    float* row = Gbuf + (size_t)u * stride;
+    if (col) atomicAdd(reinterpret_cast<float4*>(row) + c4, make_float4(x * c.x, x * c.y, x * c.z, x * c.w));
+    if (c4 == 0) atomicAdd(reinterpret_cast<float4*>(row) + K4, make_float4(x * gl, x * x * gf, 0.f, 0.f));
+  }
+}
+
+template <int G>
+__global__ void __launch_bounds__(256) update_rows_kernel(
+    const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
+    uint32_t ops, int optimizer, float lr, float eps, float* Gbuf, float* W, float* A, uint32_t* hinfo) {
+  const int K4 = k >> 2, stride = k + 4;
+  long long U = *n_uniq;
+  if (U > max_uniq) U = max_uniq;
+  const int c4 = (int)(threadIdx.x % G);
+  const long long gstep = (long long)gridDim.x * (blockDim.x / G);
+  // every group of a warp runs the same number of iterations (u may pass U in the last one)
+  const long long iters = (U + gstep - 1) / gstep;
+  long long u = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
+  for (long long it = 0; it < iters; ++it, u += gstep) {
+  const bool live = u < U;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), tail = g;
+  float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)(live ? u : 0) * stride);
+  const bool col = c4 < K4;
+  if (live) {
+    if (col) g = grow[c4];
+    tail = grow[K4];
+  }
+  __syncwarp();
+  if (!live) continue;
+  if (col) grow[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c4 == 0) { grow[K4] = make_float4(0.f, 0.f, 0.f, 0.f); hinfo[u] = 0u; }
+  const uint32_t r = __ldg(uniq_rows + u);
+  if (r == DES_ROW_NONE) continue;
+  float4* w = reinterpret_cast<float4*>(W + (size_t)r * stride);
+  float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r * stride) : nullptr;
+  auto step = [&](float& theta, float& acc, float Gd) {
+    if (optimizer == DES_OPT_ADAGRAD) {
+      acc = acc + Gd * Gd;
+      theta = theta - lr * Gd / (sqrtf(acc) + eps);
+    } else {
+      theta = theta - lr * Gd;
+    }
+  };
+  if (col && (ops & (DES_OP_FM | DES_OP_POOL | DES_OP_DENSE1))) {
+    float4 v = w[c4];
+    float4 s = a ? a[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    step(v.x, s.x, g.x - v.x * tail.y);
+    step(v.y, s.y, g.y - v.y * tail.y);
+    step(v.z, s.z, g.z - v.z * tail.y);
+    step(v.w, s.w, g.w - v.w * tail.y);
+    w[c4] = v;
+    if (a) a[c4] = s;
+  }
+  if (c4 == 0 && (ops & DES_OP_LR)) {
+    float4 v = w[K4];
+    float4 s = a ? a[K4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    step(v.x, s.x, tail.x);
+    w[K4] = v;
+    if (a) a[K4] = s;
+  }
+  }
+}
+
+static int group_for(int k) { int K4 = k / 4, G = 1; while (G < K4) G <<= 1; return G; }
+
+extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t* b,
+                                            const des_outputs_t* out, const des_grads_t* gr, void* stream) {
+  des_status_t st = des_check_batch(t, b, 1);
+  if (st != DES_OK) return st;
+  if (!out || !gr || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
+  if ((ops & DES_OP_LR) && !gr->gL) return DES_ERR_INVALID_ARG;
+  if ((ops & DES_OP_FM) && (!gr->gF || !out->out_small)) return DES_ERR_INVALID_ARG;
+  if ((ops & DES_OP_POOL) && !(ops & DES_OP_DENSE1) && !gr->gE) return DES_ERR_INVALID_ARG;
+  if ((ops & DES_OP_DENSE1) && (!t->H || !gr->gZ || !gr->gE_work || !out->pooled)) return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int B = b->batch;
+  const float* gE = (ops & DES_OP_POOL) ? gr->gE : nullptr;
+  if (ops & DES_OP_DENSE1) {
+    st = des_dense1_backward(t, out->pooled, gE, gr->gZ, gr->gE_work, B, cs);
+    if (st != DES_OK) return st;
+    gE = gr->gE_work;
+  }
+  if (b->nnz == 0) return DES_OK;
+  const int G = group_for(t->k);
+  const int nnz = (int)b->nnz;
+  const long long nbags = (long long)B * t->F;
+  // hot-key detection on a sample, replica assignment, per-occurrence destination row
+  int shift = 0;
+  while (shift < 6 && ((long long)nnz >> shift) > (1ll << 20)) ++shift;
+  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 8, cs));
+  {
+    const int n = (nnz >> shift) + 1;
+    sample_count_kernel<<<(n + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
+    DES_LAUNCH_CHECK(t);
+    hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
+                                                       t->hot_u, t->hot_ctr, t->hot_max, t->rep_max);
+    DES_LAUNCH_CHECK(t);
+    make_dest_kernel<<<(nnz + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
+                                                        t->dest);
+    DES_LAUNCH_CHECK(t);
+  }
+  {
+    const long long threads = nbags * G;
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+#define SC(GG) grad_scatter_kernel<GG><<<grid, 256, 0, cs>>>(b->offsets, b->vals, t->dest, nbags, t->F, t->k, ops, \
+                                                            out->out_small, gr->gL, gr->gF, gE, t->Gbuf)
+    switch (G) { case 1: SC(1); break; case 2: SC(2); break; case 4: SC(4); break; case 8: SC(8); break; default: SC(16); }
+#undef SC
+    DES_LAUNCH_CHECK(t);
+  }
+  hot_reduce_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hot_ctr, t->hot_max, t->hot_base, t->hot_R, t->hot_u,
+                                                     t->max_uniq, t->k, t->Gbuf);
+  DES_LAUNCH_CHECK(t);
+  {
+    const unsigned grid = (unsigned)(t->sm_count * 8);
+#define UP(GG) update_rows_kernel<GG><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops,       \
+                                                           t->cfg.optimizer, t->cfg.lr, t->cfg.eps, t->Gbuf, t->W, t->A, t->hinfo)
+    switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }
+#undef UP
+    DES_LAUNCH_CHECK(t);
+  }
+  return DES_OK;
+}
+
+// ---- whole step from host buffers ---------------------------------------------
+static void* st_alloc(des_table* t, size_t bytes) {
+  if (t->cfg.alloc) return t->cfg.alloc(bytes ? bytes : 256, t->cfg.alloc_ctx);
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes ? bytes : 256) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return p;
+}
+
+extern "C" des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
+                                      const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                                      const des_grads_t* d_grads, float* d_pooled, float* d_Z, float* h_out_small,
+                                      void* stream) {
+  if (!t || !h_offsets || (nnz > 0 && !h_ids) || !d_grads || !h_out_small) return DES_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > t->max_batch || nnz < 0 || nnz > t->max_nnz) return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  if (!t->st_ids) {   // first call: device staging sized for the largest batch (allocates, synchronises)
+    const size_t nb = (size_t)t->max_batch * t->F + 1;
+    t->st_offsets = (int32_t*)st_alloc(t, nb * 4);
+    t->st_ids = (unsigned long long*)st_alloc(t, (size_t)t->max_nnz * 8);
+    t->st_vals = (float*)st_alloc(t, (size_t)t->max_nnz * 4);
+    t->st_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+    t->st_shards = (uint8_t*)st_alloc(t, (size_t)t->max_nnz);
+    t->st_uidx = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+    t->st_uniq_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+    t->st_n_uniq = (uint32_t*)st_alloc(t, 256);
+    t->st_part_small = (float*)st_alloc(t, (size_t)t->S * t->max_batch * t->stride * 4);
+    t->st_out_small = (float*)st_alloc(t, (size_t)t->max_batch * t->stride * 4);
+    if (!t->st_offsets || !t->st_ids || !t->st_vals || !t->st_rows || !t->st_shards || !t->st_uidx ||
+        !t->st_uniq_rows || !t->st_n_uniq || !t->st_part_small || !t->st_out_small)
+      return DES_ERR_CUDA;
+  }
+  const size_t nb = (size_t)batch * t->F + 1;
+  DES_CUDA(cudaMemcpyAsync(t->st_offsets, h_offsets, nb * 4, cudaMemcpyHostToDevice, cs));
+  if (nnz) DES_CUDA(cudaMemcpyAsync(t->st_ids, h_ids, (size_t)nnz * 8, cudaMemcpyHostToDevice, cs));
+  if (h_vals && nnz) DES_CUDA(cudaMemcpyAsync(t->st_vals, h_vals, (size_t)nnz * 4, cudaMemcpyHostToDevice, cs));
+  des_batch_t b;
+  b.batch = batch; b.nnz = nnz; b.offsets = t->st_offsets; b.ids = (const uint64_t*)t->st_ids;
+  b.vals = h_vals ? t->st_vals : nullptr; b.rows = t->st_rows; b.shards = t->st_shards; b.uidx = t->st_uidx;
+  b.uniq_rows = t->st_uniq_rows; b.n_uniq = t->st_n_uniq;
+  des_partials_t p; p.part_small = t->st_part_small; p.pooled = d_pooled; p.part_pooled = nullptr; p.part_dense = nullptr;
+  des_outputs_t o; o.out_small = t->st_out_small; o.pooled = d_pooled; o.Z = d_Z;
+  des_status_t st;
+  if ((st = des_find_or_insert(t, &b, 1, stream)) != DES_OK) return st;
+  if ((st = des_forward_partials(t, ops, &b, &p, stream)) != DES_OK) return st;
+  if ((st = des_aggregate(t, ops, &b, &p, &o, stream)) != DES_OK) return st;
+  if ((st = des_backward_update(t, ops, &b, &o, d_grads, stream)) != DES_OK) return st;
+  DES_CUDA(cudaMemcpyAsync(h_out_small, t->st_out_small, (size_t)batch * t->stride * 4, cudaMemcpyDeviceToHost, cs));
+  DES_CUDA(cudaStreamSynchronize(cs));
+  return DES_OK;
+}

@@ -1,0 +1,187 @@
+// Row-split first dense layer (Section 4.3): V^T W = sum_s V_s^T W_s, where
+// V_s are the pooled blocks of the fields shard s owns and W_s the matching
+// rows of W1 (Eq. 9); its backward needs no cross-shard term (Section 3.2):
+// gE = gZ W1^T block by block, gW1 = V^T gZ.
+//
+// Operands are rounded to bfloat16 (RNE) and accumulated in fp32.  The K loop
+// of the forward runs over fields in (owning shard, field) order, so the
+// accumulator sees P_0, P_1, ... in shard order; with `part_dense` the K range
+// of every shard is a separate slice of the launch and P_s is stored.
+//
+// This is the plain shared-memory tiled version (64x64x16 tiles, 4x4 outputs
+// per thread, CUDA cores): the flops of the step are tiny next to its memory
+// traffic.
+#include "des_internal.cuh"
+
+#define TM 64
+#define TN 64
+#define TK 16
+
+enum { GEMM_FWD = 0, GEMM_DGRAD = 1, GEMM_WGRAD = 2 };
+
+struct GemmArgs {
+  int M, N, K;                 // problem
+  const float* A32;            // fwd: pooled [B][FK]   dgrad: gZ [B][H]    wgrad: pooled [B][FK]
+  const __nv_bfloat16* Bb;     // fwd/dgrad: W1 bf16 [FK][H]
+  const float* B32;            // wgrad: gZ [B][H]
+  const float* add;            // dgrad: gE [B][FK] or NULL
+  float* out;                  // [slices][M][N]
+  int k_emb, FK, H;
+  const DevMeta* meta;
+  int slices;                  // grid.z
+  int slice_by_shard;          // fwd: slice z = K range of shard z (FIELD) / all K of part_pooled[z] (HASH)
+  int partition, S, F;
+  size_t a_slice_stride;       // fwd + HASH materialise: part_pooled slice stride
+};
+
+__device__ __forceinline__ float bf16r(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+template <int MODE>
+__global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
+  __shared__ float As[TK][TM + 4];
+  __shared__ float Bs[TK][TN + 4];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN, z = blockIdx.z;
+  int k_lo = 0, k_hi = g.K;
+  const float* A32 = g.A32;
+  if (MODE == GEMM_FWD && g.slice_by_shard) {
+    if (g.partition == DES_PART_FIELD) {
+      // fields are K-ordered by owning shard: shard z owns a contiguous K range
+      int before = 0, mine = 0;
+      for (int f = 0; f < g.F; ++f) { int s = f % g.S; if (s < z) ++before; else if (s == z) ++mine; }
+      k_lo = before * g.k_emb; k_hi = k_lo + mine * g.k_emb;
+    } else {
+      A32 += (size_t)z * g.a_slice_stride;
+    }
+  } else if (MODE == GEMM_WGRAD) {
+    const int per = (g.K + g.slices - 1) / g.slices;
+    k_lo = z * per; k_hi = min(g.K, k_lo + per);
+  }
+  float acc[4][4] = {};
+  for (int kb = k_lo; kb < k_hi; kb += TK) {
+    // stage A tile [TM][TK] and B tile [TK][TN], 4 elements per thread each
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int idx = threadIdx.x + e * 256;
+      float av = 0.f, bv = 0.f;
+      if (MODE == GEMM_FWD) {
+        const int kk = kb + (idx & 15), m = m0 + (idx >> 4);
+        if (kk < k_hi && m < g.M) {
+          const int col = g.meta->field_order[kk / g.k_emb] * g.k_emb + kk % g.k_emb;
+          av = bf16r(__ldg(A32 + (size_t)m * g.FK + col));
+        }
+        As[idx & 15][idx >> 4] = av;
+        const int kk2 = kb + (idx >> 6), n = n0 + (idx & 63);
+        if (kk2 < k_hi && n < g.N) {
+          const int row = g.meta->field_order[kk2 / g.k_emb] * g.k_emb + kk2 % g.k_emb;
+          bv = __bfloat162float(g.Bb[(size_t)row * g.H + n]);
+        }
+        Bs[idx >> 6][idx & 63] = bv;
+      } else if (MODE == GEMM_DGRAD) {
+        const int kk = kb + (idx & 15), m = m0 + (idx >> 4);
+        if (kk < k_hi && m < g.M) av = __ldg(A32 + (size_t)m * g.H + kk);
+        As[idx & 15][idx >> 4] = av;
+        const int kk2 = kb + (idx & 15), n = n0 + (idx >> 4);       // W1^T: read along H
+        if (kk2 < k_hi && n < g.N) bv = __bfloat162float(g.Bb[(size_t)n * g.H + kk2]);
+        Bs[idx & 15][idx >> 4] = bv;
+      } else {
+        const int kk = kb + (idx >> 6), m = m0 + (idx & 63);        // pooled^T: read along FK
+        if (kk < k_hi && m < g.M) av = bf16r(__ldg(A32 + (size_t)kk * g.FK + m));
+        As[idx >> 6][idx & 63] = av;
+        const int kk2 = kb + (idx >> 6), n = n0 + (idx & 63);
+        if (kk2 < k_hi && n < g.N) bv = __ldg(g.B32 + (size_t)kk2 * g.H + n);
+        Bs[idx >> 6][idx & 63] = bv;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < TK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* out = g.out + (size_t)z * g.M * g.N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= g.M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= g.N) continue;
+      float v = acc[i][j];
+      if (MODE == GEMM_DGRAD && g.add) v += __ldg(g.add + (size_t)m * g.N + n);
+      out[(size_t)m * g.N + n] = v;
+    }
+  }
+}
+
+// Sum the split-K slices of gW1 in slice order, apply the optimizer to the
+// fp32 master weights, refresh the bf16 shadow.
+__global__ void w1_update_kernel(const float* __restrict__ part, int slices, size_t n, float* W1, float* acc,
+                                 __nv_bfloat16* W1b, int optimizer, float lr, float eps) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += st) {
+    float G = 0.f;
+    for (int z = 0; z < slices; ++z) G += __ldg(part + (size_t)z * n + i);
+    float w = W1[i];
+    if (optimizer == DES_OPT_ADAGRAD) {
+      float a = acc[i] + G * G;
+      acc[i] = a;
+      w -= lr * G / (sqrtf(a) + eps);
+    } else {
+      w -= lr * G;
+    }
+    W1[i] = w;
+    W1b[i] = __float2bfloat16_rn(w);
+  }
+}
+
+des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float* Z, float* part_dense,
+                                const float* part_pooled, cudaStream_t st) {
+  GemmArgs g; memset(&g, 0, sizeof(g));
+  g.M = B; g.N = t->H; g.K = t->F * t->k; g.A32 = pooled; g.Bb = t->W1b; g.k_emb = t->k; g.FK = g.K; g.H = t->H;
+  g.meta = t->meta; g.partition = t->cfg.partition; g.S = t->S; g.F = t->F;
+  g.out = Z; g.slices = 1; g.slice_by_shard = 0;
+  if (part_dense) {
+    if (t->cfg.partition == DES_PART_HASH && !part_pooled) return DES_ERR_INVALID_ARG;
+    g.out = part_dense; g.slices = t->S; g.slice_by_shard = 1;
+    if (t->cfg.partition == DES_PART_HASH) { g.A32 = part_pooled; g.a_slice_stride = (size_t)B * g.FK; }
+  }
+  dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.slices);
+  gemm_kernel<GEMM_FWD><<<grid, 256, 0, st>>>(g);
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}
+
+des_status_t des_dense1_backward(des_table* t, const float* pooled, const float* gE, const float* gZ,
+                                 float* gE_work, int B, cudaStream_t st) {
+  const int FK = t->F * t->k;
+  {  // gE_work = gE + gZ W1^T
+    GemmArgs g; memset(&g, 0, sizeof(g));
+    g.M = B; g.N = FK; g.K = t->H; g.A32 = gZ; g.Bb = t->W1b; g.add = gE; g.out = gE_work;
+    g.k_emb = t->k; g.FK = FK; g.H = t->H; g.meta = t->meta; g.slices = 1;
+    dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, 1);
+    gemm_kernel<GEMM_DGRAD><<<grid, 256, 0, st>>>(g);
+    DES_LAUNCH_CHECK(t);
+  }
+  {  // gW1 = pooled^T gZ, split over the batch
+    GemmArgs g; memset(&g, 0, sizeof(g));
+    g.M = FK; g.N = t->H; g.K = B; g.A32 = pooled; g.B32 = gZ; g.out = t->gW1_part;
+    g.k_emb = t->k; g.FK = FK; g.H = t->H; g.meta = t->meta; g.slices = t->gw1_splits;
+    dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.slices);
+    gemm_kernel<GEMM_WGRAD><<<grid, 256, 0, st>>>(g);
+    DES_LAUNCH_CHECK(t);
+    const size_t n = (size_t)FK * t->H;
+    w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, g.slices, n, t->W1, t->accW1, t->W1b,
+                                                      t->cfg.optimizer, t->cfg.lr, t->cfg.eps);
+    DES_LAUNCH_CHECK(t);
+  }
+  return DES_OK;
+}

@@ -1,0 +1,242 @@
+// Forward of the DES sparse operators.
+//
+// des_forward_partials: the sub-operators M_j of every shard —
+//   LR   M_1 = sum_{j in shard} w_j x_j                       (Eq. 2)
+//   FM   M_1 = sum v_j x_j,  M_2 = sum <v_j x_j, v_j x_j>      (Eq. 7)
+//   POOL per-field sum pooling of the latent vectors          (Section 4.3)
+// des_aggregate: (+) over shards in the order s = 0..S-1 (Eq. 1) and the
+// substitution operator F = 1/2 <(+)M_1,(+)M_1> - 1/2 (+)M_2 (Eq. 8).
+//
+// Kernel shape.  One warp walks one sample.  A row (k floats + the linear
+// weight) is read by a group of G = k/4 lanes (rounded up to a power of two)
+// with one 16-byte load per lane; the 32/G groups of the warp take different
+// bags of the sample, so a bag's pooled sum lives in one group's registers and
+// is stored once.  The per-(shard, sample) partials live in shared memory,
+// S x (k+4) floats per warp; two groups that hit the same shard in the same
+// step are serialised in group order (found with a warp match), so every sum
+// is taken in CSR order and the result is deterministic.
+#include "des_internal.cuh"
+
+#define FW_UNROLL 4
+
+template <int G>
+__global__ void __launch_bounds__(256) forward_partials_kernel(
+    const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
+    const uint8_t* __restrict__ shards, int B, int F, int S, int k, uint32_t ops, const float* __restrict__ W,
+    const DevMeta* __restrict__ meta, float* __restrict__ part_small, float* __restrict__ pooled,
+    float* __restrict__ part_pooled) {
+  extern __shared__ __align__(16) float smem[];
+  constexpr int NG = 32 / G;
+  const int K4 = k >> 2, stride = k + 4;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+  const int g = lane / G, c4 = lane % G;
+  const bool col = c4 < K4;
+  const bool want_small = part_small != nullptr;
+  float* acc = smem + (size_t)warp * S * stride;
+  const int acc_f4 = S * (K4 + 1);
+  if (want_small)
+    for (int i = lane; i < acc_f4; i += 32) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncwarp();
+  const unsigned group_lt = (g == 0) ? 0u : (0xFFFFFFFFu >> (32 - g * G));
+
+  for (int b = blockIdx.x * wpb + warp; b < B; b += gridDim.x * wpb) {
+    for (int fbase = 0; fbase < F; fbase += NG) {
+      const int f = fbase + g;
+      int lo = 0, hi = 0;
+      if (f < F) { lo = __ldg(offsets + (size_t)b * F + f); hi = __ldg(offsets + (size_t)b * F + f + 1); }
+      const int maxlen = __reduce_max_sync(0xFFFFFFFFu, hi - lo);
+      float4 pacc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = 0; i < maxlen; i += FW_UNROLL) {
+        float4 v[FW_UNROLL]; float lin[FW_UNROLL], x[FW_UNROLL]; int sh[FW_UNROLL];
+#pragma unroll
+        for (int u = 0; u < FW_UNROLL; ++u) {
+          const int j = lo + i + u;
+          v[u] = make_float4(0.f, 0.f, 0.f, 0.f); lin[u] = 0.f; x[u] = 0.f; sh[u] = -1;
+          if (j < hi) {
+            const uint32_t r = __ldg(rows + j);
+            if (r != DES_ROW_NONE) {
+              const int s = __ldg(shards + j);
+              sh[u] = s;
+              x[u] = vals ? __ldg(vals + j) : 1.f;
+              const float* wr = W + (meta->row_base[s] + r) * (size_t)stride;
+              if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
+              if (c4 == 0) lin[u] = __ldg(wr + k);
+            }
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < FW_UNROLL; ++u) {
+          if (i + u >= maxlen) break;                       // warp-uniform
+          const float xx = x[u];
+          const float4 vx = make_float4(v[u].x * xx, v[u].y * xx, v[u].z * xx, v[u].w * xx);
+          pacc.x += vx.x; pacc.y += vx.y; pacc.z += vx.z; pacc.w += vx.w;
+          if (part_pooled && sh[u] >= 0 && col) {
+            float* pp = part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) + (size_t)f * k + c4 * 4;
+            pp[0] += vx.x; pp[1] += vx.y; pp[2] += vx.z; pp[3] += vx.w;   // this group owns the bag
+          }
+          if (want_small) {
+            float sq = vx.x * vx.x + vx.y * vx.y + vx.z * vx.z + vx.w * vx.w;
+#pragma unroll
+            for (int d = 1; d < G; d <<= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, d);
+            // groups that hit the same shard in this step add one after the other
+            const unsigned peers = __match_any_sync(0xFFFFFFFFu, sh[u] >= 0 ? sh[u] : 0x100 + g);
+            const int rank = __popc(peers & group_lt) / G;
+            const int rmax = __reduce_max_sync(0xFFFFFFFFu, rank);
+            for (int r = 0; r <= rmax; ++r) {
+              if (r == rank && sh[u] >= 0) {
+                float* a = acc + sh[u] * stride;
+                if (col) {
+                  float4 t = reinterpret_cast<float4*>(a)[c4];
+                  t.x += vx.x; t.y += vx.y; t.z += vx.z; t.w += vx.w;
+                  reinterpret_cast<float4*>(a)[c4] = t;
+                }
+                if (c4 == 0) { a[k] += lin[u] * xx; a[k + 1] += sq; }
+              }
+              __syncwarp();
+            }
+          }
+        }
+      }
+      if (pooled && f < F && col)
+        reinterpret_cast<float4*>(pooled + ((size_t)b * F + f) * k)[c4] = pacc;
+    }
+    if (want_small) {
+      __syncwarp();
+      const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
+      for (int i = lane; i < acc_f4; i += 32) {
+        const int s = i / (K4 + 1), q = i % (K4 + 1);
+        float4 t = reinterpret_cast<float4*>(acc)[i];
+        reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (q == K4) { if (!lr) t.x = 0.f; if (!fm) t.y = 0.f; }
+        else if (!fm) t = make_float4(0.f, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride)[q] = t;
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// (+) over shards and F.  G lanes per sample, one float4 column each; lane 0 of
+// the group also carries the tail (R_lr, Q).  <A, A> is taken in double.
+template <int G>
+__global__ void __launch_bounds__(256) aggregate_small_kernel(const float* __restrict__ part_small, int B, int S, int k,
+                                                              uint32_t ops, float* __restrict__ out_small) {
+  const int K4 = k >> 2, stride = k + 4;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = t / G, c4 = t % G;
+  const bool live = b < B;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), tail = a;
+  if (live) {
+    for (int s = 0; s < S; ++s) {
+      const float4* p = reinterpret_cast<const float4*>(part_small + ((size_t)s * B + b) * stride);
+      if (c4 < K4) { float4 v = __ldg(p + c4); a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
+      if (c4 == 0) { float4 v = __ldg(p + K4); tail.x += v.x; tail.y += v.y; }
+    }
+  }
+  double aa = (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+#pragma unroll
+  for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
+  if (!live) return;
+  float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
+  if (c4 < K4) o[c4] = a;
+  if (c4 == 0) {
+    const float fm2 = (ops & DES_OP_FM) ? (float)(0.5 * aa - 0.5 * (double)tail.y) : 0.f;
+    o[K4] = make_float4(tail.x, fm2, tail.y, 0.f);
+  }
+}
+
+// sum over shards of a dense [S][B][n] tensor (materialised pooled / dense partials)
+__global__ void reduce_shards_kernel(const float* __restrict__ part, size_t per_shard, int S, float* __restrict__ out) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
+  for (; i < per_shard; i += st) {
+    float a = 0.f;
+    for (int s = 0; s < S; ++s) a += __ldg(part + (size_t)s * per_shard + i);
+    out[i] = a;
+  }
+}
+
+static int group_for(int k) { int K4 = k / 4, G = 1; while (G < K4) G <<= 1; return G; }
+
+extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_t* b,
+                                             const des_partials_t* part, void* stream) {
+  des_status_t st = des_check_batch(t, b, 0);
+  if (st != DES_OK) return st;
+  if (!part || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
+  const bool small = ops & (DES_OP_LR | DES_OP_FM), pool = ops & (DES_OP_POOL | DES_OP_DENSE1);
+  if (small && !part->part_small) return DES_ERR_INVALID_ARG;
+  if (pool && !part->pooled) return DES_ERR_INVALID_ARG;
+  if ((ops & DES_OP_DENSE1) && !t->H) return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int B = b->batch;
+  float* ps = small ? part->part_small : nullptr;
+  float* pl = pool ? part->pooled : nullptr;
+  float* pp = pool ? part->part_pooled : nullptr;
+  if (pp) DES_CUDA(cudaMemsetAsync(pp, 0, (size_t)t->S * B * t->F * t->k * 4, cs));
+  const size_t per_warp = small ? (size_t)t->S * t->stride * 4 : 0;
+  int wpb = 8;
+  while (wpb > 1 && per_warp * wpb > 200 * 1024) wpb >>= 1;
+  const size_t smem = per_warp * wpb;
+  int grid = (B + wpb - 1) / wpb;
+  const int G = group_for(t->k);
+#define FWD(GG)                                                                                                   \
+  do {                                                                                                            \
+    if (smem > 48 * 1024)                                                                                         \
+      DES_CUDA(cudaFuncSetAttribute(forward_partials_kernel<GG>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                    (int)smem));                                                                  \
+    forward_partials_kernel<GG><<<grid, wpb * 32, smem, cs>>>(b->offsets, b->vals, b->rows, b->shards, B, t->F,   \
+                                                              t->S, t->k, ops, t->W, t->meta, ps, pl, pp);        \
+  } while (0)
+  switch (G) {
+    case 1: FWD(1); break;
+    case 2: FWD(2); break;
+    case 4: FWD(4); break;
+    case 8: FWD(8); break;
+    default: FWD(16); break;
+  }
+#undef FWD
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}
+
+extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* b, const des_partials_t* part,
+                                      const des_outputs_t* out, void* stream) {
+  if (!t || !b || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
+  if (b->batch <= 0 || b->batch > t->max_batch) return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int B = b->batch;
+  if (ops & (DES_OP_LR | DES_OP_FM)) {
+    if (!part->part_small || !out->out_small) return DES_ERR_INVALID_ARG;
+    const int G = group_for(t->k);
+    const long long threads = (long long)B * G;
+    const int grid = (int)((threads + 255) / 256);
+    switch (G) {
+      case 1: aggregate_small_kernel<1><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
+      case 2: aggregate_small_kernel<2><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
+      case 4: aggregate_small_kernel<4><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
+      case 8: aggregate_small_kernel<8><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
+      default: aggregate_small_kernel<16><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
+    }
+    DES_LAUNCH_CHECK(t);
+  }
+  if (ops & (DES_OP_POOL | DES_OP_DENSE1)) {
+    if (!part->pooled || !out->pooled) return DES_ERR_INVALID_ARG;
+    const size_t n = (size_t)B * t->F * t->k;
+    if (part->part_pooled) {
+      // materialised per-shard pooled partials: aggregate them in shard order
+      reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part->part_pooled, n, t->S, out->pooled);
+      DES_LAUNCH_CHECK(t);
+    } else if (out->pooled != part->pooled) {
+      DES_CUDA(cudaMemcpyAsync(out->pooled, part->pooled, n * 4, cudaMemcpyDeviceToDevice, cs));
+    }
+  }
+  if (ops & DES_OP_DENSE1) {
+    if (!t->H || !out->Z) return DES_ERR_INVALID_ARG;
+    des_status_t st = des_dense1_forward(t, out->pooled, B, out->Z, part->part_dense, part->part_pooled, cs);
+    if (st != DES_OK) return st;
+    if (part->part_dense) {
+      reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part->part_dense, (size_t)B * t->H, t->S, out->Z);
+      DES_LAUNCH_CHECK(t);
+    }
+  }
+  return DES_OK;
+}

@@ -1,0 +1,257 @@
+// lookup + insert on the dynamic hash table (Section 5, "Dynamic Hash Table"),
+// including shard routing (Section 5, "Large-scale Sparse Features": weights of
+// field f live on node f mod N; Section 4.2: any balanced partition).
+//
+// One call = six short kernels, none of which waits on another thread:
+//   probe_claim   every occurrence finds its key's slot in the owning shard's
+//                 region (linear probing) or claims an empty one with a 64-bit
+//                 CAS; the slot remembers the smallest occurrence index.
+//   flag_count    occurrence j is the FIRST of its key iff slot.first_occ == j,
+//                 and the key is NEW iff its slot has no row yet; per-block
+//                 counts of firsts and of new keys per shard.
+//   scan          exclusive scan of those counts over blocks.
+//   assign        first occurrences get the batch-unique index (rank among
+//                 firsts) and, for new keys, the next shard-local row (rank
+//                 among the shard's new keys): both in CSR order, so the result
+//                 does not depend on thread scheduling.  New rows are
+//                 initialised here from the counter-based generator.
+//   resolve       every occurrence reads row and unique index from its slot.
+//   finish        slots' scratch word is reset, shard sizes are advanced.
+#include "des_internal.cuh"
+
+#define IB 1024  // threads (= occurrences) per block in every kernel of this file
+
+__device__ __forceinline__ Slot load_slot(const Slot* p) {
+  unsigned long long a, b;     // bypass L1: other SMs claim slots while we probe
+  asm volatile("ld.volatile.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p));
+  Slot s;
+  s.key = a; s.row = (uint32_t)b; s.first_occ = (uint32_t)(b >> 32);
+  return s;
+}
+
+__global__ void __launch_bounds__(IB) probe_claim_kernel(
+    const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
+    int S, int F, int partition, int insert, Slot* slots, DevMeta* meta,
+    uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards, uint32_t* __restrict__ rows) {
+  int j = blockIdx.x * IB + threadIdx.x;
+  if (j >= nnz) return;
+  unsigned long long id = ids[j];
+  uint32_t s;
+  if (partition == DES_PART_HASH) s = (uint32_t)(des_mix64(id) % (unsigned)S);
+  else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
+  shards[j] = (uint8_t)s;
+  uint32_t found = DES_SLOT_NONE;
+  uint32_t row = DES_ROW_NONE;
+  if (id == DES_KEY_EMPTY) {
+    des_raise(meta, DES_ERR_RESERVED_KEY);
+  } else {
+    const unsigned long long base = meta->slot_base[s];
+    const unsigned long long n = meta->slot_base[s + 1] - base;
+    unsigned long long pos = __umul64hi(des_mix64(id ^ 0x9E3779B97F4A7C15ull), n);
+    bool full = true;
+    for (unsigned long long probe = 0; probe < n; ++probe) {
+      Slot* sp = slots + base + pos;
+      Slot sl = load_slot(sp);
+      if (sl.key == id) { found = (uint32_t)(base + pos); row = sl.row; full = false; break; }
+      if (sl.key == DES_KEY_EMPTY) {
+        if (!insert) { full = false; break; }
+        unsigned long long old = atomicCAS(&sp->key, DES_KEY_EMPTY, id);
+        if (old == DES_KEY_EMPTY || old == id) { found = (uint32_t)(base + pos); full = false; break; }
+      }
+      pos = (pos + 1 == n) ? 0 : pos + 1;
+    }
+    if (full && insert) des_raise(meta, DES_ERR_CAPACITY);
+    if (found != DES_SLOT_NONE && insert) {
+      uint32_t* fo = &slots[found].first_occ;
+      if (*reinterpret_cast<volatile uint32_t*>(fo) > (uint32_t)j) atomicMin(fo, (uint32_t)j);
+    }
+  }
+  if (insert) slot_of[j] = found;
+  else rows[j] = row;
+}
+
+// flags: bit0 = first occurrence of its key in the batch, bit1 = key is new.
+__global__ void __launch_bounds__(IB) flag_count_kernel(
+    int nnz, int S, const Slot* __restrict__ slots, const uint32_t* __restrict__ slot_of,
+    const uint8_t* __restrict__ shards, uint8_t* __restrict__ flags, uint32_t* __restrict__ blk_cnt, int nblk_max) {
+  __shared__ uint32_t cnt[DES_MAX_SHARDS + 1];
+  if (threadIdx.x <= DES_MAX_SHARDS) cnt[threadIdx.x] = 0;
+  __syncthreads();
+  int j = blockIdx.x * IB + threadIdx.x;
+  uint8_t fl = 0;
+  if (j < nnz) {
+    uint32_t so = slot_of[j];
+    if (so != DES_SLOT_NONE) {
+      Slot sl = slots[so];
+      if (sl.first_occ == (uint32_t)j) fl = (sl.row == DES_ROW_NONE) ? 3 : 1;
+    }
+    flags[j] = fl;
+  }
+  unsigned firsts = __ballot_sync(0xFFFFFFFFu, fl & 1);
+  if ((threadIdx.x & 31) == 0 && firsts) atomicAdd(&cnt[0], __popc(firsts));
+  if (fl & 2) atomicAdd(&cnt[1 + shards[j]], 1u);
+  __syncthreads();
+  if (threadIdx.x <= S) blk_cnt[(size_t)threadIdx.x * nblk_max + blockIdx.x] = cnt[threadIdx.x];
+}
+
+// One block per sequence (sequence 0 = firsts, 1 + s = new keys of shard s):
+// in-place exclusive scan over the blocks of the batch, total to meta.
+__global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, int nblk, int nblk_max, DevMeta* meta) {
+  __shared__ uint32_t wsum[32];
+  uint32_t* seq = blk_cnt + (size_t)blockIdx.x * nblk_max;
+  const int per = (nblk + 1023) / 1024;
+  const int lo = threadIdx.x * per, hi = min(nblk, lo + per);
+  uint32_t sum = 0;
+  for (int i = lo; i < hi; ++i) sum += seq[i];
+  uint32_t incl = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if ((threadIdx.x & 31) >= d) incl += v;
+  }
+  if ((threadIdx.x & 31) == 31) wsum[threadIdx.x >> 5] = incl;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    uint32_t w = wsum[threadIdx.x], wi = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t v = __shfl_up_sync(0xFFFFFFFFu, wi, d);
+      if (threadIdx.x >= d) wi += v;
+    }
+    wsum[threadIdx.x] = wi - w;
+    if (threadIdx.x == 31) {
+      if (blockIdx.x == 0) meta->n_uniq = wi; else meta->new_total[blockIdx.x - 1] = wi;
+    }
+  }
+  __syncthreads();
+  uint32_t run = wsum[threadIdx.x >> 5] + incl - sum;
+  for (int i = lo; i < hi; ++i) { uint32_t v = seq[i]; seq[i] = run; run += v; }
+}
+
+__global__ void __launch_bounds__(IB) assign_kernel(
+    const unsigned long long* __restrict__ ids, int nnz, int S, int k, int stride, Slot* slots, DevMeta* meta,
+    const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
+    const uint32_t* __restrict__ blk_cnt, int nblk_max, uint32_t* __restrict__ uslot,
+    uint32_t* __restrict__ uniq_rows, long long max_uniq, float* __restrict__ W, float* __restrict__ A,
+    unsigned long long seed, float init_scale, float init_acc) {
+  __shared__ uint32_t wfirst[32];
+  __shared__ uint16_t wnew[32][DES_MAX_SHARDS];
+  const int j = blockIdx.x * IB + threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint8_t fl = (j < nnz) ? flags[j] : 0;
+  const uint32_t s = (j < nnz) ? shards[j] : 0;
+  for (int i = threadIdx.x; i < 32 * DES_MAX_SHARDS; i += IB) (&wnew[0][0])[i] = 0;
+  __syncthreads();
+  // rank among firsts / among the shard's new keys inside the warp (lane order = CSR order)
+  const unsigned fmask = __ballot_sync(0xFFFFFFFFu, fl & 1);
+  const unsigned lt = (1u << lane) - 1u;
+  uint32_t frank = __popc(fmask & lt);
+  const unsigned nmask_all = __ballot_sync(0xFFFFFFFFu, fl & 2);
+  uint32_t nrank = 0;
+  if (fl & 2) {
+    unsigned same = __match_any_sync(nmask_all, s);
+    nrank = __popc(same & lt);
+    if ((same >> lane) == 1u) wnew[warp][s] = (uint16_t)__popc(same);   // highest lane of the group
+  }
+  if (lane == 0) wfirst[warp] = __popc(fmask);
+  __syncthreads();
+  // exclusive prefix over warps
+  if (threadIdx.x < 32) {
+    uint32_t v = wfirst[threadIdx.x], in = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      uint32_t o = __shfl_up_sync(0xFFFFFFFFu, in, d);
+      if (threadIdx.x >= d) in += o;
+    }
+    wfirst[threadIdx.x] = in - v;
+  } else if (threadIdx.x >= 64 && threadIdx.x < 64 + S) {
+    const int sh = threadIdx.x - 64;
+    uint32_t run = 0;
+    for (int w = 0; w < 32; ++w) { uint16_t v = wnew[w][sh]; wnew[w][sh] = (uint16_t)run; run += v; }
+  }
+  __syncthreads();
+  if (!(fl & 1)) return;
+  const uint32_t so = slot_of[j];
+  const uint32_t u = blk_cnt[blockIdx.x] + wfirst[warp] + frank;
+  uint32_t local;
+  if (fl & 2) {
+    local = meta->n_rows[s] + blk_cnt[(size_t)(1 + s) * nblk_max + blockIdx.x] + wnew[warp][s] + nrank;
+    if (local >= meta->row_cap[s]) { local = DES_ROW_NONE; des_raise(meta, DES_ERR_CAPACITY); }
+    else slots[so].row = local;
+  } else {
+    local = slots[so].row;
+  }
+  slots[so].first_occ = u;
+  uslot[u] = so;
+  const unsigned long long g = meta->row_base[s] + local;
+  uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
+  if ((long long)u >= max_uniq) des_raise(meta, DES_ERR_CAPACITY);   // gradient buffer too small for this batch
+  if ((fl & 2) && local != DES_ROW_NONE) {
+    const unsigned long long id = ids[j];
+    float4* w = reinterpret_cast<float4*>(W + g * stride);
+    const int q4 = k >> 2;
+    for (int q = 0; q < q4; ++q) w[q] = des_init4(seed, id, q, init_scale);
+    w[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (A) {
+      float4* a = reinterpret_cast<float4*>(A + g * stride);
+      const float4 ia = make_float4(init_acc, init_acc, init_acc, init_acc);
+      for (int q = 0; q < q4; ++q) a[q] = ia;
+      a[q4] = make_float4(init_acc, 0.f, 0.f, 0.f);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(IB) resolve_kernel(int nnz, const Slot* __restrict__ slots,
+                                                     const uint32_t* __restrict__ slot_of,
+                                                     uint32_t* __restrict__ rows, uint32_t* __restrict__ uidx) {
+  int j = blockIdx.x * IB + threadIdx.x;
+  if (j >= nnz) return;
+  uint32_t so = slot_of[j];
+  uint32_t row = DES_ROW_NONE, u = DES_ROW_NONE;
+  if (so != DES_SLOT_NONE) { Slot sl = slots[so]; row = sl.row; u = sl.first_occ; }
+  rows[j] = row;
+  uidx[j] = (row == DES_ROW_NONE) ? DES_ROW_NONE : u;
+}
+
+__global__ void __launch_bounds__(IB) finish_kernel(int nnz, int S, Slot* slots, const uint32_t* __restrict__ uslot,
+                                                    DevMeta* meta, uint32_t* n_uniq_out) {
+  int u = blockIdx.x * IB + threadIdx.x;
+  const uint32_t U = meta->n_uniq;
+  if (u < nnz && (uint32_t)u < U) slots[uslot[u]].first_occ = DES_ROW_NONE;
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x < S) {
+    // the last block is the only writer of n_rows; other blocks never read it
+    uint32_t n = meta->n_rows[threadIdx.x] + meta->new_total[threadIdx.x];
+    meta->n_rows[threadIdx.x] = min(n, meta->row_cap[threadIdx.x]);
+  }
+  if (u == 0) *n_uniq_out = U;
+}
+
+extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b, int insert, void* stream) {
+  des_status_t st = des_check_batch(t, b, insert);
+  if (st != DES_OK) return st;
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int nnz = (int)b->nnz;
+  const int nbags = b->batch * (int)t->F;
+  if (nnz == 0) {
+    if (insert) DES_CUDA(cudaMemsetAsync(b->n_uniq, 0, 4, cs));
+    return DES_OK;
+  }
+  const int nblk = (nnz + IB - 1) / IB;
+  probe_claim_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
+                                          t->cfg.partition, insert, t->slots, t->meta, t->slot_of, b->shards, b->rows);
+  DES_LAUNCH_CHECK(t);
+  if (!insert) return DES_OK;
+  flag_count_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);
+  DES_LAUNCH_CHECK(t);
+  scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
+  DES_LAUNCH_CHECK(t);
+  assign_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, nnz, t->S, t->k, t->stride, t->slots, t->meta,
+                                     t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max, t->uslot, b->uniq_rows,
+                                     t->max_uniq, t->W, t->A, t->cfg.seed, t->cfg.init_scale, t->cfg.init_acc);
+  DES_LAUNCH_CHECK(t);
+  resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
+  DES_LAUNCH_CHECK(t);
+  finish_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->uslot, t->meta, b->n_uniq);
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}

@@ -1,0 +1,131 @@
+// Internal declarations of the DES CUDA library (sm_100a).  Nothing in here is
+// shared with the CPU oracle.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "des.h"
+
+#define DES_MAX_SHARDS 64
+#define DES_SLOT_NONE 0xFFFFFFFFu
+
+// One open-addressing slot: 16 bytes, read with a single vector load.
+//   key        DES_KEY_EMPTY until claimed by a 64-bit CAS; never changes after.
+//   row        shard-local row, DES_ROW_NONE until the key's insert call numbers it.
+//   first_occ  scratch of the running find_or_insert call: smallest occurrence
+//              index of the key in the batch, then the key's batch-unique index;
+//              DES_ROW_NONE between calls.
+struct __align__(16) Slot {
+  unsigned long long key;
+  uint32_t row;
+  uint32_t first_occ;
+};
+
+// Per-table metadata that kernels read through a pointer (broadcast loads).
+struct DevMeta {
+  unsigned long long row_base[DES_MAX_SHARDS + 1];   // first table-global row of shard s
+  unsigned long long slot_base[DES_MAX_SHARDS + 1];  // first slot of shard s's region
+  uint32_t row_cap[DES_MAX_SHARDS];                  // row capacity of shard s
+  uint32_t n_rows[DES_MAX_SHARDS];                   // rows in use
+  uint32_t new_total[DES_MAX_SHARDS];                // new keys of the running insert call
+  uint32_t n_uniq;                                   // unique keys of the running insert call
+  uint32_t err;                                      // sticky des_status_t raised on device
+  uint32_t field_order[1024];                        // fields sorted by (owning shard, field)
+};
+
+struct des_table {
+  des_config_t cfg;
+  int device;
+  uint32_t S, F, k, H, stride;       // stride = k + 4 floats per row
+  uint64_t total_rows, total_slots;
+  uint64_t h_row_base[DES_MAX_SHARDS + 1], h_slot_base[DES_MAX_SHARDS + 1];
+  int64_t max_nnz; int32_t max_batch; int64_t max_uniq;
+  uint32_t nblk_max;                 // scan-block capacity of the workspace
+  // device memory
+  Slot* slots;
+  float* W;                          // [total_rows][stride]: latent vector, linear weight, 3 pad
+  float* A;                          // same shape: Adagrad accumulators (NULL for SGD)
+  DevMeta* meta;
+  // find_or_insert workspace
+  uint32_t* slot_of;                 // [max_nnz]
+  uint8_t* flags;                    // [max_nnz]
+  uint32_t* uslot;                   // [max_nnz]
+  uint32_t* blk_cnt;                 // [(S+1)][nblk_max]
+  // backward workspace
+  float* Gbuf;                       // [max_uniq + rep_max][stride]: per-unique gradient rows, then
+                                     // hot-key replica rows; all zero between calls
+  uint32_t* hinfo;                   // [max_uniq] sampled count, then hot index; zero between calls
+  uint32_t* dest;                    // [max_nnz] gradient row of each occurrence
+  uint32_t *hot_base, *hot_R, *hot_u, *hot_ctr;   // hot list [hot_max] and its two counters
+  uint32_t hot_max, rep_max;
+  // first dense layer
+  float* W1; float* accW1;           // [F*k][H] fp32 master and state
+  __nv_bfloat16* W1b;                // bf16 shadow
+  float* gW1_part; int gw1_splits;   // [splits][F*k][H]
+  // host-step staging
+  int32_t* st_offsets; unsigned long long* st_ids; float* st_vals;
+  uint32_t* st_rows; uint8_t* st_shards; uint32_t* st_uidx; uint32_t* st_uniq_rows; uint32_t* st_n_uniq;
+  float* st_part_small; float* st_out_small;
+  uint64_t launches;
+  int sm_count;
+};
+
+#define DES_CUDA(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return DES_ERR_CUDA; } while (0)
+#define DES_LAUNCH_CHECK(t) do { (t)->launches++; if (cudaGetLastError() != cudaSuccess) return DES_ERR_CUDA; } while (0)
+
+// ---- device helpers ---------------------------------------------------------
+
+// Table mixer: the three xor-shift / odd-multiply rounds of the splitmix64
+// finaliser; a bijection on 64-bit words.
+__host__ __device__ __forceinline__ unsigned long long des_mix64(unsigned long long z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27; z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+// Philox4x32-10 block function.
+__device__ __forceinline__ uint4 des_philox(uint4 c, uint2 key) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ key.x, lo1, hi0 ^ c.w ^ key.y, lo0);
+    key.x += 0x9E3779B9u; key.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// Uniform in [-scale, scale) from the top 24 bits; exact up to the last multiply.
+__device__ __forceinline__ float des_u24(uint32_t r, float scale) {
+  float x = __fmul_rn(__uint2float_rn(r >> 8), 1.0f / 8388608.0f);
+  return __fmul_rn(__fsub_rn(x, 1.0f), scale);
+}
+
+// Four consecutive components 4q..4q+3 of the initial latent vector of `id`.
+__device__ __forceinline__ float4 des_init4(unsigned long long seed, unsigned long long id, uint32_t q, float scale) {
+  uint4 r = des_philox(make_uint4(q, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)),
+                       make_uint2((uint32_t)id, (uint32_t)(id >> 32)));
+  return make_float4(des_u24(r.x, scale), des_u24(r.y, scale), des_u24(r.z, scale), des_u24(r.w, scale));
+}
+
+// Index of the bag that holds occurrence j: largest i with offsets[i] <= j
+// among bags that are not past the end (handles empty bags).
+__device__ __forceinline__ int des_bag_of(const int32_t* __restrict__ offsets, int nbags, int j) {
+  int lo = 0, hi = nbags;             // invariant: offsets[lo] <= j < offsets[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (__ldg(offsets + mid) <= j) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ void des_raise(DevMeta* meta, uint32_t code) { atomicCAS(&meta->err, 0u, code); }
+
+// shared declarations across translation units
+des_status_t des_check_batch(const des_table* t, const des_batch_t* b, int need_dedup);
+des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float* Z, float* part_dense,
+                                const float* part_pooled, cudaStream_t st);
+des_status_t des_dense1_backward(des_table* t, const float* pooled, const float* gE, const float* gZ,
+                                 float* gE_work, int B, cudaStream_t st);

@@ -1,0 +1,296 @@
+// Table life cycle and inspection: allocation of slots / rows / state /
+// workspace, status, size, export, row read-back (Section 5, "Dynamic Hash
+// Table": the storage behind lookup / insert / update).
+#include <new>
+#include <string.h>
+
+#include "des_internal.cuh"
+
+static void* dalloc(const des_config_t& c, size_t bytes) {
+  if (bytes == 0) bytes = 256;
+  if (c.alloc) return c.alloc(bytes, c.alloc_ctx);
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return p;
+}
+static void dfree(const des_config_t& c, void* p) {
+  if (!p) return;
+  if (c.dealloc) c.dealloc(p, c.alloc_ctx); else cudaFree(p);
+}
+
+__global__ void fill_f32_kernel(float* p, size_t n, float v) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += st) p[i] = v;
+}
+
+extern "C" const char* des_status_string(des_status_t s) {
+  switch (s) {
+    case DES_OK: return "ok";
+    case DES_ERR_INVALID_ARG: return "invalid argument";
+    case DES_ERR_RESERVED_KEY: return "reserved key (all ones) in the batch";
+    case DES_ERR_CAPACITY: return "a shard is out of slots or rows";
+    case DES_ERR_UNSUPPORTED: return "unsupported";
+    case DES_ERR_CUDA: return "CUDA runtime error or no device";
+    case DES_ERR_NOT_FOUND: return "not found";
+  }
+  return "?";
+}
+
+extern "C" des_status_t des_table_destroy(des_table_t* t) {
+  if (!t) return DES_OK;
+  cudaSetDevice(t->device);
+  cudaDeviceSynchronize();
+  void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->Gbuf, t->hinfo, t->dest, t->hot_base,
+                  t->hot_R, t->hot_u, t->hot_ctr,
+                  t->W1, t->accW1, t->W1b, t->gW1_part, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
+                  t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
+  for (void* p : ptrs) dfree(t->cfg, p);
+  delete t;
+  return DES_OK;
+}
+
+extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** out) {
+  if (!out) return DES_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!cfg) return DES_ERR_INVALID_ARG;
+  const des_config_t& c = *cfg;
+  if (c.num_shards < 1 || c.num_shards > DES_MAX_SHARDS || c.num_fields < 1 || c.num_fields > 1024 ||
+      c.emb_dim < 4 || c.emb_dim > 64 || (c.emb_dim & 3) || (c.hidden & 3) || c.partition > DES_PART_FIELD ||
+      c.optimizer > DES_OPT_ADAGRAD || c.max_rows == 0 || !(c.max_load > 0.f && c.max_load <= 0.9f) ||
+      c.max_nnz <= 0 || c.max_nnz >= (1ll << 31) || c.max_batch <= 0 || c.max_uniq < 0 ||
+      (int64_t)c.max_batch * c.num_fields >= (1ll << 31))
+    return DES_ERR_INVALID_ARG;
+  if ((c.alloc == nullptr) != (c.dealloc == nullptr)) return DES_ERR_INVALID_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return DES_ERR_CUDA; }
+  des_table* t = new (std::nothrow) des_table();
+  if (!t) return DES_ERR_CUDA;
+  memset(t, 0, sizeof(*t));
+  t->cfg = c; t->cfg.h_rows_per_shard = nullptr; t->device = dev;
+  t->S = c.num_shards; t->F = c.num_fields; t->k = c.emb_dim; t->H = c.hidden; t->stride = c.emb_dim + 4;
+  t->max_nnz = c.max_nnz; t->max_batch = c.max_batch; t->max_uniq = c.max_uniq ? c.max_uniq : c.max_nnz;
+  if (t->max_uniq > t->max_nnz) t->max_uniq = t->max_nnz;
+  cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  DevMeta hm; memset(&hm, 0, sizeof(hm));
+  uint64_t rows = 0, slots = 0;
+  for (uint32_t s = 0; s < t->S; ++s) {
+    uint64_t cap = c.h_rows_per_shard ? c.h_rows_per_shard[s]
+                                      : (uint64_t)((double)(c.max_rows / t->S) * 1.05) + 1024;
+    if (cap == 0) cap = 1;
+    uint64_t ns = (uint64_t)((double)cap / (double)c.max_load) + 1;
+    if (cap >= 0xFFFFFFF0ull) { delete t; return DES_ERR_INVALID_ARG; }
+    t->h_row_base[s] = rows; t->h_slot_base[s] = slots;
+    hm.row_base[s] = rows; hm.slot_base[s] = slots; hm.row_cap[s] = (uint32_t)cap;
+    rows += cap; slots += ns;
+  }
+  t->h_row_base[t->S] = rows; t->h_slot_base[t->S] = slots;
+  hm.row_base[t->S] = rows; hm.slot_base[t->S] = slots;
+  if (rows >= 0xFFFFFFF0ull || slots >= 0xFFFFFFF0ull) { delete t; return DES_ERR_INVALID_ARG; }
+  t->total_rows = rows; t->total_slots = slots;
+  // fields sorted by (owning shard under FIELD, field): the K order of the row-split GEMM
+  {
+    uint32_t n = 0;
+    for (uint32_t s = 0; s < t->S; ++s)
+      for (uint32_t f = 0; f < t->F; ++f)
+        if (f % t->S == s) hm.field_order[n++] = f;
+  }
+  t->nblk_max = (uint32_t)((t->max_nnz + 1023) / 1024) + 1;
+  const size_t rowbytes = (size_t)t->stride * 4;
+  const size_t FKH = (size_t)t->F * t->k * t->H;
+  bool ok = true;
+  auto A = [&](auto*& p, size_t bytes) {
+    p = (typename std::remove_reference<decltype(p)>::type)dalloc(c, bytes);
+    if (!p) ok = false;
+  };
+  A(t->slots, slots * sizeof(Slot));
+  A(t->W, rows * rowbytes);
+  if (c.optimizer == DES_OPT_ADAGRAD) A(t->A, rows * rowbytes);
+  A(t->meta, sizeof(DevMeta));
+  A(t->slot_of, (size_t)t->max_nnz * 4);
+  A(t->flags, (size_t)t->max_nnz);
+  A(t->uslot, (size_t)t->max_nnz * 4);
+  A(t->blk_cnt, (size_t)(t->S + 1) * t->nblk_max * 4);
+  t->hot_max = 65536;
+  t->rep_max = (uint32_t)(t->max_nnz / 256 + t->hot_max + 1024);
+  A(t->Gbuf, ((size_t)t->max_uniq + t->rep_max) * rowbytes);
+  A(t->hinfo, (size_t)t->max_uniq * 4);
+  A(t->dest, (size_t)t->max_nnz * 4);
+  A(t->hot_base, (size_t)t->hot_max * 4);
+  A(t->hot_R, (size_t)t->hot_max * 4);
+  A(t->hot_u, (size_t)t->hot_max * 4);
+  A(t->hot_ctr, 256);
+  if (t->H) {
+    A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
+    t->gw1_splits = 32;
+    A(t->gW1_part, (size_t)t->gw1_splits * FKH * 4);
+  }
+  if (!ok) { des_table_destroy(t); return DES_ERR_CUDA; }
+  bool cu = true;
+  cu &= cudaMemset(t->slots, 0xFF, slots * sizeof(Slot)) == cudaSuccess;
+  cu &= cudaMemset(t->Gbuf, 0, ((size_t)t->max_uniq + t->rep_max) * rowbytes) == cudaSuccess;
+  cu &= cudaMemset(t->hinfo, 0, (size_t)t->max_uniq * 4) == cudaSuccess;
+  cu &= cudaMemcpy(t->meta, &hm, sizeof(hm), cudaMemcpyHostToDevice) == cudaSuccess;
+  if (t->H) {
+    cu &= cudaMemset(t->W1, 0, FKH * 4) == cudaSuccess;
+    cu &= cudaMemset(t->W1b, 0, FKH * 2) == cudaSuccess;
+    fill_f32_kernel<<<256, 256>>>(t->accW1, FKH, c.init_acc);
+    cu &= cudaGetLastError() == cudaSuccess;
+  }
+  cu &= cudaDeviceSynchronize() == cudaSuccess;
+  if (!cu) { cudaGetLastError(); des_table_destroy(t); return DES_ERR_CUDA; }
+  *out = t;
+  return DES_OK;
+}
+
+extern "C" des_status_t des_table_status(des_table_t* t) {
+  if (!t) return DES_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DES_ERR_CUDA;
+  uint32_t e = 0;
+  DES_CUDA(cudaMemcpy(&e, &t->meta->err, 4, cudaMemcpyDeviceToHost));
+  return (des_status_t)e;
+}
+
+extern "C" des_status_t des_table_size(des_table_t* t, uint64_t* h) {
+  if (!t || !h) return DES_ERR_INVALID_ARG;
+  uint32_t n[DES_MAX_SHARDS];
+  DES_CUDA(cudaDeviceSynchronize());
+  DES_CUDA(cudaMemcpy(n, t->meta->n_rows, sizeof(n), cudaMemcpyDeviceToHost));
+  for (uint32_t s = 0; s < t->S; ++s) h[s] = n[s];
+  return DES_OK;
+}
+
+extern "C" des_status_t des_table_row_base(des_table_t* t, uint64_t* h) {
+  if (!t || !h) return DES_ERR_INVALID_ARG;
+  for (uint32_t s = 0; s <= t->S; ++s) h[s] = t->h_row_base[s];
+  return DES_OK;
+}
+
+extern "C" uint64_t des_table_launch_count(des_table_t* t) { return t ? t->launches : 0; }
+
+__global__ void export_kernel(const Slot* __restrict__ slots, unsigned long long nslots, const DevMeta* __restrict__ meta,
+                              int S, int k, int stride, const float* __restrict__ W, const float* __restrict__ A,
+                              unsigned long long* keys, uint8_t* shards, uint32_t* rows, float* emb, float* lin,
+                              float* acc_emb, float* acc_lin, unsigned long long cap, unsigned long long* counter) {
+  unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  unsigned long long st = (unsigned long long)gridDim.x * blockDim.x;
+  for (; i < nslots; i += st) {
+    Slot sl = slots[i];
+    if (sl.key == DES_KEY_EMPTY || sl.row == DES_ROW_NONE) continue;
+    int s = 0;
+    while (s + 1 < S && meta->slot_base[s + 1] <= i) ++s;
+    unsigned long long o = atomicAdd(counter, 1ull);
+    if (o >= cap) continue;
+    unsigned long long g = meta->row_base[s] + sl.row;
+    if (keys) keys[o] = sl.key;
+    if (shards) shards[o] = (uint8_t)s;
+    if (rows) rows[o] = sl.row;
+    for (int c = 0; c < k; ++c) {
+      if (emb) emb[o * k + c] = W[g * stride + c];
+      if (acc_emb) acc_emb[o * k + c] = A ? A[g * stride + c] : 0.f;
+    }
+    if (lin) lin[o] = W[g * stride + k];
+    if (acc_lin) acc_lin[o] = A ? A[g * stride + k] : 0.f;
+  }
+}
+
+extern "C" des_status_t des_table_export(des_table_t* t, uint64_t* d_keys, uint8_t* d_shards, uint32_t* d_rows,
+                                         float* d_emb, float* d_lin, float* d_acc_emb, float* d_acc_lin,
+                                         uint64_t cap, uint64_t* h_n_out) {
+  if (!t || !h_n_out) return DES_ERR_INVALID_ARG;
+  unsigned long long* ctr = nullptr;
+  DES_CUDA(cudaMalloc(&ctr, 8));
+  cudaMemset(ctr, 0, 8);
+  export_kernel<<<t->sm_count * 8, 256>>>(t->slots, t->total_slots, t->meta, t->S, t->k, t->stride, t->W, t->A,
+                                          (unsigned long long*)d_keys, d_shards, d_rows, d_emb, d_lin, d_acc_emb,
+                                          d_acc_lin, cap, ctr);
+  t->launches++;
+  cudaError_t e = cudaDeviceSynchronize();
+  unsigned long long n = 0;
+  if (e == cudaSuccess) e = cudaMemcpy(&n, ctr, 8, cudaMemcpyDeviceToHost);
+  cudaFree(ctr);
+  if (e != cudaSuccess) return DES_ERR_CUDA;
+  *h_n_out = n;
+  return DES_OK;
+}
+
+__global__ void read_rows_kernel(const uint32_t* __restrict__ grows, long long n, int k, int stride,
+                                 unsigned long long total_rows, const float* __restrict__ W,
+                                 const float* __restrict__ A, float* emb, float* lin, float* acc_emb, float* acc_lin) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t g = grows[i];
+  bool ok = g != DES_ROW_NONE && g < total_rows;
+  for (int c = 0; c < k; ++c) {
+    if (emb) emb[i * k + c] = ok ? W[(size_t)g * stride + c] : 0.f;
+    if (acc_emb) acc_emb[i * k + c] = (ok && A) ? A[(size_t)g * stride + c] : 0.f;
+  }
+  if (lin) lin[i] = ok ? W[(size_t)g * stride + k] : 0.f;
+  if (acc_lin) acc_lin[i] = (ok && A) ? A[(size_t)g * stride + k] : 0.f;
+}
+
+extern "C" des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n, float* d_emb,
+                                            float* d_lin, float* d_acc_emb, float* d_acc_lin, void* stream) {
+  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;
+  read_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}
+
+__global__ void write_rows_kernel(const uint32_t* __restrict__ grows, long long n, int k, int stride,
+                                  unsigned long long total_rows, float* W, float* A, const float* __restrict__ emb,
+                                  const float* __restrict__ lin, const float* __restrict__ acc_emb,
+                                  const float* __restrict__ acc_lin) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t g = grows[i];
+  if (g == DES_ROW_NONE || g >= total_rows) return;
+  for (int c = 0; c < k; ++c) {
+    if (emb) W[(size_t)g * stride + c] = emb[i * k + c];
+    if (acc_emb && A) A[(size_t)g * stride + c] = acc_emb[i * k + c];
+  }
+  if (lin) W[(size_t)g * stride + k] = lin[i];
+  if (acc_lin && A) A[(size_t)g * stride + k] = acc_lin[i];
+}
+
+extern "C" des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                             const float* d_emb, const float* d_lin, const float* d_acc_emb,
+                                             const float* d_acc_lin, void* stream) {
+  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;
+  write_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}
+
+// ---- first dense layer weights ----------------------------------------------
+__global__ void w1_shadow_kernel(const float* __restrict__ W1, __nv_bfloat16* __restrict__ W1b, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
+  for (; i < n; i += st) W1b[i] = __float2bfloat16_rn(W1[i]);
+}
+
+extern "C" des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream) {
+  if (!t || !d_W1 || !t->H) return DES_ERR_INVALID_ARG;
+  size_t n = (size_t)t->F * t->k * t->H;
+  DES_CUDA(cudaMemcpyAsync(t->W1, d_W1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  w1_shadow_kernel<<<256, 256, 0, (cudaStream_t)stream>>>(t->W1, t->W1b, n);
+  DES_LAUNCH_CHECK(t);
+  return DES_OK;
+}
+
+extern "C" des_status_t des_dense1_get(des_table_t* t, float* d_W1, void* stream) {
+  if (!t || !d_W1 || !t->H) return DES_ERR_INVALID_ARG;
+  size_t n = (size_t)t->F * t->k * t->H;
+  DES_CUDA(cudaMemcpyAsync(d_W1, t->W1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return DES_OK;
+}
+
+des_status_t des_check_batch(const des_table* t, const des_batch_t* b, int need_dedup) {
+  if (!t || !b) return DES_ERR_INVALID_ARG;
+  if (b->batch <= 0 || b->batch > t->max_batch || b->nnz < 0 || b->nnz > t->max_nnz) return DES_ERR_INVALID_ARG;
+  if (!b->offsets || !b->rows || !b->shards || (b->nnz > 0 && !b->ids)) return DES_ERR_INVALID_ARG;
+  if (need_dedup && (!b->uidx || !b->uniq_rows || !b->n_uniq)) return DES_ERR_INVALID_ARG;
+  return DES_OK;
+}

@@ -1,0 +1,243 @@
+"""Shared driver of the parity tests: runs one DES step on the CPU oracle and
+on the CUDA library (through the C ABI binding) from the same seeded batch, and
+compares everything the step produces.
+
+Tolerances
+  integer outputs (shards, rows, unique indices, key set, init bits): exact;
+  float32 forward outputs: |d| <= 1e-5 |ref| + 1e-6 + 2e-6 * sum_j |t_j| for the
+    per-sample sums (M_1 of LR and FM, A, R_lr): in the multi-hot workloads one
+    hot id occurs hundreds of times in a sample, its row is added again and
+    again to a growing float32 accumulator, and when the other terms cancel the
+    (small) result cannot stay within 1e-5 of itself in float32; the last term
+    measures the error against the size of the summands instead (condition-
+    aware bound; it is zero-cost for the well-conditioned elements);
+  summed per-key gradients G: |dG| <= 1e-5 |G| + 1e-6 + 2e-7 * sum_j |g_j|: a hot
+    key sums thousands of O(1) terms of both signs; the scatter keeps every
+    float32 chain to a few hundred additions and combines them in double, hence
+    the ten times smaller constant.
+  updated weights / optimizer state: the forward tolerance plus what dG does to
+    ONE optimizer application (SGD: lr dG; Adagrad: lr dG / (sqrt(acc) + eps)
+    for the weight, 2|G| dG + dG^2 for the accumulator) — Adagrad divides by
+    sqrt(acc), so a gradient that cancels to ~eps moves the weight by O(lr)
+    for a rounding-sized dG;
+  anything downstream of the bf16 first-layer GEMM: 2e-2 relative plus 1e-3 of
+    the tensor's largest magnitude (elements that cancel to ~0).
+After every step the CUDA table's touched rows are overwritten with the
+oracle's (des_table_write_rows), so each step is compared from identical state
+and tolerated differences do not compound; `resync=False` keeps the drift."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import Oracle
+from paper_1909_04823_b200 import synth
+from paper_1909_04823_b200.synth import OP_DENSE1, OP_FM, OP_LR, OP_POOL, PART_FIELD
+
+RTOL, ATOL, SUMTOL, SUMTOL_FWD = 1e-5, 1e-6, 2e-7, 2e-6
+
+
+def close32(got, ref, what, rtol=RTOL, atol=ATOL, extra=None):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    err = np.abs(got - ref)
+    tol = rtol * np.abs(ref) + atol
+    if extra is not None:
+        tol = tol + extra
+    if not np.all(err <= tol):
+        i = np.unravel_index(np.argmax(err - tol), err.shape)
+        raise AssertionError(f"{what}: worst at {i}: got {got[i]!r} ref {ref[i]!r} err {err[i]:.3e} tol {tol[i]:.3e}; "
+                             f"{int((err > tol).sum())} of {err.size} out of tolerance")
+
+
+def close_gemm(got, ref, what, extra=None):
+    ref = np.asarray(ref, dtype=np.float64)
+    close32(got, ref, what, rtol=2e-2, atol=1e-3 * max(float(np.abs(ref).max()), 1e-30), extra=extra)
+
+
+def u32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().numpy().view(np.uint32)
+
+
+def rows_per_shard_for(w, cap_total):
+    """Row capacity per shard: even under HASH; by field vocabulary under FIELD."""
+    if w.partition != PART_FIELD:
+        return None
+    per_field = []
+    for f in range(w.fields):
+        per_field.append(64 if f < w.bucket_fields else cap_total // max(1, w.fields - w.bucket_fields))
+    out = [256] * w.shards
+    for f, n in enumerate(per_field):
+        out[f % w.shards] += int(n * 1.05) + 64
+    return out
+
+
+class Pair:
+    """Oracle table + CUDA table for one workload."""
+
+    def __init__(self, w, max_rows, max_nnz, max_batch=None, max_uniq=0, resync=True):
+        from paper_1909_04823_b200.binding import Table
+        self.w = w
+        self.o = Oracle.for_workload(w)
+        self.t = Table.for_workload(w, max_rows=max_rows, max_nnz=max_nnz, max_batch=max_batch or w.batch,
+                                    rows_per_shard=rows_per_shard_for(w, max_rows), max_uniq=max_uniq)
+        self.row_base = np.array(self.t.row_base(), dtype=np.int64)
+        self.resync = resync
+        self.drifted = False        # True once un-resynced differences may have accumulated
+        if w.hidden:
+            W1 = synth.dense1_weights(w)
+            self.o.dense1_set(W1)
+            self.t.dense1_set(torch.from_numpy(W1).cuda())
+
+    def close(self):
+        self.t.close(); self.o.close()
+
+    # ------------------------------------------------------------------
+    def insert_only(self, batch):
+        from paper_1909_04823_b200.binding import DeviceBatch
+        fi = self.o.find_or_insert(batch)
+        db = DeviceBatch.from_synth(batch)
+        self.t.find_or_insert(db, True)
+        self.compare_index(batch, fi, db)
+        return fi, db
+
+    def compare_index(self, batch, fi, db):
+        n = batch.nnz
+        assert self.t.status() == 0
+        assert np.array_equal(db.shards.cpu().numpy()[:n], fi["shards"]), "shards"
+        assert np.array_equal(u32(db.rows)[:n], fi["rows"]), "rows"
+        assert np.array_equal(u32(db.uidx)[:n], fi["uidx"]), "uidx"
+        U = int(db.n_uniq.item())
+        assert U == fi["U"], ("n_uniq", U, fi["U"])
+        want = self.row_base[fi["uniq_shard"].astype(np.int64)] + fi["uniq_row"].astype(np.int64)
+        assert np.array_equal(u32(db.uniq_rows)[:U].astype(np.int64), want), "uniq_rows"
+        assert self.t.size() == [int(v) for v in self.o.size()], "table size"
+
+    def compare_rows(self, fi, db, exact=False, gemm=False, what="rows", G=None):
+        U = fi["U"]
+        ref = self.o.read_rows(fi["uniq_shard"], fi["uniq_row"])
+        got = self.t.read_rows(db.uniq_rows[:U])
+        torch.cuda.synchronize()
+        sgd = self.w.optimizer == synth.OPT_SGD
+        for name in ("emb", "lin", "acc_emb", "acc_lin"):
+            g = got[name].cpu().numpy()
+            if sgd and name.startswith("acc"):
+                continue
+            if exact:
+                assert np.array_equal(g.view(np.uint32), ref[name].view(np.uint32)), f"{what}.{name} bits"
+                continue
+            extra = None
+            if G is not None:
+                emb = name.endswith("emb")
+                Gk = (G["Gv"] if emb else G["Gw"]).astype(np.float64)
+                dG = RTOL * np.abs(Gk) + ATOL + SUMTOL * (G["Sv"] if emb else G["Sw"])
+                if gemm:
+                    dG = dG + 2e-2 * np.abs(Gk) + 1e-3 * max(float(np.abs(Gk).max()), 1e-30)
+                if name.startswith("acc"):
+                    extra = 2.0 * np.abs(Gk) * dG + dG * dG
+                elif sgd:
+                    extra = self.w.lr * dG
+                else:
+                    acc = ref["acc_" + name].astype(np.float64)
+                    extra = self.w.lr * dG / (np.sqrt(acc) + self.w.eps)
+            (close_gemm if gemm else close32)(g, ref[name], f"{what}.{name}", extra=extra)
+        return ref
+
+    # ------------------------------------------------------------------
+    def step(self, batch, grads, ops=None, materialise=False, check_init=False):
+        """One full step on both sides with every intermediate compared."""
+        from paper_1909_04823_b200.binding import DeviceBatch
+        w = self.w
+        ops = w.ops if ops is None else ops
+        B, F, k, S, H = batch.batch, w.fields, w.emb_dim, w.shards, w.hidden
+        dev = "cuda"
+        cmp = close_gemm if self.drifted else close32
+        # ---- index
+        fi = self.o.find_or_insert(batch)
+        db = DeviceBatch.from_synth(batch)
+        self.t.find_or_insert(db, True)
+        self.compare_index(batch, fi, db)
+        if check_init:
+            self.compare_rows(fi, db, exact=True, what="initial rows")
+        # ---- forward
+        op = self.o.forward_partials(ops, batch, fi, want_pooled=True, want_dense=bool(ops & OP_DENSE1))
+        oa = self.o.aggregate(B, op)
+        sabs = self.o.forward_original(ops & ~OP_DENSE1, batch)["Sabs"]
+        xa, xl = SUMTOL_FWD * sabs[:, :k], SUMTOL_FWD * sabs[:, k]
+        part_small = torch.full((S, B, k + 4), float("nan"), device=dev)
+        pooled = torch.full((B, F * k), float("nan"), device=dev)
+        part_pooled = torch.empty((S, B, F * k), device=dev) if materialise else None
+        part_dense = torch.empty((S, B, H), device=dev) if (materialise and (ops & OP_DENSE1)) else None
+        out_small = torch.full((B, k + 4), float("nan"), device=dev)
+        Z = torch.full((B, max(H, 1)), float("nan"), device=dev)
+        self.t.forward_partials(ops, db, part_small, pooled, part_pooled, part_dense)
+        self.t.aggregate(ops, db, part_small, pooled, part_pooled, part_dense, out_small, pooled, Z)
+        torch.cuda.synchronize()
+        assert self.t.status() == 0
+        ps = part_small.cpu().numpy()
+        osm = out_small.cpu().numpy()
+        if ops & OP_FM:
+            cmp(ps[:, :, :k], op["part_small"][:, :, :k], "part_small.M1_fm", extra=xa[None])
+            cmp(ps[:, :, k + 1], op["part_small"][:, :, k + 1], "part_small.M2_fm",
+                extra=SUMTOL_FWD * op["part_small"][:, :, k + 1])
+            cmp(osm[:, :k], oa["A"], "A", extra=xa)
+            cmp(osm[:, k + 2], oa["Q"], "Q", extra=SUMTOL_FWD * oa["Q"])
+            # fm2 = (<A,A> - Q)/2 subtracts two float32-rounded inputs of size <A,A>/2 and Q/2
+            AA = np.sum(oa["A"] ** 2, axis=1)
+            cmp(osm[:, k + 1], oa["fm2"], "fm2",
+                extra=SUMTOL_FWD * (AA + np.abs(oa["Q"])) + np.sum(np.abs(oa["A"]) * xa, axis=1))
+        if ops & OP_LR:
+            cmp(ps[:, :, k], op["part_small"][:, :, k], "part_small.M1_lr", extra=xl[None])
+            cmp(osm[:, k], oa["lr"], "R_lr", extra=xl)
+        if ops & (OP_LR | OP_FM):
+            assert not np.any(ps[:, :, k + 2:]) and not np.any(osm[:, k + 3]), "padding must be zero"
+        if ops & (OP_POOL | OP_DENSE1):
+            cmp(pooled.cpu().numpy(), oa["pooled"], "pooled")
+            if materialise:
+                cmp(part_pooled.cpu().numpy(), op["part_pooled"], "part_pooled")
+        if ops & OP_DENSE1:
+            close_gemm(Z.cpu().numpy(), oa["Z"], "Z")
+            if materialise:
+                close_gemm(part_dense.cpu().numpy(), op["part_dense"], "part_dense")
+        # ---- backward + update
+        g = grads
+        gdev = {n: torch.from_numpy(v).to(dev) for n, v in g.items()}
+        gE_work = torch.empty((B, F * k), device=dev) if (ops & OP_DENSE1) else None
+        ob = self.o.backward_update(ops, batch, fi, oa["A"].astype(np.float32),
+                                    oa["pooled"].astype(np.float32) if oa["pooled"] is not None else None,
+                                    g.get("gL"), g.get("gF"), g.get("gE") if (ops & OP_POOL) else None,
+                                    g.get("gZ") if (ops & OP_DENSE1) else None)
+        if self.resync:
+            # stage-wise parity: the CUDA backward starts from the same aggregated forward
+            # results as the oracle's (its own were compared above), so that differences
+            # tolerated in the forward do not leak into the gradient comparison
+            o32 = np.zeros((B, k + 4), dtype=np.float32)
+            o32[:, :k] = oa["A"].astype(np.float32)
+            out_small = torch.from_numpy(o32).to(dev)
+            if oa["pooled"] is not None:
+                pooled = torch.from_numpy(oa["pooled"].astype(np.float32)).to(dev)
+        self.t.backward_update(ops, db, out_small, pooled, Z, gdev.get("gL"), gdev.get("gF"),
+                               gdev.get("gE") if (ops & OP_POOL) else None,
+                               gdev.get("gZ") if (ops & OP_DENSE1) else None, gE_work)
+        torch.cuda.synchronize()
+        assert self.t.status() == 0
+        gemm = bool(ops & OP_DENSE1) or self.drifted
+        W1o = None
+        if ops & OP_DENSE1:
+            close_gemm(gE_work.cpu().numpy(), ob["gE_total"], "gE_total")
+            W1o, _ = self.o.dense1_get()
+            close_gemm(self.t.dense1_get().cpu().numpy(), W1o, "W1")
+        ref = self.compare_rows(fi, db, gemm=gemm, what="updated rows", G=ob)
+        if self.resync:
+            U = fi["U"]
+            td = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+            sgd = w.optimizer == synth.OPT_SGD
+            self.t.write_rows(db.uniq_rows[:U], td(ref["emb"]), td(ref["lin"]),
+                              None if sgd else td(ref["acc_emb"]), None if sgd else td(ref["acc_lin"]))
+            if W1o is not None:
+                self.t.dense1_set(td(W1o))
+            torch.cuda.synchronize()
+        else:
+            self.drifted = True
+        return dict(fi=fi, db=db, oracle_agg=oa, out_small=osm, oracle_bwd=ob)
