@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the DES sparse step (find-or-insert, per-shard partials, shard
+reduction + F, backward scatter + optimizer) on synthetic CTR-shaped batches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+One JSON line on stdout (rank 0).  `value` = samples/s of the whole job with
+the batch already resident in HBM; `e2e` = the same step through des_step_host
+from pinned host buffers (H2D of the batch and D2H of the aggregated outputs
+inside the timed region); `roofline` = the kernel with the largest share of the
+step against the measured HBM copy bandwidth; `cpu_baseline` = the CPU oracle,
+as it stands, on a bounded sample of the same batch.
+
+With N > 1 (launched by torch.distributed.run) every rank runs its own replica
+of the table on its own batches — the path has no exchange between GPUs — and
+the job's samples/s is N * B over the slowest rank's time ("weak" scaling)."""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1909_04823_b200 import synth  # noqa: E402
+from paper_1909_04823_b200.synth import OP_DENSE1, OP_FM, OP_LR, OP_POOL, PART_FIELD  # noqa: E402
+
+METRIC = "samples/sec per DES fwd+bwd sparse step"
+UNIT = "samples/s"
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def rows_per_shard(w, cap_total):
+    if w.partition != PART_FIELD:
+        return None
+    cat = max(1, w.fields - w.bucket_fields)
+    out = [256] * w.shards
+    for f in range(w.fields):
+        n = 64 if f < w.bucket_fields else cap_total // cat
+        out[f % w.shards] += int(n * 1.05) + 64
+    return out
+
+
+def sub_batch(b, n_samples):
+    """The first n_samples samples of a batch (a bounded sample for the CPU leg)."""
+    F = b.fields
+    end = int(b.offsets[n_samples * F])
+    return synth.Batch(n_samples, F, b.offsets[:n_samples * F + 1].copy(), b.ids[:end].copy(),
+                       None if b.vals is None else b.vals[:end].copy())
+
+
+# ---------------------------------------------------------------------------
+def oracle_step(o, w, b, g):
+    fi = o.find_or_insert(b)
+    part = o.forward_partials(w.ops, b, fi, want_pooled=bool(w.ops & (OP_POOL | OP_DENSE1)),
+                              want_dense=bool(w.ops & OP_DENSE1))
+    agg = o.aggregate(b.batch, part)
+    pooled = None if agg["pooled"] is None else agg["pooled"].astype(np.float32)
+    o.backward_update(w.ops, b, fi, agg["A"].astype(np.float32), pooled, g.get("gL"), g.get("gF"),
+                      g.get("gE") if (w.ops & OP_POOL) else None, g.get("gZ") if (w.ops & OP_DENSE1) else None)
+
+
+def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0):
+    """Times the CPU oracle on the first Bs samples of `batch`, Bs sized so that
+    one step takes about budget_s seconds.  Returns (samples/s, Bs, seconds per step)."""
+    from oracle import Oracle
+    if w.hidden:
+        W1 = synth.dense1_weights(w)
+
+    def run(bs, n):
+        sb = sub_batch(batch, bs)
+        g = {k_: v[:bs] for k_, v in grads.items()}
+        o = Oracle.for_workload(w)
+        if w.hidden:
+            o.dense1_set(W1)
+        ts = []
+        for _ in range(n):
+            t0 = time.perf_counter()
+            oracle_step(o, w, sb, g)
+            ts.append(time.perf_counter() - t0)
+        o.close()
+        return ts
+
+    probe = max(1, min(batch.batch, 8))
+    t = run(probe, 1)[0]
+    per_sample = max(t / probe, 1e-7)
+    bs = int(max(1, min(batch.batch, budget_s / per_sample)))
+    ts = run(bs, warmup + steps)[warmup:]
+    sec = float(np.mean(ts))
+    return bs / sec, bs, sec
+
+
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.f.name):
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for n_, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n_)
+        os.unlink(self.f.name)
+        if sm:
+            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+# ---------------------------------------------------------------------------
+def kernel_bytes(name, st):
+    """Algorithmic bytes one launch of `name` must move (what the method needs,
+    each datum once; see the design notes for the derivation)."""
+    nnz, B, F, k, S, U, R = st["nnz"], st["B"], st["F"], st["k"], st["S"], st["U"], st["rep_rows"]
+    row = 4 * k + 16
+    state = 1 if st["adagrad"] else 0
+    small = bool(st["ops"] & (OP_LR | OP_FM))
+    pool = bool(st["ops"] & (OP_POOL | OP_DENSE1))
+    if name == "probe_claim_kernel":
+        return 8 * nnz + 16 * U + 4 * nnz + nnz
+    if name == "flag_count_kernel":
+        return 4 * nnz + 16 * U + nnz + nnz
+    if name == "assign_kernel":
+        return nnz + nnz + 4 * U + 8 * U + 4 * U
+    if name == "resolve_kernel":
+        return 4 * nnz + 16 * U + 8 * nnz
+    if name == "forward_partials_kernel":
+        return 4 * (B * F + 1) + 5 * nnz + row * U + (4 * S * B * (k + 4) if small else 0) + (4 * B * F * k if pool else 0)
+    if name == "aggregate_small_kernel":
+        return 4 * S * B * (k + 4) + 4 * B * (k + 4)
+    if name == "make_dest_kernel":
+        return 8 * nnz + 4 * U
+    if name == "grad_scatter_kernel":
+        return 4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + 2 * row * (U + R)
+    if name == "hot_reduce_kernel":
+        return 2 * row * R
+    if name == "update_rows_kernel":
+        return U * (2 * row + 2 * row * (1 + state) + 8)
+    return None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, help="workload 1..5 (default: 5, the large multi-hot one)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--vocab", type=int, default=0, help="override the number of pre-populated keys (config 5)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = synth.config(args.config)
+    if world > 1:
+        w = w.scaled(seed=w.seed + 1000 * rank)     # every replica has its own data stream
+
+    # ------------------------------------------------------------------ reference arm: the CPU oracle
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        ww = w
+        if ww.vocab > 20_000_000 or ww.prepopulate > 20_000_000:
+            # the sample touches a few thousand keys; their rows are a pure function of the id, so the
+            # oracle needs no pre-populated table to reproduce the first step of the full workload
+            pass
+        st = synth.Stream(ww)
+        b = st.next_batch()
+        g = synth.upstream_grads(ww, b.batch, 0)
+        budget = min(args.cpu_budget, 120.0 / max(1, args.steps + args.warmup))
+        v, bs, sec = time_oracle(ww, b, g, budget_s=budget, steps=max(1, args.steps), warmup=args.warmup)
+        cores = 1
+        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": {"workload": ww.name, "batch": ww.batch, "fields": ww.fields, "emb_dim": ww.emb_dim,
+                           "shards": ww.shards, "sample": f"first {bs} of {ww.batch} samples per step"},
+                "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                 "sample": f"first {bs} of {ww.batch} samples of one batch, table holding the keys it touches"},
+                "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line), flush=True)
+        return 0
+
+    # ------------------------------------------------------------------ our arm
+    import torch
+    import torch.distributed as dist
+    from paper_1909_04823_b200.binding import DeviceBatch, Table
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DES path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    hbm_peak, peak_kind = measured_peaks()
+
+    # ---- size the table for the memory that is actually free
+    free_b, total_b = torch.cuda.mem_get_info()
+    prepop = w.prepopulate
+    vocab = w.vocab
+    if args.config == 5:
+        if args.vocab:
+            prepop = vocab = args.vocab
+        per_key = 2 * (4 * w.emb_dim + 16) * 1.06 + 16 * 2.2      # rows + state + slots at load 0.5
+        fit = int((free_b - 14e9) / per_key)
+        if fit < prepop:
+            prepop = vocab = max(1_000_000, (fit // 1_000_000) * 1_000_000)
+            log(f"[bench] only {free_b / 1e9:.0f} GB free: table scaled to {prepop} keys")
+        w = w.scaled(vocab=vocab, prepopulate=prepop)
+    stream = synth.Stream(w)
+    n_batches = 2 if args.config != 4 else min(args.steps + args.warmup, 12)
+    t0 = time.time()
+    batches = [stream.next_batch() for _ in range(n_batches)]
+    log(f"[bench] generated {n_batches} batches of {w.name}: nnz {batches[0].nnz} in {time.time() - t0:.1f}s")
+    max_nnz = int(max(b.nnz for b in batches) * 1.02) + 1024
+    if args.config == 4:
+        max_rows = int(prepop + (args.steps + args.warmup + 2) * batches[0].nnz * w.p_new * 1.3) + 100000
+    elif args.config == 5:
+        max_rows = prepop
+    else:
+        max_rows = int(sum(len(np.unique(b.ids)) for b in batches) * (3 + args.steps)) + 100000
+        max_rows = min(max_rows, 40_000_000)
+    uniq0 = int(len(np.unique(batches[0].ids)))
+    max_uniq = min(max_nnz, int(uniq0 * 1.5) + 4096)
+    t = Table.for_workload(w, max_rows=max_rows, max_nnz=max(max_nnz, w.batch * w.fields), max_batch=w.batch,
+                           rows_per_shard=rows_per_shard(w, max_rows), max_uniq=max_uniq)
+    if w.hidden:
+        t.dense1_set(torch.from_numpy(synth.dense1_weights(w)).to(dev))
+
+    # ---- pre-population (not timed)
+    if prepop:
+        t0 = time.time()
+        per_call = w.batch * w.fields
+        for ids in stream.prepopulation_ids(chunk=per_call * 8):
+            d_all = torch.from_numpy(ids.view(np.int64)).to(dev)
+            for lo in range(0, ids.size, per_call):
+                n = min(per_call, ids.size - lo)
+                pb = synth.prepopulation_batch(ids[lo:lo + n], w.fields)
+                db = DeviceBatch(pb.offsets, d_all[lo:lo + n], None, pb.batch, dev)
+                t.find_or_insert(db, True)
+        t.check_status()
+        log(f"[bench] pre-populated {sum(t.size())} keys in {time.time() - t0:.1f}s")
+
+    B, F, k, S, H = w.batch, w.fields, w.emb_dim, w.shards, w.hidden
+    dbs = [DeviceBatch.from_synth(b, dev) for b in batches]
+    g_host = synth.upstream_grads(w, B, 0)
+    gd = {n_: torch.from_numpy(v).to(dev) for n_, v in g_host.items()}
+    small = bool(w.ops & (OP_LR | OP_FM)); pool = bool(w.ops & (OP_POOL | OP_DENSE1))
+    part_small = torch.zeros((S, B, k + 4), device=dev) if small else None
+    pooled = torch.zeros((B, F * k), device=dev) if pool else None
+    out_small = torch.zeros((B, k + 4), device=dev)
+    Z = torch.zeros((B, H), device=dev) if H else None
+    gE_work = torch.zeros((B, F * k), device=dev) if (w.ops & OP_DENSE1) else None
+    gE = gd.get("gE") if (w.ops & OP_POOL) else None
+    gZ = gd.get("gZ") if (w.ops & OP_DENSE1) else None
+
+    def step(i):
+        db = dbs[i % len(dbs)]
+        t.find_or_insert(db, True)
+        t.forward_partials(w.ops, db, part_small, pooled)
+        t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
+        t.backward_update(w.ops, db, out_small, pooled, Z, gd.get("gL"), gd.get("gF"), gE, gZ, gE_work)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    t.check_status()
+    barrier()
+    launches0 = t.launch_count()
+    t.profile_enable(True)
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    prof = t.profile_read()
+    t.profile_enable(False)
+    launches = t.launch_count() - launches0
+    t.check_status()
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    value = world * B / (ms_step / 1e3)
+
+    # ---- per-kernel shares and the roofline of the dominant kernel
+    per = {}
+    for name, ms in prof:
+        a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += ms
+    U = int(dbs[0].n_uniq.item())
+    stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, U=U, ops=w.ops, adagrad=(w.optimizer == synth.OPT_ADAGRAD),
+                 rep_rows=0)
+    tot_k = sum(v[1] for v in per.values()) or 1.0
+    kernels = []
+    for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
+        by = kernel_bytes(name, stats)
+        avg = ms / n_
+        kernels.append({"kernel": name, "launches": n_, "ms_per_launch": round(avg, 4), "share": round(ms / tot_k, 4),
+                        "alg_gbs": None if by is None else round(by / avg / 1e6, 1)})
+    top = kernels[0] if kernels else None
+    roofline = None
+    if top and top["alg_gbs"] is not None:
+        roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
+                    "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4), "traffic": None,
+                    "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
+    step_bytes = sum((kernel_bytes(kk["kernel"], stats) or 0) * kk["launches"] for kk in kernels) / args.steps
+
+    # ---- end to end from pinned host buffers
+    e2e = None
+    try:
+        if args.no_e2e:
+            raise RuntimeError("skipped by --no-e2e")
+        hb = batches[0]
+        h_off = torch.from_numpy(hb.offsets).pin_memory()
+        h_ids = torch.from_numpy(hb.ids.view(np.int64)).pin_memory()
+        h_out = torch.empty((B, k + 4), dtype=torch.float32).pin_memory()
+
+        def step_host():
+            t.step_host(w.ops, B, hb.nnz, h_off, h_ids, None, h_out, d_pooled=pooled, d_Z=Z, gL=gd.get("gL"),
+                        gF=gd.get("gF"), gE=gE, gZ=gZ, gE_work=gE_work)
+        for _ in range(max(1, min(args.warmup, 3))):
+            step_host()
+        barrier()
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record()
+        for _ in range(n_e2e):
+            step_host()
+        e1.record()
+        barrier()
+        ms_e = e0.elapsed_time(e1) / n_e2e
+        if world > 1:
+            tt = torch.tensor([ms_e], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_e = float(tt.item())
+        e2e = {"value": world * B / (ms_e / 1e3), "unit": UNIT, "ms_per_step": ms_e,
+               "h2d_bytes_per_step": int(h_off.numel() * 4 + h_ids.numel() * 8),
+               "d2h_bytes_per_step": int(h_out.numel() * 4)}
+    except Exception as ex:  # keep the device-resident number even if the host path fails
+        log(f"[bench] e2e failed: {ex!r}")
+    t.check_status()
+
+    # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        try:
+            v, bs, sec = time_oracle(w, batches[0], g_host, budget_s=args.cpu_budget)
+            cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                   "sample": f"first {bs} of {B} samples of one batch ({sec:.1f} s), table holding the keys it touches"}
+        except Exception as ex:
+            log(f"[bench] cpu baseline failed: {ex!r}")
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name, "batch": B, "fields": F, "emb_dim": k, "shards": S,
+                           "nnz_per_step": batches[0].nnz, "unique_keys_per_step": U, "table_keys": sum(t.size()),
+                           "ops": w.ops, "optimizer": "adagrad" if w.optimizer else "sgd",
+                           "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+                           "l2": "inputs larger than L2 (no flush)" if batches[0].nnz * 8 > 126e6 else
+                                 "small workload: inputs fit in L2, two batches alternate, no flush"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline,
+                "hbm": {"alg_bytes_per_step": int(step_bytes), "alg_gbs": round(step_bytes / ms_step / 1e6, 1),
+                        "frac_of_measured_copy": round(step_bytes / ms_step / 1e6 / hbm_peak, 4),
+                        "frac_of_nominal_8000": round(step_bytes / ms_step / 1e6 / 8000.0, 4)},
+                "kernels": kernels, "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    t.close()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

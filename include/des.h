@@ -247,6 +247,15 @@ des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t 
                            const des_grads_t* d_grads, float* d_pooled, float* d_Z,
                            float* h_out_small, void* stream);
 
+/* Per-launch timing for benchmarks.  While enabled, the library records a CUDA
+ * event on the call's stream behind every kernel it launches (and one at the
+ * entry of every call); des_profile_read synchronises and returns, in launch
+ * order, each kernel's name (static string) and the milliseconds between its
+ * event and the previous one, then clears the record.  At most 16384 events
+ * are kept between reads.  Off by default; costs one event record per launch. */
+des_status_t des_profile_enable(des_table_t* t, int on);
+des_status_t des_profile_read(des_table_t* t, const char** h_names, float* h_ms, int cap, int* h_n);
+
 /* Number of kernel launches the library has issued for this table so far. */
 uint64_t des_table_launch_count(des_table_t* t);
 

@@ -25,7 +25,7 @@ STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
            "des_aggregate", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
-           "des_step_host", "des_table_launch_count", "des_status_string"]
+           "des_step_host", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
 
 
 class DesError(RuntimeError):
@@ -101,6 +101,9 @@ def load():
                                     C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]
         L.des_table_launch_count.argtypes = [C.c_void_p]
+        L.des_profile_enable.argtypes = [C.c_void_p, C.c_int]
+        L.des_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int,
+                                       C.POINTER(C.c_int)]
         L.des_table_launch_count.restype = C.c_uint64
         L.des_status_string.restype = C.c_char_p
         _lib = L
@@ -291,3 +294,15 @@ class Table:
         n = int(global_rows.numel())
         self._check(self.L.des_table_write_rows(self.h, _ptr(global_rows), n, _ptr(emb), _ptr(lin), _ptr(acc_emb),
                                                 _ptr(acc_lin), _stream()), "des_table_write_rows")
+
+    def profile_enable(self, on: bool = True):
+        self._check(self.L.des_profile_enable(self.h, 1 if on else 0), "des_profile_enable")
+
+    def profile_read(self):
+        """-> list of (kernel name, ms) in launch order since the last read."""
+        cap = 16384
+        names = (C.c_char_p * cap)()
+        ms = (C.c_float * cap)()
+        n = C.c_int(0)
+        self._check(self.L.des_profile_read(self.h, names, ms, cap, C.byref(n)), "des_profile_read")
+        return [(names[i].decode(), float(ms[i])) for i in range(min(n.value, cap))]

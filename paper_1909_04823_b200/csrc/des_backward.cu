@@ -28,6 +28,7 @@
 
 #define HOT_MIN 512u      // estimated occurrences from which a key is treated as hot
 #define HOT_CHAIN 256u    // target number of additions per replica row
+#define HOT_RCHUNK 64u    // replica rows summed by one warp of the reduction
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
   x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
@@ -49,9 +50,13 @@ __global__ void __launch_bounds__(256) sample_count_kernel(const uint32_t* __res
 __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const uint32_t* __restrict__ n_uniq,
                                                          long long max_uniq, int shift, uint32_t* hot_base,
                                                          uint32_t* hot_R, uint32_t* hot_u, uint32_t* ctr,
-                                                         uint32_t h_max, uint32_t rep_max) {
+                                                         uint32_t h_max, uint32_t rep_max, DevMeta* meta,
+                                                         uint32_t* hot_work, uint32_t work_max) {
   long long U = *n_uniq;
-  if (U > max_uniq) U = max_uniq;
+  if (U > max_uniq) {           // the gradient buffer cannot hold this batch: report, update what fits
+    if (blockIdx.x == 0 && threadIdx.x == 0) des_raise(meta, DES_ERR_CAPACITY);
+    U = max_uniq;
+  }
   for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (long long)gridDim.x * blockDim.x) {
     const uint32_t est = hinfo[u] << shift;
     uint32_t h = DES_ROW_NONE;
@@ -60,8 +65,16 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
       const uint32_t hh = atomicAdd(&ctr[0], 1u);
       if (hh < h_max) {
         const uint32_t base = atomicAdd(&ctr[1], R);
-        if (base + R <= rep_max) { hot_base[hh] = base; hot_R[hh] = R; hot_u[hh] = (uint32_t)u; h = hh; }
-        else hot_R[hh] = 0;
+        const uint32_t nchunk = (R + HOT_RCHUNK - 1) / HOT_RCHUNK;
+        bool ok = base + R <= rep_max;
+        uint32_t wbase = 0;
+        if (ok) { wbase = atomicAdd(&ctr[2], nchunk); ok = wbase + nchunk <= work_max; }
+        if (ok) {
+          hot_base[hh] = base; hot_R[hh] = R; hot_u[hh] = (uint32_t)u; h = hh;
+          for (uint32_t i = 0; i < nchunk; ++i) hot_work[wbase + i] = (hh << 18) | i;
+        } else {
+          hot_R[hh] = 0;
+        }
       }
     }
     hinfo[u] = h;
@@ -85,36 +98,52 @@ __global__ void __launch_bounds__(256) make_dest_kernel(const uint32_t* __restri
   dest[j] = d;
 }
 
-// One block per hot key: sum its replica rows in double (fixed order inside a
-// thread, tree across threads), add into the key's gradient row, clear the replicas.
-__global__ void __launch_bounds__(256) hot_reduce_kernel(const uint32_t* __restrict__ ctr, uint32_t h_max,
+// Replica reduction, stage 1: one warp per work item = HOT_RCHUNK replica rows
+// of one hot key.  Columns are spread over the lanes, sums are taken in double
+// and added (double atomics, a few hundred per key at most) to the key's row of
+// hot_acc; the replica rows are cleared for the next step.
+__global__ void __launch_bounds__(256) hot_reduce_kernel(const uint32_t* __restrict__ ctr, uint32_t work_max,
+                                                         const uint32_t* __restrict__ hot_work,
                                                          const uint32_t* __restrict__ hot_base,
+                                                         const uint32_t* __restrict__ hot_R, long long max_uniq,
+                                                         int k, float* __restrict__ Gbuf, double* __restrict__ hot_acc) {
+  const int stride = k + 4, lane = threadIdx.x & 31;
+  uint32_t nw = ctr[2];
+  if (nw > work_max) nw = work_max;
+  const uint32_t wstep = gridDim.x * (blockDim.x >> 5);
+  for (uint32_t wi = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wi < nw; wi += wstep) {
+    const uint32_t item = hot_work[wi], h = item >> 18, chunk = item & 0x3FFFFu;
+    const uint32_t R = hot_R[h];
+    const uint32_t r_lo = chunk * HOT_RCHUNK, r_hi = min(R, r_lo + HOT_RCHUNK);
+    float* rep = Gbuf + ((size_t)max_uniq + hot_base[h]) * stride;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+    for (uint32_t r = r_lo; r < r_hi; ++r) {
+      float* row = rep + (size_t)r * stride;
+      if (lane < stride) { a0 += (double)row[lane]; row[lane] = 0.f; }
+      if (lane + 32 < stride) { a1 += (double)row[lane + 32]; row[lane + 32] = 0.f; }
+      if (lane + 64 < stride) { a2 += (double)row[lane + 64]; row[lane + 64] = 0.f; }
+    }
+    double* dst = hot_acc + (size_t)h * stride;
+    if (lane < stride) atomicAdd(dst + lane, a0);
+    if (lane + 32 < stride) atomicAdd(dst + lane + 32, a1);
+    if (lane + 64 < stride) atomicAdd(dst + lane + 64, a2);
+  }
+}
+
+// Stage 2: the double sums go into the hot keys' gradient rows; hot_acc is cleared.
+__global__ void __launch_bounds__(256) hot_finish_kernel(const uint32_t* __restrict__ ctr, uint32_t h_max,
                                                          const uint32_t* __restrict__ hot_R,
-                                                         const uint32_t* __restrict__ hot_u, long long max_uniq,
-                                                         int k, float* Gbuf) {
-  __shared__ double red[256];
+                                                         const uint32_t* __restrict__ hot_u, int k,
+                                                         float* __restrict__ Gbuf, double* __restrict__ hot_acc) {
   const int stride = k + 4;
   uint32_t nh = ctr[0];
   if (nh > h_max) nh = h_max;
-  for (uint32_t h = blockIdx.x; h < nh; h += gridDim.x) {
-    const uint32_t R = hot_R[h];
-    if (R == 0) continue;
-    float* rep = Gbuf + ((size_t)max_uniq + hot_base[h]) * stride;
-    float* dst = Gbuf + (size_t)hot_u[h] * stride;
-    // thread t handles column t % stride of rows t / stride, t / stride + rows_par, ...
-    const int rows_par = 256 / stride;                       // stride <= 68
-    const int c = threadIdx.x % stride, r0 = threadIdx.x / stride;
-    double a = 0.0;
-    if (r0 < rows_par)
-      for (uint32_t r = r0; r < R; r += rows_par) { a += (double)rep[(size_t)r * stride + c]; rep[(size_t)r * stride + c] = 0.f; }
-    red[threadIdx.x] = a;
-    __syncthreads();
-    if (threadIdx.x < stride) {
-      double t = 0.0;
-      for (int q = 0; q < rows_par; ++q) t += red[q * stride + threadIdx.x];
-      dst[threadIdx.x] += (float)t;
-    }
-    __syncthreads();
+  const long long n = (long long)nh * stride;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const uint32_t h = (uint32_t)(i / stride), c = (uint32_t)(i % stride);
+    if (hot_R[h] == 0) continue;
+    Gbuf[(size_t)hot_u[h] * stride + c] += (float)hot_acc[i];
+    hot_acc[i] = 0.0;
   }
 }
 
@@ -156,35 +185,24 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
   }
 }
 
+#define UP_UNROLL 4
+
+// One optimizer application per unique key.  A group of G lanes owns a key (one
+// 16-byte column each, lane 0 also the linear weight); it works on UP_UNROLL
+// keys at a time so that their gradient rows, row numbers, weights and state
+// are all in flight together: the kernel is a pure stream of 272-byte rows.
 template <int G>
 __global__ void __launch_bounds__(256) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
-    uint32_t ops, int optimizer, float lr, float eps, float* Gbuf, float* W, float* A, uint32_t* hinfo) {
+    uint32_t ops, int optimizer, float lr, float eps, float* __restrict__ Gbuf, float* __restrict__ W,
+    float* __restrict__ A, uint32_t* __restrict__ hinfo) {
   const int K4 = k >> 2, stride = k + 4;
   long long U = *n_uniq;
   if (U > max_uniq) U = max_uniq;
   const int c4 = (int)(threadIdx.x % G);
+  const bool col = c4 < K4, lead = c4 == 0;
+  const bool upd_v = ops & (DES_OP_FM | DES_OP_POOL | DES_OP_DENSE1), upd_w = ops & DES_OP_LR;
   const long long gstep = (long long)gridDim.x * (blockDim.x / G);
-  // every group of a warp runs the same number of iterations (u may pass U in the last one)
-  const long long iters = (U + gstep - 1) / gstep;
-  long long u = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
-  for (long long it = 0; it < iters; ++it, u += gstep) {
-  const bool live = u < U;
-  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), tail = g;
-  float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)(live ? u : 0) * stride);
-  const bool col = c4 < K4;
-  if (live) {
-    if (col) g = grow[c4];
-    tail = grow[K4];
-  }
-  __syncwarp();
-  if (!live) continue;
-  if (col) grow[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (c4 == 0) { grow[K4] = make_float4(0.f, 0.f, 0.f, 0.f); hinfo[u] = 0u; }
-  const uint32_t r = __ldg(uniq_rows + u);
-  if (r == DES_ROW_NONE) continue;
-  float4* w = reinterpret_cast<float4*>(W + (size_t)r * stride);
-  float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r * stride) : nullptr;
   auto step = [&](float& theta, float& acc, float Gd) {
     if (optimizer == DES_OPT_ADAGRAD) {
       acc = acc + Gd * Gd;
@@ -193,23 +211,60 @@ __global__ void __launch_bounds__(256) update_rows_kernel(
       theta = theta - lr * Gd;
     }
   };
-  if (col && (ops & (DES_OP_FM | DES_OP_POOL | DES_OP_DENSE1))) {
-    float4 v = w[c4];
-    float4 s = a ? a[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
-    step(v.x, s.x, g.x - v.x * tail.y);
-    step(v.y, s.y, g.y - v.y * tail.y);
-    step(v.z, s.z, g.z - v.z * tail.y);
-    step(v.w, s.w, g.w - v.w * tail.y);
-    w[c4] = v;
-    if (a) a[c4] = s;
-  }
-  if (c4 == 0 && (ops & DES_OP_LR)) {
-    float4 v = w[K4];
-    float4 s = a ? a[K4] : make_float4(0.f, 0.f, 0.f, 0.f);
-    step(v.x, s.x, tail.x);
-    w[K4] = v;
-    if (a) a[K4] = s;
-  }
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  // every lane of a warp runs the same number of iterations (keys past U are masked off)
+  const long long iters = (U + gstep * UP_UNROLL - 1) / (gstep * UP_UNROLL);
+  long long u0 = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
+  for (long long it = 0; it < iters; ++it, u0 += gstep * UP_UNROLL) {
+    uint32_t r[UP_UNROLL];
+    float4 g[UP_UNROLL], tail[UP_UNROLL], v[UP_UNROLL], s[UP_UNROLL], vt[UP_UNROLL], st[UP_UNROLL];
+#pragma unroll
+    for (int q = 0; q < UP_UNROLL; ++q) {
+      const long long u = u0 + q * gstep;
+      r[q] = (u < U) ? __ldg(uniq_rows + u) : DES_ROW_NONE;
+      g[q] = zero; tail[q] = zero;
+      if (u < U) {
+        const float4* grow = reinterpret_cast<const float4*>(Gbuf + (size_t)u * stride);
+        if (col) g[q] = grow[c4];
+        tail[q] = grow[K4];
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < UP_UNROLL; ++q) {
+      v[q] = zero; s[q] = zero; vt[q] = zero; st[q] = zero;
+      if (r[q] != DES_ROW_NONE) {
+        const float4* w = reinterpret_cast<const float4*>(W + (size_t)r[q] * stride);
+        const float4* a = A ? reinterpret_cast<const float4*>(A + (size_t)r[q] * stride) : nullptr;
+        if (col && upd_v) { v[q] = w[c4]; if (a) s[q] = a[c4]; }
+        if (lead && upd_w) { vt[q] = w[K4]; if (a) st[q] = a[K4]; }
+      }
+    }
+    __syncwarp();   // all lanes of a group have read the gradient row before its lead lane clears it
+#pragma unroll
+    for (int q = 0; q < UP_UNROLL; ++q) {
+      const long long u = u0 + q * gstep;
+      if (u >= U) continue;
+      float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)u * stride);
+      if (col) grow[c4] = zero;
+      if (lead) { grow[K4] = zero; hinfo[u] = 0u; }
+      if (r[q] == DES_ROW_NONE) continue;
+      float4* w = reinterpret_cast<float4*>(W + (size_t)r[q] * stride);
+      float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r[q] * stride) : nullptr;
+      if (col && upd_v) {
+        const float t1 = tail[q].y;
+        step(v[q].x, s[q].x, g[q].x - v[q].x * t1);
+        step(v[q].y, s[q].y, g[q].y - v[q].y * t1);
+        step(v[q].z, s[q].z, g[q].z - v[q].z * t1);
+        step(v[q].w, s[q].w, g[q].w - v[q].w * t1);
+        w[c4] = v[q];
+        if (a) a[c4] = s[q];
+      }
+      if (lead && upd_w) {
+        step(vt[q].x, st[q].x, tail[q].x);
+        w[K4] = vt[q];
+        if (a) a[K4] = st[q];
+      }
+    }
   }
 }
 
@@ -225,6 +280,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   if ((ops & DES_OP_POOL) && !(ops & DES_OP_DENSE1) && !gr->gE) return DES_ERR_INVALID_ARG;
   if ((ops & DES_OP_DENSE1) && (!t->H || !gr->gZ || !gr->gE_work || !out->pooled)) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
   const int B = b->batch;
   const float* gE = (ops & DES_OP_POOL) ? gr->gE : nullptr;
   if (ops & DES_OP_DENSE1) {
@@ -239,17 +295,18 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   // hot-key detection on a sample, replica assignment, per-occurrence destination row
   int shift = 0;
   while (shift < 6 && ((long long)nnz >> shift) > (1ll << 20)) ++shift;
-  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 8, cs));
+  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 16, cs));
   {
     const int n = (nnz >> shift) + 1;
     sample_count_kernel<<<(n + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "sample_count_kernel");
     hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
-                                                       t->hot_u, t->hot_ctr, t->hot_max, t->rep_max);
-    DES_LAUNCH_CHECK(t);
+                                                       t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
+                                                       t->hot_work, t->work_max);
+    DES_LAUNCH_CHECK(t, "hot_select_kernel");
     make_dest_kernel<<<(nnz + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
                                                         t->dest);
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "make_dest_kernel");
   }
   {
     const long long threads = nbags * G;
@@ -258,18 +315,21 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
                                                             out->out_small, gr->gL, gr->gF, gE, t->Gbuf)
     switch (G) { case 1: SC(1); break; case 2: SC(2); break; case 4: SC(4); break; case 8: SC(8); break; default: SC(16); }
 #undef SC
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "grad_scatter_kernel");
   }
-  hot_reduce_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hot_ctr, t->hot_max, t->hot_base, t->hot_R, t->hot_u,
-                                                     t->max_uniq, t->k, t->Gbuf);
-  DES_LAUNCH_CHECK(t);
+  hot_reduce_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->hot_ctr, t->work_max, t->hot_work, t->hot_base, t->hot_R,
+                                                     t->max_uniq, t->k, t->Gbuf, t->hot_acc);
+  DES_LAUNCH_CHECK(t, "hot_reduce_kernel");
+  hot_finish_kernel<<<t->sm_count * 2, 256, 0, cs>>>(t->hot_ctr, t->hot_max, t->hot_R, t->hot_u, t->k, t->Gbuf,
+                                                     t->hot_acc);
+  DES_LAUNCH_CHECK(t, "hot_finish_kernel");
   {
     const unsigned grid = (unsigned)(t->sm_count * 8);
 #define UP(GG) update_rows_kernel<GG><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops,       \
                                                            t->cfg.optimizer, t->cfg.lr, t->cfg.eps, t->Gbuf, t->W, t->A, t->hinfo)
     switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }
 #undef UP
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "update_rows_kernel");
   }
   return DES_OK;
 }

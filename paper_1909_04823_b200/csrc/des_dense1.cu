@@ -156,7 +156,7 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
   }
   dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.slices);
   gemm_kernel<GEMM_FWD><<<grid, 256, 0, st>>>(g);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "gemm_kernel");
   return DES_OK;
 }
 
@@ -169,7 +169,7 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
     g.k_emb = t->k; g.FK = FK; g.H = t->H; g.meta = t->meta; g.slices = 1;
     dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, 1);
     gemm_kernel<GEMM_DGRAD><<<grid, 256, 0, st>>>(g);
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "gemm_kernel");
   }
   {  // gW1 = pooled^T gZ, split over the batch
     GemmArgs g; memset(&g, 0, sizeof(g));
@@ -177,11 +177,11 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
     g.k_emb = t->k; g.FK = FK; g.H = t->H; g.meta = t->meta; g.slices = t->gw1_splits;
     dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.slices);
     gemm_kernel<GEMM_WGRAD><<<grid, 256, 0, st>>>(g);
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "gemm_kernel");
     const size_t n = (size_t)FK * t->H;
     w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, g.slices, n, t->W1, t->accW1, t->W1b,
                                                       t->cfg.optimizer, t->cfg.lr, t->cfg.eps);
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "w1_update_kernel");
   }
   return DES_OK;
 }

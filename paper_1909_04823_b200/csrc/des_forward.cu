@@ -7,20 +7,22 @@
 // des_aggregate: (+) over shards in the order s = 0..S-1 (Eq. 1) and the
 // substitution operator F = 1/2 <(+)M_1,(+)M_1> - 1/2 (+)M_2 (Eq. 8).
 //
-// Kernel shape.  One warp walks one sample.  A row (k floats + the linear
-// weight) is read by a group of G = k/4 lanes (rounded up to a power of two)
-// with one 16-byte load per lane; the 32/G groups of the warp take different
-// bags of the sample, so a bag's pooled sum lives in one group's registers and
-// is stored once.  The per-(shard, sample) partials live in shared memory,
-// S x (k+4) floats per warp; two groups that hit the same shard in the same
-// step are serialised in group order (found with a warp match), so every sum
-// is taken in CSR order and the result is deterministic.
+// Kernel shape.  One warp walks one sample, bag by bag.  A row (k floats + the
+// linear weight) is read by a group of G = k/4 lanes (rounded up to a power of
+// two) with one 16-byte load per lane; the NG = 32/G groups of the warp split
+// the occurrences of a bag BY SHARD: group g takes the occurrences whose shard
+// is congruent to g modulo NG.  The per-(shard, sample) partials live in shared
+// memory, S x (k+4) floats per warp, and because a shard's accumulator row is
+// only ever touched by its owning group, in occurrence order, there are no
+// conflicts to resolve and the result is deterministic.  A bag's pooled sum is
+// the sum of the groups' partial sums (a few shuffles per bag).  Each group
+// keeps FW_UNROLL row loads in flight.
 #include "des_internal.cuh"
 
 #define FW_UNROLL 4
 
 template <int G>
-__global__ void __launch_bounds__(256) forward_partials_kernel(
+__global__ void __launch_bounds__(384) forward_partials_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
     const uint8_t* __restrict__ shards, int B, int F, int S, int k, uint32_t ops, const float* __restrict__ W,
     const DevMeta* __restrict__ meta, float* __restrict__ part_small, float* __restrict__ pooled,
@@ -37,54 +39,57 @@ __global__ void __launch_bounds__(256) forward_partials_kernel(
   if (want_small)
     for (int i = lane; i < acc_f4; i += 32) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   __syncwarp();
-  const unsigned group_lt = (g == 0) ? 0u : (0xFFFFFFFFu >> (32 - g * G));
 
   for (int b = blockIdx.x * wpb + warp; b < B; b += gridDim.x * wpb) {
-    for (int fbase = 0; fbase < F; fbase += NG) {
-      const int f = fbase + g;
-      int lo = 0, hi = 0;
-      if (f < F) { lo = __ldg(offsets + (size_t)b * F + f); hi = __ldg(offsets + (size_t)b * F + f + 1); }
-      const int maxlen = __reduce_max_sync(0xFFFFFFFFu, hi - lo);
+    for (int f = 0; f < F; ++f) {
+      const int lo = __ldg(offsets + (size_t)b * F + f), hi = __ldg(offsets + (size_t)b * F + f + 1);
       float4 pacc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int i = 0; i < maxlen; i += FW_UNROLL) {
-        float4 v[FW_UNROLL]; float lin[FW_UNROLL], x[FW_UNROLL]; int sh[FW_UNROLL];
+      for (int base = lo; base < hi; base += 32) {
+        // every lane fetches one occurrence of the chunk; groups then pick their shards' entries
+        const int j = base + lane;
+        uint32_t my_row = DES_ROW_NONE; int my_s = 0; float my_x = 1.f;
+        if (j < hi) {
+          my_row = __ldg(rows + j); my_s = __ldg(shards + j);
+          if (vals) my_x = __ldg(vals + j);
+        }
+        const int key = (my_row == DES_ROW_NONE) ? -1 : ((want_small ? my_s : lane) & (NG - 1));
+        unsigned m = 0;
 #pragma unroll
-        for (int u = 0; u < FW_UNROLL; ++u) {
-          const int j = lo + i + u;
-          v[u] = make_float4(0.f, 0.f, 0.f, 0.f); lin[u] = 0.f; x[u] = 0.f; sh[u] = -1;
-          if (j < hi) {
-            const uint32_t r = __ldg(rows + j);
-            if (r != DES_ROW_NONE) {
-              const int s = __ldg(shards + j);
-              sh[u] = s;
-              x[u] = vals ? __ldg(vals + j) : 1.f;
+        for (int q = 0; q < NG; ++q) {
+          const unsigned mq = __ballot_sync(0xFFFFFFFFu, key == q);
+          if (q == g) m = mq;
+        }
+        while (__any_sync(0xFFFFFFFFu, m != 0)) {
+          float4 v[FW_UNROLL]; float lin[FW_UNROLL], x[FW_UNROLL]; int sh[FW_UNROLL];
+#pragma unroll
+          for (int u = 0; u < FW_UNROLL; ++u) {
+            const int src = m ? (__ffs(m) - 1) : -1;
+            m &= m - 1;                                     // 0 stays 0
+            const uint32_t r = __shfl_sync(0xFFFFFFFFu, my_row, src < 0 ? 0 : src);
+            const int s = __shfl_sync(0xFFFFFFFFu, my_s, src < 0 ? 0 : src);
+            x[u] = __shfl_sync(0xFFFFFFFFu, my_x, src < 0 ? 0 : src);
+            sh[u] = src < 0 ? -1 : s;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f); lin[u] = 0.f;
+            if (src >= 0) {
               const float* wr = W + (meta->row_base[s] + r) * (size_t)stride;
               if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
               if (c4 == 0) lin[u] = __ldg(wr + k);
             }
           }
-        }
 #pragma unroll
-        for (int u = 0; u < FW_UNROLL; ++u) {
-          if (i + u >= maxlen) break;                       // warp-uniform
-          const float xx = x[u];
-          const float4 vx = make_float4(v[u].x * xx, v[u].y * xx, v[u].z * xx, v[u].w * xx);
-          pacc.x += vx.x; pacc.y += vx.y; pacc.z += vx.z; pacc.w += vx.w;
-          if (part_pooled && sh[u] >= 0 && col) {
-            float* pp = part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) + (size_t)f * k + c4 * 4;
-            pp[0] += vx.x; pp[1] += vx.y; pp[2] += vx.z; pp[3] += vx.w;   // this group owns the bag
-          }
-          if (want_small) {
-            float sq = vx.x * vx.x + vx.y * vx.y + vx.z * vx.z + vx.w * vx.w;
+          for (int u = 0; u < FW_UNROLL; ++u) {
+            const float xx = x[u];
+            const float4 vx = make_float4(v[u].x * xx, v[u].y * xx, v[u].z * xx, v[u].w * xx);
+            pacc.x += vx.x; pacc.y += vx.y; pacc.z += vx.z; pacc.w += vx.w;
+            if (part_pooled && sh[u] >= 0 && col)
+              atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) +
+                                                  (size_t)f * k) + c4, vx);
+            if (want_small) {
+              float sq = vx.x * vx.x + vx.y * vx.y + vx.z * vx.z + vx.w * vx.w;
 #pragma unroll
-            for (int d = 1; d < G; d <<= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, d);
-            // groups that hit the same shard in this step add one after the other
-            const unsigned peers = __match_any_sync(0xFFFFFFFFu, sh[u] >= 0 ? sh[u] : 0x100 + g);
-            const int rank = __popc(peers & group_lt) / G;
-            const int rmax = __reduce_max_sync(0xFFFFFFFFu, rank);
-            for (int r = 0; r <= rmax; ++r) {
-              if (r == rank && sh[u] >= 0) {
-                float* a = acc + sh[u] * stride;
+              for (int d = 1; d < G; d <<= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, d);
+              if (sh[u] >= 0) {
+                float* a = acc + sh[u] * stride;             // row owned by this group
                 if (col) {
                   float4 t = reinterpret_cast<float4*>(a)[c4];
                   t.x += vx.x; t.y += vx.y; t.z += vx.z; t.w += vx.w;
@@ -92,13 +97,18 @@ __global__ void __launch_bounds__(256) forward_partials_kernel(
                 }
                 if (c4 == 0) { a[k] += lin[u] * xx; a[k + 1] += sq; }
               }
-              __syncwarp();
             }
           }
         }
       }
-      if (pooled && f < F && col)
-        reinterpret_cast<float4*>(pooled + ((size_t)b * F + f) * k)[c4] = pacc;
+      if (pooled) {
+#pragma unroll
+        for (int d = G; d < 32; d <<= 1) {
+          pacc.x += __shfl_xor_sync(0xFFFFFFFFu, pacc.x, d); pacc.y += __shfl_xor_sync(0xFFFFFFFFu, pacc.y, d);
+          pacc.z += __shfl_xor_sync(0xFFFFFFFFu, pacc.z, d); pacc.w += __shfl_xor_sync(0xFFFFFFFFu, pacc.w, d);
+        }
+        if (g == 0 && col) reinterpret_cast<float4*>(pooled + ((size_t)b * F + f) * k)[c4] = pacc;
+      }
     }
     if (want_small) {
       __syncwarp();
@@ -167,14 +177,15 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   if (pool && !part->pooled) return DES_ERR_INVALID_ARG;
   if ((ops & DES_OP_DENSE1) && !t->H) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
   const int B = b->batch;
   float* ps = small ? part->part_small : nullptr;
   float* pl = pool ? part->pooled : nullptr;
   float* pp = pool ? part->part_pooled : nullptr;
   if (pp) DES_CUDA(cudaMemsetAsync(pp, 0, (size_t)t->S * B * t->F * t->k * 4, cs));
   const size_t per_warp = small ? (size_t)t->S * t->stride * 4 : 0;
-  int wpb = 8;
-  while (wpb > 1 && per_warp * wpb > 200 * 1024) wpb >>= 1;
+  int wpb = 12;
+  while (wpb > 1 && per_warp * wpb > 208 * 1024) --wpb;
   const size_t smem = per_warp * wpb;
   int grid = (B + wpb - 1) / wpb;
   const int G = group_for(t->k);
@@ -194,7 +205,7 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
     default: FWD(16); break;
   }
 #undef FWD
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "forward_partials_kernel");
   return DES_OK;
 }
 
@@ -203,6 +214,7 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
   if (!t || !b || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
   if (b->batch <= 0 || b->batch > t->max_batch) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
   const int B = b->batch;
   if (ops & (DES_OP_LR | DES_OP_FM)) {
     if (!part->part_small || !out->out_small) return DES_ERR_INVALID_ARG;
@@ -216,7 +228,7 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
       case 8: aggregate_small_kernel<8><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
       default: aggregate_small_kernel<16><<<grid, 256, 0, cs>>>(part->part_small, B, t->S, t->k, ops, out->out_small); break;
     }
-    DES_LAUNCH_CHECK(t);
+    DES_LAUNCH_CHECK(t, "aggregate_small_kernel");
   }
   if (ops & (DES_OP_POOL | DES_OP_DENSE1)) {
     if (!part->pooled || !out->pooled) return DES_ERR_INVALID_ARG;
@@ -224,7 +236,7 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
     if (part->part_pooled) {
       // materialised per-shard pooled partials: aggregate them in shard order
       reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part->part_pooled, n, t->S, out->pooled);
-      DES_LAUNCH_CHECK(t);
+      DES_LAUNCH_CHECK(t, "reduce_shards_kernel");
     } else if (out->pooled != part->pooled) {
       DES_CUDA(cudaMemcpyAsync(out->pooled, part->pooled, n * 4, cudaMemcpyDeviceToDevice, cs));
     }
@@ -235,7 +247,7 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
     if (st != DES_OK) return st;
     if (part->part_dense) {
       reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part->part_dense, (size_t)B * t->H, t->S, out->Z);
-      DES_LAUNCH_CHECK(t);
+      DES_LAUNCH_CHECK(t, "reduce_shards_kernel");
     }
   }
   return DES_OK;

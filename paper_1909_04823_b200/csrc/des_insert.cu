@@ -185,7 +185,6 @@ __global__ void __launch_bounds__(IB) assign_kernel(
   uslot[u] = so;
   const unsigned long long g = meta->row_base[s] + local;
   uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
-  if ((long long)u >= max_uniq) des_raise(meta, DES_ERR_CAPACITY);   // gradient buffer too small for this batch
   if ((fl & 2) && local != DES_ROW_NONE) {
     const unsigned long long id = ids[j];
     float4* w = reinterpret_cast<float4*>(W + g * stride);
@@ -230,6 +229,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   des_status_t st = des_check_batch(t, b, insert);
   if (st != DES_OK) return st;
   cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
   const int nnz = (int)b->nnz;
   const int nbags = b->batch * (int)t->F;
   if (nnz == 0) {
@@ -239,19 +239,19 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   const int nblk = (nnz + IB - 1) / IB;
   probe_claim_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
                                           t->cfg.partition, insert, t->slots, t->meta, t->slot_of, b->shards, b->rows);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "probe_claim_kernel");
   if (!insert) return DES_OK;
   flag_count_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "flag_count_kernel");
   scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "scan_blocks_kernel");
   assign_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, nnz, t->S, t->k, t->stride, t->slots, t->meta,
                                      t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max, t->uslot, b->uniq_rows,
                                      t->max_uniq, t->W, t->A, t->cfg.seed, t->cfg.init_scale, t->cfg.init_acc);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "assign_kernel");
   resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "resolve_kernel");
   finish_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->uslot, t->meta, b->n_uniq);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "finish_kernel");
   return DES_OK;
 }

@@ -58,7 +58,9 @@ struct des_table {
   uint32_t* hinfo;                   // [max_uniq] sampled count, then hot index; zero between calls
   uint32_t* dest;                    // [max_nnz] gradient row of each occurrence
   uint32_t *hot_base, *hot_R, *hot_u, *hot_ctr;   // hot list [hot_max] and its two counters
-  uint32_t hot_max, rep_max;
+  uint32_t* hot_work;                // [work_max] (hot index << 18 | chunk) items of the replica reduction
+  double* hot_acc;                   // [hot_max][stride] double sums of the replicas; zero between calls
+  uint32_t hot_max, rep_max, work_max;
   // first dense layer
   float* W1; float* accW1;           // [F*k][H] fp32 master and state
   __nv_bfloat16* W1b;                // bf16 shadow
@@ -69,10 +71,19 @@ struct des_table {
   float* st_part_small; float* st_out_small;
   uint64_t launches;
   int sm_count;
+  // optional per-launch timing (des_profile_*): one event after every launch, and one at API entry
+  int prof_on, prof_n;
+  cudaStream_t cur_stream;
+  cudaEvent_t* prof_ev;              // [DES_PROF_MAX]
+  const char** prof_name;            // [DES_PROF_MAX], NULL = API-entry marker
 };
+#define DES_PROF_MAX 16384
 
 #define DES_CUDA(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return DES_ERR_CUDA; } while (0)
-#define DES_LAUNCH_CHECK(t) do { (t)->launches++; if (cudaGetLastError() != cudaSuccess) return DES_ERR_CUDA; } while (0)
+// after every kernel launch: count it, check the launch, and (when profiling) drop an event behind it
+int des_prof_mark(des_table* t, const char* name, int check);
+void des_api_begin(des_table* t, cudaStream_t cs);
+#define DES_LAUNCH_CHECK(t, name) do { if (des_prof_mark((t), (name), 1)) return DES_ERR_CUDA; } while (0)
 
 // ---- device helpers ---------------------------------------------------------
 

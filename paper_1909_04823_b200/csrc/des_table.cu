@@ -23,6 +23,51 @@ __global__ void fill_f32_kernel(float* p, size_t n, float v) {
   for (; i < n; i += st) p[i] = v;
 }
 
+int des_prof_mark(des_table* t, const char* name, int check) {
+  if (name) t->launches++;
+  if (check && cudaGetLastError() != cudaSuccess) return 1;
+  if (t->prof_on && t->prof_n < DES_PROF_MAX) {
+    t->prof_name[t->prof_n] = name;
+    cudaEventRecord(t->prof_ev[t->prof_n], t->cur_stream);
+    t->prof_n++;
+  }
+  return 0;
+}
+
+void des_api_begin(des_table* t, cudaStream_t cs) {
+  t->cur_stream = cs;
+  if (t->prof_on) des_prof_mark(t, nullptr, 0);
+}
+
+extern "C" des_status_t des_profile_enable(des_table_t* t, int on) {
+  if (!t) return DES_ERR_INVALID_ARG;
+  if (on && !t->prof_ev) {
+    t->prof_ev = new (std::nothrow) cudaEvent_t[DES_PROF_MAX];
+    t->prof_name = new (std::nothrow) const char*[DES_PROF_MAX];
+    if (!t->prof_ev || !t->prof_name) return DES_ERR_CUDA;
+    for (int i = 0; i < DES_PROF_MAX; ++i) DES_CUDA(cudaEventCreate(&t->prof_ev[i]));
+  }
+  t->prof_on = on ? 1 : 0;
+  t->prof_n = 0;
+  return DES_OK;
+}
+
+extern "C" des_status_t des_profile_read(des_table_t* t, const char** h_names, float* h_ms, int cap, int* h_n) {
+  if (!t || !h_n || !t->prof_ev) return DES_ERR_INVALID_ARG;
+  DES_CUDA(cudaDeviceSynchronize());
+  int n = 0;
+  for (int i = 1; i < t->prof_n; ++i) {
+    if (!t->prof_name[i]) continue;
+    float ms = 0.f;
+    DES_CUDA(cudaEventElapsedTime(&ms, t->prof_ev[i - 1], t->prof_ev[i]));
+    if (n < cap) { if (h_names) h_names[n] = t->prof_name[i]; if (h_ms) h_ms[n] = ms; }
+    ++n;
+  }
+  *h_n = n;
+  t->prof_n = 0;
+  return DES_OK;
+}
+
 extern "C" const char* des_status_string(des_status_t s) {
   switch (s) {
     case DES_OK: return "ok";
@@ -41,10 +86,12 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->Gbuf, t->hinfo, t->dest, t->hot_base,
-                  t->hot_R, t->hot_u, t->hot_ctr,
+                  t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc,
                   t->W1, t->accW1, t->W1b, t->gW1_part, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
   for (void* p : ptrs) dfree(t->cfg, p);
+  if (t->prof_ev) { for (int i = 0; i < DES_PROF_MAX; ++i) cudaEventDestroy(t->prof_ev[i]); delete[] t->prof_ev; }
+  delete[] t->prof_name;
   delete t;
   return DES_OK;
 }
@@ -110,7 +157,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->flags, (size_t)t->max_nnz);
   A(t->uslot, (size_t)t->max_nnz * 4);
   A(t->blk_cnt, (size_t)(t->S + 1) * t->nblk_max * 4);
-  t->hot_max = 65536;
+  t->hot_max = 16384;
   t->rep_max = (uint32_t)(t->max_nnz / 256 + t->hot_max + 1024);
   A(t->Gbuf, ((size_t)t->max_uniq + t->rep_max) * rowbytes);
   A(t->hinfo, (size_t)t->max_uniq * 4);
@@ -119,6 +166,9 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->hot_R, (size_t)t->hot_max * 4);
   A(t->hot_u, (size_t)t->hot_max * 4);
   A(t->hot_ctr, 256);
+  t->work_max = t->rep_max / 64 + t->hot_max;
+  A(t->hot_work, (size_t)t->work_max * 4);
+  A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);
   if (t->H) {
     A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
     t->gw1_splits = 32;
@@ -129,6 +179,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   cu &= cudaMemset(t->slots, 0xFF, slots * sizeof(Slot)) == cudaSuccess;
   cu &= cudaMemset(t->Gbuf, 0, ((size_t)t->max_uniq + t->rep_max) * rowbytes) == cudaSuccess;
   cu &= cudaMemset(t->hinfo, 0, (size_t)t->max_uniq * 4) == cudaSuccess;
+  cu &= cudaMemset(t->hot_acc, 0, (size_t)t->hot_max * t->stride * 8) == cudaSuccess;
   cu &= cudaMemcpy(t->meta, &hm, sizeof(hm), cudaMemcpyHostToDevice) == cudaSuccess;
   if (t->H) {
     cu &= cudaMemset(t->W1, 0, FKH * 4) == cudaSuccess;
@@ -200,10 +251,11 @@ extern "C" des_status_t des_table_export(des_table_t* t, uint64_t* d_keys, uint8
   unsigned long long* ctr = nullptr;
   DES_CUDA(cudaMalloc(&ctr, 8));
   cudaMemset(ctr, 0, 8);
+  des_api_begin(t, 0);
   export_kernel<<<t->sm_count * 8, 256>>>(t->slots, t->total_slots, t->meta, t->S, t->k, t->stride, t->W, t->A,
                                           (unsigned long long*)d_keys, d_shards, d_rows, d_emb, d_lin, d_acc_emb,
                                           d_acc_lin, cap, ctr);
-  t->launches++;
+  des_prof_mark(t, "export_kernel", 0);
   cudaError_t e = cudaDeviceSynchronize();
   unsigned long long n = 0;
   if (e == cudaSuccess) e = cudaMemcpy(&n, ctr, 8, cudaMemcpyDeviceToHost);
@@ -232,9 +284,10 @@ extern "C" des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_gl
                                             float* d_lin, float* d_acc_emb, float* d_acc_lin, void* stream) {
   if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
   if (n == 0) return DES_OK;
+  des_api_begin(t, (cudaStream_t)stream);
   read_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "read_rows_kernel");
   return DES_OK;
 }
 
@@ -259,9 +312,10 @@ extern "C" des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_g
                                              const float* d_acc_lin, void* stream) {
   if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
   if (n == 0) return DES_OK;
+  des_api_begin(t, (cudaStream_t)stream);
   write_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "write_rows_kernel");
   return DES_OK;
 }
 
@@ -274,9 +328,10 @@ __global__ void w1_shadow_kernel(const float* __restrict__ W1, __nv_bfloat16* __
 extern "C" des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream) {
   if (!t || !d_W1 || !t->H) return DES_ERR_INVALID_ARG;
   size_t n = (size_t)t->F * t->k * t->H;
+  des_api_begin(t, (cudaStream_t)stream);
   DES_CUDA(cudaMemcpyAsync(t->W1, d_W1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   w1_shadow_kernel<<<256, 256, 0, (cudaStream_t)stream>>>(t->W1, t->W1b, n);
-  DES_LAUNCH_CHECK(t);
+  DES_LAUNCH_CHECK(t, "w1_shadow_kernel");
   return DES_OK;
 }
 
