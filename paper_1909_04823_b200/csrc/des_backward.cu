@@ -235,34 +235,40 @@ __global__ void __launch_bounds__(256) update_rows_kernel(
       if (r[q] != DES_ROW_NONE) {
         const float4* w = reinterpret_cast<const float4*>(W + (size_t)r[q] * stride);
         const float4* a = A ? reinterpret_cast<const float4*>(A + (size_t)r[q] * stride) : nullptr;
-        if (col && upd_v) { v[q] = w[c4]; if (a) s[q] = a[c4]; }
-        if (lead && upd_w) { vt[q] = w[K4]; if (a) st[q] = a[K4]; }
+        if (col) { v[q] = w[c4]; if (a && upd_v) s[q] = a[c4]; }
+        if (lead) { vt[q] = w[K4]; if (a && upd_w) st[q] = a[K4]; }
       }
     }
     __syncwarp();   // all lanes of a group have read the gradient row before its lead lane clears it
 #pragma unroll
     for (int q = 0; q < UP_UNROLL; ++q) {
       const long long u = u0 + q * gstep;
-      if (u >= U) continue;
-      float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)u * stride);
-      if (col) grow[c4] = zero;
-      if (lead) { grow[K4] = zero; hinfo[u] = 0u; }
-      if (r[q] == DES_ROW_NONE) continue;
-      float4* w = reinterpret_cast<float4*>(W + (size_t)r[q] * stride);
-      float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r[q] * stride) : nullptr;
-      if (col && upd_v) {
+      const bool live = u < U, mapped = r[q] != DES_ROW_NONE;
+      if (live) {
+        float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)u * stride);
+        if (col) grow[c4] = zero;
+        if (lead) { grow[K4] = zero; hinfo[u] = 0u; }
+      }
+      if (mapped && col && upd_v) {
         const float t1 = tail[q].y;
         step(v[q].x, s[q].x, g[q].x - v[q].x * t1);
         step(v[q].y, s[q].y, g[q].y - v[q].y * t1);
         step(v[q].z, s[q].z, g[q].z - v[q].z * t1);
         step(v[q].w, s[q].w, g[q].w - v[q].w * t1);
-        w[c4] = v[q];
-        if (a) a[c4] = s[q];
       }
-      if (lead && upd_w) {
-        step(vt[q].x, st[q].x, tail[q].x);
+      // squared norm of the (new) latent vector, kept in the row's tail for the forward's M_2
+      float n2 = v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
+#pragma unroll
+      for (int d = 1; d < G; d <<= 1) n2 += __shfl_xor_sync(0xFFFFFFFFu, n2, d);
+      if (!mapped) continue;
+      float4* w = reinterpret_cast<float4*>(W + (size_t)r[q] * stride);
+      float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r[q] * stride) : nullptr;
+      if (col && upd_v) { w[c4] = v[q]; if (a) a[c4] = s[q]; }
+      if (lead) {
+        if (upd_w) step(vt[q].x, st[q].x, tail[q].x);
+        vt[q].y = n2;
         w[K4] = vt[q];
-        if (a) a[K4] = st[q];
+        if (a && upd_w) a[K4] = st[q];
       }
     }
   }

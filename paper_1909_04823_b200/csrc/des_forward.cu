@@ -16,29 +16,33 @@
 // only ever touched by its owning group, in occurrence order, there are no
 // conflicts to resolve and the result is deterministic.  A bag's pooled sum is
 // the sum of the groups' partial sums (a few shuffles per bag).  Each group
-// keeps FW_UNROLL row loads in flight.
+// keeps FW_UNROLL row loads in flight.  M_2 needs |v|^2 of every row: the table
+// keeps it next to the linear weight in the row's 16-byte tail (refreshed by the
+// update kernel), so the forward adds x^2 |v|^2 without a cross-lane reduction.
 #include "des_internal.cuh"
 
 #define FW_UNROLL 4
 
-template <int G>
+template <int G, bool HAS_VALS, bool MATERIALISE>
 __global__ void __launch_bounds__(384) forward_partials_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
     const uint8_t* __restrict__ shards, int B, int F, int S, int k, uint32_t ops, const float* __restrict__ W,
     const DevMeta* __restrict__ meta, float* __restrict__ part_small, float* __restrict__ pooled,
     float* __restrict__ part_pooled) {
   extern __shared__ __align__(16) float smem[];
+  __shared__ uint32_t row_base[DES_MAX_SHARDS];
   constexpr int NG = 32 / G;
   const int K4 = k >> 2, stride = k + 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
   const int g = lane / G, c4 = lane % G;
-  const bool col = c4 < K4;
+  const bool col = c4 < K4, lead = c4 == 0;
   const bool want_small = part_small != nullptr;
   float* acc = smem + (size_t)warp * S * stride;
   const int acc_f4 = S * (K4 + 1);
+  if (threadIdx.x < S) row_base[threadIdx.x] = (uint32_t)meta->row_base[threadIdx.x];
   if (want_small)
     for (int i = lane; i < acc_f4; i += 32) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-  __syncwarp();
+  __syncthreads();
 
   for (int b = blockIdx.x * wpb + warp; b < B; b += gridDim.x * wpb) {
     for (int f = 0; f < F; ++f) {
@@ -47,12 +51,14 @@ __global__ void __launch_bounds__(384) forward_partials_kernel(
       for (int base = lo; base < hi; base += 32) {
         // every lane fetches one occurrence of the chunk; groups then pick their shards' entries
         const int j = base + lane;
-        uint32_t my_row = DES_ROW_NONE; int my_s = 0; float my_x = 1.f;
+        uint32_t my_grow = DES_ROW_NONE; int my_s = 0; float my_x = 1.f;
         if (j < hi) {
-          my_row = __ldg(rows + j); my_s = __ldg(shards + j);
-          if (vals) my_x = __ldg(vals + j);
+          const uint32_t r = __ldg(rows + j);
+          my_s = __ldg(shards + j);
+          if (r != DES_ROW_NONE) my_grow = row_base[my_s] + r;      // table-global row
+          if (HAS_VALS) my_x = __ldg(vals + j);
         }
-        const int key = (my_row == DES_ROW_NONE) ? -1 : ((want_small ? my_s : lane) & (NG - 1));
+        const int key = (my_grow == DES_ROW_NONE) ? -1 : ((want_small ? my_s : lane) & (NG - 1));
         unsigned m = 0;
 #pragma unroll
         for (int q = 0; q < NG; ++q) {
@@ -60,42 +66,44 @@ __global__ void __launch_bounds__(384) forward_partials_kernel(
           if (q == g) m = mq;
         }
         while (__any_sync(0xFFFFFFFFu, m != 0)) {
-          float4 v[FW_UNROLL]; float lin[FW_UNROLL], x[FW_UNROLL]; int sh[FW_UNROLL];
+          float4 v[FW_UNROLL], tl[FW_UNROLL]; float x[FW_UNROLL]; int sh[FW_UNROLL];
 #pragma unroll
           for (int u = 0; u < FW_UNROLL; ++u) {
-            const int src = m ? (__ffs(m) - 1) : -1;
+            const bool have = m != 0;
+            const int src = have ? (__ffs(m) - 1) : 0;
             m &= m - 1;                                     // 0 stays 0
-            const uint32_t r = __shfl_sync(0xFFFFFFFFu, my_row, src < 0 ? 0 : src);
-            const int s = __shfl_sync(0xFFFFFFFFu, my_s, src < 0 ? 0 : src);
-            x[u] = __shfl_sync(0xFFFFFFFFu, my_x, src < 0 ? 0 : src);
-            sh[u] = src < 0 ? -1 : s;
-            v[u] = make_float4(0.f, 0.f, 0.f, 0.f); lin[u] = 0.f;
-            if (src >= 0) {
-              const float* wr = W + (meta->row_base[s] + r) * (size_t)stride;
-              if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
-              if (c4 == 0) lin[u] = __ldg(wr + k);
+            const uint32_t gr = __shfl_sync(0xFFFFFFFFu, my_grow, src);
+            const int s = __shfl_sync(0xFFFFFFFFu, my_s, src);
+            x[u] = HAS_VALS ? __shfl_sync(0xFFFFFFFFu, my_x, src) : 1.f;
+            sh[u] = have ? s : -1;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f); tl[u] = v[u];
+            if (have) {
+              const float4* wr = reinterpret_cast<const float4*>(W + (size_t)gr * stride);
+              if (col) v[u] = __ldg(wr + c4);
+              if (lead && want_small) tl[u] = __ldg(wr + K4);      // (linear weight, |v|^2, 0, 0)
             }
           }
 #pragma unroll
           for (int u = 0; u < FW_UNROLL; ++u) {
-            const float xx = x[u];
-            const float4 vx = make_float4(v[u].x * xx, v[u].y * xx, v[u].z * xx, v[u].w * xx);
+            float4 vx = v[u];
+            if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
             pacc.x += vx.x; pacc.y += vx.y; pacc.z += vx.z; pacc.w += vx.w;
-            if (part_pooled && sh[u] >= 0 && col)
-              atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) +
-                                                  (size_t)f * k) + c4, vx);
-            if (want_small) {
-              float sq = vx.x * vx.x + vx.y * vx.y + vx.z * vx.z + vx.w * vx.w;
-#pragma unroll
-              for (int d = 1; d < G; d <<= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, d);
-              if (sh[u] >= 0) {
+            if (sh[u] >= 0) {
+              if (MATERIALISE && col)
+                atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) +
+                                                    (size_t)f * k) + c4, vx);
+              if (want_small) {
                 float* a = acc + sh[u] * stride;             // row owned by this group
                 if (col) {
                   float4 t = reinterpret_cast<float4*>(a)[c4];
                   t.x += vx.x; t.y += vx.y; t.z += vx.z; t.w += vx.w;
                   reinterpret_cast<float4*>(a)[c4] = t;
                 }
-                if (c4 == 0) { a[k] += lin[u] * xx; a[k + 1] += sq; }
+                if (lead) {
+                  float2 t = *reinterpret_cast<float2*>(a + k);
+                  t.x += tl[u].x * x[u]; t.y += tl[u].y * x[u] * x[u];
+                  *reinterpret_cast<float2*>(a + k) = t;
+                }
               }
             }
           }
@@ -189,13 +197,18 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   const size_t smem = per_warp * wpb;
   int grid = (B + wpb - 1) / wpb;
   const int G = group_for(t->k);
-#define FWD(GG)                                                                                                   \
+#define FWD3(GG, HV, MT)                                                                                          \
   do {                                                                                                            \
     if (smem > 48 * 1024)                                                                                         \
-      DES_CUDA(cudaFuncSetAttribute(forward_partials_kernel<GG>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
-                                    (int)smem));                                                                  \
-    forward_partials_kernel<GG><<<grid, wpb * 32, smem, cs>>>(b->offsets, b->vals, b->rows, b->shards, B, t->F,   \
-                                                              t->S, t->k, ops, t->W, t->meta, ps, pl, pp);        \
+      DES_CUDA(cudaFuncSetAttribute(forward_partials_kernel<GG, HV, MT>,                                          \
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));                     \
+    forward_partials_kernel<GG, HV, MT><<<grid, wpb * 32, smem, cs>>>(                                            \
+        b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->k, ops, t->W, t->meta, ps, pl, pp);            \
+  } while (0)
+#define FWD(GG)                                                                                                   \
+  do {                                                                                                            \
+    if (pp) { if (b->vals) FWD3(GG, true, true); else FWD3(GG, false, true); }                                    \
+    else { if (b->vals) FWD3(GG, true, false); else FWD3(GG, false, false); }                                     \
   } while (0)
   switch (G) {
     case 1: FWD(1); break;
@@ -204,6 +217,7 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
     case 8: FWD(8); break;
     default: FWD(16); break;
   }
+#undef FWD3
 #undef FWD
   DES_LAUNCH_CHECK(t, "forward_partials_kernel");
   return DES_OK;

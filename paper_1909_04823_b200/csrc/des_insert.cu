@@ -189,8 +189,13 @@ __global__ void __launch_bounds__(IB) assign_kernel(
     const unsigned long long id = ids[j];
     float4* w = reinterpret_cast<float4*>(W + g * stride);
     const int q4 = k >> 2;
-    for (int q = 0; q < q4; ++q) w[q] = des_init4(seed, id, q, init_scale);
-    w[q4] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float n2 = 0.f;
+    for (int q = 0; q < q4; ++q) {
+      const float4 v = des_init4(seed, id, q, init_scale);
+      n2 += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      w[q] = v;
+    }
+    w[q4] = make_float4(0.f, n2, 0.f, 0.f);   // linear weight, squared norm of the latent vector
     if (A) {
       float4* a = reinterpret_cast<float4*>(A + g * stride);
       const float4 ia = make_float4(init_acc, init_acc, init_acc, init_acc);

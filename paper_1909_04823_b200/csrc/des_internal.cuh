@@ -44,7 +44,7 @@ struct des_table {
   uint32_t nblk_max;                 // scan-block capacity of the workspace
   // device memory
   Slot* slots;
-  float* W;                          // [total_rows][stride]: latent vector, linear weight, 3 pad
+  float* W;                          // [total_rows][stride]: latent vector v[k], linear weight, |v|^2, 2 pad
   float* A;                          // same shape: Adagrad accumulators (NULL for SGD)
   DevMeta* meta;
   // find_or_insert workspace

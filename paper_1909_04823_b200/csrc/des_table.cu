@@ -299,10 +299,14 @@ __global__ void write_rows_kernel(const uint32_t* __restrict__ grows, long long 
   if (i >= n) return;
   uint32_t g = grows[i];
   if (g == DES_ROW_NONE || g >= total_rows) return;
+  float n2 = 0.f;
   for (int c = 0; c < k; ++c) {
     if (emb) W[(size_t)g * stride + c] = emb[i * k + c];
     if (acc_emb && A) A[(size_t)g * stride + c] = acc_emb[i * k + c];
+    const float v = W[(size_t)g * stride + c];
+    n2 += v * v;
   }
+  W[(size_t)g * stride + k + 1] = n2;
   if (lin) W[(size_t)g * stride + k] = lin[i];
   if (acc_lin && A) A[(size_t)g * stride + k] = acc_lin[i];
 }
