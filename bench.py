@@ -61,6 +61,26 @@ def rows_per_shard(w, cap_total):
     return out
 
 
+def per_rank_workload(w, rank, world):
+    """Replicas are independent: rank r draws its own batches (seed offset), same shapes."""
+    return w if world == 1 else w.scaled(seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(value, world, device=None):
+    """Slowest rank's time (the job's step time) — torch.distributed MAX all-reduce."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(batch, world, ms_step):
+    return world * batch / (ms_step / 1e3)
+
+
 def sub_batch(b, n_samples):
     """The first n_samples samples of a batch (a bounded sample for the CPU leg)."""
     F = b.fields
@@ -121,7 +141,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "50"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -206,8 +226,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     w = synth.config(args.config)
-    if world > 1:
-        w = w.scaled(seed=w.seed + 1000 * rank)     # every replica has its own data stream
+    w = per_rank_workload(w, rank, world)           # every replica has its own data stream
 
     # ------------------------------------------------------------------ reference arm: the CPU oracle
     if args.impl == "reference":
@@ -321,13 +340,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None     # sampling from the warm-up on, every 50 ms
     for i in range(args.warmup):
         step(i)
     t.check_status()
     barrier()
     launches0 = t.launch_count()
     t.profile_enable(True)
-    sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
@@ -340,12 +359,9 @@ def main():
     t.profile_enable(False)
     launches = t.launch_count() - launches0
     t.check_status()
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    value = world * B / (ms_step / 1e3)
+    value = job_throughput(B, world, ms_step)
 
     # ---- per-kernel shares and the roofline of the dominant kernel
     per = {}
@@ -392,11 +408,8 @@ def main():
         e1.record()
         barrier()
         ms_e = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            tt = torch.tensor([ms_e], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_e = float(tt.item())
-        e2e = {"value": world * B / (ms_e / 1e3), "unit": UNIT, "ms_per_step": ms_e,
+        ms_e = max_over_ranks(ms_e, world, dev)
+        e2e = {"value": job_throughput(B, world, ms_e), "unit": UNIT, "ms_per_step": ms_e,
                "h2d_bytes_per_step": int(h_off.numel() * 4 + h_ids.numel() * 8),
                "d2h_bytes_per_step": int(h_out.numel() * 4)}
     except Exception as ex:  # keep the device-resident number even if the host path fails

@@ -40,9 +40,14 @@ __global__ void __launch_bounds__(256) sample_count_kernel(const uint32_t* __res
                                                            long long max_uniq, uint32_t* hinfo) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const long long j = ((long long)i << shift) + (shift ? (hash_u32((uint32_t)i) & ((1u << shift) - 1u)) : 0u);
-  if (j >= nnz) return;
-  const uint32_t u = __ldg(uidx + j);
-  if (u != DES_ROW_NONE && (long long)u < max_uniq) atomicAdd(hinfo + u, 1u);
+  uint32_t u = DES_ROW_NONE;
+  if (j < nnz) u = __ldg(uidx + j);
+  const bool ok = u != DES_ROW_NONE && (long long)u < max_uniq;
+  // one atomic per distinct key of the warp (a hot key fills several lanes)
+  const unsigned act = __ballot_sync(0xFFFFFFFFu, ok);
+  if (!ok) return;
+  const unsigned same = __match_any_sync(act, u);
+  if ((threadIdx.x & 31) == __ffs(same) - 1) atomicAdd(hinfo + u, (uint32_t)__popc(same));
 }
 
 // Turns the sampled counts into the hot list: hinfo[u] becomes the key's hot

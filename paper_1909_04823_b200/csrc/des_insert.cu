@@ -2,7 +2,7 @@
 // including shard routing (Section 5, "Large-scale Sparse Features": weights of
 // field f live on node f mod N; Section 4.2: any balanced partition).
 //
-// One call = six short kernels, none of which waits on another thread:
+// One call = seven short kernels, none of which waits on another thread:
 //   probe_claim   every occurrence finds its key's slot in the owning shard's
 //                 region (linear probing) or claims an empty one with a 64-bit
 //                 CAS; the slot remembers the smallest occurrence index.
@@ -13,8 +13,10 @@
 //   assign        first occurrences get the batch-unique index (rank among
 //                 firsts) and, for new keys, the next shard-local row (rank
 //                 among the shard's new keys): both in CSR order, so the result
-//                 does not depend on thread scheduling.  New rows are
-//                 initialised here from the counter-based generator.
+//                 does not depend on thread scheduling.
+//   apply_first   one thread per unique key writes these numbers into the
+//                 key's slot and initialises new rows from the counter-based
+//                 generator.
 //   resolve       every occurrence reads row and unique index from its slot.
 //   finish        slots' scratch word is reset, shard sizes are advanced.
 #include "des_internal.cuh"
@@ -128,12 +130,13 @@ __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, in
   for (int i = lo; i < hi; ++i) { uint32_t v = seq[i]; seq[i] = run; run += v; }
 }
 
+// Ranks only: first_j[u] = occurrence index of unique key u (bit 31 set for a new
+// key) and, for a new key, its shard-local row in uniq_rows[u].  The random slot
+// accesses are left to apply_first_kernel, which runs one thread per unique key.
 __global__ void __launch_bounds__(IB) assign_kernel(
-    const unsigned long long* __restrict__ ids, int nnz, int S, int k, int stride, Slot* slots, DevMeta* meta,
-    const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
-    const uint32_t* __restrict__ blk_cnt, int nblk_max, uint32_t* __restrict__ uslot,
-    uint32_t* __restrict__ uniq_rows, long long max_uniq, float* __restrict__ W, float* __restrict__ A,
-    unsigned long long seed, float init_scale, float init_acc) {
+    int nnz, int S, DevMeta* meta, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
+    const uint32_t* __restrict__ blk_cnt, int nblk_max, uint32_t* __restrict__ first_j,
+    uint32_t* __restrict__ uniq_rows) {
   __shared__ uint32_t wfirst[32];
   __shared__ uint16_t wnew[32][DES_MAX_SHARDS];
   const int j = blockIdx.x * IB + threadIdx.x;
@@ -171,36 +174,60 @@ __global__ void __launch_bounds__(IB) assign_kernel(
   }
   __syncthreads();
   if (!(fl & 1)) return;
-  const uint32_t so = slot_of[j];
   const uint32_t u = blk_cnt[blockIdx.x] + wfirst[warp] + frank;
-  uint32_t local;
   if (fl & 2) {
-    local = meta->n_rows[s] + blk_cnt[(size_t)(1 + s) * nblk_max + blockIdx.x] + wnew[warp][s] + nrank;
+    uint32_t local = meta->n_rows[s] + blk_cnt[(size_t)(1 + s) * nblk_max + blockIdx.x] + wnew[warp][s] + nrank;
     if (local >= meta->row_cap[s]) { local = DES_ROW_NONE; des_raise(meta, DES_ERR_CAPACITY); }
-    else slots[so].row = local;
+    uniq_rows[u] = local;
+    first_j[u] = (uint32_t)j | 0x80000000u;
   } else {
-    local = slots[so].row;
+    first_j[u] = (uint32_t)j;
   }
-  slots[so].first_occ = u;
-  uslot[u] = so;
-  const unsigned long long g = meta->row_base[s] + local;
-  uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
-  if ((fl & 2) && local != DES_ROW_NONE) {
-    const unsigned long long id = ids[j];
-    float4* w = reinterpret_cast<float4*>(W + g * stride);
-    const int q4 = k >> 2;
-    float n2 = 0.f;
-    for (int q = 0; q < q4; ++q) {
-      const float4 v = des_init4(seed, id, q, init_scale);
-      n2 += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-      w[q] = v;
+}
+
+// One thread per unique key of the batch: number new keys' slots and initialise
+// their rows, publish the key's batch-unique index in its slot (read back by
+// every occurrence in resolve_kernel), record slot and table-global row.
+__global__ void __launch_bounds__(256) apply_first_kernel(
+    const unsigned long long* __restrict__ ids, int k, int stride, Slot* slots, const DevMeta* __restrict__ meta,
+    const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint32_t* __restrict__ first_j,
+    uint32_t* __restrict__ uslot, uint32_t* __restrict__ uniq_rows, float* __restrict__ W, float* __restrict__ A,
+    unsigned long long seed, float init_scale, float init_acc) {
+  const uint32_t U = meta->n_uniq;
+  for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
+    const uint32_t fj = first_j[u];
+    const bool is_new = fj >> 31;
+    const uint32_t j = fj & 0x7FFFFFFFu;
+    const uint32_t so = slot_of[j];
+    const uint32_t s = shards[j];
+    uint32_t local;
+    if (is_new) {
+      local = uniq_rows[u];
+      if (local != DES_ROW_NONE) slots[so].row = local;
+    } else {
+      local = slots[so].row;
     }
-    w[q4] = make_float4(0.f, n2, 0.f, 0.f);   // linear weight, squared norm of the latent vector
-    if (A) {
-      float4* a = reinterpret_cast<float4*>(A + g * stride);
-      const float4 ia = make_float4(init_acc, init_acc, init_acc, init_acc);
-      for (int q = 0; q < q4; ++q) a[q] = ia;
-      a[q4] = make_float4(init_acc, 0.f, 0.f, 0.f);
+    slots[so].first_occ = u;
+    uslot[u] = so;
+    const unsigned long long g = meta->row_base[s] + local;
+    uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
+    if (is_new && local != DES_ROW_NONE) {
+      const unsigned long long id = ids[j];
+      float4* w = reinterpret_cast<float4*>(W + g * stride);
+      const int q4 = k >> 2;
+      float n2 = 0.f;
+      for (int q = 0; q < q4; ++q) {
+        const float4 v = des_init4(seed, id, q, init_scale);
+        n2 += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        w[q] = v;
+      }
+      w[q4] = make_float4(0.f, n2, 0.f, 0.f);   // linear weight, squared norm of the latent vector
+      if (A) {
+        float4* a = reinterpret_cast<float4*>(A + g * stride);
+        const float4 ia = make_float4(init_acc, init_acc, init_acc, init_acc);
+        for (int q = 0; q < q4; ++q) a[q] = ia;
+        a[q4] = make_float4(init_acc, 0.f, 0.f, 0.f);
+      }
     }
   }
 }
@@ -250,10 +277,13 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   DES_LAUNCH_CHECK(t, "flag_count_kernel");
   scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
   DES_LAUNCH_CHECK(t, "scan_blocks_kernel");
-  assign_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, nnz, t->S, t->k, t->stride, t->slots, t->meta,
-                                     t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max, t->uslot, b->uniq_rows,
-                                     t->max_uniq, t->W, t->A, t->cfg.seed, t->cfg.init_scale, t->cfg.init_acc);
+  assign_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->meta, b->shards, t->flags, t->blk_cnt, t->nblk_max, t->dest,
+                                     b->uniq_rows);
   DES_LAUNCH_CHECK(t, "assign_kernel");
+  apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>((const unsigned long long*)b->ids, t->k, t->stride, t->slots,
+                                                      t->meta, t->slot_of, b->shards, t->dest, t->uslot, b->uniq_rows,
+                                                      t->W, t->A, t->cfg.seed, t->cfg.init_scale, t->cfg.init_acc);
+  DES_LAUNCH_CHECK(t, "apply_first_kernel");
   resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
   DES_LAUNCH_CHECK(t, "resolve_kernel");
   finish_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->uslot, t->meta, b->n_uniq);
