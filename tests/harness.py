@@ -60,6 +60,17 @@ def u32(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().numpy().view(np.uint32)
 
 
+def select_samples(batch, idx):
+    """A batch made of the given samples of `batch`, in the given order."""
+    F = batch.fields
+    lo = batch.offsets[np.asarray(idx) * F]
+    hi = batch.offsets[np.asarray(idx) * F + F]
+    pos = np.concatenate([np.arange(a, b_) for a, b_ in zip(lo, hi)]) if len(idx) else np.zeros(0, np.int64)
+    lens = np.concatenate([np.diff(batch.offsets[i * F:i * F + F + 1]) for i in idx])
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    return synth.Batch(len(idx), F, off, batch.ids[pos], None if batch.vals is None else batch.vals[pos])
+
+
 def rows_per_shard_for(w, cap_total):
     """Row capacity per shard: even under HASH; by field vocabulary under FIELD."""
     if w.partition != PART_FIELD:
@@ -102,14 +113,20 @@ class Pair:
         self.compare_index(batch, fi, db)
         return fi, db
 
-    def compare_index(self, batch, fi, db):
+    def compare_index(self, batch, fi, db, by_key=False):
+        """by_key: the oracle's table holds only the keys of this batch (the CUDA table
+        is pre-populated with many more), so row NUMBERS differ by construction; shards
+        and batch-unique indices must still be identical, and rows are then compared
+        through the unique index, i.e. key by key."""
         n = batch.nnz
         assert self.t.status() == 0
         assert np.array_equal(db.shards.cpu().numpy()[:n], fi["shards"]), "shards"
-        assert np.array_equal(u32(db.rows)[:n], fi["rows"]), "rows"
         assert np.array_equal(u32(db.uidx)[:n], fi["uidx"]), "uidx"
         U = int(db.n_uniq.item())
         assert U == fi["U"], ("n_uniq", U, fi["U"])
+        if by_key:
+            return
+        assert np.array_equal(u32(db.rows)[:n], fi["rows"]), "rows"
         want = self.row_base[fi["uniq_shard"].astype(np.int64)] + fi["uniq_row"].astype(np.int64)
         assert np.array_equal(u32(db.uniq_rows)[:U].astype(np.int64), want), "uniq_rows"
         assert self.t.size() == [int(v) for v in self.o.size()], "table size"
@@ -145,8 +162,11 @@ class Pair:
         return ref
 
     # ------------------------------------------------------------------
-    def step(self, batch, grads, ops=None, materialise=False, check_init=False):
-        """One full step on both sides with every intermediate compared."""
+    def step(self, batch, grads, ops=None, materialise=False, check_init=False, by_key=False,
+             pooled_samples=None):
+        """One full step on both sides with every intermediate compared.
+        pooled_samples: compare `pooled` only on these sample indices (the dense
+        per-shard pooled partial of the oracle is too large at full size)."""
         from paper_1909_04823_b200.binding import DeviceBatch
         w = self.w
         ops = w.ops if ops is None else ops
@@ -157,11 +177,12 @@ class Pair:
         fi = self.o.find_or_insert(batch)
         db = DeviceBatch.from_synth(batch)
         self.t.find_or_insert(db, True)
-        self.compare_index(batch, fi, db)
+        self.compare_index(batch, fi, db, by_key=by_key)
         if check_init:
             self.compare_rows(fi, db, exact=True, what="initial rows")
         # ---- forward
-        op = self.o.forward_partials(ops, batch, fi, want_pooled=True, want_dense=bool(ops & OP_DENSE1))
+        op = self.o.forward_partials(ops, batch, fi, want_pooled=pooled_samples is None,
+                                     want_dense=bool(ops & OP_DENSE1))
         oa = self.o.aggregate(B, op)
         sabs = self.o.forward_original(ops & ~OP_DENSE1, batch)["Sabs"]
         xa, xl = SUMTOL_FWD * sabs[:, :k], SUMTOL_FWD * sabs[:, k]
@@ -192,7 +213,12 @@ class Pair:
             cmp(osm[:, k], oa["lr"], "R_lr", extra=xl)
         if ops & (OP_LR | OP_FM):
             assert not np.any(ps[:, :, k + 2:]) and not np.any(osm[:, k + 3]), "padding must be zero"
-        if ops & (OP_POOL | OP_DENSE1):
+        if (ops & (OP_POOL | OP_DENSE1)) and pooled_samples is not None:
+            sel = np.asarray(pooled_samples)
+            sb = select_samples(batch, sel)
+            ref_p = self.o.forward_original(ops & ~OP_DENSE1, sb)["pooled"]
+            cmp(pooled[torch.from_numpy(sel).to(dev)].cpu().numpy(), ref_p, "pooled (sampled)")
+        elif ops & (OP_POOL | OP_DENSE1):
             cmp(pooled.cpu().numpy(), oa["pooled"], "pooled")
             if materialise:
                 cmp(part_pooled.cpu().numpy(), op["part_pooled"], "part_pooled")

@@ -1,0 +1,99 @@
+"""Parity at the benchmark's full size and launch configuration (the large
+multi-hot workload: 2e8 pre-populated keys, batch 16384 x 100 fields, k = 64,
+S = 64, LR + FM + pooled embeddings, Adagrad).
+
+The oracle cannot hold 2e8 rows on the host, and does not need to: until a row
+is first updated its contents are a pure function of the id, so an oracle table
+that holds only the keys of the batch produces the same forward results and the
+same per-key updates.  Row NUMBERS differ by construction and are checked by
+the property that defines them instead: the shard-local row of pre-populated
+rank r is the number of earlier ranks in the same shard.
+
+Runs one full oracle step (about a minute on one core)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1909_04823_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+M64 = (1 << 64) - 1
+
+
+def fmix64_inverse(y: np.ndarray) -> np.ndarray:
+    """Inverse of synth.fmix64 (each step is a bijection on 64-bit words)."""
+    inv1 = np.uint64(pow(0xFF51AFD7ED558CCD, -1, 1 << 64))
+    inv2 = np.uint64(pow(0xC4CEB9FE1A85EC53, -1, 1 << 64))
+    x = y.astype(np.uint64).copy()
+    with np.errstate(over="ignore"):
+        x ^= x >> np.uint64(33); x *= inv2      # x ^= x >> 33 is its own inverse for shifts >= 32
+        x ^= x >> np.uint64(33); x *= inv1
+        x ^= x >> np.uint64(33)
+    return x
+
+
+def test_fmix64_inverse_roundtrip():
+    r = np.random.default_rng(0).integers(0, 2 ** 62, 1000).astype(np.uint64)
+    assert np.array_equal(fmix64_inverse(synth.fmix64(r)), r)
+
+
+def test_full_size_step_matches_oracle():
+    from harness import Pair
+    from paper_1909_04823_b200.binding import DeviceBatch
+    w = synth.config(5)
+    free_b, _ = torch.cuda.mem_get_info()
+    per_key = 2 * (4 * w.emb_dim + 16) * 1.06 + 16 * 2.2
+    n_keys = w.prepopulate
+    fit = int((free_b - 16e9) / per_key)
+    if fit < n_keys:                                  # shared GPU with less free memory: largest table that fits
+        n_keys = max(1_000_000, (fit // 1_000_000) * 1_000_000)
+        w = w.scaled(vocab=n_keys, prepopulate=n_keys)
+    st = synth.Stream(w)
+    b = st.next_batch()
+    U_est = int(np.unique(b.ids).size)
+    p = Pair(w, max_rows=n_keys, max_nnz=max(b.nnz + 1024, w.batch * w.fields), max_uniq=int(U_est * 1.2) + 4096)
+    try:
+        # ---- pre-populate the CUDA table only (ranks 0..n-1 in order)
+        per_call = w.batch * w.fields
+        for ids in st.prepopulation_ids(chunk=per_call * 8):
+            d_all = torch.from_numpy(ids.view(np.int64)).cuda()
+            for lo in range(0, ids.size, per_call):
+                n = min(per_call, ids.size - lo)
+                pb = synth.prepopulation_batch(ids[lo:lo + n], w.fields)
+                p.t.find_or_insert(DeviceBatch(pb.offsets, d_all[lo:lo + n], None, pb.batch), True)
+        assert p.t.status() == 0 and sum(p.t.size()) == n_keys
+        # ---- the step, compared key by key; pooled on 96 sampled samples
+        sel = np.sort(np.random.default_rng(1).choice(w.batch, 96, replace=False))
+        g = synth.upstream_grads(w, b.batch, 0)
+        res = p.step(b, g, by_key=True, pooled_samples=sel)
+        assert sum(p.t.size()) == n_keys                          # nothing new was inserted
+        # ---- row numbers: rank r sits at row (#earlier ranks in its shard)
+        db = res["db"]
+        rows = db.rows.cpu().numpy().view(np.uint32)[:b.nnz]
+        shards = db.shards.cpu().numpy()[:b.nnz]
+        ranks = fmix64_inverse(b.ids)
+        assert ranks.max() < n_keys
+        want = np.empty(b.nnz, dtype=np.uint32)
+        chunk = 1 << 24
+        counts = np.zeros(w.shards, dtype=np.int64)
+        order = np.argsort(ranks, kind="stable")
+        sorted_ranks = ranks[order]
+        for lo in range(0, n_keys, chunk):
+            hi = min(n_keys, lo + chunk)
+            sh = oracle.shard_of_many(synth.fmix64(np.arange(lo, hi, dtype=np.uint64)), w.shards)
+            a, z = np.searchsorted(sorted_ranks, [lo, hi])
+            if z > a:
+                # row of rank r = counts[shard] + (#ranks of the same shard in [lo, r))
+                local = np.empty(hi - lo, dtype=np.int64)
+                for s in range(w.shards):
+                    m = np.flatnonzero(sh == s)
+                    local[m] = counts[s] + np.arange(m.size)
+                idx = (sorted_ranks[a:z] - np.uint64(lo)).astype(np.int64)
+                want[order[a:z]] = local[idx].astype(np.uint32)
+                assert np.array_equal(shards[order[a:z]], sh[idx])
+            counts += np.bincount(sh, minlength=w.shards)
+        assert np.array_equal(rows, want)
+    finally:
+        p.close()
