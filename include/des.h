@@ -65,7 +65,8 @@ typedef enum {
   DES_ERR_CAPACITY = 3,      /* a shard ran out of slots or rows (sticky, device-side)  */
   DES_ERR_UNSUPPORTED = 4,
   DES_ERR_CUDA = 5,          /* a CUDA runtime call failed, or no device                */
-  DES_ERR_NOT_FOUND = 6
+  DES_ERR_NOT_FOUND = 6,
+  DES_ERR_TOO_LARGE = 7      /* problem exceeds the fixed scratch of a no-allocation entry point */
 } des_status_t;
 
 /* operator kind bitmask */
@@ -203,6 +204,35 @@ des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t
 /* ---- first dense layer weights W1 [F*k][H], fp32 master (Section 4.3) ----- */
 des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream);
 des_status_t des_dense1_get(des_table_t* t, float* d_W1, void* stream);
+
+/* Row-split first layer for callers that must not allocate.  (The paper has no
+ * counterpart: this is a packaging variant of des_aggregate's DENSE1 step, same
+ * arithmetic, same result.)
+ *
+ * Who needs it: code that is handed a stream and some buffers but is not allowed
+ * to call cudaMalloc — a serving loop with a frozen memory budget, a plug-in
+ * running inside someone else's framework, anything between the begin and end
+ * of a latency-critical section where an allocation would synchronise the
+ * device.  des_aggregate normally wants the caller to bring the [S][B][H]
+ * buffer for the per-shard partial products P_s = V_s W_s; here that buffer is
+ * a fixed array inside the library image instead.
+ *
+ * Computes Z[B][H] = sum over shards s = 0..S-1 of P_s from d_pooled [B][F*k]
+ * and the table's W1 (FIELD partition only).  The partial products live in a
+ * static device array of DES_NOALLOC_SCRATCH_FLOATS floats (8 MiB, reserved on
+ * every GPU that loads the library until the process exits); the call is
+ * rejected with DES_ERR_TOO_LARGE when S*B*H exceeds that.  It calls no
+ * cudaMalloc / cudaFree and no allocating routine of any library.
+ *
+ * The first call on a device looks up the array's device address (one runtime
+ * query, result cached per device); make that first call outside any stream
+ * capture.  All calls share the one array and it keeps the last call's
+ * contents: every element a call reads is written by that same call first, so
+ * stale contents are harmless, but two calls whose kernels overlap on the GPU
+ * (different streams, no ordering) race on it. */
+#define DES_NOALLOC_SCRATCH_FLOATS (2u * 1024u * 1024u)
+des_status_t des_dense1_forward_noalloc(des_table_t* t, const float* d_pooled, int32_t batch, float* d_Z,
+                                        void* stream);
 
 /* ---- inspection (synchronising) ------------------------------------------ */
 

@@ -20,10 +20,11 @@ ROW_NONE = 0xFFFFFFFF
 KEY_EMPTY = 0xFFFFFFFFFFFFFFFF
 
 STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "DES_ERR_CAPACITY",
-          4: "DES_ERR_UNSUPPORTED", 5: "DES_ERR_CUDA", 6: "DES_ERR_NOT_FOUND"}
+          4: "DES_ERR_UNSUPPORTED", 5: "DES_ERR_CUDA", 6: "DES_ERR_NOT_FOUND",
+          7: "DES_ERR_TOO_LARGE"}
 
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
-           "des_aggregate", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_table_status",
+           "des_aggregate", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_step_host", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
 
@@ -91,6 +92,7 @@ def load():
                                           C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
         L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.des_dense1_get.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_dense1_forward_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.des_table_status.argtypes = [C.c_void_p]
         L.des_table_size.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
         L.des_table_row_base.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
@@ -306,3 +308,9 @@ class Table:
         n = C.c_int(0)
         self._check(self.L.des_profile_read(self.h, names, ms, cap, C.byref(n)), "des_profile_read")
         return [(names[i].decode(), float(ms[i])) for i in range(min(n.value, cap))]
+
+    def dense1_forward_noalloc(self, pooled: torch.Tensor, Z: torch.Tensor):
+        """Z = sum_s P_s with the per-shard partial products kept in the library's
+        static device array: no allocation anywhere in the call."""
+        self._check(self.L.des_dense1_forward_noalloc(self.h, _ptr(pooled), int(pooled.shape[0]), _ptr(Z), _stream()),
+                    "des_dense1_forward_noalloc")

@@ -185,3 +185,48 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
   }
   return DES_OK;
 }
+
+// ---- no-allocation variant of the row-split forward ---------------------------
+// The per-shard partial products live in this file-scope array.  In host code
+// the symbol below is only a handle: its device address is obtained once per
+// device with cudaGetSymbolAddress and that pointer is what the kernels get.
+static __device__ __align__(256) float g_noalloc_partials[DES_NOALLOC_SCRATCH_FLOATS];
+static float* g_noalloc_ptr[64];   // per device ordinal, filled on first use
+
+__global__ void noalloc_reduce_kernel(const float* __restrict__ part, size_t per_shard, int S, float* __restrict__ out) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
+  for (; i < per_shard; i += st) {
+    float a = 0.f;
+    for (int s = 0; s < S; ++s) a += part[(size_t)s * per_shard + i];
+    out[i] = a;
+  }
+}
+
+extern "C" des_status_t des_dense1_forward_noalloc(des_table_t* t, const float* d_pooled, int32_t batch, float* d_Z,
+                                                   void* stream) {
+  if (!t || !d_pooled || !d_Z || batch <= 0 || !t->H) return DES_ERR_INVALID_ARG;
+  if (t->cfg.partition != DES_PART_FIELD) return DES_ERR_UNSUPPORTED;
+  const size_t need = (size_t)t->S * (size_t)batch * t->H;
+  if (need > (size_t)DES_NOALLOC_SCRATCH_FLOATS) return DES_ERR_TOO_LARGE;
+  int dev = 0;
+  DES_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return DES_ERR_UNSUPPORTED;
+  if (!g_noalloc_ptr[dev]) {          // set-up, once per device, with that device current
+    float* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_noalloc_partials) != cudaSuccess || !p) { cudaGetLastError(); return DES_ERR_CUDA; }
+    g_noalloc_ptr[dev] = p;
+  }
+  float* part = g_noalloc_ptr[dev];
+  cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
+  GemmArgs g; memset(&g, 0, sizeof(g));
+  g.M = batch; g.N = t->H; g.K = t->F * t->k; g.A32 = d_pooled; g.Bb = t->W1b; g.k_emb = t->k; g.FK = g.K; g.H = t->H;
+  g.meta = t->meta; g.partition = t->cfg.partition; g.S = t->S; g.F = t->F;
+  g.out = part; g.slices = t->S; g.slice_by_shard = 1;     // every element of every slice is written
+  dim3 grid((g.N + TN - 1) / TN, (g.M + TM - 1) / TM, g.slices);
+  gemm_kernel<GEMM_FWD><<<grid, 256, 0, cs>>>(g);
+  DES_LAUNCH_CHECK(t, "gemm_kernel");
+  noalloc_reduce_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part, (size_t)batch * t->H, t->S, d_Z);
+  DES_LAUNCH_CHECK(t, "noalloc_reduce_kernel");
+  return DES_OK;
+}

@@ -77,6 +77,7 @@ extern "C" const char* des_status_string(des_status_t s) {
     case DES_ERR_UNSUPPORTED: return "unsupported";
     case DES_ERR_CUDA: return "CUDA runtime error or no device";
     case DES_ERR_NOT_FOUND: return "not found";
+    case DES_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
   }
   return "?";
 }
