@@ -193,8 +193,12 @@ def kernel_bytes(name, st):
         return nnz + nnz + 4 * U + 8 * U + 4 * U
     if name == "resolve_kernel":
         return 4 * nnz + 16 * U + 8 * nnz
-    if name == "forward_partials_kernel":
-        return 4 * (B * F + 1) + 5 * nnz + row * U + (4 * S * B * (k + 4) if small else 0) + (4 * B * F * k if pool else 0)
+    if name == "route_kernel":
+        return 8 * B + 2 * 5 * nnz + 8 * nnz + 4 * B * (S + 1)
+    if name == "shard_partials_kernel":
+        return 4 * B * (S + 1) + 4 * nnz + row * U + 4 * S * B * (k + 4)
+    if name == "pool_kernel":
+        return 4 * (B * F + 1) + 4 * nnz + 4 * k * U + 4 * B * F * k
     if name == "aggregate_small_kernel":
         return 4 * S * B * (k + 4) + 4 * B * (k + 4)
     if name == "make_dest_kernel":

@@ -7,131 +7,165 @@
 // des_aggregate: (+) over shards in the order s = 0..S-1 (Eq. 1) and the
 // substitution operator F = 1/2 <(+)M_1,(+)M_1> - 1/2 (+)M_2 (Eq. 8).
 //
-// Kernel shape.  One warp walks one sample, bag by bag.  A row (k floats + the
-// linear weight) is read by a group of G = k/4 lanes (rounded up to a power of
-// two) with one 16-byte load per lane; the NG = 32/G groups of the warp split
-// the occurrences of a bag BY SHARD: group g takes the occurrences whose shard
-// is congruent to g modulo NG.  The per-(shard, sample) partials live in shared
-// memory, S x (k+4) floats per warp, and because a shard's accumulator row is
-// only ever touched by its owning group, in occurrence order, there are no
-// conflicts to resolve and the result is deterministic.  A bag's pooled sum is
-// the sum of the groups' partial sums (a few shuffles per bag).  Each group
-// keeps FW_UNROLL row loads in flight.  M_2 needs |v|^2 of every row: the table
-// keeps it next to the linear weight in the row's 16-byte tail (refreshed by the
-// update kernel), so the forward adds x^2 |v|^2 without a cross-lane reduction.
+// Kernels.
+//  route_kernel   "each shard looks up its own ids": one warp per sample buckets
+//                 the sample's occurrences by owning shard with a stable counting
+//                 sort (warp match + running cursors), writing the table-global
+//                 row of every occurrence in shard-major order, the segment
+//                 bounds [B][S+1], and the same rows in CSR order for pooling.
+//  shard_partials_kernel   one group of G = k/4 lanes (rounded up to a power of
+//                 two) per (sample, shard) segment: it streams the segment's
+//                 rows with 16-byte loads, FW_UNROLL in flight, and keeps
+//                 M_1, M_1^lr, M_2 in registers until the segment ends — no
+//                 shared memory, no atomics, sums in CSR order (deterministic).
+//                 M_2 uses the |v|^2 cached in the row's 16-byte tail.
+//  pool_kernel    one group per bag: sum pooling of the latent vectors in
+//                 registers.  The per-shard pooled partial [S][B][F*k] is only
+//                 materialised (with atomics) when the caller asks for it.
 #include "des_internal.cuh"
 
-#define FW_UNROLL 4
+#define FW_UNROLL 8
 
-template <int G, bool HAS_VALS, bool MATERIALISE>
-__global__ void __launch_bounds__(384) forward_partials_kernel(
+__global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
-    const uint8_t* __restrict__ shards, int B, int F, int S, int k, uint32_t ops, const float* __restrict__ W,
-    const DevMeta* __restrict__ meta, float* __restrict__ part_small, float* __restrict__ pooled,
-    float* __restrict__ part_pooled) {
-  extern __shared__ __align__(16) float smem[];
+    const uint8_t* __restrict__ shards, int B, int F, int S, const DevMeta* __restrict__ meta,
+    uint32_t* __restrict__ grow_csr, uint32_t* __restrict__ grow_sorted, float* __restrict__ x_sorted,
+    int32_t* __restrict__ seg_off) {
   __shared__ uint32_t row_base[DES_MAX_SHARDS];
-  constexpr int NG = 32 / G;
-  const int K4 = k >> 2, stride = k + 4;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
-  const int g = lane / G, c4 = lane % G;
-  const bool col = c4 < K4, lead = c4 == 0;
-  const bool want_small = part_small != nullptr;
-  float* acc = smem + (size_t)warp * S * stride;
-  const int acc_f4 = S * (K4 + 1);
+  __shared__ int cursor[8][DES_MAX_SHARDS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x < S) row_base[threadIdx.x] = (uint32_t)meta->row_base[threadIdx.x];
-  if (want_small)
-    for (int i = lane; i < acc_f4; i += 32) reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   __syncthreads();
-
-  for (int b = blockIdx.x * wpb + warp; b < B; b += gridDim.x * wpb) {
-    for (int f = 0; f < F; ++f) {
-      const int lo = __ldg(offsets + (size_t)b * F + f), hi = __ldg(offsets + (size_t)b * F + f + 1);
-      float4 pacc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int base = lo; base < hi; base += 32) {
-        // every lane fetches one occurrence of the chunk; groups then pick their shards' entries
-        const int j = base + lane;
-        uint32_t my_grow = DES_ROW_NONE; int my_s = 0; float my_x = 1.f;
-        if (j < hi) {
-          const uint32_t r = __ldg(rows + j);
-          my_s = __ldg(shards + j);
-          if (r != DES_ROW_NONE) my_grow = row_base[my_s] + r;      // table-global row
-          if (HAS_VALS) my_x = __ldg(vals + j);
-        }
-        const int key = (my_grow == DES_ROW_NONE) ? -1 : ((want_small ? my_s : lane) & (NG - 1));
-        unsigned m = 0;
-#pragma unroll
-        for (int q = 0; q < NG; ++q) {
-          const unsigned mq = __ballot_sync(0xFFFFFFFFu, key == q);
-          if (q == g) m = mq;
-        }
-        while (__any_sync(0xFFFFFFFFu, m != 0)) {
-          float4 v[FW_UNROLL], tl[FW_UNROLL]; float x[FW_UNROLL]; int sh[FW_UNROLL];
-#pragma unroll
-          for (int u = 0; u < FW_UNROLL; ++u) {
-            const bool have = m != 0;
-            const int src = have ? (__ffs(m) - 1) : 0;
-            m &= m - 1;                                     // 0 stays 0
-            const uint32_t gr = __shfl_sync(0xFFFFFFFFu, my_grow, src);
-            const int s = __shfl_sync(0xFFFFFFFFu, my_s, src);
-            x[u] = HAS_VALS ? __shfl_sync(0xFFFFFFFFu, my_x, src) : 1.f;
-            sh[u] = have ? s : -1;
-            v[u] = make_float4(0.f, 0.f, 0.f, 0.f); tl[u] = v[u];
-            if (have) {
-              const float4* wr = reinterpret_cast<const float4*>(W + (size_t)gr * stride);
-              if (col) v[u] = __ldg(wr + c4);
-              if (lead && want_small) tl[u] = __ldg(wr + K4);      // (linear weight, |v|^2, 0, 0)
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < FW_UNROLL; ++u) {
-            float4 vx = v[u];
-            if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
-            pacc.x += vx.x; pacc.y += vx.y; pacc.z += vx.z; pacc.w += vx.w;
-            if (sh[u] >= 0) {
-              if (MATERIALISE && col)
-                atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)sh[u] * B + b) * ((size_t)F * k) +
-                                                    (size_t)f * k) + c4, vx);
-              if (want_small) {
-                float* a = acc + sh[u] * stride;             // row owned by this group
-                if (col) {
-                  float4 t = reinterpret_cast<float4*>(a)[c4];
-                  t.x += vx.x; t.y += vx.y; t.z += vx.z; t.w += vx.w;
-                  reinterpret_cast<float4*>(a)[c4] = t;
-                }
-                if (lead) {
-                  float2 t = *reinterpret_cast<float2*>(a + k);
-                  t.x += tl[u].x * x[u]; t.y += tl[u].y * x[u] * x[u];
-                  *reinterpret_cast<float2*>(a + k) = t;
-                }
-              }
-            }
-          }
-        }
+  int* cur = cursor[warp];
+  const unsigned lt = (1u << lane) - 1u;
+  for (int b = blockIdx.x * 8 + warp; b < B; b += gridDim.x * 8) {
+    const int lo = __ldg(offsets + (size_t)b * F), hi = __ldg(offsets + (size_t)(b + 1) * F);
+    for (int s = lane; s < S; s += 32) cur[s] = 0;
+    __syncwarp();
+    // pass 1: occurrences per shard (mapped rows only); CSR-order rows for the pooling kernel
+    for (int base = lo; base < hi; base += 32) {
+      const int j = base + lane;
+      int key = -1 - lane;
+      if (j < hi) {
+        const uint32_t r = __ldg(rows + j);
+        const int s = __ldg(shards + j);
+        grow_csr[j] = (r == DES_ROW_NONE) ? DES_ROW_NONE : row_base[s] + r;
+        if (r != DES_ROW_NONE) key = s;
       }
-      if (pooled) {
-#pragma unroll
-        for (int d = G; d < 32; d <<= 1) {
-          pacc.x += __shfl_xor_sync(0xFFFFFFFFu, pacc.x, d); pacc.y += __shfl_xor_sync(0xFFFFFFFFu, pacc.y, d);
-          pacc.z += __shfl_xor_sync(0xFFFFFFFFu, pacc.z, d); pacc.w += __shfl_xor_sync(0xFFFFFFFFu, pacc.w, d);
-        }
-        if (g == 0 && col) reinterpret_cast<float4*>(pooled + ((size_t)b * F + f) * k)[c4] = pacc;
-      }
-    }
-    if (want_small) {
+      const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+      if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
       __syncwarp();
-      const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
-      for (int i = lane; i < acc_f4; i += 32) {
-        const int s = i / (K4 + 1), q = i % (K4 + 1);
-        float4 t = reinterpret_cast<float4*>(acc)[i];
-        reinterpret_cast<float4*>(acc)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (q == K4) { if (!lr) t.x = 0.f; if (!fm) t.y = 0.f; }
-        else if (!fm) t = make_float4(0.f, 0.f, 0.f, 0.f);
-        reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride)[q] = t;
+    }
+    // exclusive scan over shards -> segment starts (lane 0 walks the <= 64 counters)
+    if (lane == 0) {
+      int run = lo;
+      int32_t* so = seg_off + (size_t)b * (S + 1);
+      for (int s = 0; s < S; ++s) { const int c = cur[s]; cur[s] = run; so[s] = run; run += c; }
+      so[S] = run;
+    }
+    __syncwarp();
+    // pass 2: stable placement
+    for (int base = lo; base < hi; base += 32) {
+      const int j = base + lane;
+      int key = -1 - lane; uint32_t gr = 0;
+      if (j < hi) {
+        const uint32_t r = __ldg(rows + j);
+        const int s = __ldg(shards + j);
+        if (r != DES_ROW_NONE) { key = s; gr = row_base[s] + r; }
       }
+      const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+      if (key >= 0) {
+        const int pos = cur[key] + __popc(same & lt);
+        grow_sorted[pos] = gr;
+        if (vals) x_sorted[pos] = __ldg(vals + j);
+      }
+      __syncwarp();
+      if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
       __syncwarp();
     }
   }
+}
+
+template <int G, bool HAS_VALS>
+__global__ void __launch_bounds__(256) shard_partials_kernel(
+    const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted, const int32_t* __restrict__ seg_off,
+    int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small) {
+  const int K4 = k >> 2, stride = k + 4;
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long seg = t / G;                       // = b * S + s
+  const int c4 = (int)(t % G);
+  if (seg >= (long long)B * S) return;
+  const int b = (int)(seg / S), s = (int)(seg % S);
+  const bool col = c4 < K4, lead = c4 == 0;
+  if (!col && !lead) return;
+  const int lo = __ldg(seg_off + (size_t)b * (S + 1) + s), hi = __ldg(seg_off + (size_t)b * (S + 1) + s + 1);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float m1lr = 0.f, m2 = 0.f;
+  for (int i0 = lo; i0 < hi; i0 += FW_UNROLL) {
+    float4 v[FW_UNROLL]; float2 tl[FW_UNROLL]; float x[FW_UNROLL];
+#pragma unroll
+    for (int u = 0; u < FW_UNROLL; ++u) {
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f); tl[u] = make_float2(0.f, 0.f); x[u] = 1.f;
+      if (i0 + u < hi) {
+        const float* wr = W + (size_t)__ldg(grow_sorted + i0 + u) * stride;
+        if (HAS_VALS) x[u] = __ldg(x_sorted + i0 + u);
+        if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
+        if (lead) tl[u] = __ldg(reinterpret_cast<const float2*>(wr + k));      // (w, |v|^2)
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < FW_UNROLL; ++u) {
+      if (HAS_VALS) {
+        acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
+        m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
+      } else {
+        acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+        m1lr += tl[u].x; m2 += tl[u].y;
+      }
+    }
+  }
+  const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
+  float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
+  if (col) dst[c4] = fm ? acc : make_float4(0.f, 0.f, 0.f, 0.f);
+  if (lead) dst[K4] = make_float4(lr ? m1lr : 0.f, fm ? m2 : 0.f, 0.f, 0.f);
+}
+
+template <int G, bool HAS_VALS, bool MATERIALISE>
+__global__ void __launch_bounds__(256) pool_kernel(
+    const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ grow_csr,
+    const uint8_t* __restrict__ shards, long long nbags, int B, int F, int k, const float* __restrict__ W,
+    float* __restrict__ pooled, float* __restrict__ part_pooled) {
+  const int K4 = k >> 2, stride = k + 4;
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long bag = t / G;
+  const int c4 = (int)(t % G);
+  if (bag >= nbags || c4 >= K4) return;
+  const int lo = __ldg(offsets + bag), hi = __ldg(offsets + bag + 1);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i0 = lo; i0 < hi; i0 += FW_UNROLL) {
+    float4 v[FW_UNROLL]; float x[FW_UNROLL];
+#pragma unroll
+    for (int u = 0; u < FW_UNROLL; ++u) {
+      v[u] = make_float4(0.f, 0.f, 0.f, 0.f); x[u] = 1.f;
+      if (i0 + u < hi) {
+        const uint32_t gr = __ldg(grow_csr + i0 + u);
+        if (HAS_VALS) x[u] = __ldg(vals + i0 + u);
+        if (gr != DES_ROW_NONE) v[u] = __ldg(reinterpret_cast<const float4*>(W + (size_t)gr * stride) + c4);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < FW_UNROLL; ++u) {
+      float4 vx = v[u];
+      if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
+      acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
+      if (MATERIALISE && i0 + u < hi && __ldg(grow_csr + i0 + u) != DES_ROW_NONE) {
+        const int s = __ldg(shards + i0 + u);
+        const long long b = bag / F, f = bag % F;
+        atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)s * B + b) * ((size_t)F * k) + (size_t)f * k) + c4, vx);
+      }
+    }
+  }
+  reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
 }
 
 // (+) over shards and F.  G lanes per sample, one float4 column each; lane 0 of
@@ -191,38 +225,38 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   float* pl = pool ? part->pooled : nullptr;
   float* pp = pool ? part->part_pooled : nullptr;
   if (pp) DES_CUDA(cudaMemsetAsync(pp, 0, (size_t)t->S * B * t->F * t->k * 4, cs));
-  const size_t per_warp = small ? (size_t)t->S * t->stride * 4 : 0;
-  int wpb = 12;
-  while (wpb > 1 && per_warp * wpb > 208 * 1024) --wpb;
-  const size_t smem = per_warp * wpb;
-  int grid = (B + wpb - 1) / wpb;
   const int G = group_for(t->k);
-#define FWD3(GG, HV, MT)                                                                                          \
-  do {                                                                                                            \
-    if (smem > 48 * 1024)                                                                                         \
-      DES_CUDA(cudaFuncSetAttribute(forward_partials_kernel<GG, HV, MT>,                                          \
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));                     \
-    forward_partials_kernel<GG, HV, MT><<<grid, wpb * 32, smem, cs>>>(                                            \
-        b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->k, ops, t->W, t->meta, ps, pl, pp);            \
-  } while (0)
-#define FWD(GG)                                                                                                   \
-  do {                                                                                                            \
-    if (pp) { if (b->vals) FWD3(GG, true, true); else FWD3(GG, false, true); }                                    \
-    else { if (b->vals) FWD3(GG, true, false); else FWD3(GG, false, false); }                                     \
-  } while (0)
-  switch (G) {
-    case 1: FWD(1); break;
-    case 2: FWD(2); break;
-    case 4: FWD(4); break;
-    case 8: FWD(8); break;
-    default: FWD(16); break;
+  // routing: rows of every occurrence in shard-major order per sample (workspace shared with find_or_insert,
+  // which has finished with it by the time a forward can run on the same stream)
+  uint32_t* grow_csr = t->uslot;
+  uint32_t* grow_sorted = t->slot_of;
+  float* x_sorted = reinterpret_cast<float*>(t->dest);
+  route_kernel<<<(B + 7) / 8 < t->sm_count * 8 ? (B + 7) / 8 : t->sm_count * 8, 256, 0, cs>>>(
+      b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, grow_csr, grow_sorted, x_sorted, t->seg_off);
+  DES_LAUNCH_CHECK(t, "route_kernel");
+  if (ps) {
+    const long long threads = (long long)B * t->S * G;
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+#define SP(GG) do { if (b->vals) shard_partials_kernel<GG, true><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, t->k, ops, t->W, ps); \
+                    else shard_partials_kernel<GG, false><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, t->k, ops, t->W, ps); } while (0)
+    switch (G) { case 1: SP(1); break; case 2: SP(2); break; case 4: SP(4); break; case 8: SP(8); break; default: SP(16); }
+#undef SP
+    DES_LAUNCH_CHECK(t, "shard_partials_kernel");
   }
-#undef FWD3
-#undef FWD
-  DES_LAUNCH_CHECK(t, "forward_partials_kernel");
+  if (pl) {
+    const long long nbags = (long long)B * t->F;
+    const long long threads = nbags * G;
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+#define PK3(GG, HV, MT) pool_kernel<GG, HV, MT><<<grid, 256, 0, cs>>>(b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, t->k, t->W, pl, pp)
+#define PK(GG) do { if (pp) { if (b->vals) PK3(GG, true, true); else PK3(GG, false, true); } \
+                    else { if (b->vals) PK3(GG, true, false); else PK3(GG, false, false); } } while (0)
+    switch (G) { case 1: PK(1); break; case 2: PK(2); break; case 4: PK(4); break; case 8: PK(8); break; default: PK(16); }
+#undef PK
+#undef PK3
+    DES_LAUNCH_CHECK(t, "pool_kernel");
+  }
   return DES_OK;
 }
-
 extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* b, const des_partials_t* part,
                                       const des_outputs_t* out, void* stream) {
   if (!t || !b || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;

@@ -52,6 +52,7 @@ struct des_table {
   uint8_t* flags;                    // [max_nnz]
   uint32_t* uslot;                   // [max_nnz]
   uint32_t* blk_cnt;                 // [(S+1)][nblk_max]
+  int32_t* seg_off;                  // [max_batch][S+1] forward routing: (sample, shard) segment bounds
   // backward workspace
   float* Gbuf;                       // [max_uniq + rep_max][stride]: per-unique gradient rows, then
                                      // hot-key replica rows; all zero between calls

@@ -86,7 +86,7 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   if (!t) return DES_OK;
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
-  void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->Gbuf, t->hinfo, t->dest, t->hot_base,
+  void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
                   t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc,
                   t->W1, t->accW1, t->W1b, t->gW1_part, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
@@ -158,6 +158,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->flags, (size_t)t->max_nnz);
   A(t->uslot, (size_t)t->max_nnz * 4);
   A(t->blk_cnt, (size_t)(t->S + 1) * t->nblk_max * 4);
+  A(t->seg_off, (size_t)t->max_batch * (t->S + 1) * 4);
   t->hot_max = 16384;
   t->rep_max = (uint32_t)(t->max_nnz / 256 + t->hot_max + 1024);
   A(t->Gbuf, ((size_t)t->max_uniq + t->rep_max) * rowbytes);
