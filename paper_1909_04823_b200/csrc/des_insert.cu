@@ -31,45 +31,73 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
   return s;
 }
 
-__global__ void __launch_bounds__(IB) probe_claim_kernel(
+#define PROBE_ILP 4   // occurrences per thread: their probe chains are independent, so 4 slot loads are in flight
+
+struct SlotGeom { unsigned long long slot_base[DES_MAX_SHARDS + 1]; };   // kernel parameter: constant-bank reads
+
+__global__ void __launch_bounds__(256) probe_claim_kernel(
     const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
-    int S, int F, int partition, int insert, Slot* slots, DevMeta* meta,
+    int S, int F, int partition, int insert, Slot* slots, DevMeta* meta, const __grid_constant__ SlotGeom geom,
     uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards, uint32_t* __restrict__ rows) {
-  int j = blockIdx.x * IB + threadIdx.x;
-  if (j >= nnz) return;
-  unsigned long long id = ids[j];
-  uint32_t s;
-  if (partition == DES_PART_HASH) s = (uint32_t)(des_mix64(id) % (unsigned)S);
-  else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
-  shards[j] = (uint8_t)s;
-  uint32_t found = DES_SLOT_NONE;
-  uint32_t row = DES_ROW_NONE;
-  if (id == DES_KEY_EMPTY) {
-    des_raise(meta, DES_ERR_RESERVED_KEY);
-  } else {
-    const unsigned long long base = meta->slot_base[s];
-    const unsigned long long n = meta->slot_base[s + 1] - base;
-    unsigned long long pos = __umul64hi(des_mix64(id ^ 0x9E3779B97F4A7C15ull), n);
-    bool full = true;
-    for (unsigned long long probe = 0; probe < n; ++probe) {
-      Slot* sp = slots + base + pos;
-      Slot sl = load_slot(sp);
-      if (sl.key == id) { found = (uint32_t)(base + pos); row = sl.row; full = false; break; }
-      if (sl.key == DES_KEY_EMPTY) {
-        if (!insert) { full = false; break; }
-        unsigned long long old = atomicCAS(&sp->key, DES_KEY_EMPTY, id);
-        if (old == DES_KEY_EMPTY || old == id) { found = (uint32_t)(base + pos); full = false; break; }
+  // occurrence j = tile * (256 * PROBE_ILP) + q * 256 + thread: every access of a warp is contiguous
+  const int j0 = blockIdx.x * (256 * PROBE_ILP) + threadIdx.x;
+  unsigned long long id[PROBE_ILP], base[PROBE_ILP], n[PROBE_ILP], pos[PROBE_ILP];
+  uint32_t found[PROBE_ILP], row[PROBE_ILP], seen_fo[PROBE_ILP];
+  bool busy[PROBE_ILP];
+  unsigned long long nmax = 0;
+#pragma unroll
+  for (int q = 0; q < PROBE_ILP; ++q) {
+    const int j = j0 + q * 256;
+    busy[q] = false; found[q] = DES_SLOT_NONE; row[q] = DES_ROW_NONE; id[q] = 0; base[q] = 0; n[q] = 1; pos[q] = 0;
+    seen_fo[q] = DES_ROW_NONE;
+    if (j >= nnz) continue;
+    id[q] = ids[j];
+    uint32_t s;
+    if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S);
+    else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
+    shards[j] = (uint8_t)s;
+    if (id[q] == DES_KEY_EMPTY) { des_raise(meta, DES_ERR_RESERVED_KEY); continue; }
+    base[q] = geom.slot_base[s];
+    n[q] = geom.slot_base[s + 1] - base[q];
+    pos[q] = __umul64hi(des_mix64(id[q] ^ 0x9E3779B97F4A7C15ull), n[q]);
+    busy[q] = true;
+    nmax = max(nmax, n[q]);
+  }
+  for (unsigned long long probe = 0; probe < nmax; ++probe) {
+    Slot sl[PROBE_ILP];
+    bool any = false;
+#pragma unroll
+    for (int q = 0; q < PROBE_ILP; ++q)
+      if (busy[q]) { sl[q] = load_slot(slots + base[q] + pos[q]); any = true; }
+    if (!any) break;
+#pragma unroll
+    for (int q = 0; q < PROBE_ILP; ++q) {
+      if (!busy[q]) continue;
+      Slot* sp = slots + base[q] + pos[q];
+      if (sl[q].key == id[q]) {
+        found[q] = (uint32_t)(base[q] + pos[q]); row[q] = sl[q].row; seen_fo[q] = sl[q].first_occ;
+        busy[q] = false; continue;
       }
-      pos = (pos + 1 == n) ? 0 : pos + 1;
-    }
-    if (full && insert) des_raise(meta, DES_ERR_CAPACITY);
-    if (found != DES_SLOT_NONE && insert) {
-      uint32_t* fo = &slots[found].first_occ;
-      if (*reinterpret_cast<volatile uint32_t*>(fo) > (uint32_t)j) atomicMin(fo, (uint32_t)j);
+      if (sl[q].key == DES_KEY_EMPTY) {
+        if (!insert) { busy[q] = false; continue; }
+        const unsigned long long old = atomicCAS(&sp->key, DES_KEY_EMPTY, id[q]);
+        if (old == DES_KEY_EMPTY || old == id[q]) { found[q] = (uint32_t)(base[q] + pos[q]); busy[q] = false; continue; }
+      }
+      pos[q] = (pos[q] + 1 == n[q]) ? 0 : pos[q] + 1;
+      if (probe + 1 >= n[q]) { busy[q] = false; if (insert) des_raise(meta, DES_ERR_CAPACITY); }   // region is full
     }
   }
-  if (insert) slot_of[j] = found;
-  else rows[j] = row;
+#pragma unroll
+  for (int q = 0; q < PROBE_ILP; ++q) {
+    const int j = j0 + q * 256;
+    if (j >= nnz) continue;
+    // the slot's scratch word as seen by the probe may be stale, but only ever too LARGE:
+    // skipping the atomic when it is already smaller than j is safe
+    if (found[q] != DES_SLOT_NONE && insert && seen_fo[q] > (uint32_t)j)
+      atomicMin(&slots[found[q]].first_occ, (uint32_t)j);
+    if (insert) slot_of[j] = found[q];
+    else rows[j] = row[q];
+  }
 }
 
 // flags: bit0 = first occurrence of its key in the batch, bit1 = key is new.
@@ -269,8 +297,10 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
     return DES_OK;
   }
   const int nblk = (nnz + IB - 1) / IB;
-  probe_claim_kernel<<<nblk, IB, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
-                                          t->cfg.partition, insert, t->slots, t->meta, t->slot_of, b->shards, b->rows);
+  SlotGeom geom;
+  for (uint32_t s = 0; s <= t->S; ++s) geom.slot_base[s] = t->h_slot_base[s];
+  probe_claim_kernel<<<(nnz + 256 * PROBE_ILP - 1) / (256 * PROBE_ILP), 256, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
+                                          t->cfg.partition, insert, t->slots, t->meta, geom, t->slot_of, b->shards, b->rows);
   DES_LAUNCH_CHECK(t, "probe_claim_kernel");
   if (!insert) return DES_OK;
   flag_count_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);

@@ -97,6 +97,14 @@ __host__ __device__ __forceinline__ unsigned long long des_mix64(unsigned long l
   return z;
 }
 
+// h mod S for a small S (<= 64), exactly, with 32-bit divisions only:
+// h = hi * 2^32 + lo  =>  h mod S = ((hi mod S) * (2^32 mod S) + lo mod S) mod S.
+__device__ __forceinline__ uint32_t des_mod_small(unsigned long long h, uint32_t S) {
+  const uint32_t hi = (uint32_t)(h >> 32), lo = (uint32_t)h;
+  const uint32_t two32 = (0xFFFFFFFFu % S + 1u) % S;
+  return ((hi % S) * two32 + lo % S) % S;
+}
+
 // Philox4x32-10 block function.
 __device__ __forceinline__ uint4 des_philox(uint4 c, uint2 key) {
 #pragma unroll
