@@ -198,14 +198,15 @@ class Oracle:
         Gv = np.zeros((U, k), dtype=np.float32)
         gEt = np.zeros((B, F * k), dtype=np.float32)
         Sw = np.zeros(U); Sv = np.zeros((U, k))
+        gW1 = np.zeros((F * k, self.H), dtype=np.float32) if (self.H and gZ is not None) else None
         self.L.orc_backward_update(self.h, C.c_uint32(ops), _p(batch.offsets, C.c_int32),
                                    _p(batch.vals, C.c_float), _p(fi["rows"], C.c_uint32),
                                    _p(fi["shards"], C.c_uint8), _p(fi["uidx"], C.c_uint32),
                                    C.c_int32(B), C.c_int64(U), _p(A, C.c_float), _p(pooled, C.c_float),
                                    _p(gL, C.c_float), _p(gF, C.c_float), _p(gE, C.c_float), _p(gZ, C.c_float),
                                    _p(Gw, C.c_float), _p(Gv, C.c_float), _p(gEt, C.c_float),
-                                   _p(Sw, C.c_double), _p(Sv, C.c_double))
-        return dict(Gw=Gw, Gv=Gv, gE_total=gEt, Sw=Sw, Sv=Sv)
+                                   _p(Sw, C.c_double), _p(Sv, C.c_double), _p(gW1, C.c_float))
+        return dict(Gw=Gw, Gv=Gv, gE_total=gEt, Sw=Sw, Sv=Sv, gW1=gW1)
 
     def read_rows(self, shard, row):
         shard = np.ascontiguousarray(shard, dtype=np.uint8)

@@ -394,12 +394,14 @@ void orc_aggregate(void* p, int32_t B, const double* part_small, const double* p
 // the forward (float32).  Optional outputs: Gw[U], Gv[U][k] (the summed
 // gradients, rounded to float32), gE_total[B][F*k], and Sw[U], Sv[U][k]: the sums
 // of the ABSOLUTE values of the same per-occurrence terms (the scale against
-// which a float32 summation error is measured when the terms cancel).
+// which a float32 summation error is measured when the terms cancel); gW1[F*k][H]:
+// the first layer's weight gradient before the optimizer.
 void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const float* vals,
                          const uint32_t* rows, const uint8_t* shards, const uint32_t* uidx,
                          int32_t B, int64_t U, const float* A, const float* pooled,
                          const float* gL, const float* gF, const float* gE, const float* gZ,
-                         float* Gw_out, float* Gv_out, float* gE_total_out, double* Sw_out, double* Sv_out) {
+                         float* Gw_out, float* Gv_out, float* gE_total_out, double* Sw_out, double* Sv_out,
+                         float* gW1_out) {
   Table* t = (Table*)p;
   const uint32_t F = t->F, k = t->k, H = t->H;
   const size_t FK = (size_t)F * k;
@@ -458,6 +460,7 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
         double g = 0;
         for (int32_t b = 0; b < B; ++b)
           g += (double)bf16_round(pooled[(size_t)b * FK + i]) * (double)gZ[(size_t)b * H + h2];
+        if (gW1_out) gW1_out[i * H + h2] = (float)g;
         apply_opt(*t, t->W1[i * H + h2], t->accW1[i * H + h2], g);
       }
   }

@@ -8,10 +8,16 @@
 // accumulator sees P_0, P_1, ... in shard order; with `part_dense` the K range
 // of every shard is a separate slice of the launch and P_s is stored.
 //
-// This is the plain shared-memory tiled version (64x64x16 tiles, 4x4 outputs
-// per thread, CUDA cores): the flops of the step are tiny next to its memory
-// traffic.
+// Fast path: the three GEMMs (Z = V W, gE = gZ W1^T, gW1 = V^T gZ) run on the
+// tcgen05 tensor cores (des_tc_gemm*.cu: bf16 operands by TMA, fp32 accumulators
+// in tensor memory) after a float -> bf16 pass over V and gZ.  The kernel in
+// this file is the plain shared-memory tiled CUDA-core version (64x64x16 tiles,
+// 4x4 outputs per thread): it serves the materialised per-shard partials P_s
+// (slices of the K range) and shapes the TMA path cannot take (a K or N extent
+// that is not a multiple of 8).
 #include "des_internal.cuh"
+#define DES_TC_GEMM_DECL_ONLY
+#include "des_tc_gemm.cuh"
 
 #define TM 64
 #define TN 64
@@ -143,8 +149,31 @@ __global__ void w1_update_kernel(const float* __restrict__ part, int slices, siz
   }
 }
 
+__global__ void cvt_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
+  size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4, st = (size_t)gridDim.x * blockDim.x * 4;
+  for (; i + 3 < n; i += st) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(dst + i) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+  }
+}
+
+static des_status_t to_bf16(des_table* t, const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st) {
+  cvt_bf16_kernel<<<t->sm_count * 4, 256, 0, st>>>(src, dst, n);     // n is a multiple of 4 (k and H are)
+  DES_LAUNCH_CHECK(t, "cvt_bf16_kernel");
+  return DES_OK;
+}
+
 des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float* Z, float* part_dense,
                                 const float* part_pooled, cudaStream_t st) {
+  if (!part_dense && t->use_tc) {
+    const int FK = t->F * t->k;
+    des_status_t e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
+    if (e != DES_OK) return e;
+    const int rc = des_tc_gemm_fwd(B, t->H, FK, t->pooled_b, t->W1b, Z, Z, 0.f, t->gemm_ws, t->gemm_ws_bytes, st);
+    if (rc == 0) { DES_LAUNCH_CHECK(t, "tc_gemm_fwd"); return DES_OK; }
+    if (rc != 1) return DES_ERR_CUDA;
+  }
   GemmArgs g; memset(&g, 0, sizeof(g));
   g.M = B; g.N = t->H; g.K = t->F * t->k; g.A32 = pooled; g.Bb = t->W1b; g.k_emb = t->k; g.FK = g.K; g.H = t->H;
   g.meta = t->meta; g.partition = t->cfg.partition; g.S = t->S; g.F = t->F;
@@ -163,6 +192,25 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
 des_status_t des_dense1_backward(des_table* t, const float* pooled, const float* gE, const float* gZ,
                                  float* gE_work, int B, cudaStream_t st) {
   const int FK = t->F * t->k;
+  if (t->use_tc) {
+    des_status_t e = to_bf16(t, gZ, t->gZ_b, (size_t)B * t->H, st);
+    if (e == DES_OK) e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
+    if (e != DES_OK) return e;
+    const int rc1 = des_tc_gemm_dgrad(B, FK, t->H, t->gZ_b, t->W1b, gE ? gE : gE_work, gE_work, gE ? 1.f : 0.f,
+                                      t->gemm_ws, t->gemm_ws_bytes, st);
+    if (rc1 == 0) {
+      DES_LAUNCH_CHECK(t, "tc_gemm_dgrad");
+      const int rc2 = des_tc_gemm_wgrad(FK, t->H, B, t->pooled_b, t->gZ_b, t->gW1_part, t->gW1_part, 0.f, t->gemm_ws,
+                                        t->gemm_ws_bytes, st);
+      if (rc2 != 0) return DES_ERR_CUDA;           // same alignment rules as the dgrad: cannot differ
+      DES_LAUNCH_CHECK(t, "tc_gemm_wgrad");
+      w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, 1, (size_t)FK * t->H, t->W1, t->accW1, t->W1b,
+                                                        t->cfg.optimizer, t->cfg.lr, t->cfg.eps);
+      DES_LAUNCH_CHECK(t, "w1_update_kernel");
+      return DES_OK;
+    }
+    if (rc1 != 1) return DES_ERR_CUDA;
+  }
   {  // gE_work = gE + gZ W1^T
     GemmArgs g; memset(&g, 0, sizeof(g));
     g.M = B; g.N = FK; g.K = t->H; g.A32 = gZ; g.Bb = t->W1b; g.add = gE; g.out = gE_work;

@@ -25,6 +25,7 @@
 #include "des_internal.cuh"
 
 #define FW_UNROLL 8
+#define SP_UNROLL 4
 
 __global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
@@ -101,10 +102,10 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
   const int lo = __ldg(seg_off + (size_t)b * (S + 1) + s), hi = __ldg(seg_off + (size_t)b * (S + 1) + s + 1);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float m1lr = 0.f, m2 = 0.f;
-  for (int i0 = lo; i0 < hi; i0 += FW_UNROLL) {
-    float4 v[FW_UNROLL]; float2 tl[FW_UNROLL]; float x[FW_UNROLL];
+  for (int i0 = lo; i0 < hi; i0 += SP_UNROLL) {
+    float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
 #pragma unroll
-    for (int u = 0; u < FW_UNROLL; ++u) {
+    for (int u = 0; u < SP_UNROLL; ++u) {
       v[u] = make_float4(0.f, 0.f, 0.f, 0.f); tl[u] = make_float2(0.f, 0.f); x[u] = 1.f;
       if (i0 + u < hi) {
         const float* wr = W + (size_t)__ldg(grow_sorted + i0 + u) * stride;
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
       }
     }
 #pragma unroll
-    for (int u = 0; u < FW_UNROLL; ++u) {
+    for (int u = 0; u < SP_UNROLL; ++u) {
       if (HAS_VALS) {
         acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
         m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];

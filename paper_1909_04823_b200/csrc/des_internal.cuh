@@ -66,6 +66,9 @@ struct des_table {
   float* W1; float* accW1;           // [F*k][H] fp32 master and state
   __nv_bfloat16* W1b;                // bf16 shadow
   float* gW1_part; int gw1_splits;   // [splits][F*k][H]
+  int use_tc;                        // tensor-core GEMM path usable for this table's shapes
+  __nv_bfloat16 *pooled_b, *gZ_b;    // bf16 copies of V [max_batch][F*k] and gZ [max_batch][H]
+  void* gemm_ws; size_t gemm_ws_bytes;
   // host-step staging
   int32_t* st_offsets; unsigned long long* st_ids; float* st_vals;
   uint32_t* st_rows; uint8_t* st_shards; uint32_t* st_uidx; uint32_t* st_uniq_rows; uint32_t* st_n_uniq;

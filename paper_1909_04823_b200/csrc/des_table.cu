@@ -88,7 +88,7 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
                   t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc,
-                  t->W1, t->accW1, t->W1b, t->gW1_part, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
+                  t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
   for (void* p : ptrs) dfree(t->cfg, p);
   if (t->prof_ev) { for (int i = 0; i < DES_PROF_MAX; ++i) cudaEventDestroy(t->prof_ev[i]); delete[] t->prof_ev; }
@@ -175,6 +175,12 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
     A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
     t->gw1_splits = 32;
     A(t->gW1_part, (size_t)t->gw1_splits * FKH * 4);
+    // TMA needs 16-byte rows: every contiguous extent of a bf16 operand a multiple of 8
+    t->use_tc = ((t->F * t->k) % 8 == 0) && (t->H % 8 == 0);
+    A(t->pooled_b, (size_t)t->max_batch * t->F * t->k * 2);
+    A(t->gZ_b, (size_t)t->max_batch * t->H * 2);
+    t->gemm_ws_bytes = 8u << 20;
+    A(t->gemm_ws, t->gemm_ws_bytes);
   }
   if (!ok) { des_table_destroy(t); return DES_ERR_CUDA; }
   bool cu = true;

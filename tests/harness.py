@@ -157,7 +157,7 @@ class Pair:
                     extra = self.w.lr * dG
                 else:
                     acc = ref["acc_" + name].astype(np.float64)
-                    extra = self.w.lr * dG / (np.sqrt(acc) + self.w.eps)
+                    extra = self.w.lr * np.minimum(2.0, 2.0 * dG / (np.sqrt(acc) + self.w.eps))
             (close_gemm if gemm else close32)(g, ref[name], f"{what}.{name}", extra=extra)
         return ref
 
@@ -252,8 +252,17 @@ class Pair:
         W1o = None
         if ops & OP_DENSE1:
             close_gemm(gE_work.cpu().numpy(), ob["gE_total"], "gE_total")
-            W1o, _ = self.o.dense1_get()
-            close_gemm(self.t.dense1_get().cpu().numpy(), W1o, "W1")
+            W1o, accW1o = self.o.dense1_get()
+            # same reasoning as for the rows: a 2e-2-relative error of the weight gradient, pushed
+            # through one optimizer application (Adagrad divides by sqrt(acc))
+            Gk = ob["gW1"].astype(np.float64)
+            dG = 2e-2 * np.abs(Gk) + 1e-3 * max(float(np.abs(Gk).max()), 1e-30)
+            if w.optimizer == synth.OPT_SGD:
+                extra = w.lr * dG
+            else:
+                # G / sqrt(acc) is bounded by 1 and, for dG below |G|, moves by at most ~2 dG / sqrt(acc)
+                extra = w.lr * np.minimum(2.0, 2.0 * dG / (np.sqrt(accW1o.astype(np.float64)) + w.eps))
+            close_gemm(self.t.dense1_get().cpu().numpy(), W1o, "W1", extra=extra)
         ref = self.compare_rows(fi, db, gemm=gemm, what="updated rows", G=ob)
         if self.resync:
             U = fi["U"]
