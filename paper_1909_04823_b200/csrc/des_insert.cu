@@ -272,17 +272,17 @@ __global__ void __launch_bounds__(IB) resolve_kernel(int nnz, const Slot* __rest
   uidx[j] = (row == DES_ROW_NONE) ? DES_ROW_NONE : u;
 }
 
-__global__ void __launch_bounds__(IB) finish_kernel(int nnz, int S, Slot* slots, const uint32_t* __restrict__ uslot,
-                                                    DevMeta* meta, uint32_t* n_uniq_out) {
-  int u = blockIdx.x * IB + threadIdx.x;
+__global__ void __launch_bounds__(256) finish_kernel(int S, Slot* slots, const uint32_t* __restrict__ uslot,
+                                                     DevMeta* meta, uint32_t* n_uniq_out) {
   const uint32_t U = meta->n_uniq;
-  if (u < nnz && (uint32_t)u < U) slots[uslot[u]].first_occ = DES_ROW_NONE;
-  if (blockIdx.x == gridDim.x - 1 && threadIdx.x < S) {
-    // the last block is the only writer of n_rows; other blocks never read it
+  for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x)
+    slots[uslot[u]].first_occ = DES_ROW_NONE;
+  if (blockIdx.x == 0 && threadIdx.x < S) {
+    // block 0 is the only writer of n_rows; no other block of this kernel reads it
     uint32_t n = meta->n_rows[threadIdx.x] + meta->new_total[threadIdx.x];
     meta->n_rows[threadIdx.x] = min(n, meta->row_cap[threadIdx.x]);
   }
-  if (u == 0) *n_uniq_out = U;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *n_uniq_out = U;
 }
 
 extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b, int insert, void* stream) {
@@ -316,7 +316,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   DES_LAUNCH_CHECK(t, "apply_first_kernel");
   resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
   DES_LAUNCH_CHECK(t, "resolve_kernel");
-  finish_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->uslot, t->meta, b->n_uniq);
+  finish_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->S, t->slots, t->uslot, t->meta, b->n_uniq);
   DES_LAUNCH_CHECK(t, "finish_kernel");
   return DES_OK;
 }

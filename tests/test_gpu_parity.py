@@ -239,3 +239,11 @@ def test_multi_step_without_resync_stays_close():
             b = st.next_batch()
     finally:
         p.close()
+
+
+def test_cfg5_multihot_million_occurrences():
+    # a batch above one million occurrences: the backward samples its hot-key counts (1 in 2)
+    # instead of counting every occurrence, and every kernel runs several waves
+    w = synth.config(5).scaled(batch=640, vocab=50000, prepopulate=50000, init_scale=0.05)
+    assert synth.Stream(w).next_batch().nnz > (1 << 20)
+    _run(w, 2, max_rows=120000, prepop=1)
