@@ -41,13 +41,15 @@ def log(*a):
 
 
 def measured_peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, "measured" | "fallback")"""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         try:
-            return float(json.load(open(p))["hbm_gbs"]), "measured"
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", 1400.0)), "measured"
         except Exception:
             pass
-    return 6650.0, "fallback"
+    return 6650.0, 1400.0, "fallback"
 
 
 def rows_per_shard(w, cap_total):
@@ -177,6 +179,20 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
+# profiles/memory_counters_cfg5_batch_small_table.md: the benchmark's own batch on a 4e6-key table (the
+# 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
+# the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
+NCU_DRAM_TRAFFIC = {
+    ("cfg5", "grad_scatter_kernel"): 1949e6,
+    ("cfg5", "shard_partials_kernel"): 1071e6,
+    ("cfg5", "pool_kernel"): 1207e6,
+    ("cfg5", "update_rows_kernel"): 1936e6,
+    ("cfg5", "probe_claim_kernel"): 599e6,
+    ("cfg5", "route_kernel"): 697e6,
+}
+
+
 def kernel_bytes(name, st):
     """Algorithmic bytes one launch of `name` must move (what the method needs,
     each datum once; see the design notes for the derivation)."""
@@ -209,6 +225,15 @@ def kernel_bytes(name, st):
         return 2 * row * R
     if name == "update_rows_kernel":
         return U * (2 * row + 2 * row * (1 + state) + 8)
+    if name == "cvt_bf16_kernel":          # three launches per step: pooled (forward), gZ and pooled (backward)
+        return 6 * (2 * B * F * k + B * st["H"]) // 3
+    return None
+
+
+def kernel_flops(name, st):
+    """Dense flops of one launch (tensor-core GEMMs of the row-split first layer)."""
+    if name in ("tc_gemm_fwd", "tc_gemm_dgrad", "tc_gemm_wgrad"):
+        return 2 * st["B"] * st["F"] * st["k"] * st["H"]
     return None
 
 
@@ -270,7 +295,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
-    hbm_peak, peak_kind = measured_peaks()
+    hbm_peak, tc_peak, peak_kind = measured_peaks()
 
     # ---- size the table for the memory that is actually free
     free_b, total_b = torch.cuda.mem_get_info()
@@ -372,21 +397,32 @@ def main():
     for name, ms in prof:
         a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += ms
     U = int(dbs[0].n_uniq.item())
-    stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, U=U, ops=w.ops, adagrad=(w.optimizer == synth.OPT_ADAGRAD),
-                 rep_rows=0)
+    stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, H=H, U=U, ops=w.ops,
+                 adagrad=(w.optimizer == synth.OPT_ADAGRAD), rep_rows=0)
     tot_k = sum(v[1] for v in per.values()) or 1.0
     kernels = []
     for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
         by = kernel_bytes(name, stats)
+        fl = kernel_flops(name, stats)
         avg = ms / n_
         kernels.append({"kernel": name, "launches": n_, "ms_per_launch": round(avg, 4), "share": round(ms / tot_k, 4),
-                        "alg_gbs": None if by is None else round(by / avg / 1e6, 1)})
-    top = kernels[0] if kernels else None
+                        "alg_gbs": None if by is None else round(by / avg / 1e6, 1),
+                        "tflops": None if fl is None else round(fl / avg / 1e9, 1)})
+    # the kernel with the largest share of the timed region that has a byte / flop model
     roofline = None
-    if top and top["alg_gbs"] is not None:
-        roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
-                    "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4), "traffic": None,
-                    "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
+    for top in kernels:
+        if top["alg_gbs"] is not None:
+            roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
+                        "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4),
+                        "traffic": NCU_DRAM_TRAFFIC.get((w.name.split("_")[0], top["kernel"])),
+                        "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
+            break
+        if top["tflops"] is not None:
+            roofline = {"bound": "tensor", "kernel": top["kernel"], "achieved": top["tflops"], "peak": tc_peak,
+                        "unit": "TFLOP/s", "frac": round(top["tflops"] / tc_peak, 4), "traffic": None,
+                        "peak_kind": f"of {peak_kind} (sustained bf16)", "ms_per_launch": top["ms_per_launch"],
+                        "share": top["share"]}
+            break
     step_bytes = sum((kernel_bytes(kk["kernel"], stats) or 0) * kk["launches"] for kk in kernels) / args.steps
 
     # ---- end to end from pinned host buffers

@@ -35,7 +35,7 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
 
 struct SlotGeom { unsigned long long slot_base[DES_MAX_SHARDS + 1]; };   // kernel parameter: constant-bank reads
 
-__global__ void __launch_bounds__(256) probe_claim_kernel(
+__global__ void __launch_bounds__(256, 4) probe_claim_kernel(
     const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
     int S, int F, int partition, int insert, Slot* slots, DevMeta* meta, const __grid_constant__ SlotGeom geom,
     uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards, uint32_t* __restrict__ rows) {
