@@ -247,6 +247,8 @@ def main():
     ap.add_argument("--vocab", type=int, default=0, help="override the number of pre-populated keys (config 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--fused", action="store_true",
+                    help="use des_forward_fused (per-shard partials kept on chip) instead of partials + aggregate")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -360,8 +362,11 @@ def main():
     def step(i):
         db = dbs[i % len(dbs)]
         t.find_or_insert(db, True)
-        t.forward_partials(w.ops, db, part_small, pooled)
-        t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
+        if args.fused:
+            t.forward_fused(w.ops, db, None, pooled, out_small, Z)
+        else:
+            t.forward_partials(w.ops, db, part_small, pooled)
+            t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
         t.backward_update(w.ops, db, out_small, pooled, Z, gd.get("gL"), gd.get("gF"), gE, gZ, gE_work)
 
     def barrier():
@@ -474,6 +479,8 @@ def main():
                            "nnz_per_step": batches[0].nnz, "unique_keys_per_step": U, "table_keys": sum(t.size()),
                            "ops": w.ops, "optimizer": "adagrad" if w.optimizer else "sgd",
                            "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+                           "forward": "fused (per-shard partials on chip)" if args.fused else
+                                      "per-shard partials materialised, then aggregated",
                            "l2": "inputs larger than L2 (no flush)" if batches[0].nnz * 8 > 126e6 else
                                  "small workload: inputs fit in L2, two batches alternate, no flush"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),

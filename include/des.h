@@ -192,6 +192,16 @@ des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_
 des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* batch,
                            const des_partials_t* part, const des_outputs_t* out, void* stream);
 
+/* des_forward_partials + des_aggregate in one call, with the per-shard partial
+ * results of LR / FM kept on chip: every sample's partials are formed shard by
+ * shard in registers, aggregated in the same fixed shard order and passed
+ * through F without ever being written (Algorithm 1 with the aggregation made
+ * an on-chip reduction).  Results are bit-identical to the two-call path.
+ * part->part_small may be NULL (or given, to receive the partials as well);
+ * part->part_pooled and part->part_dense must be NULL. */
+des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* batch,
+                               const des_partials_t* part, const des_outputs_t* out, void* stream);
+
 /* Mirror of the forward (Section 3.2): per-occurrence gradients
  *   g_w(j) = x_j gL[b],  g_v(j) = x_j ( gF[b] (A[b] - v_j x_j) + gE[b][f] ),
  * summed per unique key, then one SGD / Adagrad application per key with the

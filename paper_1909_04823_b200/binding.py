@@ -24,7 +24,7 @@ STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "
           7: "DES_ERR_TOO_LARGE"}
 
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
-           "des_aggregate", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_forward_noalloc", "des_table_status",
+           "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_step_host", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
 
@@ -88,6 +88,8 @@ def load():
                                            C.POINTER(des_partials_t), C.c_void_p]
         L.des_aggregate.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
                                     C.POINTER(des_outputs_t), C.c_void_p]
+        L.des_forward_fused.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
+                                        C.POINTER(des_outputs_t), C.c_void_p]
         L.des_backward_update.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
                                           C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
         L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -217,6 +219,13 @@ class Table:
         o = des_outputs_t(_ptr(out_small), _ptr(out_pooled if out_pooled is not None else pooled), _ptr(Z))
         self._check(self.L.des_aggregate(self.h, ops, C.byref(cb), C.byref(p), C.byref(o), _stream()),
                     "des_aggregate")
+
+    def forward_fused(self, ops, batch, part_small=None, pooled=None, out_small=None, Z=None):
+        cb = batch.c()
+        p = des_partials_t(_ptr(part_small), _ptr(pooled), None, None)
+        o = des_outputs_t(_ptr(out_small), _ptr(pooled), _ptr(Z))
+        self._check(self.L.des_forward_fused(self.h, ops, C.byref(cb), C.byref(p), C.byref(o), _stream()),
+                    "des_forward_fused")
 
     def backward_update(self, ops, batch, out_small=None, pooled=None, Z=None, gL=None, gF=None, gE=None,
                         gZ=None, gE_work=None):

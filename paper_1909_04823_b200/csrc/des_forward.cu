@@ -14,11 +14,12 @@
 //                 row of every occurrence in shard-major order, the segment
 //                 bounds [B][S+1], and the same rows in CSR order for pooling.
 //  shard_partials_kernel   one group of G = k/4 lanes (rounded up to a power of
-//                 two) per (sample, shard) segment: it streams the segment's
-//                 rows with 16-byte loads, FW_UNROLL in flight, and keeps
-//                 M_1, M_1^lr, M_2 in registers until the segment ends — no
-//                 shared memory, no atomics, sums in CSR order (deterministic).
-//                 M_2 uses the |v|^2 cached in the row's 16-byte tail.
+//                 two) per sample walks the sample's (sample, shard) segments in
+//                 shard order: it streams a segment's rows with 16-byte loads,
+//                 SP_UNROLL in flight, and keeps M_1, M_1^lr, M_2 in registers
+//                 until the segment ends — no shared memory, no atomics, sums in
+//                 CSR order (deterministic).  M_2 uses the |v|^2 cached in the
+//                 row's 16-byte tail.  Fused variant: (+) over shards and F on chip.
 //  pool_kernel    one group per bag: sum pooling of the latent vectors in
 //                 registers.  The per-shard pooled partial [S][B][F*k] is only
 //                 materialised (with atomics) when the caller asks for it.
@@ -87,48 +88,76 @@ __global__ void __launch_bounds__(256) route_kernel(
   }
 }
 
-template <int G, bool HAS_VALS>
+// One group of G lanes per SAMPLE walks the sample's S segments in shard order.
+// Every group has the same amount of work (a sample's occurrences), whatever the
+// skew between shards.  part_small (optional) receives each segment's partial
+// sums as soon as the segment ends; with FUSED the aggregation (+) over shards
+// and the substitution operator F are applied on chip, in the same shard order
+// and with the same arithmetic as aggregate_small_kernel, and out_small is
+// written directly — the per-shard partials then never touch memory.
+template <int G, bool HAS_VALS, bool FUSED>
 __global__ void __launch_bounds__(256) shard_partials_kernel(
     const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted, const int32_t* __restrict__ seg_off,
-    int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small) {
+    int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small,
+    float* __restrict__ out_small) {
   const int K4 = k >> 2, stride = k + 4;
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long seg = t / G;                       // = b * S + s
+  const long long b = t / G;
   const int c4 = (int)(t % G);
-  if (seg >= (long long)B * S) return;
-  const int b = (int)(seg / S), s = (int)(seg % S);
-  const bool col = c4 < K4, lead = c4 == 0;
-  if (!col && !lead) return;
-  const int lo = __ldg(seg_off + (size_t)b * (S + 1) + s), hi = __ldg(seg_off + (size_t)b * (S + 1) + s + 1);
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float m1lr = 0.f, m2 = 0.f;
-  for (int i0 = lo; i0 < hi; i0 += SP_UNROLL) {
-    float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
+  const bool live = b < B;
+  const bool col = live && c4 < K4, lead = live && c4 == 0;
+  const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 A = zero4; float R = 0.f, Q = 0.f;            // FUSED: (+)M_1, (+)M_1^lr, (+)M_2
+  if (col || lead) {
+    const int32_t* so = seg_off + (size_t)b * (S + 1);
+    int hi = __ldg(so);
+    for (int s = 0; s < S; ++s) {
+      const int lo = hi;
+      hi = __ldg(so + s + 1);
+      float4 acc = zero4;
+      float m1lr = 0.f, m2 = 0.f;
+      for (int i0 = lo; i0 < hi; i0 += SP_UNROLL) {
+        float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
 #pragma unroll
-    for (int u = 0; u < SP_UNROLL; ++u) {
-      v[u] = make_float4(0.f, 0.f, 0.f, 0.f); tl[u] = make_float2(0.f, 0.f); x[u] = 1.f;
-      if (i0 + u < hi) {
-        const float* wr = W + (size_t)__ldg(grow_sorted + i0 + u) * stride;
-        if (HAS_VALS) x[u] = __ldg(x_sorted + i0 + u);
-        if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
-        if (lead) tl[u] = __ldg(reinterpret_cast<const float2*>(wr + k));      // (w, |v|^2)
-      }
-    }
+        for (int u = 0; u < SP_UNROLL; ++u) {
+          v[u] = zero4; tl[u] = make_float2(0.f, 0.f); x[u] = 1.f;
+          if (i0 + u < hi) {
+            const float* wr = W + (size_t)__ldg(grow_sorted + i0 + u) * stride;
+            if (HAS_VALS) x[u] = __ldg(x_sorted + i0 + u);
+            if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
+            if (lead) tl[u] = __ldg(reinterpret_cast<const float2*>(wr + k));      // (w, |v|^2)
+          }
+        }
 #pragma unroll
-    for (int u = 0; u < SP_UNROLL; ++u) {
-      if (HAS_VALS) {
-        acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
-        m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
-      } else {
-        acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
-        m1lr += tl[u].x; m2 += tl[u].y;
+        for (int u = 0; u < SP_UNROLL; ++u) {
+          if (HAS_VALS) {
+            acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
+            m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
+          } else {
+            acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+            m1lr += tl[u].x; m2 += tl[u].y;
+          }
+        }
       }
+      if (!fm) { acc = zero4; m2 = 0.f; }
+      if (!lr) m1lr = 0.f;
+      if (part_small) {
+        float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
+        if (col) dst[c4] = acc;
+        if (lead) dst[K4] = make_float4(m1lr, m2, 0.f, 0.f);
+      }
+      if (FUSED) { A.x += acc.x; A.y += acc.y; A.z += acc.z; A.w += acc.w; R += m1lr; Q += m2; }
     }
   }
-  const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
-  float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
-  if (col) dst[c4] = fm ? acc : make_float4(0.f, 0.f, 0.f, 0.f);
-  if (lead) dst[K4] = make_float4(lr ? m1lr : 0.f, fm ? m2 : 0.f, 0.f, 0.f);
+  if (FUSED) {
+    double aa = (double)A.x * A.x + (double)A.y * A.y + (double)A.z * A.z + (double)A.w * A.w;
+#pragma unroll
+    for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
+    float4* o = reinterpret_cast<float4*>(out_small + (size_t)(live ? b : 0) * stride);
+    if (col) o[c4] = A;
+    if (lead) o[K4] = make_float4(R, fm ? (float)(0.5 * aa - 0.5 * (double)Q) : 0.f, Q, 0.f);
+  }
 }
 
 template <int G, bool HAS_VALS, bool MATERIALISE>
@@ -210,13 +239,15 @@ __global__ void reduce_shards_kernel(const float* __restrict__ part, size_t per_
 
 static int group_for(int k) { int K4 = k / 4, G = 1; while (G < K4) G <<= 1; return G; }
 
-extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_t* b,
-                                             const des_partials_t* part, void* stream) {
+// shared by des_forward_partials (fused_out == NULL) and des_forward_fused
+static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t* b, const des_partials_t* part,
+                                 float* fused_out, void* stream) {
   des_status_t st = des_check_batch(t, b, 0);
   if (st != DES_OK) return st;
   if (!part || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
   const bool small = ops & (DES_OP_LR | DES_OP_FM), pool = ops & (DES_OP_POOL | DES_OP_DENSE1);
-  if (small && !part->part_small) return DES_ERR_INVALID_ARG;
+  if (small && !part->part_small && !fused_out) return DES_ERR_INVALID_ARG;
+  if (!small) fused_out = nullptr;
   if (pool && !part->pooled) return DES_ERR_INVALID_ARG;
   if ((ops & DES_OP_DENSE1) && !t->H) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
@@ -235,13 +266,16 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   route_kernel<<<(B + 7) / 8 < t->sm_count * 8 ? (B + 7) / 8 : t->sm_count * 8, 256, 0, cs>>>(
       b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, grow_csr, grow_sorted, x_sorted, t->seg_off);
   DES_LAUNCH_CHECK(t, "route_kernel");
-  if (ps) {
-    const long long threads = (long long)B * t->S * G;
+  if (ps || fused_out) {
+    const long long threads = (long long)B * G;
     const unsigned grid = (unsigned)((threads + 255) / 256);
-#define SP(GG) do { if (b->vals) shard_partials_kernel<GG, true><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, t->k, ops, t->W, ps); \
-                    else shard_partials_kernel<GG, false><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, t->k, ops, t->W, ps); } while (0)
+#define SP3(GG, HV, FU) shard_partials_kernel<GG, HV, FU><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, \
+                                                                              t->k, ops, t->W, ps, fused_out)
+#define SP(GG) do { if (fused_out) { if (b->vals) SP3(GG, true, true); else SP3(GG, false, true); } \
+                    else { if (b->vals) SP3(GG, true, false); else SP3(GG, false, false); } } while (0)
     switch (G) { case 1: SP(1); break; case 2: SP(2); break; case 4: SP(4); break; case 8: SP(8); break; default: SP(16); }
 #undef SP
+#undef SP3
     DES_LAUNCH_CHECK(t, "shard_partials_kernel");
   }
   if (pl) {
@@ -258,6 +292,23 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   }
   return DES_OK;
 }
+extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_t* b,
+                                             const des_partials_t* part, void* stream) {
+  return forward_impl(t, ops, b, part, nullptr, stream);
+}
+
+extern "C" des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* b,
+                                          const des_partials_t* part, const des_outputs_t* out, void* stream) {
+  if (!t || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
+  if ((ops & (DES_OP_LR | DES_OP_FM)) && !out->out_small) return DES_ERR_INVALID_ARG;
+  if (part->part_pooled || part->part_dense) return DES_ERR_INVALID_ARG;      // materialised partials: use the two-call path
+  des_status_t st = forward_impl(t, ops, b, part, out->out_small, stream);
+  if (st != DES_OK) return st;
+  // what is left of the aggregation: hand the pooled block over and run the first layer
+  const uint32_t rest = ops & ~(uint32_t)(DES_OP_LR | DES_OP_FM);
+  return rest ? des_aggregate(t, rest, b, part, out, stream) : DES_OK;
+}
+
 extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* b, const des_partials_t* part,
                                       const des_outputs_t* out, void* stream) {
   if (!t || !b || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;

@@ -196,6 +196,20 @@ class Pair:
         self.t.aggregate(ops, db, part_small, pooled, part_pooled, part_dense, out_small, pooled, Z)
         torch.cuda.synchronize()
         assert self.t.status() == 0
+        if not materialise:
+            # the fused call (partials kept on chip) must reproduce the two-call path bit for bit
+            f_small = torch.full((B, k + 4), float("nan"), device=dev)
+            f_pooled = torch.full((B, F * k), float("nan"), device=dev)
+            f_Z = torch.full((B, max(H, 1)), float("nan"), device=dev)
+            self.t.forward_fused(ops, db, None, f_pooled, f_small, f_Z)
+            torch.cuda.synchronize()
+            assert self.t.status() == 0
+            if ops & (OP_LR | OP_FM):
+                assert torch.equal(f_small.view(torch.int32), out_small.view(torch.int32)), "fused out_small"
+            if ops & (OP_POOL | OP_DENSE1):
+                assert torch.equal(f_pooled.view(torch.int32), pooled.view(torch.int32)), "fused pooled"
+            if ops & OP_DENSE1:
+                assert torch.equal(f_Z.view(torch.int32), Z.view(torch.int32)), "fused Z"
         ps = part_small.cpu().numpy()
         osm = out_small.cpu().numpy()
         if ops & OP_FM:
