@@ -75,7 +75,12 @@ enum { DES_OP_LR = 1, DES_OP_FM = 2, DES_OP_POOL = 4, DES_OP_DENSE1 = 8 };
  * balances", Section 4.2); FIELD = field mod S (Section 5, "Large-scale
  * Sparse Features"; required for a weight-disjoint row split, Section 4.3). */
 enum { DES_PART_HASH = 0, DES_PART_FIELD = 1 };
-enum { DES_OPT_SGD = 0, DES_OPT_ADAGRAD = 1 };
+/* optimizer of the latent vectors and of the first dense layer; the order-1
+ * (linear) weights follow it unless lin_optimizer says FTRL (Section 6,
+ * "Parameter Settings": FTRL for order-1 components, AdaGrad or Adam for the
+ * embedding and DNN components). */
+enum { DES_OPT_SGD = 0, DES_OPT_ADAGRAD = 1, DES_OPT_ADAM = 2 };
+enum { DES_LIN_SAME = 0, DES_LIN_FTRL = 1 };
 
 #define DES_KEY_EMPTY 0xFFFFFFFFFFFFFFFFull /* reserved id                         */
 #define DES_ROW_NONE  0xFFFFFFFFu           /* "no row": missing key / failed insert */
@@ -98,6 +103,15 @@ typedef struct {
   float    lr, eps, init_acc; /* theta -= lr*G            (SGD)
                                  a += G*G; theta -= lr*G/(sqrt(a)+eps)   (Adagrad),
                                  a starts at init_acc                                */
+  uint32_t lin_optimizer;/* DES_LIN_*: optimizer of the order-1 weights                */
+  float    beta1, beta2; /* Adam (lazy: only the keys of the batch move; one global step
+                            count t per backward call):  m = b1 m + (1-b1) G;
+                            v = b2 v + (1-b2) G*G;
+                            theta -= lr * (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + eps)       */
+  float    ftrl_alpha, ftrl_beta, ftrl_l1, ftrl_l2; /* FTRL-Proximal per coordinate:
+                            sigma = (sqrt(n+G*G) - sqrt(n))/alpha; z += G - sigma*w;
+                            n += G*G; w = |z| <= l1 ? 0 :
+                            -(z - sign(z) l1) / ((beta + sqrt(n))/alpha + l2)           */
   int64_t  max_nnz;      /* largest nnz of any batch (sizes the workspace)            */
   int32_t  max_batch;    /* largest B of any batch                                    */
   int64_t  max_uniq;     /* largest number of distinct keys in one batch (sizes the
@@ -214,6 +228,12 @@ des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t
 /* ---- first dense layer weights W1 [F*k][H], fp32 master (Section 4.3) ----- */
 des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream);
 des_status_t des_dense1_get(des_table_t* t, float* d_W1, void* stream);
+/* Optimizer state of W1, same shape as W1: state1 = Adagrad accumulator or Adam
+ * first moment, state2 = Adam second moment.  Either pointer may be NULL; a
+ * non-NULL pointer for a state the configured optimizer does not keep is
+ * DES_ERR_INVALID_ARG.  Device pointers; copies are enqueued on `stream`. */
+des_status_t des_dense1_get_state(des_table_t* t, float* d_state1, float* d_state2, void* stream);
+des_status_t des_dense1_set_state(des_table_t* t, const float* d_state1, const float* d_state2, void* stream);
 
 /* Row-split first layer for callers that must not allocate.  (The paper has no
  * counterpart: this is a packaging variant of des_aggregate's DENSE1 step, same
@@ -271,6 +291,16 @@ des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_global_rows, 
 des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
                                   const float* d_emb, const float* d_lin, const float* d_acc_emb,
                                   const float* d_acc_lin, void* stream);
+
+/* Second optimizer-state slot of the same rows (what des_table_read_rows /
+ * write_rows do for the first): Adam's v of the latent vectors [n][k] and the
+ * second state word of the linear weight [n] (Adam's v, FTRL's z; the first
+ * word — Adagrad's accumulator, Adam's m, FTRL's n — is `acc_lin`).  Any
+ * pointer may be NULL; parts the configured optimizers do not keep read as 0. */
+des_status_t des_table_read_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                   float* d_acc2_emb, float* d_lin2, void* stream);
+des_status_t des_table_write_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                    const float* d_acc2_emb, const float* d_lin2, void* stream);
 
 /* ---- whole step from host buffers ---------------------------------------- */
 

@@ -48,7 +48,8 @@ def lib():
         for name in ("orc_dense1_set", "orc_dense1_get", "orc_size", "orc_find_or_insert",
                      "orc_forward_original", "orc_fm_pairs", "orc_forward_partials", "orc_aggregate",
                      "orc_backward_update", "orc_read_rows", "orc_poke", "orc_philox4x32_10",
-                     "orc_shard_of_many", "orc_comm_saving"):
+                     "orc_shard_of_many", "orc_comm_saving", "orc_set_opt", "orc_read_state2",
+                     "orc_dense1_get_state2"):
             getattr(L, name).argtypes = None
     return _lib
 
@@ -96,10 +97,20 @@ class Oracle:
                                               C.c_float(init_scale), C.c_float(lr), C.c_float(eps),
                                               C.c_float(init_acc)))
 
+    def set_opt(self, lin_optimizer=0, beta1=0.9, beta2=0.999, ftrl_alpha=0.05, ftrl_beta=1.0, ftrl_l1=0.0,
+                ftrl_l2=0.0):
+        """Optimizer settings beyond the constructor's; call before the first insert."""
+        self.L.orc_set_opt(self.h, C.c_uint32(lin_optimizer), C.c_float(beta1), C.c_float(beta2),
+                           C.c_float(ftrl_alpha), C.c_float(ftrl_beta), C.c_float(ftrl_l1), C.c_float(ftrl_l2))
+
     @classmethod
     def for_workload(cls, w):
-        return cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, w.seed,
-                   w.init_scale, w.lr, w.eps, w.init_acc)
+        o = cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, w.seed,
+                w.init_scale, w.lr, w.eps, w.init_acc)
+        o.set_opt(getattr(w, "lin_optimizer", 0), getattr(w, "beta1", 0.9), getattr(w, "beta2", 0.999),
+                  getattr(w, "ftrl_alpha", 0.05), getattr(w, "ftrl_beta", 1.0), getattr(w, "ftrl_l1", 0.0),
+                  getattr(w, "ftrl_l2", 0.0))
+        return o
 
     def close(self):
         if self.h:
@@ -219,6 +230,20 @@ class Oracle:
                              _p(keys, C.c_uint64), _p(emb, C.c_float), _p(lin, C.c_float),
                              _p(ae, C.c_float), _p(al, C.c_float))
         return dict(keys=keys, emb=emb, lin=lin, acc_emb=ae, acc_lin=al)
+
+    def read_state2(self, shard, row):
+        shard = np.ascontiguousarray(shard, dtype=np.uint8)
+        row = np.ascontiguousarray(row, dtype=np.uint32)
+        n, k = shard.shape[0], self.k
+        a2 = np.empty((n, k), dtype=np.float32); l2 = np.empty(n, dtype=np.float32)
+        self.L.orc_read_state2(self.h, C.c_int64(n), _p(shard, C.c_uint8), _p(row, C.c_uint32),
+                               _p(a2, C.c_float), _p(l2, C.c_float))
+        return dict(acc2_emb=a2, lin2=l2)
+
+    def dense1_get_state2(self):
+        a2 = np.empty((self.F * self.k, self.H), dtype=np.float32)
+        self.L.orc_dense1_get_state2(self.h, _p(a2, C.c_float))
+        return a2
 
     def poke(self, shard, row, col, value, set_=False):
         self.L.orc_poke(self.h, C.c_uint32(shard), C.c_uint32(row), C.c_uint32(col), C.c_float(value),

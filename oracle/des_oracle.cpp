@@ -42,7 +42,8 @@ namespace {
 const uint32_t ROW_NONE = 0xFFFFFFFFu;
 enum { OP_LR = 1, OP_FM = 2, OP_POOL = 4, OP_DENSE1 = 8 };
 enum { PART_HASH = 0, PART_FIELD = 1 };
-enum { OPT_SGD = 0, OPT_ADAGRAD = 1 };
+enum { OPT_SGD = 0, OPT_ADAGRAD = 1, OPT_ADAM = 2 };
+enum { LIN_SAME = 0, LIN_FTRL = 1 };
 
 // reading: the table's 64-bit mixer (splitmix64 finaliser steps)
 uint64_t mix64(uint64_t z) {
@@ -100,13 +101,19 @@ struct Shard {
   std::unordered_map<uint64_t, uint32_t> map;   // key -> shard-local row
   std::vector<uint64_t> keys;                   // row -> key
   std::vector<float> emb, lin, acc_emb, acc_lin;
+  std::vector<float> acc2_emb, lin2;            // second state word: Adam's v; linear weight: Adam's v / FTRL's z
 };
 
 struct Table {
   uint32_t S, F, k, H, partition, optimizer;
   uint64_t seed; float init_scale, lr, eps, init_acc;
   std::vector<Shard> sh;
-  std::vector<float> W1, accW1;                 // [F*k][H]
+  std::vector<float> W1, accW1, acc2W1;         // [F*k][H]
+  uint32_t lin_optimizer = LIN_SAME;
+  float beta1 = 0.9f, beta2 = 0.999f, ftrl_alpha = 0.05f, ftrl_beta = 1.0f, ftrl_l1 = 0.f, ftrl_l2 = 0.f;
+  int64_t step = 0;                             // backward calls so far (Adam's t)
+  float state_init() const { return optimizer == OPT_ADAGRAD ? init_acc : 0.0f; }
+  float lin_state_init() const { return (lin_optimizer == LIN_FTRL || optimizer != OPT_ADAGRAD) ? 0.0f : init_acc; }
   uint32_t shard_of(uint64_t id, uint32_t field) const {
     return partition == PART_HASH ? (uint32_t)(mix64(id) % S) : field % S;
   }
@@ -117,16 +124,40 @@ struct Table {
     h.keys.push_back(id);
     for (uint32_t c = 0; c < k; ++c) h.emb.push_back(init_value(seed, id, c, init_scale));
     h.lin.push_back(0.0f);
-    for (uint32_t c = 0; c < k; ++c) h.acc_emb.push_back(init_acc);
-    h.acc_lin.push_back(init_acc);
+    for (uint32_t c = 0; c < k; ++c) { h.acc_emb.push_back(state_init()); h.acc2_emb.push_back(0.0f); }
+    h.acc_lin.push_back(lin_state_init());
+    h.lin2.push_back(0.0f);
     return row;
   }
 };
 
-inline void apply_opt(const Table& t, float& theta, float& acc, double Gd) {
+// FTRL-Proximal per coordinate (McMahan et al. 2013, "Ad Click Prediction"), the
+// optimizer the paper runs on the order-1 weights (Section 6, "Parameter
+// Settings"): state n (sum of squared gradients) and z.
+inline void apply_ftrl(const Table& t, float& w, float& n, float& z, double Gd) {
+  const double G = (double)(float)Gd, n0 = (double)n;
+  const double sigma = (std::sqrt(n0 + G * G) - std::sqrt(n0)) / (double)t.ftrl_alpha;
+  const float zf = (float)((double)z + G - sigma * (double)w);
+  const float nf = (float)(n0 + G * G);
+  z = zf; n = nf;
+  const double zz = (double)zf, l1 = (double)t.ftrl_l1;
+  if (std::fabs(zz) <= l1) { w = 0.0f; return; }
+  const double sgn = zz > 0 ? 1.0 : -1.0;
+  w = (float)(-(zz - sgn * l1) / (((double)t.ftrl_beta + std::sqrt((double)nf)) / (double)t.ftrl_alpha + (double)t.ftrl_l2));
+}
+
+// acc / acc2: first and second state word (Adagrad: accumulator / unused; Adam: m / v).
+inline void apply_opt(const Table& t, float& theta, float& acc, float& acc2, double Gd) {
   float G = (float)Gd;                          // summed gradient, rounded once
   if (t.optimizer == OPT_SGD) {
     theta = (float)((double)theta - (double)t.lr * (double)G);
+  } else if (t.optimizer == OPT_ADAM) {         // reading: lazy Adam, one global step count per backward call
+    const double b1 = (double)t.beta1, b2 = (double)t.beta2;
+    const float m = (float)(b1 * (double)acc + (1.0 - b1) * (double)G);
+    const float v = (float)(b2 * (double)acc2 + (1.0 - b2) * (double)G * (double)G);
+    acc = m; acc2 = v;
+    const double c1 = 1.0 - std::pow(b1, (double)t.step), c2 = 1.0 - std::pow(b2, (double)t.step);
+    theta = (float)((double)theta - (double)t.lr * ((double)m / c1) / (std::sqrt((double)v / c2) + (double)t.eps));
   } else {                                      // reading: eps outside the root
     float a = (float)((double)acc + (double)G * (double)G);
     acc = a;
@@ -166,10 +197,22 @@ void* orc_create(uint32_t S, uint32_t F, uint32_t k, uint32_t H, uint32_t partit
   t->S = S; t->F = F; t->k = k; t->H = H; t->partition = partition; t->optimizer = optimizer;
   t->seed = seed; t->init_scale = init_scale; t->lr = lr; t->eps = eps; t->init_acc = init_acc;
   t->sh.resize(S);
-  if (H) { t->W1.assign((size_t)F * k * H, 0.0f); t->accW1.assign((size_t)F * k * H, init_acc); }
+  if (H) {
+    t->W1.assign((size_t)F * k * H, 0.0f);
+    t->accW1.assign((size_t)F * k * H, t->state_init());
+    t->acc2W1.assign((size_t)F * k * H, 0.0f);
+  }
   return t;
 }
 void orc_destroy(void* p) { delete (Table*)p; }
+
+// Optimizer settings beyond the constructor's (call before the first insert).
+void orc_set_opt(void* p, uint32_t lin_optimizer, float beta1, float beta2, float ftrl_alpha, float ftrl_beta,
+                 float ftrl_l1, float ftrl_l2) {
+  Table* t = (Table*)p;
+  t->lin_optimizer = lin_optimizer; t->beta1 = beta1; t->beta2 = beta2;
+  t->ftrl_alpha = ftrl_alpha; t->ftrl_beta = ftrl_beta; t->ftrl_l1 = ftrl_l1; t->ftrl_l2 = ftrl_l2;
+}
 
 void orc_dense1_set(void* p, const float* W1) { Table* t = (Table*)p; std::memcpy(t->W1.data(), W1, t->W1.size() * 4); }
 void orc_dense1_get(void* p, float* W1, float* acc) {
@@ -420,6 +463,7 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
     }
     if (gE_total_out) std::memcpy(gE_total_out, gEt.data(), gEt.size() * 4);
   }
+  t->step += 1;                                  // Adam's global step count
   std::vector<double> Gw((size_t)U, 0.0), Gv((size_t)U * k, 0.0);
   std::vector<double> Sw((size_t)U, 0.0), Sv((size_t)U * k, 0.0);
   std::vector<uint8_t> us((size_t)U); std::vector<uint32_t> ur((size_t)U);
@@ -445,10 +489,14 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
   for (int64_t u = 0; u < U; ++u) {
     Shard& h = t->sh[us[u]];
     uint32_t row = ur[u];
-    if (ops & OP_LR) apply_opt(*t, h.lin[row], h.acc_lin[row], Gw[u]);
+    if (ops & OP_LR) {
+      if (t->lin_optimizer == LIN_FTRL) apply_ftrl(*t, h.lin[row], h.acc_lin[row], h.lin2[row], Gw[u]);
+      else apply_opt(*t, h.lin[row], h.acc_lin[row], h.lin2[row], Gw[u]);
+    }
     if (ops & (OP_FM | OP_POOL | OP_DENSE1))
       for (uint32_t c = 0; c < k; ++c)
-        apply_opt(*t, h.emb[(size_t)row * k + c], h.acc_emb[(size_t)row * k + c], Gv[(size_t)u * k + c]);
+        apply_opt(*t, h.emb[(size_t)row * k + c], h.acc_emb[(size_t)row * k + c], h.acc2_emb[(size_t)row * k + c],
+                  Gv[(size_t)u * k + c]);
     if (Sw_out) Sw_out[u] = Sw[u];
     if (Sv_out) for (uint32_t c = 0; c < k; ++c) Sv_out[(size_t)u * k + c] = Sv[(size_t)u * k + c];
     if (Gw_out) Gw_out[u] = (float)Gw[u];
@@ -461,7 +509,7 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
         for (int32_t b = 0; b < B; ++b)
           g += (double)bf16_round(pooled[(size_t)b * FK + i]) * (double)gZ[(size_t)b * H + h2];
         if (gW1_out) gW1_out[i * H + h2] = (float)g;
-        apply_opt(*t, t->W1[i * H + h2], t->accW1[i * H + h2], g);
+        apply_opt(*t, t->W1[i * H + h2], t->accW1[i * H + h2], t->acc2W1[i * H + h2], g);
       }
   }
 }
@@ -480,6 +528,23 @@ void orc_read_rows(void* p, int64_t n, const uint8_t* shard, const uint32_t* row
     if (acc_emb) std::memcpy(acc_emb + (size_t)i * k, &h.acc_emb[(size_t)r * k], k * 4);
     if (acc_lin) acc_lin[i] = h.acc_lin[r];
   }
+}
+
+// Second optimizer-state word of rows given by (shard, row).
+void orc_read_state2(void* p, int64_t n, const uint8_t* shard, const uint32_t* row, float* acc2_emb, float* lin2) {
+  Table* t = (Table*)p;
+  const uint32_t k = t->k;
+  for (int64_t i = 0; i < n; ++i) {
+    const Shard& h = t->sh[shard[i]];
+    uint32_t r = row[i];
+    if (acc2_emb) std::memcpy(acc2_emb + (size_t)i * k, &h.acc2_emb[(size_t)r * k], k * 4);
+    if (lin2) lin2[i] = h.lin2[r];
+  }
+}
+
+void orc_dense1_get_state2(void* p, float* acc2) {
+  Table* t = (Table*)p;
+  std::memcpy(acc2, t->acc2W1.data(), t->acc2W1.size() * 4);
 }
 
 // Test hook: add delta to one stored weight (col < k: latent component,

@@ -15,7 +15,8 @@ from . import build as _build
 
 OP_LR, OP_FM, OP_POOL, OP_DENSE1 = 1, 2, 4, 8
 PART_HASH, PART_FIELD = 0, 1
-OPT_SGD, OPT_ADAGRAD = 0, 1
+OPT_SGD, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2
+LIN_SAME, LIN_FTRL = 0, 1
 ROW_NONE = 0xFFFFFFFF
 KEY_EMPTY = 0xFFFFFFFFFFFFFFFF
 
@@ -24,8 +25,9 @@ STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "
           7: "DES_ERR_TOO_LARGE"}
 
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
-           "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_forward_noalloc", "des_table_status",
+           "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
+           "des_table_read_state2", "des_table_write_state2",
            "des_step_host", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
 
 
@@ -42,6 +44,8 @@ class des_config_t(C.Structure):
                 ("h_rows_per_shard", C.POINTER(C.c_uint64)),
                 ("seed", C.c_uint64), ("init_scale", C.c_float),
                 ("lr", C.c_float), ("eps", C.c_float), ("init_acc", C.c_float),
+                ("lin_optimizer", C.c_uint32), ("beta1", C.c_float), ("beta2", C.c_float),
+                ("ftrl_alpha", C.c_float), ("ftrl_beta", C.c_float), ("ftrl_l1", C.c_float), ("ftrl_l2", C.c_float),
                 ("max_nnz", C.c_int64), ("max_batch", C.c_int32), ("max_uniq", C.c_int64),
                 ("alloc", C.c_void_p), ("dealloc", C.c_void_p), ("alloc_ctx", C.c_void_p)]
 
@@ -94,6 +98,8 @@ def load():
                                           C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
         L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.des_dense1_get.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_dense1_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_dense1_set_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.des_dense1_forward_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.des_table_status.argtypes = [C.c_void_p]
         L.des_table_size.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
@@ -101,6 +107,8 @@ def load():
         L.des_table_export.argtypes = [C.c_void_p] + [C.c_void_p] * 7 + [C.c_uint64, C.POINTER(C.c_uint64)]
         L.des_table_read_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
         L.des_table_write_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
+        L.des_table_read_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_table_write_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.des_step_host.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]
@@ -159,7 +167,8 @@ class Table:
 
     def __init__(self, num_shards, num_fields, emb_dim, hidden=0, partition=PART_HASH, optimizer=OPT_SGD,
                  max_rows=1 << 20, max_load=0.5, rows_per_shard=None, seed=0, init_scale=0.01, lr=0.01,
-                 eps=1e-8, init_acc=0.0, max_nnz=1 << 20, max_batch=1 << 16, max_uniq=0):
+                 eps=1e-8, init_acc=0.0, max_nnz=1 << 20, max_batch=1 << 16, max_uniq=0, lin_optimizer=LIN_SAME,
+                 beta1=0.9, beta2=0.999, ftrl_alpha=0.05, ftrl_beta=1.0, ftrl_l1=0.0, ftrl_l2=0.0):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_1909_04823_b200 needs a CUDA device; there is no CPU path")
         self.L = load()
@@ -174,6 +183,8 @@ class Table:
             self._rps = (C.c_uint64 * num_shards)(*[int(v) for v in rows_per_shard])
             cfg.h_rows_per_shard = C.cast(self._rps, C.POINTER(C.c_uint64))
         cfg.seed, cfg.init_scale, cfg.lr, cfg.eps, cfg.init_acc = int(seed), init_scale, lr, eps, init_acc
+        cfg.lin_optimizer, cfg.beta1, cfg.beta2 = lin_optimizer, beta1, beta2
+        cfg.ftrl_alpha, cfg.ftrl_beta, cfg.ftrl_l1, cfg.ftrl_l2 = ftrl_alpha, ftrl_beta, ftrl_l1, ftrl_l2
         cfg.max_nnz, cfg.max_batch, cfg.max_uniq = int(max_nnz), int(max_batch), int(max_uniq)
         self.h = C.c_void_p()
         self._check(self.L.des_table_create(C.byref(cfg), C.byref(self.h)), "des_table_create")
@@ -182,7 +193,9 @@ class Table:
     def for_workload(cls, w, max_rows, max_nnz, max_batch=None, rows_per_shard=None, max_uniq=0, max_load=0.5):
         return cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, max_rows=max_rows,
                    max_load=max_load, rows_per_shard=rows_per_shard, seed=w.seed, init_scale=w.init_scale,
-                   lr=w.lr, eps=w.eps, init_acc=w.init_acc, max_nnz=max_nnz,
+                   lr=w.lr, eps=w.eps, init_acc=w.init_acc, lin_optimizer=w.lin_optimizer, beta1=w.beta1,
+                   beta2=w.beta2, ftrl_alpha=w.ftrl_alpha, ftrl_beta=w.ftrl_beta, ftrl_l1=w.ftrl_l1,
+                   ftrl_l2=w.ftrl_l2, max_nnz=max_nnz,
                    max_batch=max_batch or w.batch, max_uniq=max_uniq)
 
     def _check(self, code, where):
@@ -323,3 +336,26 @@ class Table:
         static device array: no allocation anywhere in the call."""
         self._check(self.L.des_dense1_forward_noalloc(self.h, _ptr(pooled), int(pooled.shape[0]), _ptr(Z), _stream()),
                     "des_dense1_forward_noalloc")
+
+    def read_state2(self, global_rows: torch.Tensor):
+        n = int(global_rows.numel())
+        a2 = torch.empty((n, self.k), dtype=torch.float32, device="cuda")
+        l2 = torch.empty(n, dtype=torch.float32, device="cuda")
+        self._check(self.L.des_table_read_state2(self.h, _ptr(global_rows), n, _ptr(a2), _ptr(l2), _stream()),
+                    "des_table_read_state2")
+        return dict(acc2_emb=a2, lin2=l2)
+
+    def write_state2(self, global_rows: torch.Tensor, acc2_emb=None, lin2=None):
+        n = int(global_rows.numel())
+        self._check(self.L.des_table_write_state2(self.h, _ptr(global_rows), n, _ptr(acc2_emb), _ptr(lin2), _stream()),
+                    "des_table_write_state2")
+
+    def dense1_get_state(self, want2=False):
+        n = (self.F * self.k, self.H)
+        s1 = torch.empty(n, dtype=torch.float32, device="cuda")
+        s2 = torch.empty(n, dtype=torch.float32, device="cuda") if want2 else None
+        self._check(self.L.des_dense1_get_state(self.h, _ptr(s1), _ptr(s2), _stream()), "des_dense1_get_state")
+        return s1, s2
+
+    def dense1_set_state(self, s1=None, s2=None):
+        self._check(self.L.des_dense1_set_state(self.h, _ptr(s1), _ptr(s2), _stream()), "des_dense1_set_state")

@@ -196,33 +196,34 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
 // 16-byte column each, lane 0 also the linear weight); it works on UP_UNROLL
 // keys at a time so that their gradient rows, row numbers, weights and state
 // are all in flight together: the kernel is a pure stream of 272-byte rows.
+// Advances Adam's step count and recomputes the bias corrections 1 - beta^t in double.
+__global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
+  const unsigned long long t = meta->opt_step + 1;
+  meta->opt_step = t;
+  meta->adam_c1 = (float)(1.0 - pow((double)beta1, (double)t));
+  meta->adam_c2 = (float)(1.0 - pow((double)beta2, (double)t));
+}
+
 template <int G>
 __global__ void __launch_bounds__(256) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
-    uint32_t ops, int optimizer, float lr, float eps, float* __restrict__ Gbuf, float* __restrict__ W,
-    float* __restrict__ A, uint32_t* __restrict__ hinfo) {
+    uint32_t ops, const OptParams opt_in, const DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
+    float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2, uint32_t* __restrict__ hinfo) {
   const int K4 = k >> 2, stride = k + 4;
+  const OptParams opt = des_opt_load(opt_in, meta);
   long long U = *n_uniq;
   if (U > max_uniq) U = max_uniq;
   const int c4 = (int)(threadIdx.x % G);
   const bool col = c4 < K4, lead = c4 == 0;
   const bool upd_v = ops & (DES_OP_FM | DES_OP_POOL | DES_OP_DENSE1), upd_w = ops & DES_OP_LR;
   const long long gstep = (long long)gridDim.x * (blockDim.x / G);
-  auto step = [&](float& theta, float& acc, float Gd) {
-    if (optimizer == DES_OPT_ADAGRAD) {
-      acc = acc + Gd * Gd;
-      theta = theta - lr * Gd / (sqrtf(acc) + eps);
-    } else {
-      theta = theta - lr * Gd;
-    }
-  };
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
   // every lane of a warp runs the same number of iterations (keys past U are masked off)
   const long long iters = (U + gstep * UP_UNROLL - 1) / (gstep * UP_UNROLL);
   long long u0 = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
   for (long long it = 0; it < iters; ++it, u0 += gstep * UP_UNROLL) {
     uint32_t r[UP_UNROLL];
-    float4 g[UP_UNROLL], tail[UP_UNROLL], v[UP_UNROLL], s[UP_UNROLL], vt[UP_UNROLL], st[UP_UNROLL];
+    float4 g[UP_UNROLL], tail[UP_UNROLL], v[UP_UNROLL], s[UP_UNROLL], s2[UP_UNROLL], vt[UP_UNROLL], st[UP_UNROLL];
 #pragma unroll
     for (int q = 0; q < UP_UNROLL; ++q) {
       const long long u = u0 + q * gstep;
@@ -236,11 +237,12 @@ __global__ void __launch_bounds__(256) update_rows_kernel(
     }
 #pragma unroll
     for (int q = 0; q < UP_UNROLL; ++q) {
-      v[q] = zero; s[q] = zero; vt[q] = zero; st[q] = zero;
+      v[q] = zero; s[q] = zero; s2[q] = zero; vt[q] = zero; st[q] = zero;
       if (r[q] != DES_ROW_NONE) {
         const float4* w = reinterpret_cast<const float4*>(W + (size_t)r[q] * stride);
         const float4* a = A ? reinterpret_cast<const float4*>(A + (size_t)r[q] * stride) : nullptr;
-        if (col) { v[q] = w[c4]; if (a && upd_v) s[q] = a[c4]; }
+        const float4* a2 = A2 ? reinterpret_cast<const float4*>(A2 + (size_t)r[q] * stride) : nullptr;
+        if (col) { v[q] = w[c4]; if (a && upd_v) s[q] = a[c4]; if (a2 && upd_v) s2[q] = a2[c4]; }
         if (lead) { vt[q] = w[K4]; if (a && upd_w) st[q] = a[K4]; }
       }
     }
@@ -256,10 +258,10 @@ __global__ void __launch_bounds__(256) update_rows_kernel(
       }
       if (mapped && col && upd_v) {
         const float t1 = tail[q].y;
-        step(v[q].x, s[q].x, g[q].x - v[q].x * t1);
-        step(v[q].y, s[q].y, g[q].y - v[q].y * t1);
-        step(v[q].z, s[q].z, g[q].z - v[q].z * t1);
-        step(v[q].w, s[q].w, g[q].w - v[q].w * t1);
+        des_opt_step(opt, v[q].x, s[q].x, s2[q].x, g[q].x - v[q].x * t1);
+        des_opt_step(opt, v[q].y, s[q].y, s2[q].y, g[q].y - v[q].y * t1);
+        des_opt_step(opt, v[q].z, s[q].z, s2[q].z, g[q].z - v[q].z * t1);
+        des_opt_step(opt, v[q].w, s[q].w, s2[q].w, g[q].w - v[q].w * t1);
       }
       // squared norm of the (new) latent vector, kept in the row's tail for the forward's M_2
       float n2 = v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
@@ -268,9 +270,16 @@ __global__ void __launch_bounds__(256) update_rows_kernel(
       if (!mapped) continue;
       float4* w = reinterpret_cast<float4*>(W + (size_t)r[q] * stride);
       float4* a = A ? reinterpret_cast<float4*>(A + (size_t)r[q] * stride) : nullptr;
-      if (col && upd_v) { w[c4] = v[q]; if (a) a[c4] = s[q]; }
+      if (col && upd_v) {
+        w[c4] = v[q];
+        if (a) a[c4] = s[q];
+        if (A2) reinterpret_cast<float4*>(A2 + (size_t)r[q] * stride)[c4] = s2[q];
+      }
       if (lead) {
-        if (upd_w) step(vt[q].x, st[q].x, tail[q].x);
+        if (upd_w) {     // linear weight: its two state words sit side by side in the state row's tail
+          if (opt.lin_optimizer == DES_LIN_FTRL) des_ftrl_step(opt, vt[q].x, st[q].x, st[q].y, tail[q].x);
+          else des_opt_step(opt, vt[q].x, st[q].x, st[q].y, tail[q].x);
+        }
         vt[q].y = n2;
         w[K4] = vt[q];
         if (a && upd_w) a[K4] = st[q];
@@ -293,6 +302,11 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   cudaStream_t cs = (cudaStream_t)stream;
   des_api_begin(t, cs);
   const int B = b->batch;
+  const OptParams opt = des_opt_params(t);
+  if (opt.optimizer == DES_OPT_ADAM) {               // one optimizer step per backward call (Adam's t)
+    adam_tick_kernel<<<1, 1, 0, cs>>>(t->meta, opt.beta1, opt.beta2);
+    DES_LAUNCH_CHECK(t, "adam_tick_kernel");
+  }
   const float* gE = (ops & DES_OP_POOL) ? gr->gE : nullptr;
   if (ops & DES_OP_DENSE1) {
     st = des_dense1_backward(t, out->pooled, gE, gr->gZ, gr->gE_work, B, cs);
@@ -337,7 +351,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   {
     const unsigned grid = (unsigned)(t->sm_count * 8);
 #define UP(GG) update_rows_kernel<GG><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops,       \
-                                                           t->cfg.optimizer, t->cfg.lr, t->cfg.eps, t->Gbuf, t->W, t->A, t->hinfo)
+                                                           opt, t->meta, t->Gbuf, t->W, t->A, t->A2, t->hinfo)
     switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }
 #undef UP
     DES_LAUNCH_CHECK(t, "update_rows_kernel");

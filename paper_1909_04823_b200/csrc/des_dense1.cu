@@ -131,19 +131,18 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs g) {
 // Sum the split-K slices of gW1 in slice order, apply the optimizer to the
 // fp32 master weights, refresh the bf16 shadow.
 __global__ void w1_update_kernel(const float* __restrict__ part, int slices, size_t n, float* W1, float* acc,
-                                 __nv_bfloat16* W1b, int optimizer, float lr, float eps) {
+                                 float* acc2, __nv_bfloat16* W1b, const OptParams opt_in,
+                                 const DevMeta* __restrict__ meta) {
+  const OptParams opt = des_opt_load(opt_in, meta);
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
   for (; i < n; i += st) {
     float G = 0.f;
     for (int z = 0; z < slices; ++z) G += __ldg(part + (size_t)z * n + i);
     float w = W1[i];
-    if (optimizer == DES_OPT_ADAGRAD) {
-      float a = acc[i] + G * G;
-      acc[i] = a;
-      w -= lr * G / (sqrtf(a) + eps);
-    } else {
-      w -= lr * G;
-    }
+    float s1 = acc[i], s2 = acc2 ? acc2[i] : 0.f;
+    des_opt_step(opt, w, s1, s2, G);
+    acc[i] = s1;
+    if (acc2) acc2[i] = s2;
     W1[i] = w;
     W1b[i] = __float2bfloat16_rn(w);
   }
@@ -204,8 +203,8 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
                                         t->gemm_ws_bytes, st);
       if (rc2 != 0) return DES_ERR_CUDA;           // same alignment rules as the dgrad: cannot differ
       DES_LAUNCH_CHECK(t, "tc_gemm_wgrad");
-      w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, 1, (size_t)FK * t->H, t->W1, t->accW1, t->W1b,
-                                                        t->cfg.optimizer, t->cfg.lr, t->cfg.eps);
+      w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, 1, (size_t)FK * t->H, t->W1, t->accW1, t->acc2W1,
+                                                        t->W1b, des_opt_params(t), t->meta);
       DES_LAUNCH_CHECK(t, "w1_update_kernel");
       return DES_OK;
     }
@@ -227,8 +226,8 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
     gemm_kernel<GEMM_WGRAD><<<grid, 256, 0, st>>>(g);
     DES_LAUNCH_CHECK(t, "gemm_kernel");
     const size_t n = (size_t)FK * t->H;
-    w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, g.slices, n, t->W1, t->accW1, t->W1b,
-                                                      t->cfg.optimizer, t->cfg.lr, t->cfg.eps);
+    w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, g.slices, n, t->W1, t->accW1, t->acc2W1,
+                                                      t->W1b, des_opt_params(t), t->meta);
     DES_LAUNCH_CHECK(t, "w1_update_kernel");
   }
   return DES_OK;

@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(256) apply_first_kernel(
     const unsigned long long* __restrict__ ids, int k, int stride, Slot* slots, const DevMeta* __restrict__ meta,
     const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint32_t* __restrict__ first_j,
     uint32_t* __restrict__ uslot, uint32_t* __restrict__ uniq_rows, float* __restrict__ W, float* __restrict__ A,
-    unsigned long long seed, float init_scale, float init_acc) {
+    float* __restrict__ A2, unsigned long long seed, float init_scale, float state_init, float lin_state_init) {
   const uint32_t U = meta->n_uniq;
   for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
     const uint32_t fj = first_j[u];
@@ -252,9 +252,13 @@ __global__ void __launch_bounds__(256) apply_first_kernel(
       w[q4] = make_float4(0.f, n2, 0.f, 0.f);   // linear weight, squared norm of the latent vector
       if (A) {
         float4* a = reinterpret_cast<float4*>(A + g * stride);
-        const float4 ia = make_float4(init_acc, init_acc, init_acc, init_acc);
+        const float4 ia = make_float4(state_init, state_init, state_init, state_init);
         for (int q = 0; q < q4; ++q) a[q] = ia;
-        a[q4] = make_float4(init_acc, 0.f, 0.f, 0.f);
+        a[q4] = make_float4(lin_state_init, 0.f, 0.f, 0.f);
+      }
+      if (A2) {
+        float4* a2 = reinterpret_cast<float4*>(A2 + g * stride);
+        for (int q = 0; q <= q4; ++q) a2[q] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
   }
@@ -312,7 +316,10 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   DES_LAUNCH_CHECK(t, "assign_kernel");
   apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>((const unsigned long long*)b->ids, t->k, t->stride, t->slots,
                                                       t->meta, t->slot_of, b->shards, t->dest, t->uslot, b->uniq_rows,
-                                                      t->W, t->A, t->cfg.seed, t->cfg.init_scale, t->cfg.init_acc);
+                                                      t->W, t->A, t->A2, t->cfg.seed, t->cfg.init_scale,
+                                                      t->cfg.optimizer == DES_OPT_ADAGRAD ? t->cfg.init_acc : 0.f,
+                                                      (t->cfg.lin_optimizer == DES_LIN_FTRL ||
+                                                       t->cfg.optimizer != DES_OPT_ADAGRAD) ? 0.f : t->cfg.init_acc);
   DES_LAUNCH_CHECK(t, "apply_first_kernel");
   resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
   DES_LAUNCH_CHECK(t, "resolve_kernel");

@@ -32,6 +32,8 @@ struct DevMeta {
   uint32_t n_uniq;                                   // unique keys of the running insert call
   uint32_t err;                                      // sticky des_status_t raised on device
   uint32_t field_order[1024];                        // fields sorted by (owning shard, field)
+  unsigned long long opt_step;                       // backward calls so far (Adam's t), advanced on device
+  float adam_c1, adam_c2;                            // 1 - beta1^t, 1 - beta2^t for the running step
 };
 
 struct des_table {
@@ -45,7 +47,9 @@ struct des_table {
   // device memory
   Slot* slots;
   float* W;                          // [total_rows][stride]: latent vector v[k], linear weight, |v|^2, 2 pad
-  float* A;                          // same shape: Adagrad accumulators (NULL for SGD)
+  float* A;                          // same shape, first optimizer-state word: Adagrad accumulator / Adam m;
+                                     // tail = (linear weight's state 1, state 2): Adagrad acc | Adam m, v | FTRL n, z
+  float* A2;                         // same shape, second state word of the latent vector (Adam v); NULL otherwise
   DevMeta* meta;
   // find_or_insert workspace
   uint32_t* slot_of;                 // [max_nnz]
@@ -64,6 +68,7 @@ struct des_table {
   uint32_t hot_max, rep_max, work_max;
   // first dense layer
   float* W1; float* accW1;           // [F*k][H] fp32 master and state
+  float* acc2W1;                     // Adam's second moment of W1 (NULL otherwise)
   __nv_bfloat16* W1b;                // bf16 shadow
   float* gW1_part; int gw1_splits;   // [splits][F*k][H]
   int use_tc;                        // tensor-core GEMM path usable for this table's shapes
@@ -145,6 +150,51 @@ __device__ __forceinline__ int des_bag_of(const int32_t* __restrict__ offsets, i
 }
 
 __device__ __forceinline__ void des_raise(DevMeta* meta, uint32_t code) { atomicCAS(&meta->err, 0u, code); }
+
+// Optimizer parameters handed to the update kernels by value.
+struct OptParams {
+  int optimizer, lin_optimizer;
+  float lr, eps;
+  float beta1, beta2, c1, c2;          // Adam: c1 = 1 - beta1^t, c2 = 1 - beta2^t (filled on device, see des_opt_load)
+  float ftrl_alpha, ftrl_beta, ftrl_l1, ftrl_l2;
+};
+
+// One application of SGD / Adagrad / Adam to one parameter.  s1, s2: first and
+// second state word (Adagrad: accumulator, -; Adam: m, v).
+__device__ __forceinline__ void des_opt_step(const OptParams& o, float& theta, float& s1, float& s2, float G) {
+  if (o.optimizer == DES_OPT_ADAGRAD) {
+    s1 = s1 + G * G;
+    theta = theta - o.lr * G / (sqrtf(s1) + o.eps);
+  } else if (o.optimizer == DES_OPT_ADAM) {
+    s1 = o.beta1 * s1 + (1.f - o.beta1) * G;
+    s2 = o.beta2 * s2 + (1.f - o.beta2) * G * G;
+    theta = theta - o.lr * (s1 / o.c1) / (sqrtf(s2 / o.c2) + o.eps);
+  } else {
+    theta = theta - o.lr * G;
+  }
+}
+
+// FTRL-Proximal on one coordinate: state n (sum of squared gradients) and z.
+__device__ __forceinline__ void des_ftrl_step(const OptParams& o, float& w, float& n, float& z, float G) {
+  const float n1 = n + G * G;
+  const float sigma = (sqrtf(n1) - sqrtf(n)) / o.ftrl_alpha;
+  z = z + G - sigma * w;
+  n = n1;
+  if (fabsf(z) <= o.ftrl_l1) { w = 0.f; return; }
+  const float sgn = z > 0.f ? 1.f : -1.f;
+  w = -(z - sgn * o.ftrl_l1) / ((o.ftrl_beta + sqrtf(n1)) / o.ftrl_alpha + o.ftrl_l2);
+}
+
+OptParams des_opt_params(des_table* t);
+
+// The launch carries the configured constants; Adam's bias corrections live in
+// device memory (advanced by one small kernel per backward call) so that a
+// backward captured into a CUDA graph keeps counting steps when replayed.
+__device__ __forceinline__ OptParams des_opt_load(const OptParams& o, const DevMeta* __restrict__ meta) {
+  OptParams r = o;
+  if (o.optimizer == DES_OPT_ADAM) { r.c1 = meta->adam_c1; r.c2 = meta->adam_c2; }
+  return r;
+}
 
 // shared declarations across translation units
 des_status_t des_check_batch(const des_table* t, const des_batch_t* b, int need_dedup);

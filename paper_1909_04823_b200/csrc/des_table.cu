@@ -2,6 +2,7 @@
 // workspace, status, size, export, row read-back (Section 5, "Dynamic Hash
 // Table": the storage behind lookup / insert / update).
 #include <new>
+#include <math.h>
 #include <string.h>
 
 #include "des_internal.cuh"
@@ -21,6 +22,16 @@ static void dfree(const des_config_t& c, void* p) {
 __global__ void fill_f32_kernel(float* p, size_t n, float v) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
   for (; i < n; i += st) p[i] = v;
+}
+
+OptParams des_opt_params(des_table* t) {
+  OptParams o;
+  const des_config_t& c = t->cfg;
+  o.optimizer = (int)c.optimizer; o.lin_optimizer = (int)c.lin_optimizer;
+  o.lr = c.lr; o.eps = c.eps; o.beta1 = c.beta1; o.beta2 = c.beta2;
+  o.c1 = 1.f; o.c2 = 1.f;
+  o.ftrl_alpha = c.ftrl_alpha; o.ftrl_beta = c.ftrl_beta; o.ftrl_l1 = c.ftrl_l1; o.ftrl_l2 = c.ftrl_l2;
+  return o;
 }
 
 int des_prof_mark(des_table* t, const char* name, int check) {
@@ -86,7 +97,7 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   if (!t) return DES_OK;
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
-  void* ptrs[] = {t->slots, t->W, t->A, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
+  void* ptrs[] = {t->slots, t->W, t->A, t->A2, t->acc2W1, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
                   t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc,
                   t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
@@ -104,11 +115,15 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   const des_config_t& c = *cfg;
   if (c.num_shards < 1 || c.num_shards > DES_MAX_SHARDS || c.num_fields < 1 || c.num_fields > 1024 ||
       c.emb_dim < 4 || c.emb_dim > 64 || (c.emb_dim & 3) || (c.hidden & 3) || c.partition > DES_PART_FIELD ||
-      c.optimizer > DES_OPT_ADAGRAD || c.max_rows == 0 || !(c.max_load > 0.f && c.max_load <= 0.9f) ||
+      c.optimizer > DES_OPT_ADAM || c.lin_optimizer > DES_LIN_FTRL || c.max_rows == 0 || !(c.max_load > 0.f && c.max_load <= 0.9f) ||
       c.max_nnz <= 0 || c.max_nnz >= (1ll << 31) || c.max_batch <= 0 || c.max_uniq < 0 ||
       (int64_t)c.max_batch * c.num_fields >= (1ll << 31))
     return DES_ERR_INVALID_ARG;
   if ((c.alloc == nullptr) != (c.dealloc == nullptr)) return DES_ERR_INVALID_ARG;
+  if (c.optimizer == DES_OPT_ADAM && !(c.beta1 >= 0.f && c.beta1 < 1.f && c.beta2 >= 0.f && c.beta2 < 1.f))
+    return DES_ERR_INVALID_ARG;
+  if (c.lin_optimizer == DES_LIN_FTRL && !(c.ftrl_alpha > 0.f && c.ftrl_beta >= 0.f && c.ftrl_l1 >= 0.f && c.ftrl_l2 >= 0.f))
+    return DES_ERR_INVALID_ARG;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return DES_ERR_CUDA; }
   des_table* t = new (std::nothrow) des_table();
@@ -152,7 +167,8 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   };
   A(t->slots, slots * sizeof(Slot));
   A(t->W, rows * rowbytes);
-  if (c.optimizer == DES_OPT_ADAGRAD) A(t->A, rows * rowbytes);
+  if (c.optimizer != DES_OPT_SGD || c.lin_optimizer == DES_LIN_FTRL) A(t->A, rows * rowbytes);
+  if (c.optimizer == DES_OPT_ADAM) A(t->A2, rows * rowbytes);
   A(t->meta, sizeof(DevMeta));
   A(t->slot_of, (size_t)t->max_nnz * 4);
   A(t->flags, (size_t)t->max_nnz);
@@ -173,6 +189,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);
   if (t->H) {
     A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
+    if (c.optimizer == DES_OPT_ADAM) A(t->acc2W1, FKH * 4);
     t->gw1_splits = 32;
     A(t->gW1_part, (size_t)t->gw1_splits * FKH * 4);
     // TMA needs 16-byte rows: every contiguous extent of a bf16 operand a multiple of 8
@@ -192,7 +209,8 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   if (t->H) {
     cu &= cudaMemset(t->W1, 0, FKH * 4) == cudaSuccess;
     cu &= cudaMemset(t->W1b, 0, FKH * 2) == cudaSuccess;
-    fill_f32_kernel<<<256, 256>>>(t->accW1, FKH, c.init_acc);
+    fill_f32_kernel<<<256, 256>>>(t->accW1, FKH, c.optimizer == DES_OPT_ADAGRAD ? c.init_acc : 0.f);
+    if (t->acc2W1) cu &= cudaMemset(t->acc2W1, 0, FKH * 4) == cudaSuccess;
     cu &= cudaGetLastError() == cudaSuccess;
   }
   cu &= cudaDeviceSynchronize() == cudaSuccess;
@@ -331,6 +349,46 @@ extern "C" des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_g
   return DES_OK;
 }
 
+__global__ void state2_kernel(const uint32_t* __restrict__ grows, long long n, int k, int stride,
+                              unsigned long long total_rows, float* A, float* A2, float* acc2_emb, float* lin2,
+                              int write) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t g = grows[i];
+  const bool ok = g != DES_ROW_NONE && g < total_rows;
+  if (write) {
+    if (!ok) return;
+    if (acc2_emb && A2) for (int c = 0; c < k; ++c) A2[(size_t)g * stride + c] = acc2_emb[i * k + c];
+    if (lin2 && A) A[(size_t)g * stride + k + 1] = lin2[i];
+  } else {
+    if (acc2_emb) for (int c = 0; c < k; ++c) acc2_emb[i * k + c] = (ok && A2) ? A2[(size_t)g * stride + c] : 0.f;
+    if (lin2) lin2[i] = (ok && A) ? A[(size_t)g * stride + k + 1] : 0.f;
+  }
+}
+
+extern "C" des_status_t des_table_read_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                              float* d_acc2_emb, float* d_lin2, void* stream) {
+  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;
+  des_api_begin(t, (cudaStream_t)stream);
+  state2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      d_global_rows, n, t->k, t->stride, t->total_rows, t->A, t->A2, d_acc2_emb, d_lin2, 0);
+  DES_LAUNCH_CHECK(t, "state2_kernel");
+  return DES_OK;
+}
+
+extern "C" des_status_t des_table_write_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
+                                               const float* d_acc2_emb, const float* d_lin2, void* stream) {
+  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;
+  des_api_begin(t, (cudaStream_t)stream);
+  state2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      d_global_rows, n, t->k, t->stride, t->total_rows, t->A, t->A2, const_cast<float*>(d_acc2_emb),
+      const_cast<float*>(d_lin2), 1);
+  DES_LAUNCH_CHECK(t, "state2_kernel");
+  return DES_OK;
+}
+
 // ---- first dense layer weights ----------------------------------------------
 __global__ void w1_shadow_kernel(const float* __restrict__ W1, __nv_bfloat16* __restrict__ W1b, size_t n) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
@@ -351,6 +409,25 @@ extern "C" des_status_t des_dense1_get(des_table_t* t, float* d_W1, void* stream
   if (!t || !d_W1 || !t->H) return DES_ERR_INVALID_ARG;
   size_t n = (size_t)t->F * t->k * t->H;
   DES_CUDA(cudaMemcpyAsync(d_W1, t->W1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return DES_OK;
+}
+
+// Optimizer state of W1: first word (Adagrad accumulator / Adam m) and second word (Adam v).
+extern "C" des_status_t des_dense1_get_state(des_table_t* t, float* d_state1, float* d_state2, void* stream) {
+  if (!t || !t->H) return DES_ERR_INVALID_ARG;
+  if ((d_state1 && !t->accW1) || (d_state2 && !t->acc2W1)) return DES_ERR_INVALID_ARG;
+  size_t n = (size_t)t->F * t->k * t->H;
+  if (d_state1) DES_CUDA(cudaMemcpyAsync(d_state1, t->accW1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  if (d_state2) DES_CUDA(cudaMemcpyAsync(d_state2, t->acc2W1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return DES_OK;
+}
+
+extern "C" des_status_t des_dense1_set_state(des_table_t* t, const float* d_state1, const float* d_state2, void* stream) {
+  if (!t || !t->H) return DES_ERR_INVALID_ARG;
+  if ((d_state1 && !t->accW1) || (d_state2 && !t->acc2W1)) return DES_ERR_INVALID_ARG;
+  size_t n = (size_t)t->F * t->k * t->H;
+  if (d_state1) DES_CUDA(cudaMemcpyAsync(t->accW1, d_state1, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  if (d_state2) DES_CUDA(cudaMemcpyAsync(t->acc2W1, d_state2, n * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return DES_OK;
 }
 

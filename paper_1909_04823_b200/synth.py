@@ -22,7 +22,8 @@ import numpy as np
 
 OP_LR, OP_FM, OP_POOL, OP_DENSE1 = 1, 2, 4, 8
 PART_HASH, PART_FIELD = 0, 1
-OPT_SGD, OPT_ADAGRAD = 0, 1
+OPT_SGD, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2
+LIN_SAME, LIN_FTRL = 0, 1
 
 _U64 = np.uint64
 
@@ -93,6 +94,13 @@ class Workload:
     lr: float = 0.01
     eps: float = 1e-8
     init_acc: float = 0.0
+    lin_optimizer: int = 0     # LIN_SAME: order-1 weights follow `optimizer`; LIN_FTRL
+    beta1: float = 0.9
+    beta2: float = 0.999
+    ftrl_alpha: float = 0.05
+    ftrl_beta: float = 1.0
+    ftrl_l1: float = 0.0
+    ftrl_l2: float = 0.0
     init_scale: float = 0.01
     steps: int = 1
     # id law

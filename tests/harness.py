@@ -96,6 +96,7 @@ class Pair:
         self.row_base = np.array(self.t.row_base(), dtype=np.int64)
         self.resync = resync
         self.drifted = False        # True once un-resynced differences may have accumulated
+        self.nstep = 0              # backward calls so far (Adam's bias-correction step)
         if w.hidden:
             W1 = synth.dense1_weights(w)
             self.o.dense1_set(W1)
@@ -131,34 +132,75 @@ class Pair:
         assert np.array_equal(u32(db.uniq_rows)[:U].astype(np.int64), want), "uniq_rows"
         assert self.t.size() == [int(v) for v in self.o.size()], "table size"
 
-    def compare_rows(self, fi, db, exact=False, gemm=False, what="rows", G=None):
+    def _adam_tol(self, G, dG, m, v):
+        """Bounds on |d theta|, |d m|, |d v| of one Adam application when the summed gradient moves
+        by at most dG; m, v: the oracle's moments AFTER the application."""
+        w, t = self.w, max(self.nstep, 1)
+        c1, c2 = 1.0 - w.beta1 ** t, 1.0 - w.beta2 ** t
+        dm = (1.0 - w.beta1) * dG
+        dv = (1.0 - w.beta2) * (2.0 * np.abs(G) * dG + dG * dG)
+        rt = np.sqrt(v / c2)
+        drt = np.minimum(dv / c2 / (2.0 * rt + 1e-300), np.sqrt(dv / c2))
+        den = rt + w.eps
+        r = np.abs(m) / c1 / den
+        dth = 2.0 * (dm / c1 / den + r * drt / den)
+        return w.lr * np.minimum(dth, 2.0 * r + 2.0), dm, dv
+
+    def _ftrl_tol(self, G, dG, w_old, w_new, n_new):
+        """Bounds on |d w|, |d n|, |d z| of one FTRL-Proximal application."""
+        w = self.w
+        dn = 2.0 * np.abs(G) * dG + dG * dG
+        rt = np.sqrt(n_new)
+        drt = np.minimum(dn / (2.0 * rt + 1e-300), np.sqrt(dn))
+        dz = dG + drt / w.ftrl_alpha * np.abs(w_old)
+        D = (w.ftrl_beta + rt) / w.ftrl_alpha + w.ftrl_l2
+        dw = 2.0 * (dz / D + np.abs(w_new) * (drt / w.ftrl_alpha) / D)
+        return dw, dn, dz
+
+    def compare_rows(self, fi, db, exact=False, gemm=False, what="rows", G=None, before=None):
         U = fi["U"]
+        w = self.w
         ref = self.o.read_rows(fi["uniq_shard"], fi["uniq_row"])
         got = self.t.read_rows(db.uniq_rows[:U])
+        adam = w.optimizer == synth.OPT_ADAM
+        ftrl = w.lin_optimizer == synth.LIN_FTRL
+        if adam or ftrl:
+            ref.update(self.o.read_state2(fi["uniq_shard"], fi["uniq_row"]))
+            got.update(self.t.read_state2(db.uniq_rows[:U]))
         torch.cuda.synchronize()
-        sgd = self.w.optimizer == synth.OPT_SGD
-        for name in ("emb", "lin", "acc_emb", "acc_lin"):
-            g = got[name].cpu().numpy()
-            if sgd and name.startswith("acc"):
-                continue
-            if exact:
-                assert np.array_equal(g.view(np.uint32), ref[name].view(np.uint32)), f"{what}.{name} bits"
-                continue
-            extra = None
-            if G is not None:
-                emb = name.endswith("emb")
+        sgd = w.optimizer == synth.OPT_SGD
+        names = ["emb", "lin", "acc_emb", "acc_lin"] + (["acc2_emb"] if adam else []) + (["lin2"] if adam or ftrl else [])
+        tol = {}
+        if G is not None:
+            for emb in (True, False):
                 Gk = (G["Gv"] if emb else G["Gw"]).astype(np.float64)
                 dG = RTOL * np.abs(Gk) + ATOL + SUMTOL * (G["Sv"] if emb else G["Sw"])
                 if gemm:
                     dG = dG + 2e-2 * np.abs(Gk) + 1e-3 * max(float(np.abs(Gk).max()), 1e-30)
-                if name.startswith("acc"):
-                    extra = 2.0 * np.abs(Gk) * dG + dG * dG
+                th, s1, s2 = ("emb", "acc_emb", "acc2_emb") if emb else ("lin", "acc_lin", "lin2")
+                if ftrl and not emb:
+                    tol[th], tol[s1], tol[s2] = self._ftrl_tol(Gk, dG, before["lin"].astype(np.float64),
+                                                               ref["lin"].astype(np.float64),
+                                                               ref["acc_lin"].astype(np.float64))
+                elif adam:
+                    tol[th], tol[s1], tol[s2] = self._adam_tol(Gk, dG, ref[s1].astype(np.float64),
+                                                               ref[s2].astype(np.float64))
                 elif sgd:
-                    extra = self.w.lr * dG
+                    tol[th] = w.lr * dG
                 else:
-                    acc = ref["acc_" + name].astype(np.float64)
-                    extra = self.w.lr * np.minimum(2.0, 2.0 * dG / (np.sqrt(acc) + self.w.eps))
-            (close_gemm if gemm else close32)(g, ref[name], f"{what}.{name}", extra=extra)
+                    acc = ref[s1].astype(np.float64)
+                    tol[s1] = 2.0 * np.abs(Gk) * dG + dG * dG
+                    tol[th] = w.lr * np.minimum(2.0, 2.0 * dG / (np.sqrt(acc) + w.eps))
+        for name in names:
+            g = got[name].cpu().numpy()
+            if sgd and name == "acc_emb":
+                continue
+            if sgd and name == "acc_lin" and not ftrl:
+                continue
+            if exact:
+                assert np.array_equal(g.view(np.uint32), ref[name].view(np.uint32)), f"{what}.{name} bits"
+                continue
+            (close_gemm if gemm else close32)(g, ref[name], f"{what}.{name}", extra=tol.get(name))
         return ref
 
     # ------------------------------------------------------------------
@@ -244,6 +286,8 @@ class Pair:
         g = grads
         gdev = {n: torch.from_numpy(v).to(dev) for n, v in g.items()}
         gE_work = torch.empty((B, F * k), device=dev) if (ops & OP_DENSE1) else None
+        before = self.o.read_rows(fi["uniq_shard"], fi["uniq_row"]) if w.lin_optimizer == synth.LIN_FTRL else None
+        self.nstep += 1
         ob = self.o.backward_update(ops, batch, fi, oa["A"].astype(np.float32),
                                     oa["pooled"].astype(np.float32) if oa["pooled"] is not None else None,
                                     g.get("gL"), g.get("gF"), g.get("gE") if (ops & OP_POOL) else None,
@@ -267,25 +311,37 @@ class Pair:
         if ops & OP_DENSE1:
             close_gemm(gE_work.cpu().numpy(), ob["gE_total"], "gE_total")
             W1o, accW1o = self.o.dense1_get()
+            acc2W1o = self.o.dense1_get_state2() if w.optimizer == synth.OPT_ADAM else None
             # same reasoning as for the rows: a 2e-2-relative error of the weight gradient, pushed
             # through one optimizer application (Adagrad divides by sqrt(acc))
             Gk = ob["gW1"].astype(np.float64)
             dG = 2e-2 * np.abs(Gk) + 1e-3 * max(float(np.abs(Gk).max()), 1e-30)
             if w.optimizer == synth.OPT_SGD:
                 extra = w.lr * dG
+            elif w.optimizer == synth.OPT_ADAM:
+                extra, dm, dv = self._adam_tol(Gk, dG, accW1o.astype(np.float64), acc2W1o.astype(np.float64))
+                s1, s2 = self.t.dense1_get_state(want2=True)
+                close_gemm(s1.cpu().numpy(), accW1o, "W1.m", extra=dm)
+                close_gemm(s2.cpu().numpy(), acc2W1o, "W1.v", extra=dv)
             else:
                 # G / sqrt(acc) is bounded by 1 and, for dG below |G|, moves by at most ~2 dG / sqrt(acc)
                 extra = w.lr * np.minimum(2.0, 2.0 * dG / (np.sqrt(accW1o.astype(np.float64)) + w.eps))
             close_gemm(self.t.dense1_get().cpu().numpy(), W1o, "W1", extra=extra)
-        ref = self.compare_rows(fi, db, gemm=gemm, what="updated rows", G=ob)
+        ref = self.compare_rows(fi, db, gemm=gemm, what="updated rows", G=ob, before=before)
         if self.resync:
             U = fi["U"]
             td = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
             sgd = w.optimizer == synth.OPT_SGD
+            ftrl = w.lin_optimizer == synth.LIN_FTRL
             self.t.write_rows(db.uniq_rows[:U], td(ref["emb"]), td(ref["lin"]),
-                              None if sgd else td(ref["acc_emb"]), None if sgd else td(ref["acc_lin"]))
+                              None if sgd else td(ref["acc_emb"]), None if (sgd and not ftrl) else td(ref["acc_lin"]))
+            if "lin2" in ref:
+                self.t.write_state2(db.uniq_rows[:U], td(ref["acc2_emb"]) if "acc2_emb" in ref and w.optimizer == synth.OPT_ADAM else None,
+                                    td(ref["lin2"]))
             if W1o is not None:
                 self.t.dense1_set(td(W1o))
+                if not sgd:
+                    self.t.dense1_set_state(td(accW1o), None if acc2W1o is None else td(acc2W1o))
             torch.cuda.synchronize()
         else:
             self.drifted = True

@@ -323,3 +323,136 @@ def test_paper_table2_comm_saving():
         got = 100.0 * oracle.comm_saving(B, U, 8, 256, 4800 * 256 * 4)
         for gv, want in zip(got, r[2:5]):
             assert f"{gv:.3f}" == want
+
+
+# --------------------------------------------------------------------------- Adam / FTRL
+def _one_key_per_sample(keys, F=1):
+    n = len(keys)
+    return synth.Batch(n, F, np.arange(n + 1, dtype=np.int32), np.asarray(keys, dtype=np.uint64), None)
+
+
+def test_adam_equals_library_adam_when_every_key_is_touched():
+    # With every key in every batch the lazy per-key Adam is plain dense Adam.
+    from paper_1909_04823_b200.synth import OPT_ADAM
+    n, k, lr, eps = 7, 4, 0.05, 1e-8
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    b = _one_key_per_sample(keys)
+    o = Oracle(3, 1, k, 0, PART_HASH, OPT_ADAM, seed=5, init_scale=0.5, lr=lr, eps=eps)
+    o.set_opt(0, 0.9, 0.999)
+    f = o.find_or_insert(b)
+    assert f["U"] == n and np.array_equal(f["uidx"], np.arange(n))
+    P = torch.tensor(o.read_rows(f["uniq_shard"], f["uniq_row"])["emb"], dtype=torch.float64, requires_grad=True)
+    Pl = torch.zeros(n, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([P, Pl], lr=lr, betas=(0.9, 0.999), eps=eps)
+    rng = np.random.default_rng(3)
+    for step in range(6):
+        gE = rng.standard_normal((n, k)).astype(np.float32)
+        gL = rng.standard_normal(n).astype(np.float32)
+        o.backward_update(OP_LR | OP_POOL, b, f, np.zeros((n, k)), None, gL, None, gE)
+        P.grad = torch.from_numpy(gE.astype(np.float64)); Pl.grad = torch.from_numpy(gL.astype(np.float64))
+        opt.step()
+        r = o.read_rows(f["uniq_shard"], f["uniq_row"])
+        np.testing.assert_allclose(r["emb"], P.detach().numpy(), rtol=2e-5, atol=2e-7)
+        np.testing.assert_allclose(r["lin"], Pl.detach().numpy(), rtol=2e-5, atol=2e-7)
+    st = opt.state[P]
+    r2 = o.read_state2(f["uniq_shard"], f["uniq_row"])
+    np.testing.assert_allclose(r["acc_emb"], st["exp_avg"].numpy(), rtol=2e-5, atol=1e-7)
+    np.testing.assert_allclose(r2["acc2_emb"], st["exp_avg_sq"].numpy(), rtol=2e-5, atol=1e-9)
+    np.testing.assert_allclose(r2["lin2"], opt.state[Pl]["exp_avg_sq"].numpy(), rtol=2e-5, atol=1e-9)
+
+
+def test_adam_is_lazy_with_one_global_step_count():
+    # Keys absent from a batch keep value and moments; bias correction uses the number of
+    # backward calls so far.  The library's sparse Adam has exactly these semantics (its
+    # epsilon sits at a slightly different place, far below the tolerance here).
+    from paper_1909_04823_b200.synth import OPT_ADAM
+    n, k, lr = 9, 4, 0.03
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    o = Oracle(2, 1, k, 0, PART_HASH, OPT_ADAM, seed=6, init_scale=0.5, lr=lr, eps=1e-8)
+    o.set_opt(0, 0.9, 0.999)
+    fall = o.find_or_insert(_one_key_per_sample(keys))
+    P = torch.tensor(o.read_rows(fall["uniq_shard"], fall["uniq_row"])["emb"], dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SparseAdam([P], lr=lr, betas=(0.9, 0.999), eps=1e-8)
+    rng = np.random.default_rng(4)
+    for step in range(8):
+        sub = np.sort(rng.choice(n, size=rng.integers(1, n), replace=False))
+        b = _one_key_per_sample(keys[sub])
+        f = o.find_or_insert(b)
+        gE = rng.standard_normal((len(sub), k)).astype(np.float32)
+        before = o.read_rows(fall["uniq_shard"], fall["uniq_row"])
+        o.backward_update(OP_POOL, b, f, np.zeros((len(sub), k)), None, None, None, gE)
+        after = o.read_rows(fall["uniq_shard"], fall["uniq_row"])
+        rest = np.setdiff1d(np.arange(n), sub)
+        for name in ("emb", "acc_emb"):
+            assert np.array_equal(before[name][rest], after[name][rest])
+        P.grad = torch.sparse_coo_tensor(torch.from_numpy(sub)[None], torch.from_numpy(gE.astype(np.float64)), (n, k), check_invariants=False)
+        opt.step()
+        np.testing.assert_allclose(after["emb"], P.detach().numpy(), rtol=2e-5, atol=2e-7)
+
+
+def _ftrl_oracle(alpha, beta, l1, l2, n=6):
+    from paper_1909_04823_b200.synth import LIN_FTRL
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    o = Oracle(2, 1, 4, 0, PART_HASH, OPT_SGD, seed=7, init_scale=0.5, lr=0.1, eps=1e-8)
+    o.set_opt(LIN_FTRL, 0.9, 0.999, alpha, beta, l1, l2)
+    b = _one_key_per_sample(keys)
+    f = o.find_or_insert(b)
+    return o, b, f
+
+
+def test_ftrl_without_regularisation_is_per_coordinate_gradient_descent():
+    # l1 = l2 = beta = 0: FTRL-Proximal coincides with w <- w - (alpha / sqrt(n_t)) g_t.
+    alpha, n = 0.2, 6
+    o, b, f = _ftrl_oracle(alpha, 0.0, 0.0, 0.0, n)
+    rng = np.random.default_rng(8)
+    w = np.zeros(n); nn = np.zeros(n)
+    for step in range(10):
+        gL = rng.standard_normal(n).astype(np.float32)
+        o.backward_update(OP_LR, b, f, np.zeros((n, 4)), None, gL, None, None)
+        g = gL.astype(np.float64)
+        nn += g * g
+        w -= alpha / np.sqrt(nn) * g
+        np.testing.assert_allclose(o.read_rows(f["uniq_shard"], f["uniq_row"])["lin"], w, rtol=1e-4, atol=1e-6)
+    np.testing.assert_allclose(o.read_rows(f["uniq_shard"], f["uniq_row"])["acc_lin"], nn, rtol=1e-5)
+
+
+def test_ftrl_weight_minimises_the_proximal_objective():
+    # Definition: w_{t+1} = argmin_w  g_{1:t} w + 1/2 sum_s sigma_s (w - w_s)^2 + (beta / 2 alpha) w^2
+    #                                 + l1 |w| + (l2 / 2) w^2,   sigma_s = (sqrt(n_s) - sqrt(n_{s-1})) / alpha.
+    from scipy.optimize import minimize_scalar
+    alpha, beta, l1, l2, n = 0.3, 1.0, 0.4, 0.05, 5
+    o, b, f = _ftrl_oracle(alpha, beta, l1, l2, n)
+    rng = np.random.default_rng(9)
+    gs, ws, zero_seen, nonzero_seen = [], [np.zeros(n)], 0, 0
+    for step in range(9):
+        gL = (rng.standard_normal(n) * (0.3 if step < 2 else 1.0)).astype(np.float32)
+        o.backward_update(OP_LR, b, f, np.zeros((n, 4)), None, gL, None, None)
+        gs.append(gL.astype(np.float64))
+        got = o.read_rows(f["uniq_shard"], f["uniq_row"])["lin"].astype(np.float64)
+        G = np.array(gs)
+        rootn = np.sqrt(np.cumsum(G * G, axis=0))
+        sig = np.diff(np.concatenate([np.zeros((1, n)), rootn]), axis=0) / alpha
+        W = np.array(ws)
+        for i in range(n):
+            obj = lambda x: (G[:, i].sum() * x + 0.5 * np.sum(sig[:, i] * (x - W[:, i]) ** 2)
+                             + 0.5 * beta / alpha * x * x + l1 * abs(x) + 0.5 * l2 * x * x)
+            res = minimize_scalar(obj, bounds=(-5, 5), method="bounded", options=dict(xatol=1e-10))
+            assert abs(got[i] - res.x) < 2e-6, (step, i, got[i], res.x)
+            assert obj(got[i]) <= obj(res.x) + 1e-12
+            zero_seen += got[i] == 0.0
+            nonzero_seen += got[i] != 0.0
+        ws.append(got)
+    assert zero_seen >= 3 and nonzero_seen >= 10      # both branches of the soft threshold were exercised
+
+
+def test_ftrl_l1_keeps_small_weights_at_exact_zero():
+    o, b, f = _ftrl_oracle(0.1, 1.0, 100.0, 0.0, 6)
+    rng = np.random.default_rng(10)
+    tot = np.zeros(6)
+    for step in range(5):
+        gL = rng.standard_normal(6).astype(np.float32)
+        o.backward_update(OP_LR, b, f, np.zeros((6, 4)), None, gL, None, None)
+        tot += gL
+        assert not np.any(o.read_rows(f["uniq_shard"], f["uniq_row"])["lin"])
+    # with every weight still zero, z is the plain gradient sum
+    np.testing.assert_allclose(o.read_state2(f["uniq_shard"], f["uniq_row"])["lin2"], tot, rtol=1e-5, atol=1e-6)
