@@ -29,6 +29,9 @@
 #define HOT_MIN 512u      // estimated occurrences from which a key is treated as hot
 #define HOT_CHAIN 256u    // target number of additions per replica row
 #define HOT_RCHUNK 64u    // replica rows summed by one warp of the reduction
+#define SUPER_T 16u       // keys whose occurrences are summed in registers instead of by atomics
+#define SUPER_R 64u       // replica rows of such a key (they only take one partial sum per lane group)
+#define SUPER_TAG 0xFFFFFF00u   // dest[j] = SUPER_TAG | slot for an occurrence of such a key
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
   x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
                                                          long long max_uniq, int shift, uint32_t* hot_base,
                                                          uint32_t* hot_R, uint32_t* hot_u, uint32_t* ctr,
                                                          uint32_t h_max, uint32_t rep_max, DevMeta* meta,
-                                                         uint32_t* hot_work, uint32_t work_max) {
+                                                         uint32_t* hot_work, uint32_t work_max, uint32_t super_min) {
   long long U = *n_uniq;
   if (U > max_uniq) {           // the gradient buffer cannot hold this batch: report, update what fits
     if (blockIdx.x == 0 && threadIdx.x == 0) des_raise(meta, DES_ERR_CAPACITY);
@@ -66,7 +69,12 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
     const uint32_t est = hinfo[u] << shift;
     uint32_t h = DES_ROW_NONE;
     if (est >= HOT_MIN) {
-      const uint32_t R = (est + HOT_CHAIN - 1) / HOT_CHAIN;
+      // the few keys that own a large share of the batch (super_min = 0: feature off) take one of
+      // SUPER_T slots: ctr[3] = slots claimed, ctr[4 + slot] = hot index; hinfo carries slot + 1 in bits 24..
+      bool sup = false;
+      uint32_t ts = 0;
+      if (super_min && est >= super_min) { ts = atomicAdd(&ctr[3], 1u); sup = ts < SUPER_T; }
+      const uint32_t R = sup ? SUPER_R : (est + HOT_CHAIN - 1) / HOT_CHAIN;
       const uint32_t hh = atomicAdd(&ctr[0], 1u);
       if (hh < h_max) {
         const uint32_t base = atomicAdd(&ctr[1], R);
@@ -75,12 +83,14 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
         uint32_t wbase = 0;
         if (ok) { wbase = atomicAdd(&ctr[2], nchunk); ok = wbase + nchunk <= work_max; }
         if (ok) {
-          hot_base[hh] = base; hot_R[hh] = R; hot_u[hh] = (uint32_t)u; h = hh;
+          hot_base[hh] = base; hot_R[hh] = R; hot_u[hh] = (uint32_t)u;
+          h = hh | (sup ? (ts + 1u) << 24 : 0u);
           for (uint32_t i = 0; i < nchunk; ++i) hot_work[wbase + i] = (hh << 18) | i;
         } else {
           hot_R[hh] = 0;
         }
       }
+      if (sup) ctr[4 + ts] = (h == DES_ROW_NONE) ? DES_ROW_NONE : (h & 0xFFFFFFu);
     }
     hinfo[u] = h;
   }
@@ -97,8 +107,14 @@ __global__ void __launch_bounds__(256) make_dest_kernel(const uint32_t* __restri
   const uint32_t u = __ldg(uidx + j);
   uint32_t d = DES_ROW_NONE;
   if (u != DES_ROW_NONE && (long long)u < max_uniq) {
-    const uint32_t h = __ldg(hinfo + u);
-    d = (h == DES_ROW_NONE) ? u : (uint32_t)max_uniq + __ldg(hot_base + h) + hash_u32((uint32_t)j) % __ldg(hot_R + h);
+    const uint32_t hv = __ldg(hinfo + u);
+    if (hv == DES_ROW_NONE) {
+      d = u;
+    } else if (hv >> 24) {
+      d = SUPER_TAG | ((hv >> 24) - 1u);
+    } else {
+      d = (uint32_t)max_uniq + __ldg(hot_base + hv) + hash_u32((uint32_t)j) % __ldg(hot_R + hv);
+    }
   }
   dest[j] = d;
 }
@@ -152,20 +168,28 @@ __global__ void __launch_bounds__(256) hot_finish_kernel(const uint32_t* __restr
   }
 }
 
-template <int G>
+// SUPER (16-lane groups only): occurrences of the few keys that own a large share of a skewed
+// batch (dest = SUPER_TAG | slot) send no atomics.  Lane t of the group counts the bag's
+// occurrences of slot t — every lane sees every dest[j] anyway — and the counts go to
+// super_cnt[bag][16]; super_dense_kernel turns them into the keys' gradient sums.
+template <int G, bool SUPER>
 __global__ void __launch_bounds__(256) grad_scatter_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ dest,
     long long nbags, int F, int k, uint32_t ops, const float* __restrict__ out_small,
-    const float* __restrict__ gL, const float* __restrict__ gF, const float* __restrict__ gE, float* Gbuf) {
+    const float* __restrict__ gL, const float* __restrict__ gF, const float* __restrict__ gE, float* Gbuf,
+    uint16_t* __restrict__ super_cnt) {
   const int K4 = k >> 2, stride = k + 4;
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long bag = t / G;
   const int c4 = (int)(t % G);
   if (bag >= nbags) return;
   const int lo = __ldg(offsets + bag), hi = __ldg(offsets + bag + 1);
-  if (lo == hi) return;
+  if (lo == hi) {
+    if (SUPER) super_cnt[bag * 16 + c4] = 0;
+    return;
+  }
   const bool col = c4 < K4;
-  if (!col && c4 != 0) return;
+  if (!SUPER && !col && c4 != 0) return;
   const long long b = bag / F;
   const float gf = (ops & DES_OP_FM) ? __ldg(gF + b) : 0.f;
   const float gl = (ops & DES_OP_LR) ? __ldg(gL + b) : 0.f;
@@ -180,22 +204,150 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
       c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
     }
   }
+  uint32_t cnt = 0;
+  const uint32_t mine = SUPER_TAG | (uint32_t)c4;
   for (int j = lo; j < hi; ++j) {
     const uint32_t u = __ldg(dest + j);
-    if (u == DES_ROW_NONE) continue;
+    if (SUPER) {
+      cnt += (u == mine);
+      if (u >= SUPER_TAG) continue;                   // counted, or no row
+    } else if (u == DES_ROW_NONE) {
+      continue;
+    }
     const float x = vals ? __ldg(vals + j) : 1.f;
     float* row = Gbuf + (size_t)u * stride;
     if (col) atomicAdd(reinterpret_cast<float4*>(row) + c4, make_float4(x * c.x, x * c.y, x * c.z, x * c.w));
     if (c4 == 0) atomicAdd(reinterpret_cast<float4*>(row) + K4, make_float4(x * gl, x * x * gf, 0.f, 0.f));
   }
+  if (SUPER) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
+}
+
+// Gradient sums of the SUPER_T marked keys as a dense product:
+//   G_t = sum over bags of count[bag][t] * c_bag,   tail_t = sum of count * (gL[b], gF[b]),
+// with c_bag rebuilt from gE and the aggregated forward exactly as in the scatter.  A CTA
+// stages SD_TILE bags (c_bag rows, counts, gL / gF) in shared memory; thread (t, c4) owns the
+// accumulator of key t, 16-byte column c4.  Each CTA adds its sums to one replica row per key
+// (summed in double by hot_reduce).  All feature values are 1 on this path.
+#define SD_TILE 32
+#define SD_THREADS 288   // 256 column threads + one warp for the linear-weight tails
+__global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
+    const uint16_t* __restrict__ super_cnt, int nbags, int F, int k, uint32_t ops,
+    const float* __restrict__ out_small, const float* __restrict__ gL, const float* __restrict__ gF,
+    const float* __restrict__ gE, float* Gbuf, const uint32_t* __restrict__ ctr,
+    const uint32_t* __restrict__ hot_base, const uint32_t* __restrict__ hot_R, long long max_uniq) {
+  uint32_t ns = __ldg(ctr + 3);
+  if (ns == 0) return;
+  if (ns > SUPER_T) ns = SUPER_T;
+  __shared__ float4 s_c[SD_TILE][16];
+  __shared__ __align__(16) float s_n[SD_TILE][16];
+  __shared__ float2 s_g[SD_TILE];
+  const int K4 = k >> 2, stride = k + 4;
+  const int tid = threadIdx.x;
+  const bool tailw = tid >= 256;                       // the extra warp
+  // staging role (threads < 256): thread (tk, c4) fetches column c4 of bags tk and tk + 16 of a tile
+  const int c4 = tid & 15, tk = (tid >> 4) & 15;
+  // multiply role (threads < 256): column c4, keys 4 kg .. 4 kg + 3, bags sub, sub + 4, ...
+  const int kg = (tid >> 4) & 3, sub = (tid >> 6) & 3;
+  // tail role (extra warp): key tt, bags th, th + 2, ...
+  const int tt = tid & 15, th = (tid >> 4) & 1;
+  const bool col = c4 < K4, fm = ops & DES_OP_FM, lr = ops & DES_OP_LR;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 acc[4] = {zero, zero, zero, zero};
+  float tw = 0.f, tq = 0.f;
+  float4 e[2], a[2];
+  float gfv[2], nv[2];
+  float2 g2;
+  auto fetch = [&](int base) {
+    if (tailw) {
+      g2 = make_float2(0.f, 0.f);
+      const int i = tid - 256;
+      if (base + i < nbags) {
+        const int b = (base + i) / F;
+        g2.x = lr ? __ldg(gL + b) : 0.f;
+        g2.y = fm ? __ldg(gF + b) : 0.f;
+      }
+      return;
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int bag = base + r * 16 + tk;
+      e[r] = zero; a[r] = zero; gfv[r] = 0.f; nv[r] = 0.f;
+      if (bag < nbags) {
+        const int b = bag / F;
+        nv[r] = (float)__ldg(super_cnt + (size_t)bag * 16 + c4);
+        if (col && gE) e[r] = __ldg(reinterpret_cast<const float4*>(gE + (size_t)bag * k) + c4);
+        if (col && fm) { a[r] = __ldg(reinterpret_cast<const float4*>(out_small + (size_t)b * stride) + c4); gfv[r] = __ldg(gF + b); }
+      }
+    }
+  };
+  const int tstep = gridDim.x * SD_TILE;
+  int base = blockIdx.x * SD_TILE;
+  if (base < nbags) fetch(base);
+  for (; base < nbags; base += tstep) {
+    __syncthreads();                                   // previous tile fully consumed
+    if (tailw) {
+      s_g[tid - 256] = g2;
+    } else {
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int i = r * 16 + tk;
+        s_c[i][c4] = make_float4(fmaf(gfv[r], a[r].x, e[r].x), fmaf(gfv[r], a[r].y, e[r].y),
+                                 fmaf(gfv[r], a[r].z, e[r].z), fmaf(gfv[r], a[r].w, e[r].w));
+        s_n[i][c4] = nv[r];
+      }
+    }
+    __syncthreads();
+    if (base + tstep < nbags) fetch(base + tstep);     // in flight while this tile is multiplied
+    if (tailw) {
+#pragma unroll 4
+      for (int i = th; i < SD_TILE; i += 2) {
+        const float f = s_n[i][tt];
+        const float2 gg = s_g[i];
+        tw = fmaf(f, gg.x, tw); tq = fmaf(f, gg.y, tq);
+      }
+    } else {
+#pragma unroll
+      for (int i = sub; i < SD_TILE; i += 4) {
+        const float4 f = *reinterpret_cast<const float4*>(&s_n[i][kg * 4]);
+        const float4 c = s_c[i][c4];
+        acc[0].x = fmaf(f.x, c.x, acc[0].x); acc[0].y = fmaf(f.x, c.y, acc[0].y);
+        acc[0].z = fmaf(f.x, c.z, acc[0].z); acc[0].w = fmaf(f.x, c.w, acc[0].w);
+        acc[1].x = fmaf(f.y, c.x, acc[1].x); acc[1].y = fmaf(f.y, c.y, acc[1].y);
+        acc[1].z = fmaf(f.y, c.z, acc[1].z); acc[1].w = fmaf(f.y, c.w, acc[1].w);
+        acc[2].x = fmaf(f.z, c.x, acc[2].x); acc[2].y = fmaf(f.z, c.y, acc[2].y);
+        acc[2].z = fmaf(f.z, c.z, acc[2].z); acc[2].w = fmaf(f.z, c.w, acc[2].w);
+        acc[3].x = fmaf(f.w, c.x, acc[3].x); acc[3].y = fmaf(f.w, c.y, acc[3].y);
+        acc[3].z = fmaf(f.w, c.z, acc[3].z); acc[3].w = fmaf(f.w, c.w, acc[3].w);
+      }
+    }
+  }
+  // each (CTA, bag subset) hands its sums to one replica row per key
+  const uint32_t salt = hash_u32(blockIdx.x * 4u + (uint32_t)(tailw ? th : sub));
+  if (tailw) {
+    if ((uint32_t)tt >= ns) return;
+    const uint32_t hh = __ldg(ctr + 4 + tt);
+    if (hh == DES_ROW_NONE) return;
+    const uint32_t R = __ldg(hot_R + hh);
+    if (R == 0) return;
+    float* row = Gbuf + ((size_t)max_uniq + __ldg(hot_base + hh) + salt % R) * stride;
+    atomicAdd(reinterpret_cast<float4*>(row) + K4, make_float4(tw, tq, 0.f, 0.f));
+    return;
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint32_t key = (uint32_t)(kg * 4 + q);
+    if (key >= ns || !col) continue;
+    const uint32_t hh = __ldg(ctr + 4 + key);
+    if (hh == DES_ROW_NONE) continue;
+    const uint32_t R = __ldg(hot_R + hh);
+    if (R == 0) continue;
+    float* row = Gbuf + ((size_t)max_uniq + __ldg(hot_base + hh) + salt % R) * stride;
+    atomicAdd(reinterpret_cast<float4*>(row) + c4, acc[q]);
+  }
 }
 
 #define UP_UNROLL 4
 
-// One optimizer application per unique key.  A group of G lanes owns a key (one
-// 16-byte column each, lane 0 also the linear weight); it works on UP_UNROLL
-// keys at a time so that their gradient rows, row numbers, weights and state
-// are all in flight together: the kernel is a pure stream of 272-byte rows.
 // Advances Adam's step count and recomputes the bias corrections 1 - beta^t in double.
 __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
   const unsigned long long t = meta->opt_step + 1;
@@ -204,6 +356,10 @@ __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
   meta->adam_c2 = (float)(1.0 - pow((double)beta2, (double)t));
 }
 
+// One optimizer application per unique key.  A group of G lanes owns a key (one
+// 16-byte column each, lane 0 also the linear weight); it works on UP_UNROLL
+// keys at a time so that their gradient rows, row numbers, weights and state
+// are all in flight together: the kernel is a pure stream of 272-byte rows.
 template <int G>
 __global__ void __launch_bounds__(256) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
@@ -320,24 +476,37 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   // hot-key detection on a sample, replica assignment, per-occurrence destination row
   int shift = 0;
   while (shift < 6 && ((long long)nnz >> shift) > (1ll << 20)) ++shift;
-  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 16, cs));
+  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 128, cs));
+  // skewed-batch scatter: 16-lane groups, unit feature values, batches large enough to fill a persistent grid
+  const bool use_super = G == 16 && !b->vals && nnz >= (1 << 20) && t->super_cnt;
+  const uint32_t super_min = use_super ? (uint32_t)(nnz >> 7) : 0u;
   {
     const int n = (nnz >> shift) + 1;
     sample_count_kernel<<<(n + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
     DES_LAUNCH_CHECK(t, "sample_count_kernel");
     hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
                                                        t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
-                                                       t->hot_work, t->work_max);
+                                                       t->hot_work, t->work_max, super_min);
     DES_LAUNCH_CHECK(t, "hot_select_kernel");
     make_dest_kernel<<<(nnz + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
                                                         t->dest);
     DES_LAUNCH_CHECK(t, "make_dest_kernel");
   }
-  {
+  if (use_super) {
+    const unsigned grid = (unsigned)((nbags * 16 + 255) / 256);
+    grad_scatter_kernel<16, true><<<grid, 256, 0, cs>>>(b->offsets, nullptr, t->dest, nbags, t->F, t->k, ops,
+                                                        out->out_small, gr->gL, gr->gF, gE, t->Gbuf, t->super_cnt);
+    DES_LAUNCH_CHECK(t, "grad_scatter_kernel");
+    super_dense_kernel<<<t->sm_count * 3, SD_THREADS, 0, cs>>>(t->super_cnt, (int)nbags, t->F, t->k, ops, out->out_small, gr->gL,
+                                                        gr->gF, gE, t->Gbuf, t->hot_ctr, t->hot_base, t->hot_R,
+                                                        t->max_uniq);
+    DES_LAUNCH_CHECK(t, "super_dense_kernel");
+  } else {
     const long long threads = nbags * G;
     const unsigned grid = (unsigned)((threads + 255) / 256);
-#define SC(GG) grad_scatter_kernel<GG><<<grid, 256, 0, cs>>>(b->offsets, b->vals, t->dest, nbags, t->F, t->k, ops, \
-                                                            out->out_small, gr->gL, gr->gF, gE, t->Gbuf)
+#define SC(GG) grad_scatter_kernel<GG, false><<<grid, 256, 0, cs>>>(b->offsets, b->vals, t->dest, nbags, t->F, t->k,  \
+                                                                   ops, out->out_small, gr->gL, gr->gF, gE, t->Gbuf, \
+                                                                   nullptr)
     switch (G) { case 1: SC(1); break; case 2: SC(2); break; case 4: SC(4); break; case 8: SC(8); break; default: SC(16); }
 #undef SC
     DES_LAUNCH_CHECK(t, "grad_scatter_kernel");

@@ -13,12 +13,12 @@
 //                 sort (warp match + running cursors), writing the table-global
 //                 row of every occurrence in shard-major order, the segment
 //                 bounds [B][S+1], and the same rows in CSR order for pooling.
-//  shard_partials_kernel   one group of G = k/4 lanes (rounded up to a power of
-//                 two) per sample walks the sample's (sample, shard) segments in
-//                 shard order: it streams a segment's rows with 16-byte loads,
-//                 SP_UNROLL in flight, and keeps M_1, M_1^lr, M_2 in registers
-//                 until the segment ends — no shared memory, no atomics, sums in
-//                 CSR order (deterministic).  M_2 uses the |v|^2 cached in the
+//  shard_partials_kernel   one warp per sample (32 / G sub-groups of G = k/4
+//                 lanes, rounded up to a power of two) walks the sample's
+//                 (sample, shard) segments in shard order: it streams a segment's
+//                 rows with 16-byte loads, SP_UNROLL in flight per lane, and keeps
+//                 M_1, M_1^lr, M_2 in registers until the segment ends — no shared
+//                 memory, no atomics, a fixed summation order (deterministic).  M_2 uses the |v|^2 cached in the
 //                 row's 16-byte tail.  Fused variant: (+) over shards and F on chip.
 //  pool_kernel    one group per bag: sum pooling of the latent vectors in
 //                 registers.  The per-shard pooled partial [S][B][F*k] is only
@@ -88,75 +88,105 @@ __global__ void __launch_bounds__(256) route_kernel(
   }
 }
 
-// One group of G lanes per SAMPLE walks the sample's S segments in shard order.
-// Every group has the same amount of work (a sample's occurrences), whatever the
-// skew between shards.  part_small (optional) receives each segment's partial
-// sums as soon as the segment ends; with FUSED the aggregation (+) over shards
-// and the substitution operator F are applied on chip, in the same shard order
-// and with the same arithmetic as aggregate_small_kernel, and out_small is
+// One WARP per sample walks the sample's S segments in shard order.  The warp is
+// split into P = 32 / G sub-groups of G lanes (one 16-byte column per lane);
+// sub-group p takes occurrences p, p + P, ... of a segment, SP_UNROLL of them in
+// flight, and the sub-groups' sums are combined by a butterfly when the segment
+// ends — so both halves of a warp always run the same trip counts, whatever the
+// skew between shards, and every warp has the same amount of work (a sample's
+// occurrences).  The loop body is kept to the loads and adds: whole iterations
+// carry no bound checks, row addresses are one multiply-add from a per-lane base,
+// and lanes without a column of their own (k not a multiple of 4 G) re-read
+// column 0 instead of branching.  part_small (optional) receives each segment's
+// partial sums as soon as the segment ends; with FUSED the aggregation (+) over
+// shards and the substitution operator F are applied on chip, in the same shard
+// order and with the same arithmetic as aggregate_small_kernel, and out_small is
 // written directly — the per-shard partials then never touch memory.
 template <int G, bool HAS_VALS, bool FUSED>
 __global__ void __launch_bounds__(256) shard_partials_kernel(
     const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted, const int32_t* __restrict__ seg_off,
     int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small,
     float* __restrict__ out_small) {
+  constexpr int P = 32 / G;
   const int K4 = k >> 2, stride = k + 4;
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long b = t / G;
-  const int c4 = (int)(t % G);
-  const bool live = b < B;
-  const bool col = live && c4 < K4, lead = live && c4 == 0;
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (b >= B) return;                                  // whole warp
+  const int c4 = lane % G, p = lane / G;
+  const bool col = c4 < K4;
   const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  const unsigned rowB = (unsigned)stride * 4u;         // bytes per row
+  const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
+  const char* Wt = reinterpret_cast<const char*>(W + k);                       // (w, |v|^2)
   float4 A = zero4; float R = 0.f, Q = 0.f;            // FUSED: (+)M_1, (+)M_1^lr, (+)M_2
-  if (col || lead) {
-    const int32_t* so = seg_off + (size_t)b * (S + 1);
-    int hi = __ldg(so);
-    for (int s = 0; s < S; ++s) {
-      const int lo = hi;
-      hi = __ldg(so + s + 1);
-      float4 acc = zero4;
-      float m1lr = 0.f, m2 = 0.f;
-      for (int i0 = lo; i0 < hi; i0 += SP_UNROLL) {
-        float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
+  const int32_t* so = seg_off + (size_t)b * (S + 1);
+  int hi = __ldg(so);
+  for (int s = 0; s < S; ++s) {
+    const int lo = hi;
+    hi = __ldg(so + s + 1);
+    float4 acc = zero4;
+    float m1lr = 0.f, m2 = 0.f;
+    int i0 = lo;
+    for (; i0 + SP_UNROLL * P <= hi; i0 += SP_UNROLL * P) {
+      float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
 #pragma unroll
-        for (int u = 0; u < SP_UNROLL; ++u) {
-          v[u] = zero4; tl[u] = make_float2(0.f, 0.f); x[u] = 1.f;
-          if (i0 + u < hi) {
-            const float* wr = W + (size_t)__ldg(grow_sorted + i0 + u) * stride;
-            if (HAS_VALS) x[u] = __ldg(x_sorted + i0 + u);
-            if (col) v[u] = __ldg(reinterpret_cast<const float4*>(wr) + c4);
-            if (lead) tl[u] = __ldg(reinterpret_cast<const float2*>(wr + k));      // (w, |v|^2)
-          }
-        }
+      for (int u = 0; u < SP_UNROLL; ++u) {
+        const int i = i0 + u * P + p;
+        const size_t off = (size_t)__ldg(grow_sorted + i) * rowB;
+        if (HAS_VALS) x[u] = __ldg(x_sorted + i);
+        v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
+        tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
+      }
 #pragma unroll
-        for (int u = 0; u < SP_UNROLL; ++u) {
-          if (HAS_VALS) {
-            acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
-            m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
-          } else {
-            acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
-            m1lr += tl[u].x; m2 += tl[u].y;
-          }
+      for (int u = 0; u < SP_UNROLL; ++u) {
+        if (HAS_VALS) {
+          acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
+          m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
+        } else {
+          acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+          m1lr += tl[u].x; m2 += tl[u].y;
         }
       }
-      if (!fm) { acc = zero4; m2 = 0.f; }
-      if (!lr) m1lr = 0.f;
-      if (part_small) {
-        float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
-        if (col) dst[c4] = acc;
-        if (lead) dst[K4] = make_float4(m1lr, m2, 0.f, 0.f);
-      }
-      if (FUSED) { A.x += acc.x; A.y += acc.y; A.z += acc.z; A.w += acc.w; R += m1lr; Q += m2; }
     }
+    for (; i0 < hi; i0 += P) {                         // ragged end of the segment
+      const int i = i0 + p;
+      if (i < hi) {
+        const size_t off = (size_t)__ldg(grow_sorted + i) * rowB;
+        const float x = HAS_VALS ? __ldg(x_sorted + i) : 1.f;
+        const float4 v = __ldg(reinterpret_cast<const float4*>(Wc + off));
+        const float2 tl = __ldg(reinterpret_cast<const float2*>(Wt + off));
+        if (HAS_VALS) {
+          acc.x += v.x * x; acc.y += v.y * x; acc.z += v.z * x; acc.w += v.w * x;
+          m1lr += tl.x * x; m2 += tl.y * x * x;
+        } else {
+          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+          m1lr += tl.x; m2 += tl.y;
+        }
+      }
+    }
+#pragma unroll
+    for (int d = G; d < 32; d <<= 1) {                 // combine the sub-groups (same result in every lane)
+      acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
+      acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
+      m1lr += __shfl_xor_sync(0xFFFFFFFFu, m1lr, d); m2 += __shfl_xor_sync(0xFFFFFFFFu, m2, d);
+    }
+    if (!fm) { acc = zero4; m2 = 0.f; }
+    if (!lr) m1lr = 0.f;
+    if (part_small && p == 0) {
+      float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
+      if (col) dst[c4] = acc;
+      if (c4 == 0) dst[K4] = make_float4(m1lr, m2, 0.f, 0.f);
+    }
+    if (FUSED) { A.x += acc.x; A.y += acc.y; A.z += acc.z; A.w += acc.w; R += m1lr; Q += m2; }
   }
   if (FUSED) {
-    double aa = (double)A.x * A.x + (double)A.y * A.y + (double)A.z * A.z + (double)A.w * A.w;
+    double aa = col ? (double)A.x * A.x + (double)A.y * A.y + (double)A.z * A.z + (double)A.w * A.w : 0.0;
 #pragma unroll
     for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
-    float4* o = reinterpret_cast<float4*>(out_small + (size_t)(live ? b : 0) * stride);
-    if (col) o[c4] = A;
-    if (lead) o[K4] = make_float4(R, fm ? (float)(0.5 * aa - 0.5 * (double)Q) : 0.f, Q, 0.f);
+    float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
+    if (p == 0 && col) o[c4] = A;
+    if (lane == 0) o[K4] = make_float4(R, fm ? (float)(0.5 * aa - 0.5 * (double)Q) : 0.f, Q, 0.f);
   }
 }
 
@@ -267,8 +297,7 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
       b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, grow_csr, grow_sorted, x_sorted, t->seg_off);
   DES_LAUNCH_CHECK(t, "route_kernel");
   if (ps || fused_out) {
-    const long long threads = (long long)B * G;
-    const unsigned grid = (unsigned)((threads + 255) / 256);
+    const unsigned grid = (unsigned)((B + 7) / 8);      // one warp per sample
 #define SP3(GG, HV, FU) shard_partials_kernel<GG, HV, FU><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, \
                                                                               t->k, ops, t->W, ps, fused_out)
 #define SP(GG) do { if (fused_out) { if (b->vals) SP3(GG, true, true); else SP3(GG, false, true); } \

@@ -98,7 +98,7 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->A2, t->acc2W1, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
-                  t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc,
+                  t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc, t->super_cnt,
                   t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
   for (void* p : ptrs) dfree(t->cfg, p);
@@ -187,6 +187,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   t->work_max = t->rep_max / 64 + t->hot_max;
   A(t->hot_work, (size_t)t->work_max * 4);
   A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);
+  if (t->k > 28 && t->max_nnz >= (1 << 20)) A(t->super_cnt, (size_t)t->max_batch * t->F * 16 * 2);
   if (t->H) {
     A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
     if (c.optimizer == DES_OPT_ADAM) A(t->acc2W1, FKH * 4);
