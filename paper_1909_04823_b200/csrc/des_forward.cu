@@ -30,7 +30,7 @@
 
 __global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
-    const uint8_t* __restrict__ shards, int B, int F, int S, const DevMeta* __restrict__ meta,
+    const uint8_t* __restrict__ shards, int B, int F, int S, const DevMeta* __restrict__ meta, uint32_t null_row,
     uint32_t* __restrict__ grow_csr, uint32_t* __restrict__ grow_sorted, float* __restrict__ x_sorted,
     int32_t* __restrict__ seg_off) {
   __shared__ uint32_t row_base[DES_MAX_SHARDS];
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(256) route_kernel(
       if (j < hi) {
         const uint32_t r = __ldg(rows + j);
         const int s = __ldg(shards + j);
-        grow_csr[j] = (r == DES_ROW_NONE) ? DES_ROW_NONE : row_base[s] + r;
+        grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
         if (r != DES_ROW_NONE) key = s;
       }
       const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
@@ -190,42 +190,64 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
   }
 }
 
-template <int G, bool HAS_VALS, bool MATERIALISE>
+template <int G, int P, bool HAS_VALS, bool MATERIALISE>
 __global__ void __launch_bounds__(256) pool_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ grow_csr,
     const uint8_t* __restrict__ shards, long long nbags, int B, int F, int k, const float* __restrict__ W,
-    float* __restrict__ pooled, float* __restrict__ part_pooled) {
+    uint32_t null_row, float* __restrict__ pooled, float* __restrict__ part_pooled) {
+  constexpr int LB = G * P;                            // lanes per bag
   const int K4 = k >> 2, stride = k + 4;
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long bag = t / G;
-  const int c4 = (int)(t % G);
-  if (bag >= nbags || c4 >= K4) return;
-  const int lo = __ldg(offsets + bag), hi = __ldg(offsets + bag + 1);
+  const long long bag = t / LB;
+  const int sub = (int)(t % LB), c4 = sub % G, p = sub / G;
+  const bool live = bag < nbags, col = c4 < K4;
+  int lo = 0, hi = 0;
+  if (live) { lo = __ldg(offsets + bag); hi = __ldg(offsets + bag + 1); }
+  const unsigned rowB = (unsigned)stride * 4u;
+  const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int i0 = lo; i0 < hi; i0 += FW_UNROLL) {
-    float4 v[FW_UNROLL]; float x[FW_UNROLL];
+  // per-shard copy of the pooled sum (tests only): every real occurrence is also added to its shard's block
+  auto materialise = [&](int i, uint32_t gr, const float4& vx) {
+    if (MATERIALISE && col && gr != null_row) {
+      const int s = __ldg(shards + i);
+      const long long b = bag / F, f = bag % F;
+      atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)s * B + b) * ((size_t)F * k) + (size_t)f * k) + c4, vx);
+    }
+  };
+  int i0 = lo;
+  for (; i0 + FW_UNROLL * P <= hi; i0 += FW_UNROLL * P) {
+    float4 v[FW_UNROLL]; float x[FW_UNROLL]; uint32_t gr[FW_UNROLL];
 #pragma unroll
     for (int u = 0; u < FW_UNROLL; ++u) {
-      v[u] = make_float4(0.f, 0.f, 0.f, 0.f); x[u] = 1.f;
-      if (i0 + u < hi) {
-        const uint32_t gr = __ldg(grow_csr + i0 + u);
-        if (HAS_VALS) x[u] = __ldg(vals + i0 + u);
-        if (gr != DES_ROW_NONE) v[u] = __ldg(reinterpret_cast<const float4*>(W + (size_t)gr * stride) + c4);
-      }
+      const int i = i0 + u * P + p;
+      gr[u] = __ldg(grow_csr + i);
+      if (HAS_VALS) x[u] = __ldg(vals + i);
+      v[u] = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr[u] * rowB));
     }
 #pragma unroll
     for (int u = 0; u < FW_UNROLL; ++u) {
       float4 vx = v[u];
       if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
       acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
-      if (MATERIALISE && i0 + u < hi && __ldg(grow_csr + i0 + u) != DES_ROW_NONE) {
-        const int s = __ldg(shards + i0 + u);
-        const long long b = bag / F, f = bag % F;
-        atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)s * B + b) * ((size_t)F * k) + (size_t)f * k) + c4, vx);
-      }
+      materialise(i0 + u * P + p, gr[u], vx);
     }
   }
-  reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+  for (; i0 < hi; i0 += P) {                           // ragged end of the bag
+    const int i = i0 + p;
+    if (i < hi) {
+      const uint32_t gr = __ldg(grow_csr + i);
+      float4 vx = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr * rowB));
+      if (HAS_VALS) { const float x = __ldg(vals + i); vx.x *= x; vx.y *= x; vx.z *= x; vx.w *= x; }
+      acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
+      materialise(i, gr, vx);
+    }
+  }
+#pragma unroll
+  for (int d = G; d < LB; d <<= 1) {                   // combine the bag's sub-groups
+    acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
+    acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
+  }
+  if (live && p == 0 && col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
 }
 
 // (+) over shards and F.  G lanes per sample, one float4 column each; lane 0 of
@@ -294,7 +316,8 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   uint32_t* grow_sorted = t->slot_of;
   float* x_sorted = reinterpret_cast<float*>(t->dest);
   route_kernel<<<(B + 7) / 8 < t->sm_count * 8 ? (B + 7) / 8 : t->sm_count * 8, 256, 0, cs>>>(
-      b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, grow_csr, grow_sorted, x_sorted, t->seg_off);
+      b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, (uint32_t)t->total_rows, grow_csr, grow_sorted,
+      x_sorted, t->seg_off);
   DES_LAUNCH_CHECK(t, "route_kernel");
   if (ps || fused_out) {
     const unsigned grid = (unsigned)((B + 7) / 8);      // one warp per sample
@@ -309,14 +332,19 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   }
   if (pl) {
     const long long nbags = (long long)B * t->F;
-    const long long threads = nbags * G;
+    // long bags: a whole warp per bag (its halves take alternate occurrences); short bags: G lanes per bag
+    const bool wide = b->nnz >= 4 * nbags;
+    const long long threads = nbags * (wide ? 32 : G);
     const unsigned grid = (unsigned)((threads + 255) / 256);
-#define PK3(GG, HV, MT) pool_kernel<GG, HV, MT><<<grid, 256, 0, cs>>>(b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, t->k, t->W, pl, pp)
+#define PK4(GG, PP, HV, MT) pool_kernel<GG, PP, HV, MT><<<grid, 256, 0, cs>>>(b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, \
+                                                                             t->k, t->W, (uint32_t)t->total_rows, pl, pp)
+#define PK3(GG, HV, MT) do { if (wide) PK4(GG, 32 / GG, HV, MT); else PK4(GG, 1, HV, MT); } while (0)
 #define PK(GG) do { if (pp) { if (b->vals) PK3(GG, true, true); else PK3(GG, false, true); } \
                     else { if (b->vals) PK3(GG, true, false); else PK3(GG, false, false); } } while (0)
     switch (G) { case 1: PK(1); break; case 2: PK(2); break; case 4: PK(4); break; case 8: PK(8); break; default: PK(16); }
 #undef PK
 #undef PK3
+#undef PK4
     DES_LAUNCH_CHECK(t, "pool_kernel");
   }
   return DES_OK;

@@ -166,7 +166,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
     if (!p) ok = false;
   };
   A(t->slots, slots * sizeof(Slot));
-  A(t->W, rows * rowbytes);
+  A(t->W, (rows + 1) * rowbytes);          // one all-zero row behind the table stands for "no row" in gathers
   if (c.optimizer != DES_OPT_SGD || c.lin_optimizer == DES_LIN_FTRL) A(t->A, rows * rowbytes);
   if (c.optimizer == DES_OPT_ADAM) A(t->A2, rows * rowbytes);
   A(t->meta, sizeof(DevMeta));
@@ -203,6 +203,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   if (!ok) { des_table_destroy(t); return DES_ERR_CUDA; }
   bool cu = true;
   cu &= cudaMemset(t->slots, 0xFF, slots * sizeof(Slot)) == cudaSuccess;
+  cu &= cudaMemset(t->W + rows * t->stride, 0, rowbytes) == cudaSuccess;
   cu &= cudaMemset(t->Gbuf, 0, ((size_t)t->max_uniq + t->rep_max) * rowbytes) == cudaSuccess;
   cu &= cudaMemset(t->hinfo, 0, (size_t)t->max_uniq * 4) == cudaSuccess;
   cu &= cudaMemset(t->hot_acc, 0, (size_t)t->hot_max * t->stride * 8) == cudaSuccess;
