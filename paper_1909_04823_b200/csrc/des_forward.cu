@@ -16,7 +16,7 @@
 //  shard_partials_kernel   one warp per sample (32 / G sub-groups of G = k/4
 //                 lanes, rounded up to a power of two) walks the sample's
 //                 (sample, shard) segments in shard order: it streams a segment's
-//                 rows with 16-byte loads, SP_UNROLL in flight per lane, and keeps
+//                 rows with 16-byte loads and keeps
 //                 M_1, M_1^lr, M_2 in registers until the segment ends — no shared
 //                 memory, no atomics, a fixed summation order (deterministic).  M_2 uses the |v|^2 cached in the
 //                 row's 16-byte tail.  Fused variant: (+) over shards and F on chip.
@@ -25,8 +25,6 @@
 //                 materialised (with atomics) when the caller asks for it.
 #include "des_internal.cuh"
 
-#define FW_UNROLL 8
-#define SP_UNROLL 4
 
 __global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
@@ -88,9 +86,58 @@ __global__ void __launch_bounds__(256) route_kernel(
   }
 }
 
+// U rows per lane in flight: occurrences i, i + P, ... of a (sample, shard) segment.
+template <int U, int P, bool HAS_VALS>
+__device__ __forceinline__ void sp_step(const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted,
+                                        int i, const char* __restrict__ Wc, const char* __restrict__ Wt, unsigned rowB,
+                                        float4& acc, float& m1lr, float& m2) {
+  float4 v[U]; float2 tl[U]; float x[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const size_t off = (size_t)__ldg(grow_sorted + i + u * P) * rowB;
+    if (HAS_VALS) x[u] = __ldg(x_sorted + i + u * P);
+    v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
+    tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    if (HAS_VALS) {
+      acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
+      m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
+    } else {
+      acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+      m1lr += tl[u].x; m2 += tl[u].y;
+    }
+  }
+}
+
+// Same for a bag: U rows per lane, optionally also added to the per-shard copy of the pooled sum
+// (MATERIALISE, tests only).
+template <int U, int P, bool HAS_VALS, bool MATERIALISE>
+__device__ __forceinline__ void pool_step(const uint32_t* __restrict__ grow_csr, const float* __restrict__ vals,
+                                          const uint8_t* __restrict__ shards, int i, const char* __restrict__ Wc,
+                                          unsigned rowB, uint32_t null_row, float* __restrict__ part_block, size_t shard_pitch,
+                                          bool col, float4& acc) {
+  float4 v[U]; float x[U]; uint32_t gr[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    gr[u] = __ldg(grow_csr + i + u * P);
+    if (HAS_VALS) x[u] = __ldg(vals + i + u * P);
+    v[u] = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr[u] * rowB));
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    float4 vx = v[u];
+    if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
+    acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
+    if (MATERIALISE && col && gr[u] != null_row)
+      atomicAdd(reinterpret_cast<float4*>(part_block + (size_t)__ldg(shards + i + u * P) * shard_pitch), vx);
+  }
+}
+
 // One WARP per sample walks the sample's S segments in shard order.  The warp is
 // split into P = 32 / G sub-groups of G lanes (one 16-byte column per lane);
-// sub-group p takes occurrences p, p + P, ... of a segment, SP_UNROLL of them in
+// sub-group p takes occurrences p, p + P, ... of a segment, two of them in
 // flight, and the sub-groups' sums are combined by a butterfly when the segment
 // ends — so both halves of a warp always run the same trip counts, whatever the
 // skew between shards, and every warp has the same amount of work (a sample's
@@ -127,44 +174,13 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
     hi = __ldg(so + s + 1);
     float4 acc = zero4;
     float m1lr = 0.f, m2 = 0.f;
+    // whole blocks of 2 and 1 occurrences per lane (no bound checks), then one checked step; segments are
+    // short (a sample's occurrences spread over S shards), so deeper unrolling only adds ragged steps
     int i0 = lo;
-    for (; i0 + SP_UNROLL * P <= hi; i0 += SP_UNROLL * P) {
-      float4 v[SP_UNROLL]; float2 tl[SP_UNROLL]; float x[SP_UNROLL];
-#pragma unroll
-      for (int u = 0; u < SP_UNROLL; ++u) {
-        const int i = i0 + u * P + p;
-        const size_t off = (size_t)__ldg(grow_sorted + i) * rowB;
-        if (HAS_VALS) x[u] = __ldg(x_sorted + i);
-        v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
-        tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
-      }
-#pragma unroll
-      for (int u = 0; u < SP_UNROLL; ++u) {
-        if (HAS_VALS) {
-          acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
-          m1lr += tl[u].x * x[u]; m2 += tl[u].y * x[u] * x[u];
-        } else {
-          acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
-          m1lr += tl[u].x; m2 += tl[u].y;
-        }
-      }
-    }
-    for (; i0 < hi; i0 += P) {                         // ragged end of the segment
-      const int i = i0 + p;
-      if (i < hi) {
-        const size_t off = (size_t)__ldg(grow_sorted + i) * rowB;
-        const float x = HAS_VALS ? __ldg(x_sorted + i) : 1.f;
-        const float4 v = __ldg(reinterpret_cast<const float4*>(Wc + off));
-        const float2 tl = __ldg(reinterpret_cast<const float2*>(Wt + off));
-        if (HAS_VALS) {
-          acc.x += v.x * x; acc.y += v.y * x; acc.z += v.z * x; acc.w += v.w * x;
-          m1lr += tl.x * x; m2 += tl.y * x * x;
-        } else {
-          acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-          m1lr += tl.x; m2 += tl.y;
-        }
-      }
-    }
+    for (; i0 + 2 * P <= hi; i0 += 2 * P)
+      sp_step<2, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
+    if (i0 + P <= hi) { sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2); i0 += P; }
+    if (i0 + p < hi) sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
 #pragma unroll
     for (int d = G; d < 32; d <<= 1) {                 // combine the sub-groups (same result in every lane)
       acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
@@ -206,42 +222,18 @@ __global__ void __launch_bounds__(256) pool_kernel(
   const unsigned rowB = (unsigned)stride * 4u;
   const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  // per-shard copy of the pooled sum (tests only): every real occurrence is also added to its shard's block
-  auto materialise = [&](int i, uint32_t gr, const float4& vx) {
-    if (MATERIALISE && col && gr != null_row) {
-      const int s = __ldg(shards + i);
-      const long long b = bag / F, f = bag % F;
-      atomicAdd(reinterpret_cast<float4*>(part_pooled + ((size_t)s * B + b) * ((size_t)F * k) + (size_t)f * k) + c4, vx);
-    }
-  };
+  // MATERIALISE: this lane's column of block (shard 0, sample, field) of part_pooled [S][B][F*k]
+  float* part_block = nullptr;
+  const size_t shard_pitch = (size_t)B * F * k;
+  if (MATERIALISE && live) part_block = part_pooled + (size_t)bag * k + (col ? c4 : 0) * 4;
   int i0 = lo;
-  for (; i0 + FW_UNROLL * P <= hi; i0 += FW_UNROLL * P) {
-    float4 v[FW_UNROLL]; float x[FW_UNROLL]; uint32_t gr[FW_UNROLL];
-#pragma unroll
-    for (int u = 0; u < FW_UNROLL; ++u) {
-      const int i = i0 + u * P + p;
-      gr[u] = __ldg(grow_csr + i);
-      if (HAS_VALS) x[u] = __ldg(vals + i);
-      v[u] = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr[u] * rowB));
-    }
-#pragma unroll
-    for (int u = 0; u < FW_UNROLL; ++u) {
-      float4 vx = v[u];
-      if (HAS_VALS) { vx.x *= x[u]; vx.y *= x[u]; vx.z *= x[u]; vx.w *= x[u]; }
-      acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
-      materialise(i0 + u * P + p, gr[u], vx);
-    }
-  }
-  for (; i0 < hi; i0 += P) {                           // ragged end of the bag
-    const int i = i0 + p;
-    if (i < hi) {
-      const uint32_t gr = __ldg(grow_csr + i);
-      float4 vx = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr * rowB));
-      if (HAS_VALS) { const float x = __ldg(vals + i); vx.x *= x; vx.y *= x; vx.z *= x; vx.w *= x; }
-      acc.x += vx.x; acc.y += vx.y; acc.z += vx.z; acc.w += vx.w;
-      materialise(i, gr, vx);
-    }
-  }
+#define POOL_STEP(U) pool_step<U, P, HAS_VALS, MATERIALISE>(grow_csr, vals, shards, i0 + p, Wc, rowB, null_row, part_block, \
+                                                           shard_pitch, col, acc)
+  for (; i0 + 4 * P <= hi; i0 += 4 * P) POOL_STEP(4);
+  if (i0 + 2 * P <= hi) { POOL_STEP(2); i0 += 2 * P; }
+  if (i0 + P <= hi) { POOL_STEP(1); i0 += P; }
+  if (i0 + p < hi) POOL_STEP(1);
+#undef POOL_STEP
 #pragma unroll
   for (int d = G; d < LB; d <<= 1) {                   // combine the bag's sub-groups
     acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
