@@ -168,58 +168,90 @@ __global__ void __launch_bounds__(256) hot_finish_kernel(const uint32_t* __restr
   }
 }
 
-// SUPER (16-lane groups only): occurrences of the few keys that own a large share of a skewed
-// batch (dest = SUPER_TAG | slot) send no atomics.  Lane t of the group counts the bag's
-// occurrences of slot t — every lane sees every dest[j] anyway — and the counts go to
-// super_cnt[bag][16]; super_dense_kernel turns them into the keys' gradient sums.
-template <int G, bool SUPER>
+// U occurrences i, i + P, ... of a bag: one vector atomic per lane into the occurrence's gradient
+// row (lane 0 of the sub-group also adds the linear-weight tail).  SUPER: occurrences marked
+// dest = SUPER_TAG | slot send nothing; lane t counts those of slot t.
+template <int U, int P, bool HAS_VALS, bool SUPER>
+__device__ __forceinline__ void scatter_step(const uint32_t* __restrict__ dest, const float* __restrict__ vals, int i,
+                                             char* gcol, char* gtail, unsigned rowB, bool col, bool lead,
+                                             const float4& c, float gl, float gf, uint32_t mine, uint32_t& cnt) {
+  uint32_t d[U]; float x[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    d[u] = __ldg(dest + i + u * P);
+    if (HAS_VALS) x[u] = __ldg(vals + i + u * P);
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    if (SUPER) cnt += (d[u] == mine);
+    const bool ok = SUPER ? d[u] < SUPER_TAG : d[u] != DES_ROW_NONE;   // SUPER_TAG.. also covers "no row"
+    if (ok) {
+      const size_t off = (size_t)d[u] * rowB;
+      if (HAS_VALS) {
+        const float xx = x[u];
+        if (col) atomicAdd(reinterpret_cast<float4*>(gcol + off), make_float4(xx * c.x, xx * c.y, xx * c.z, xx * c.w));
+        if (lead) atomicAdd(reinterpret_cast<float4*>(gtail + off), make_float4(xx * gl, xx * xx * gf, 0.f, 0.f));
+      } else {
+        if (col) atomicAdd(reinterpret_cast<float4*>(gcol + off), c);
+        if (lead) atomicAdd(reinterpret_cast<float4*>(gtail + off), make_float4(gl, gf, 0.f, 0.f));
+      }
+    }
+  }
+}
+
+// One bag per G * P lanes: P sub-groups of G lanes (one 16-byte column each) take alternate
+// occurrences of the bag.  c_bag is formed once per bag; the loop body is the destination load
+// and the atomics.  SUPER (G = 16 only): occurrences of the few keys that own a large share of a
+// skewed batch send no atomics; lane t counts the bag's occurrences of slot t and the counts go
+// to super_cnt[bag][16]; super_dense_kernel turns them into the keys' gradient sums.
+template <int G, int P, bool HAS_VALS, bool SUPER>
 __global__ void __launch_bounds__(256) grad_scatter_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ dest,
     long long nbags, int F, int k, uint32_t ops, const float* __restrict__ out_small,
     const float* __restrict__ gL, const float* __restrict__ gF, const float* __restrict__ gE, float* Gbuf,
     uint16_t* __restrict__ super_cnt) {
+  constexpr int LB = G * P;
   const int K4 = k >> 2, stride = k + 4;
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long bag = t / G;
-  const int c4 = (int)(t % G);
-  if (bag >= nbags) return;
-  const int lo = __ldg(offsets + bag), hi = __ldg(offsets + bag + 1);
-  if (lo == hi) {
-    if (SUPER) super_cnt[bag * 16 + c4] = 0;
-    return;
-  }
-  const bool col = c4 < K4;
-  if (!SUPER && !col && c4 != 0) return;
-  const long long b = bag / F;
-  const float gf = (ops & DES_OP_FM) ? __ldg(gF + b) : 0.f;
-  const float gl = (ops & DES_OP_LR) ? __ldg(gL + b) : 0.f;
+  const long long bag = t / LB;
+  const int sub = (int)(t % LB), c4 = sub % G, p = sub / G;
+  const bool live = bag < nbags, col = c4 < K4, lead = c4 == 0;
+  int lo = 0, hi = 0;
+  if (live) { lo = __ldg(offsets + bag); hi = __ldg(offsets + bag + 1); }
   float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (col) {
-    if (ops & DES_OP_FM) {
-      const float4 a = __ldg(reinterpret_cast<const float4*>(out_small + b * stride) + c4);
-      c = make_float4(gf * a.x, gf * a.y, gf * a.z, gf * a.w);
-    }
-    if (gE) {
-      const float4 e = __ldg(reinterpret_cast<const float4*>(gE + bag * k) + c4);
-      c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
+  float gf = 0.f, gl = 0.f;
+  if (lo < hi) {
+    const long long b = bag / F;
+    if (ops & DES_OP_FM) gf = __ldg(gF + b);
+    if (ops & DES_OP_LR) gl = __ldg(gL + b);
+    if (col) {
+      if (ops & DES_OP_FM) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(out_small + b * stride) + c4);
+        c = make_float4(gf * a.x, gf * a.y, gf * a.z, gf * a.w);
+      }
+      if (gE) {
+        const float4 e = __ldg(reinterpret_cast<const float4*>(gE + bag * k) + c4);
+        c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
+      }
     }
   }
+  const unsigned rowB = (unsigned)stride * 4u;
+  char* gcol = reinterpret_cast<char*>(Gbuf) + c4 * 16;
+  char* gtail = reinterpret_cast<char*>(Gbuf + k);
   uint32_t cnt = 0;
   const uint32_t mine = SUPER_TAG | (uint32_t)c4;
-  for (int j = lo; j < hi; ++j) {
-    const uint32_t u = __ldg(dest + j);
-    if (SUPER) {
-      cnt += (u == mine);
-      if (u >= SUPER_TAG) continue;                   // counted, or no row
-    } else if (u == DES_ROW_NONE) {
-      continue;
-    }
-    const float x = vals ? __ldg(vals + j) : 1.f;
-    float* row = Gbuf + (size_t)u * stride;
-    if (col) atomicAdd(reinterpret_cast<float4*>(row) + c4, make_float4(x * c.x, x * c.y, x * c.z, x * c.w));
-    if (c4 == 0) atomicAdd(reinterpret_cast<float4*>(row) + K4, make_float4(x * gl, x * x * gf, 0.f, 0.f));
+  int i0 = lo;
+#define SC_STEP(U) scatter_step<U, P, HAS_VALS, SUPER>(dest, vals, i0 + p, gcol, gtail, rowB, col, lead, c, gl, gf, mine, cnt)
+  for (; i0 + 4 * P <= hi; i0 += 4 * P) SC_STEP(4);
+  if (i0 + 2 * P <= hi) { SC_STEP(2); i0 += 2 * P; }
+  if (i0 + P <= hi) { SC_STEP(1); i0 += P; }
+  if (i0 + p < hi) SC_STEP(1);
+#undef SC_STEP
+  if (SUPER) {
+#pragma unroll
+    for (int d = G; d < LB; d <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+    if (live && p == 0) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
   }
-  if (SUPER) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
 }
 
 // Gradient sums of the SUPER_T marked keys as a dense product:
@@ -492,24 +524,30 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
                                                         t->dest);
     DES_LAUNCH_CHECK(t, "make_dest_kernel");
   }
-  if (use_super) {
-    const unsigned grid = (unsigned)((nbags * 16 + 255) / 256);
-    grad_scatter_kernel<16, true><<<grid, 256, 0, cs>>>(b->offsets, nullptr, t->dest, nbags, t->F, t->k, ops,
-                                                        out->out_small, gr->gL, gr->gF, gE, t->Gbuf, t->super_cnt);
-    DES_LAUNCH_CHECK(t, "grad_scatter_kernel");
-    super_dense_kernel<<<t->sm_count * 3, SD_THREADS, 0, cs>>>(t->super_cnt, (int)nbags, t->F, t->k, ops, out->out_small, gr->gL,
-                                                        gr->gF, gE, t->Gbuf, t->hot_ctr, t->hot_base, t->hot_R,
-                                                        t->max_uniq);
-    DES_LAUNCH_CHECK(t, "super_dense_kernel");
-  } else {
-    const long long threads = nbags * G;
+  {
+    // long bags: a whole warp per bag (its sub-groups take alternate occurrences); short bags: G lanes per bag
+    const bool wide = (long long)nnz >= 4 * nbags;
+    const long long threads = nbags * (wide ? 32 : G);
     const unsigned grid = (unsigned)((threads + 255) / 256);
-#define SC(GG) grad_scatter_kernel<GG, false><<<grid, 256, 0, cs>>>(b->offsets, b->vals, t->dest, nbags, t->F, t->k,  \
-                                                                   ops, out->out_small, gr->gL, gr->gF, gE, t->Gbuf, \
-                                                                   nullptr)
-    switch (G) { case 1: SC(1); break; case 2: SC(2); break; case 4: SC(4); break; case 8: SC(8); break; default: SC(16); }
+#define SC4(GG, PP, HV, SU) grad_scatter_kernel<GG, PP, HV, SU><<<grid, 256, 0, cs>>>(                                  \
+        b->offsets, b->vals, t->dest, nbags, t->F, t->k, ops, out->out_small, gr->gL, gr->gF, gE, t->Gbuf, t->super_cnt)
+#define SC3(GG, HV) do { if (wide) SC4(GG, 32 / GG, HV, false); else SC4(GG, 1, HV, false); } while (0)
+#define SC(GG) do { if (b->vals) SC3(GG, true); else SC3(GG, false); } while (0)
+    if (use_super) {
+      if (wide) SC4(16, 2, false, true); else SC4(16, 1, false, true);
+    } else {
+      switch (G) { case 1: SC(1); break; case 2: SC(2); break; case 4: SC(4); break; case 8: SC(8); break; default: SC(16); }
+    }
 #undef SC
+#undef SC3
+#undef SC4
     DES_LAUNCH_CHECK(t, "grad_scatter_kernel");
+  }
+  if (use_super) {
+    super_dense_kernel<<<t->sm_count * 3, SD_THREADS, 0, cs>>>(t->super_cnt, (int)nbags, t->F, t->k, ops, out->out_small,
+                                                               gr->gL, gr->gF, gE, t->Gbuf, t->hot_ctr, t->hot_base,
+                                                               t->hot_R, t->max_uniq);
+    DES_LAUNCH_CHECK(t, "super_dense_kernel");
   }
   hot_reduce_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->hot_ctr, t->work_max, t->hot_work, t->hot_base, t->hot_R,
                                                      t->max_uniq, t->k, t->Gbuf, t->hot_acc);
