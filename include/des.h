@@ -36,8 +36,8 @@
  *   and frees it in des_table_destroy.
  * - All device work is enqueued on the caller's stream (a cudaStream_t passed
  *   as void*; NULL = the legacy default stream).  Only des_table_status,
- *   des_table_size, des_table_export, des_dense1_get/set on host pointers and
- *   des_step_host synchronise.
+ *   des_table_size, des_table_export, des_dense1_get/set on host pointers,
+ *   des_step_host and des_step_host_wait synchronise.
  * - Device-side problems (reserved key, full shard) never fault: the
  *   offending occurrences get row DES_ROW_NONE, are skipped by every later
  *   kernel, and a sticky error word is raised that des_table_status returns.
@@ -316,6 +316,24 @@ des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t 
                            const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
                            const des_grads_t* d_grads, float* d_pooled, float* d_Z,
                            float* h_out_small, void* stream);
+
+/* The same step for callers that feed batches back to back (Section 5: batch
+ * building and the optimizer phase follow each other every iteration).
+ * des_step_host_submit returns as soon as the step is enqueued: the host
+ * buffers are copied on a stream of the table's own into one of two staging
+ * slots, the kernels and the read-back of out_small run on `stream` once the
+ * copy has landed, so the copy of step i+1 overlaps the kernels of step i.
+ * *ticket names the slot; des_step_host_wait(ticket) blocks until that step is
+ * over (h_out_small written).  At most two steps are in flight: a third submit
+ * first waits for the step that used its slot.  Host buffers (inputs and
+ * h_out_small) must stay untouched until the step's wait returns, and must be
+ * pinned for the overlap to happen; all submits of a table must use the same
+ * `stream`, which orders the steps.  Results are those of des_step_host. */
+des_status_t des_step_host_submit(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
+                                  const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                                  const des_grads_t* d_grads, float* d_pooled, float* d_Z,
+                                  float* h_out_small, void* stream, int32_t* ticket);
+des_status_t des_step_host_wait(des_table_t* t, int32_t ticket);
 
 /* Per-launch timing for benchmarks.  While enabled, the library records a CUDA
  * event on the call's stream behind every kernel it launches (and one at the

@@ -28,7 +28,7 @@ EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_f
            "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_table_read_state2", "des_table_write_state2",
-           "des_step_host", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
+           "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
 
 
 class DesError(RuntimeError):
@@ -112,6 +112,10 @@ def load():
         L.des_step_host.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p]
+        L.des_step_host_submit.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.POINTER(C.c_int32)]
+        L.des_step_host_wait.argtypes = [C.c_void_p, C.c_int32]
         L.des_table_launch_count.argtypes = [C.c_void_p]
         L.des_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.des_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int,
@@ -254,6 +258,19 @@ class Table:
         self._check(self.L.des_step_host(self.h, ops, batch_size, nnz, _ptr(h_offsets), _ptr(h_ids),
                                          _ptr(h_vals), C.byref(g), _ptr(d_pooled), _ptr(d_Z),
                                          _ptr(h_out_small), _stream()), "des_step_host")
+
+    def step_host_submit(self, ops, batch_size, nnz, h_offsets, h_ids, h_vals, h_out_small, d_pooled=None, d_Z=None,
+                         gL=None, gF=None, gE=None, gZ=None, gE_work=None) -> int:
+        """Pipelined des_step_host: returns a ticket for step_host_wait."""
+        g = des_grads_t(_ptr(gL), _ptr(gF), _ptr(gE), _ptr(gZ), _ptr(gE_work))
+        ticket = C.c_int32(-1)
+        self._check(self.L.des_step_host_submit(self.h, ops, batch_size, nnz, _ptr(h_offsets), _ptr(h_ids),
+                                                _ptr(h_vals), C.byref(g), _ptr(d_pooled), _ptr(d_Z),
+                                                _ptr(h_out_small), _stream(), C.byref(ticket)), "des_step_host_submit")
+        return int(ticket.value)
+
+    def step_host_wait(self, ticket: int):
+        self._check(self.L.des_step_host_wait(self.h, ticket), "des_step_host_wait")
 
     # -- first dense layer ----------------------------------------------------------
     def dense1_set(self, W1: torch.Tensor):

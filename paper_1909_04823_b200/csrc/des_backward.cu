@@ -574,45 +574,118 @@ static void* st_alloc(des_table* t, size_t bytes) {
   return p;
 }
 
-extern "C" des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
-                                      const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
-                                      const des_grads_t* d_grads, float* d_pooled, float* d_Z, float* h_out_small,
-                                      void* stream) {
-  if (!t || !h_offsets || (nnz > 0 && !h_ids) || !d_grads || !h_out_small) return DES_ERR_INVALID_ARG;
-  if (batch <= 0 || batch > t->max_batch || nnz < 0 || nnz > t->max_nnz) return DES_ERR_INVALID_ARG;
-  cudaStream_t cs = (cudaStream_t)stream;
-  if (!t->st_ids) {   // first call: device staging sized for the largest batch (allocates, synchronises)
-    const size_t nb = (size_t)t->max_batch * t->F + 1;
-    t->st_offsets = (int32_t*)st_alloc(t, nb * 4);
-    t->st_ids = (unsigned long long*)st_alloc(t, (size_t)t->max_nnz * 8);
-    t->st_vals = (float*)st_alloc(t, (size_t)t->max_nnz * 4);
-    t->st_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
-    t->st_shards = (uint8_t*)st_alloc(t, (size_t)t->max_nnz);
-    t->st_uidx = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
-    t->st_uniq_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
-    t->st_n_uniq = (uint32_t*)st_alloc(t, 256);
-    t->st_part_small = (float*)st_alloc(t, (size_t)t->S * t->max_batch * t->stride * 4);
-    t->st_out_small = (float*)st_alloc(t, (size_t)t->max_batch * t->stride * 4);
-    if (!t->st_offsets || !t->st_ids || !t->st_vals || !t->st_rows || !t->st_shards || !t->st_uidx ||
-        !t->st_uniq_rows || !t->st_n_uniq || !t->st_part_small || !t->st_out_small)
-      return DES_ERR_CUDA;
+// Device staging of the host-buffer step, sized for the largest batch (first call: allocates, synchronises).
+// The batch inputs (offsets, ids, values) have two slots so that the copy of one step can overlap the
+// kernels of the step before; everything the kernels produce is single (kernels of consecutive steps run
+// in order on the caller's stream).
+static des_status_t st_prepare(des_table* t) {
+  if (t->st_ids[0]) return DES_OK;
+  const size_t nb = (size_t)t->max_batch * t->F + 1;
+  for (int s = 0; s < 2; ++s) {
+    t->st_offsets[s] = (int32_t*)st_alloc(t, nb * 4);
+    t->st_ids[s] = (unsigned long long*)st_alloc(t, (size_t)t->max_nnz * 8);
+    t->st_vals[s] = (float*)st_alloc(t, (size_t)t->max_nnz * 4);
+    if (!t->st_offsets[s] || !t->st_ids[s] || !t->st_vals[s]) return DES_ERR_CUDA;
   }
+  t->st_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+  t->st_shards = (uint8_t*)st_alloc(t, (size_t)t->max_nnz);
+  t->st_uidx = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+  t->st_uniq_rows = (uint32_t*)st_alloc(t, (size_t)t->max_nnz * 4);
+  t->st_n_uniq = (uint32_t*)st_alloc(t, 256);
+  t->st_part_small = (float*)st_alloc(t, (size_t)t->S * t->max_batch * t->stride * 4);
+  t->st_out_small = (float*)st_alloc(t, (size_t)t->max_batch * t->stride * 4);
+  if (!t->st_rows || !t->st_shards || !t->st_uidx || !t->st_uniq_rows || !t->st_n_uniq || !t->st_part_small ||
+      !t->st_out_small)
+    return DES_ERR_CUDA;
+  if (cudaStreamCreateWithFlags(&t->st_copy_stream, cudaStreamNonBlocking) != cudaSuccess) return DES_ERR_CUDA;
+  for (int s = 0; s < 2; ++s) {
+    if (cudaEventCreateWithFlags(&t->st_copied[s], cudaEventDisableTiming) != cudaSuccess) return DES_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&t->st_done[s], cudaEventDisableTiming) != cudaSuccess) return DES_ERR_CUDA;
+    t->st_busy[s] = 0;
+  }
+  return DES_OK;
+}
+
+// Enqueues one whole step from host buffers: inputs go to staging slot `slot` on `copy` (the caller's
+// stream itself, or the table's copy stream), the kernels and the read-back of out_small on `cs`.
+static des_status_t st_enqueue(des_table* t, int slot, cudaStream_t copy, uint32_t ops, int32_t batch, int64_t nnz,
+                               const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                               const des_grads_t* d_grads, float* d_pooled, float* d_Z, float* h_out_small,
+                               cudaStream_t cs) {
   const size_t nb = (size_t)batch * t->F + 1;
-  DES_CUDA(cudaMemcpyAsync(t->st_offsets, h_offsets, nb * 4, cudaMemcpyHostToDevice, cs));
-  if (nnz) DES_CUDA(cudaMemcpyAsync(t->st_ids, h_ids, (size_t)nnz * 8, cudaMemcpyHostToDevice, cs));
-  if (h_vals && nnz) DES_CUDA(cudaMemcpyAsync(t->st_vals, h_vals, (size_t)nnz * 4, cudaMemcpyHostToDevice, cs));
+  DES_CUDA(cudaMemcpyAsync(t->st_offsets[slot], h_offsets, nb * 4, cudaMemcpyHostToDevice, copy));
+  if (nnz) DES_CUDA(cudaMemcpyAsync(t->st_ids[slot], h_ids, (size_t)nnz * 8, cudaMemcpyHostToDevice, copy));
+  if (h_vals && nnz) DES_CUDA(cudaMemcpyAsync(t->st_vals[slot], h_vals, (size_t)nnz * 4, cudaMemcpyHostToDevice, copy));
+  if (copy != cs) {
+    DES_CUDA(cudaEventRecord(t->st_copied[slot], copy));
+    DES_CUDA(cudaStreamWaitEvent(cs, t->st_copied[slot], 0));
+  }
   des_batch_t b;
-  b.batch = batch; b.nnz = nnz; b.offsets = t->st_offsets; b.ids = (const uint64_t*)t->st_ids;
-  b.vals = h_vals ? t->st_vals : nullptr; b.rows = t->st_rows; b.shards = t->st_shards; b.uidx = t->st_uidx;
+  b.batch = batch; b.nnz = nnz; b.offsets = t->st_offsets[slot]; b.ids = (const uint64_t*)t->st_ids[slot];
+  b.vals = h_vals ? t->st_vals[slot] : nullptr; b.rows = t->st_rows; b.shards = t->st_shards; b.uidx = t->st_uidx;
   b.uniq_rows = t->st_uniq_rows; b.n_uniq = t->st_n_uniq;
   des_partials_t p; p.part_small = t->st_part_small; p.pooled = d_pooled; p.part_pooled = nullptr; p.part_dense = nullptr;
   des_outputs_t o; o.out_small = t->st_out_small; o.pooled = d_pooled; o.Z = d_Z;
   des_status_t st;
-  if ((st = des_find_or_insert(t, &b, 1, stream)) != DES_OK) return st;
-  if ((st = des_forward_partials(t, ops, &b, &p, stream)) != DES_OK) return st;
-  if ((st = des_aggregate(t, ops, &b, &p, &o, stream)) != DES_OK) return st;
-  if ((st = des_backward_update(t, ops, &b, &o, d_grads, stream)) != DES_OK) return st;
+  if ((st = des_find_or_insert(t, &b, 1, cs)) != DES_OK) return st;
+  if ((st = des_forward_partials(t, ops, &b, &p, cs)) != DES_OK) return st;
+  if ((st = des_aggregate(t, ops, &b, &p, &o, cs)) != DES_OK) return st;
+  if ((st = des_backward_update(t, ops, &b, &o, d_grads, cs)) != DES_OK) return st;
   DES_CUDA(cudaMemcpyAsync(h_out_small, t->st_out_small, (size_t)batch * t->stride * 4, cudaMemcpyDeviceToHost, cs));
+  return DES_OK;
+}
+
+static des_status_t st_check_args(des_table* t, int32_t batch, int64_t nnz, const int32_t* h_offsets,
+                                  const uint64_t* h_ids, const des_grads_t* d_grads, const float* h_out_small) {
+  if (!t || !h_offsets || (nnz > 0 && !h_ids) || !d_grads || !h_out_small) return DES_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > t->max_batch || nnz < 0 || nnz > t->max_nnz) return DES_ERR_INVALID_ARG;
+  return DES_OK;
+}
+
+extern "C" des_status_t des_step_host(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
+                                      const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                                      const des_grads_t* d_grads, float* d_pooled, float* d_Z, float* h_out_small,
+                                      void* stream) {
+  des_status_t st = st_check_args(t, batch, nnz, h_offsets, h_ids, d_grads, h_out_small);
+  if (st != DES_OK) return st;
+  if ((st = st_prepare(t)) != DES_OK) return st;
+  cudaStream_t cs = (cudaStream_t)stream;
+  for (int s = 0; s < 2; ++s)          // steps submitted earlier own the staging slots until they finish
+    if (t->st_busy[s]) { DES_CUDA(cudaEventSynchronize(t->st_done[s])); t->st_busy[s] = 0; }
+  if ((st = st_enqueue(t, 0, cs, ops, batch, nnz, h_offsets, h_ids, h_vals, d_grads, d_pooled, d_Z, h_out_small, cs)) != DES_OK)
+    return st;
   DES_CUDA(cudaStreamSynchronize(cs));
+  return DES_OK;
+}
+
+extern "C" des_status_t des_step_host_submit(des_table_t* t, uint32_t ops, int32_t batch, int64_t nnz,
+                                             const int32_t* h_offsets, const uint64_t* h_ids, const float* h_vals,
+                                             const des_grads_t* d_grads, float* d_pooled, float* d_Z,
+                                             float* h_out_small, void* stream, int32_t* ticket) {
+  des_status_t st = st_check_args(t, batch, nnz, h_offsets, h_ids, d_grads, h_out_small);
+  if (st != DES_OK) return st;
+  if (!ticket) return DES_ERR_INVALID_ARG;
+  if ((st = st_prepare(t)) != DES_OK) return st;
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int slot = (int)(t->st_next & 1);
+  if (t->st_busy[slot]) {              // the step that last used this slot must be over before it is overwritten
+    DES_CUDA(cudaEventSynchronize(t->st_done[slot]));
+    t->st_busy[slot] = 0;
+  }
+  if ((st = st_enqueue(t, slot, t->st_copy_stream, ops, batch, nnz, h_offsets, h_ids, h_vals, d_grads, d_pooled, d_Z,
+                       h_out_small, cs)) != DES_OK)
+    return st;
+  DES_CUDA(cudaEventRecord(t->st_done[slot], cs));
+  t->st_busy[slot] = 1;
+  t->st_next += 1;
+  *ticket = slot;
+  return DES_OK;
+}
+
+extern "C" des_status_t des_step_host_wait(des_table_t* t, int32_t ticket) {
+  if (!t || ticket < 0 || ticket > 1) return DES_ERR_INVALID_ARG;
+  if (!t->st_ids[0] || !t->st_busy[ticket]) return DES_OK;
+  DES_CUDA(cudaEventSynchronize(t->st_done[ticket]));
+  t->st_busy[ticket] = 0;
   return DES_OK;
 }

@@ -76,7 +76,8 @@ struct des_table {
   __nv_bfloat16 *pooled_b, *gZ_b;    // bf16 copies of V [max_batch][F*k] and gZ [max_batch][H]
   void* gemm_ws; size_t gemm_ws_bytes;
   // host-step staging
-  int32_t* st_offsets; unsigned long long* st_ids; float* st_vals;
+  int32_t* st_offsets[2]; unsigned long long* st_ids[2]; float* st_vals[2];   // two input slots (pipelined submit)
+  cudaStream_t st_copy_stream; cudaEvent_t st_copied[2], st_done[2]; int st_busy[2]; uint64_t st_next;
   uint32_t* st_rows; uint8_t* st_shards; uint32_t* st_uidx; uint32_t* st_uniq_rows; uint32_t* st_n_uniq;
   float* st_part_small; float* st_out_small;
   uint64_t launches;

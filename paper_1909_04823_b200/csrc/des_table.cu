@@ -99,9 +99,13 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->A2, t->acc2W1, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
                   t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc, t->super_cnt,
-                  t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets, t->st_ids, t->st_vals, t->st_rows,
+                  t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets[0], t->st_ids[0], t->st_vals[0], t->st_offsets[1], t->st_ids[1], t->st_vals[1], t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
   for (void* p : ptrs) dfree(t->cfg, p);
+  if (t->st_copy_stream) {
+    cudaStreamDestroy(t->st_copy_stream);
+    for (int s = 0; s < 2; ++s) { if (t->st_copied[s]) cudaEventDestroy(t->st_copied[s]); if (t->st_done[s]) cudaEventDestroy(t->st_done[s]); }
+  }
   if (t->prof_ev) { for (int i = 0; i < DES_PROF_MAX; ++i) cudaEventDestroy(t->prof_ev[i]); delete[] t->prof_ev; }
   delete[] t->prof_name;
   delete t;
