@@ -31,60 +31,78 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
   return s;
 }
 
-#define PROBE_ILP 4   // occurrences per thread: their probe chains are independent, so 4 slot loads are in flight
+// Occurrences per thread and resident blocks per SM: one probe chain per thread at full occupancy
+// measured fastest (more chains per thread cost registers, hence warps in flight; electing one lane
+// per distinct key of a warp costs more in match instructions than the cached slot loads it saves).
+#ifndef PROBE_ILP
+#define PROBE_ILP 1
+#endif
+#ifndef PROBE_MINB
+#define PROBE_MINB 8
+#endif
 
 struct SlotGeom { unsigned long long slot_base[DES_MAX_SHARDS + 1]; };   // kernel parameter: constant-bank reads
 
-__global__ void __launch_bounds__(256, 4) probe_claim_kernel(
+__global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
     int S, int F, int partition, int insert, Slot* slots, DevMeta* meta, const __grid_constant__ SlotGeom geom,
     uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards, uint32_t* __restrict__ rows) {
-  // occurrence j = tile * (256 * PROBE_ILP) + q * 256 + thread: every access of a warp is contiguous
+  // occurrence j = tile * (256 * PROBE_ILP) + q * 256 + thread: every access of a warp is contiguous.
+  // Per occurrence the probe keeps its key, the table-global slot it looks at (DES_SLOT_NONE once it
+  // is done) and the bounds of the owning shard's slot region: all 32-bit but the key.
   const int j0 = blockIdx.x * (256 * PROBE_ILP) + threadIdx.x;
-  unsigned long long id[PROBE_ILP], base[PROBE_ILP], n[PROBE_ILP], pos[PROBE_ILP];
-  uint32_t found[PROBE_ILP], row[PROBE_ILP], seen_fo[PROBE_ILP];
-  bool busy[PROBE_ILP];
-  unsigned long long nmax = 0;
+  unsigned long long id[PROBE_ILP];
+  uint32_t cur[PROBE_ILP], lo[PROBE_ILP], hi[PROBE_ILP], found[PROBE_ILP], row[PROBE_ILP], seen_fo[PROBE_ILP];
+  uint32_t nmax = 0;
 #pragma unroll
   for (int q = 0; q < PROBE_ILP; ++q) {
     const int j = j0 + q * 256;
-    busy[q] = false; found[q] = DES_SLOT_NONE; row[q] = DES_ROW_NONE; id[q] = 0; base[q] = 0; n[q] = 1; pos[q] = 0;
-    seen_fo[q] = DES_ROW_NONE;
-    if (j >= nnz) continue;
-    id[q] = ids[j];
-    uint32_t s;
-    if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S);
-    else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
-    shards[j] = (uint8_t)s;
-    if (id[q] == DES_KEY_EMPTY) { des_raise(meta, DES_ERR_RESERVED_KEY); continue; }
-    base[q] = geom.slot_base[s];
-    n[q] = geom.slot_base[s + 1] - base[q];
-    pos[q] = __umul64hi(des_mix64(id[q] ^ 0x9E3779B97F4A7C15ull), n[q]);
-    busy[q] = true;
-    nmax = max(nmax, n[q]);
+    cur[q] = DES_SLOT_NONE; found[q] = DES_SLOT_NONE; row[q] = DES_ROW_NONE; seen_fo[q] = DES_ROW_NONE;
+    id[q] = 0; lo[q] = 0; hi[q] = 0;
+    if (j < nnz) {
+      id[q] = ids[j];
+      uint32_t s;
+      if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S);
+      else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
+      shards[j] = (uint8_t)s;
+      if (id[q] == DES_KEY_EMPTY) {
+        des_raise(meta, DES_ERR_RESERVED_KEY);
+      } else {
+        lo[q] = (uint32_t)geom.slot_base[s];
+        hi[q] = (uint32_t)geom.slot_base[s + 1];
+        const uint32_t n = hi[q] - lo[q];
+        cur[q] = lo[q] + (uint32_t)__umul64hi(des_mix64(id[q] ^ 0x9E3779B97F4A7C15ull), (unsigned long long)n);
+        nmax = max(nmax, n);
+      }
+    }
   }
-  for (unsigned long long probe = 0; probe < nmax; ++probe) {
+  for (uint32_t probe = 0; probe < nmax; ++probe) {
     Slot sl[PROBE_ILP];
     bool any = false;
 #pragma unroll
     for (int q = 0; q < PROBE_ILP; ++q)
-      if (busy[q]) { sl[q] = load_slot(slots + base[q] + pos[q]); any = true; }
+      if (cur[q] != DES_SLOT_NONE) { sl[q] = load_slot(slots + cur[q]); any = true; }
     if (!any) break;
 #pragma unroll
     for (int q = 0; q < PROBE_ILP; ++q) {
-      if (!busy[q]) continue;
-      Slot* sp = slots + base[q] + pos[q];
+      if (cur[q] == DES_SLOT_NONE) continue;
+      bool done = false;
       if (sl[q].key == id[q]) {
-        found[q] = (uint32_t)(base[q] + pos[q]); row[q] = sl[q].row; seen_fo[q] = sl[q].first_occ;
-        busy[q] = false; continue;
+        found[q] = cur[q]; row[q] = sl[q].row; seen_fo[q] = sl[q].first_occ;
+        done = true;
+      } else if (sl[q].key == DES_KEY_EMPTY) {
+        if (!insert) {
+          done = true;
+        } else {
+          const unsigned long long old = atomicCAS(&slots[cur[q]].key, DES_KEY_EMPTY, id[q]);
+          if (old == DES_KEY_EMPTY || old == id[q]) { found[q] = cur[q]; done = true; }
+        }
       }
-      if (sl[q].key == DES_KEY_EMPTY) {
-        if (!insert) { busy[q] = false; continue; }
-        const unsigned long long old = atomicCAS(&sp->key, DES_KEY_EMPTY, id[q]);
-        if (old == DES_KEY_EMPTY || old == id[q]) { found[q] = (uint32_t)(base[q] + pos[q]); busy[q] = false; continue; }
+      if (!done && probe + 1 >= hi[q] - lo[q]) {       // region is full
+        done = true;
+        if (insert) des_raise(meta, DES_ERR_CAPACITY);
       }
-      pos[q] = (pos[q] + 1 == n[q]) ? 0 : pos[q] + 1;
-      if (probe + 1 >= n[q]) { busy[q] = false; if (insert) des_raise(meta, DES_ERR_CAPACITY); }   // region is full
+      cur[q] = done ? DES_SLOT_NONE : (cur[q] + 1 == hi[q] ? lo[q] : cur[q] + 1);
     }
   }
 #pragma unroll
