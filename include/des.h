@@ -335,6 +335,48 @@ des_status_t des_step_host_submit(des_table_t* t, uint32_t ops, int32_t batch, i
                                   float* h_out_small, void* stream, int32_t* ticket);
 des_status_t des_step_host_wait(des_table_t* t, int32_t ticket);
 
+/* ---- DCN cross layer under DES (Section 4.4, paragraph on DCN) --------------- */
+
+/* y = x0 * (+)_s <x[slice s], w[slice s]> + b + x  for x0, x, y [B][d] and w, b [d]
+ * (all float32, device, row-major).  w is split along d into num_shards contiguous
+ * slices (slice s = columns floor(s d / S) .. floor((s+1) d / S) - 1); each shard's
+ * partial is one scalar per sample, (+) adds them in shard order.  d_part [S][B]
+ * (optional, may be NULL) receives the per-shard scalars, d_P [B] the aggregate
+ * (needed by the backward), d_y the layer output.  No table is involved; the call
+ * only enqueues kernels on `stream`.  DES_ERR_INVALID_ARG for NULL / non-positive
+ * arguments or num_shards > d. */
+des_status_t des_cross_forward(int32_t batch, int32_t dim, int32_t num_shards, const float* d_x0,
+                               const float* d_x, const float* d_w, const float* d_b, float* d_part,
+                               float* d_P, float* d_y, void* stream);
+
+/* Backward of the same layer for an upstream gradient d_gY [B][d]: every shard can form
+ * t_b = <gY_b, x0_b> by itself (x0 and gY are replicated), so no exchange is needed:
+ *   gx = gY + t w,  gx0 = gY P,  gw = sum_b t_b x_b,  gb = sum_b gY_b.
+ * d_gx0, d_gx [B][d]; d_gw, d_gb [d]; d_ws = caller's scratch of
+ * des_cross_workspace_floats(batch, dim) floats.  The batch sums are taken in a fixed
+ * order (run-to-run identical).  Applying gw / gb is the caller's dense optimizer. */
+des_status_t des_cross_backward(int32_t batch, int32_t dim, const float* d_x0, const float* d_x,
+                                const float* d_w, const float* d_P, const float* d_gY, float* d_gx0,
+                                float* d_gx, float* d_gw, float* d_gb, float* d_ws, void* stream);
+int64_t des_cross_workspace_floats(int32_t batch, int32_t dim);
+
+/* ---- transfer volumes (Sections 4.1-4.3) ------------------------------------ */
+
+/* Bytes one worker moves per iteration under the mesh strategy, Q = (N-1)/N (S_f + S_x),
+ * and under DES, Q = 2 (N-1)/N S_M, with the saving ratio 1 - Q_DES / Q_Mesh, for
+ * [0] LR, [1] FM order 2, [2] the DNN first layer.  S_f = key_bytes * uniq; S_w, S_V from
+ * value_bytes, emb_dim and uniq; S_W = first_layer_bytes; the partials are B, B (k + 1)
+ * and B * hidden values.  Host only, no GPU needed. */
+typedef struct {
+  int32_t workers;            /* N >= 2                                   */
+  int64_t batch, uniq;        /* samples and unique features per batch   */
+  int32_t emb_dim, hidden;    /* k and the first layer's width H         */
+  int32_t key_bytes, value_bytes;   /* 8 and 4 in the paper             */
+  double  first_layer_bytes;  /* S_W                                     */
+} des_comm_model_t;
+typedef struct { double q_mesh[3], q_des[3], saving[3]; } des_comm_volume_t;
+des_status_t des_comm_volume(const des_comm_model_t* m, des_comm_volume_t* out);
+
 /* Per-launch timing for benchmarks.  While enabled, the library records a CUDA
  * event on the call's stream behind every kernel it launches (and one at the
  * entry of every call); des_profile_read synchronises and returns, in launch

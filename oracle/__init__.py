@@ -88,6 +88,31 @@ def comm_saving(B, U, k, H, S_W):
     return out
 
 
+def cross_forward(x0, x, w, bias, S):
+    """DCN cross layer under DES -> dict(part [S][B], P [B], y [B][d], Sabs [B]) in float64."""
+    x0 = np.ascontiguousarray(x0, np.float32); x = np.ascontiguousarray(x, np.float32)
+    w = np.ascontiguousarray(w, np.float32); bias = np.ascontiguousarray(bias, np.float32)
+    B, d = x.shape
+    part = np.zeros((S, B)); P = np.zeros(B); y = np.zeros((B, d)); sabs = np.zeros(B)
+    lib().orc_cross_forward(C.c_int64(B), C.c_int64(d), C.c_int64(S), _p(x0, C.c_float), _p(x, C.c_float),
+                            _p(w, C.c_float), _p(bias, C.c_float), _p(part, C.c_double), _p(P, C.c_double),
+                            _p(y, C.c_double), _p(sabs, C.c_double))
+    return dict(part=part, P=P, y=y, Sabs=sabs)
+
+
+def cross_backward(x0, x, w, P, gY):
+    """-> dict(gx0, gx [B][d], gw, gb [d], t [B]) in float64."""
+    x0 = np.ascontiguousarray(x0, np.float32); x = np.ascontiguousarray(x, np.float32)
+    w = np.ascontiguousarray(w, np.float32); P = np.ascontiguousarray(P, np.float32)
+    gY = np.ascontiguousarray(gY, np.float32)
+    B, d = x.shape
+    gx0 = np.zeros((B, d)); gx = np.zeros((B, d)); gw = np.zeros(d); gb = np.zeros(d); t = np.zeros(B)
+    lib().orc_cross_backward(C.c_int64(B), C.c_int64(d), _p(x0, C.c_float), _p(x, C.c_float), _p(w, C.c_float),
+                             _p(P, C.c_float), _p(gY, C.c_float), _p(gx0, C.c_double), _p(gx, C.c_double),
+                             _p(gw, C.c_double), _p(gb, C.c_double), _p(t, C.c_double))
+    return dict(gx0=gx0, gx=gx, gw=gw, gb=gb, t=t)
+
+
 class Oracle:
     def __init__(self, S, F, k, H=0, partition=0, optimizer=0, seed=0, init_scale=0.01,
                  lr=0.01, eps=1e-8, init_acc=0.0):

@@ -556,4 +556,49 @@ void orc_poke(void* p, uint32_t shard, uint32_t row, uint32_t col, float value, 
   w = set ? value : w + value;
 }
 
+// DCN cross layer under DES (Section 4.4, the paragraph on DCN): the weight
+// vector w is split along its long dimension d into S contiguous slices, shard
+// s forms the scalar p_s = <x[slice s], w[slice s]> per sample, (+) adds the
+// scalars in shard order, and  y = x0 * (+)p + b + x.  Slice s holds columns
+// floor(s d / S) .. floor((s + 1) d / S) - 1.  Sabs (optional) = sum |x_i w_i|.
+void orc_cross_forward(int64_t B, int64_t d, int64_t S, const float* x0, const float* x, const float* w,
+                       const float* bias, double* part, double* P, double* y, double* Sabs) {
+  for (int64_t b = 0; b < B; ++b) {
+    double tot = 0.0, sa = 0.0;
+    for (int64_t s = 0; s < S; ++s) {
+      const int64_t lo = s * d / S, hi = (s + 1) * d / S;
+      double ps = 0.0;
+      for (int64_t i = lo; i < hi; ++i) {
+        ps += (double)x[b * d + i] * (double)w[i];
+        sa += std::fabs((double)x[b * d + i] * (double)w[i]);
+      }
+      if (part) part[s * B + b] = ps;
+      tot += ps;
+    }
+    P[b] = tot;
+    if (Sabs) Sabs[b] = sa;
+    for (int64_t i = 0; i < d; ++i)
+      y[b * d + i] = (double)x0[b * d + i] * tot + (double)bias[i] + (double)x[b * d + i];
+  }
+}
+
+// Its backward for an upstream gradient gY: with t_b = <gY_b, x0_b> (the gradient of the
+// aggregated scalar, which every shard can form by itself),
+//   gx = gY + t w,   gx0 = gY P,   gw = sum_b t_b x_b,   gb = sum_b gY_b.
+void orc_cross_backward(int64_t B, int64_t d, const float* x0, const float* x, const float* w, const float* P,
+                        const float* gY, double* gx0, double* gx, double* gw, double* gb, double* t_out) {
+  for (int64_t i = 0; i < d; ++i) { gw[i] = 0.0; gb[i] = 0.0; }
+  for (int64_t b = 0; b < B; ++b) {
+    double t = 0.0;
+    for (int64_t i = 0; i < d; ++i) t += (double)gY[b * d + i] * (double)x0[b * d + i];
+    if (t_out) t_out[b] = t;
+    for (int64_t i = 0; i < d; ++i) {
+      gx[b * d + i] = (double)gY[b * d + i] + t * (double)w[i];
+      gx0[b * d + i] = (double)gY[b * d + i] * (double)P[b];
+      gw[i] += t * (double)x[b * d + i];
+      gb[i] += (double)gY[b * d + i];
+    }
+  }
+}
+
 }  // extern "C"

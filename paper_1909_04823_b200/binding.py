@@ -28,7 +28,18 @@ EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_f
            "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_table_read_state2", "des_table_write_state2",
-           "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
+           "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_cross_forward", "des_cross_backward",
+           "des_cross_workspace_floats", "des_comm_volume", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
+
+
+class des_comm_model_t(C.Structure):
+    _fields_ = [("workers", C.c_int32), ("batch", C.c_int64), ("uniq", C.c_int64), ("emb_dim", C.c_int32),
+                ("hidden", C.c_int32), ("key_bytes", C.c_int32), ("value_bytes", C.c_int32),
+                ("first_layer_bytes", C.c_double)]
+
+
+class des_comm_volume_t(C.Structure):
+    _fields_ = [("q_mesh", C.c_double * 3), ("q_des", C.c_double * 3), ("saving", C.c_double * 3)]
 
 
 class DesError(RuntimeError):
@@ -116,6 +127,11 @@ def load():
                                            C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.POINTER(C.c_int32)]
         L.des_step_host_wait.argtypes = [C.c_void_p, C.c_int32]
+        L.des_cross_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 8
+        L.des_cross_backward.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 11
+        L.des_cross_workspace_floats.argtypes = [C.c_int32, C.c_int32]
+        L.des_cross_workspace_floats.restype = C.c_int64
+        L.des_comm_volume.argtypes = [C.POINTER(des_comm_model_t), C.POINTER(des_comm_volume_t)]
         L.des_table_launch_count.argtypes = [C.c_void_p]
         L.des_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.des_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int,
@@ -376,3 +392,41 @@ class Table:
 
     def dense1_set_state(self, s1=None, s2=None):
         self._check(self.L.des_dense1_set_state(self.h, _ptr(s1), _ptr(s2), _stream()), "des_dense1_set_state")
+
+
+# ---- DCN cross layer (no table) and transfer volumes ---------------------------------------------
+def _check_free(code, where):
+    if code != 0:
+        raise DesError(code, where)
+
+
+def cross_forward(x0: torch.Tensor, x: torch.Tensor, w: torch.Tensor, b: torch.Tensor, num_shards: int,
+                  want_part: bool = False):
+    """-> (y [B][d], P [B], part [S][B] or None)"""
+    B, d = x.shape
+    y = torch.empty_like(x)
+    P = torch.empty(B, dtype=torch.float32, device=x.device)
+    part = torch.empty((num_shards, B), dtype=torch.float32, device=x.device) if want_part else None
+    _check_free(load().des_cross_forward(B, d, num_shards, _ptr(x0), _ptr(x), _ptr(w), _ptr(b), _ptr(part), _ptr(P),
+                                        _ptr(y), _stream()), "des_cross_forward")
+    return y, P, part
+
+
+def cross_backward(x0, x, w, P, gY):
+    """-> (gx0, gx [B][d], gw, gb [d])"""
+    B, d = x.shape
+    gx0 = torch.empty_like(x); gx = torch.empty_like(x)
+    gw = torch.empty(d, dtype=torch.float32, device=x.device); gb = torch.empty_like(gw)
+    ws = torch.empty(int(load().des_cross_workspace_floats(B, d)), dtype=torch.float32, device=x.device)
+    _check_free(load().des_cross_backward(B, d, _ptr(x0), _ptr(x), _ptr(w), _ptr(P), _ptr(gY), _ptr(gx0), _ptr(gx),
+                                         _ptr(gw), _ptr(gb), _ptr(ws), _stream()), "des_cross_backward")
+    return gx0, gx, gw, gb
+
+
+def comm_volume(workers, batch, uniq, emb_dim, hidden, first_layer_bytes, key_bytes=8, value_bytes=4):
+    """Per-worker bytes under the mesh strategy and under DES, and the saving ratios: dict of 3-lists
+    (LR, FM order 2, DNN first layer).  Host only."""
+    m = des_comm_model_t(workers, batch, uniq, emb_dim, hidden, key_bytes, value_bytes, float(first_layer_bytes))
+    o = des_comm_volume_t()
+    _check_free(load().des_comm_volume(C.byref(m), C.byref(o)), "des_comm_volume")
+    return dict(q_mesh=list(o.q_mesh), q_des=list(o.q_des), saving=list(o.saving))

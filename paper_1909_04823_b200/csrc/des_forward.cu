@@ -42,19 +42,24 @@ __global__ void __launch_bounds__(256) route_kernel(
     const int lo = __ldg(offsets + (size_t)b * F), hi = __ldg(offsets + (size_t)(b + 1) * F);
     for (int s = lane; s < S; s += 32) cur[s] = 0;
     __syncwarp();
-    // pass 1: occurrences per shard (mapped rows only); CSR-order rows for the pooling kernel
-    for (int base = lo; base < hi; base += 32) {
-      const int j = base + lane;
-      int key = -1 - lane;
-      if (j < hi) {
-        const uint32_t r = __ldg(rows + j);
-        const int s = __ldg(shards + j);
-        grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
-        if (r != DES_ROW_NONE) key = s;
+    // pass 1: occurrences per shard (mapped rows only); CSR-order rows for the pooling kernel.
+    // Both passes load the next 32 occurrences before they work on the current ones.
+    {
+      uint32_t r_n = DES_ROW_NONE; int s_n = 0;
+      if (lo + lane < hi) { r_n = __ldg(rows + lo + lane); s_n = __ldg(shards + lo + lane); }
+      for (int base = lo; base < hi; base += 32) {
+        const int j = base + lane;
+        const uint32_t r = r_n; const int s = s_n;
+        if (j + 32 < hi) { r_n = __ldg(rows + j + 32); s_n = __ldg(shards + j + 32); }
+        int key = -1 - lane;
+        if (j < hi) {
+          grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
+          if (r != DES_ROW_NONE) key = s;
+        }
+        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+        if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
+        __syncwarp();
       }
-      const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
-      if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
-      __syncwarp();
     }
     // exclusive scan over shards -> segment starts (lane 0 walks the <= 64 counters)
     if (lane == 0) {
@@ -65,23 +70,31 @@ __global__ void __launch_bounds__(256) route_kernel(
     }
     __syncwarp();
     // pass 2: stable placement
-    for (int base = lo; base < hi; base += 32) {
-      const int j = base + lane;
-      int key = -1 - lane; uint32_t gr = 0;
-      if (j < hi) {
-        const uint32_t r = __ldg(rows + j);
-        const int s = __ldg(shards + j);
-        if (r != DES_ROW_NONE) { key = s; gr = row_base[s] + r; }
+    {
+      uint32_t r_n = DES_ROW_NONE; int s_n = 0; float x_n = 1.f;
+      if (lo + lane < hi) {
+        r_n = __ldg(rows + lo + lane); s_n = __ldg(shards + lo + lane);
+        if (vals) x_n = __ldg(vals + lo + lane);
       }
-      const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
-      if (key >= 0) {
-        const int pos = cur[key] + __popc(same & lt);
-        grow_sorted[pos] = gr;
-        if (vals) x_sorted[pos] = __ldg(vals + j);
+      for (int base = lo; base < hi; base += 32) {
+        const int j = base + lane;
+        const uint32_t r = r_n; const int s = s_n; const float x = x_n;
+        if (j + 32 < hi) {
+          r_n = __ldg(rows + j + 32); s_n = __ldg(shards + j + 32);
+          if (vals) x_n = __ldg(vals + j + 32);
+        }
+        int key = -1 - lane; uint32_t gr = 0;
+        if (j < hi && r != DES_ROW_NONE) { key = s; gr = row_base[s] + r; }
+        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+        if (key >= 0) {
+          const int pos = cur[key] + __popc(same & lt);
+          grow_sorted[pos] = gr;
+          if (vals) x_sorted[pos] = x;
+        }
+        __syncwarp();
+        if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
+        __syncwarp();
       }
-      __syncwarp();
-      if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
-      __syncwarp();
     }
   }
 }

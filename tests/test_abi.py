@@ -36,13 +36,33 @@ def test_struct_layouts_match_header_sizes():
     prog = r'''
 #include <stdio.h>
 #include "des.h"
-int main(void) { printf("%zu %zu %zu %zu %zu\n", sizeof(des_config_t), sizeof(des_batch_t),
-  sizeof(des_partials_t), sizeof(des_outputs_t), sizeof(des_grads_t)); return 0; }
+int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(des_config_t), sizeof(des_batch_t),
+  sizeof(des_partials_t), sizeof(des_outputs_t), sizeof(des_grads_t), sizeof(des_comm_model_t),
+  sizeof(des_comm_volume_t)); return 0; }
 '''
     with tempfile.TemporaryDirectory() as d:
         open(os.path.join(d, "a.c"), "w").write(prog)
         subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", os.path.join(d, "a"), os.path.join(d, "a.c")])
         out = subprocess.check_output([os.path.join(d, "a")]).split()
     want = [C.sizeof(binding.des_config_t), C.sizeof(binding.des_batch_t), C.sizeof(binding.des_partials_t),
-            C.sizeof(binding.des_outputs_t), C.sizeof(binding.des_grads_t)]
+            C.sizeof(binding.des_outputs_t), C.sizeof(binding.des_grads_t), C.sizeof(binding.des_comm_model_t),
+            C.sizeof(binding.des_comm_volume_t)]
     assert [int(v) for v in out] == want
+
+
+def test_comm_volume_reproduces_the_papers_table_2():
+    # Table 2 (Section 4.3): unique features per batch and saving ratios on a 4-node cluster; the
+    # product's calculator (host code of the CUDA library, no GPU needed) against the printed values.
+    from paper_1909_04823_b200 import binding
+    rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "paper_table2_comm_saving.txt"))
+            if l.strip() and l[0] != "#"]
+    assert len(rows) == 5
+    for r in rows:
+        v = binding.comm_volume(4, int(r[0]), int(r[1]), 8, 256, 4800 * 256 * 4)
+        for got, want in zip(v["saving"], r[2:5]):
+            assert f"{100.0 * got:.3f}" == want
+        # the volumes themselves: 3/4 of keys + weights against twice 3/4 of the partials
+        assert v["q_mesh"][0] == 0.75 * (8 + 4) * int(r[1]) and v["q_des"][0] == 2 * 0.75 * 4 * int(r[0])
+    import pytest
+    with pytest.raises(binding.DesError):
+        binding.comm_volume(1, 512, 1000, 8, 256, 0)          # one worker exchanges nothing

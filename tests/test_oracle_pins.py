@@ -456,3 +456,31 @@ def test_ftrl_l1_keeps_small_weights_at_exact_zero():
         assert not np.any(o.read_rows(f["uniq_shard"], f["uniq_row"])["lin"])
     # with every weight still zero, z is the plain gradient sum
     np.testing.assert_allclose(o.read_state2(f["uniq_shard"], f["uniq_row"])["lin2"], tot, rtol=1e-5, atol=1e-6)
+
+
+# --------------------------------------------------------------------------- DCN cross layer
+@pytest.mark.parametrize("S", [1, 3, 4, 16])
+def test_cross_layer_matches_the_unsplit_layer_and_autograd(S):
+    # Section 4.4 (DCN): splitting w along d and adding the shards' scalars is the plain cross layer
+    # y = x0 (x . w) + b + x; its gradients are those autograd gives for that formula.
+    rng = np.random.default_rng(12)
+    B, d = 9, 23                                            # d not a multiple of S: ragged slices
+    x0, x, gY = (rng.standard_normal((B, d)).astype(np.float32) for _ in range(3))
+    w, b = (rng.standard_normal(d).astype(np.float32) for _ in range(2))
+    f = oracle.cross_forward(x0, x, w, b, S)
+    tx0, tx, tw, tb = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (x0, x, w, b))
+    ty = tx0 * (tx @ tw)[:, None] + tb + tx
+    np.testing.assert_allclose(f["y"], ty.detach().numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(f["part"].sum(0), f["P"], rtol=1e-12, atol=1e-12)
+    # every column belongs to exactly one slice: shard s alone sees w restricted to its slice
+    for s in range(S):
+        ws = np.zeros(d, np.float32); lo, hi = s * d // S, (s + 1) * d // S; ws[lo:hi] = w[lo:hi]
+        np.testing.assert_allclose(f["part"][s], x.astype(np.float64) @ ws.astype(np.float64), rtol=1e-12, atol=1e-12)
+    ty.backward(torch.tensor(gY, dtype=torch.float64))
+    g = oracle.cross_backward(x0, x, w, f["P"].astype(np.float32), gY)
+    P32 = f["P"].astype(np.float32).astype(np.float64)      # the backward is handed the float32 aggregate
+    np.testing.assert_allclose(g["gx"], tx.grad.numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g["gw"], tw.grad.numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g["gb"], tb.grad.numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g["gx0"], gY.astype(np.float64) * P32[:, None], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g["gx0"], tx0.grad.numpy(), rtol=1e-6, atol=1e-6)
