@@ -112,6 +112,11 @@ typedef struct {
                             sigma = (sqrt(n+G*G) - sqrt(n))/alpha; z += G - sigma*w;
                             n += G*G; w = |z| <= l1 ? 0 :
                             -(z - sign(z) l1) / ((beta + sqrt(n))/alpha + l2)           */
+  uint32_t shard_world, shard_rank; /* multi-GPU (Algorithm 1: each process holds W_i): this
+                            table owns the shards s with s mod shard_world == shard_rank
+                            and ignores every other key (row DES_ROW_NONE, never inserted);
+                            shard_world 0 or 1 = owns all.  max_rows is spread over the
+                            owned shards only                                           */
   int64_t  max_nnz;      /* largest nnz of any batch (sizes the workspace)            */
   int32_t  max_batch;    /* largest B of any batch                                    */
   int64_t  max_uniq;     /* largest number of distinct keys in one batch (sizes the
@@ -224,6 +229,24 @@ des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* 
  * `out` supplies A (out_small) and pooled. */
 des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t* batch,
                                  const des_outputs_t* out, const des_grads_t* grads, void* stream);
+
+/* ---- aggregation across processes (Algorithm 1, the exchange step) ---------- */
+
+/* With the shards spread over several tables (shard_world > 1, one table per GPU, the
+ * same batch on every GPU as in Section 6), (+) runs in two levels.  des_rank_partial
+ * adds this table's per-shard small partials (des_forward_partials' part_small) in
+ * shard order into d_rank_part [B][k+4], same column layout as one shard's block:
+ * that is the message a process sends.  After the processes have exchanged their
+ * messages (an all-gather into [world][B][k+4] in rank order: NCCL, or peer copies),
+ * des_aggregate_ranks adds them in rank order and applies F (Eq. 8), writing
+ * out_small [B][k+4] exactly as des_aggregate does; every process computes the same
+ * bits.  Pooled blocks and first-layer partials Z are plain element-wise sums over
+ * processes (an all-reduce of des_aggregate's local outputs).  The backward needs no
+ * exchange (Section 3.2): every table updates the keys it owns. */
+des_status_t des_rank_partial(des_table_t* t, int32_t batch, const float* d_part_small, float* d_rank_part,
+                              void* stream);
+des_status_t des_aggregate_ranks(des_table_t* t, uint32_t ops, int32_t batch, int32_t world,
+                                 const float* d_rank_parts, float* d_out_small, void* stream);
 
 /* ---- first dense layer weights W1 [F*k][H], fp32 master (Section 4.3) ----- */
 des_status_t des_dense1_set(des_table_t* t, const float* d_W1, void* stream);

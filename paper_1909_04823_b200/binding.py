@@ -25,7 +25,7 @@ STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "
           7: "DES_ERR_TOO_LARGE"}
 
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
-           "des_aggregate", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
+           "des_aggregate", "des_rank_partial", "des_aggregate_ranks", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_table_read_state2", "des_table_write_state2",
            "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_cross_forward", "des_cross_backward",
@@ -57,6 +57,7 @@ class des_config_t(C.Structure):
                 ("lr", C.c_float), ("eps", C.c_float), ("init_acc", C.c_float),
                 ("lin_optimizer", C.c_uint32), ("beta1", C.c_float), ("beta2", C.c_float),
                 ("ftrl_alpha", C.c_float), ("ftrl_beta", C.c_float), ("ftrl_l1", C.c_float), ("ftrl_l2", C.c_float),
+                ("shard_world", C.c_uint32), ("shard_rank", C.c_uint32),
                 ("max_nnz", C.c_int64), ("max_batch", C.c_int32), ("max_uniq", C.c_int64),
                 ("alloc", C.c_void_p), ("dealloc", C.c_void_p), ("alloc_ctx", C.c_void_p)]
 
@@ -127,6 +128,8 @@ def load():
                                            C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.POINTER(C.c_int32)]
         L.des_step_host_wait.argtypes = [C.c_void_p, C.c_int32]
+        L.des_rank_partial.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.des_aggregate_ranks.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         L.des_cross_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 8
         L.des_cross_backward.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 11
         L.des_cross_workspace_floats.argtypes = [C.c_int32, C.c_int32]
@@ -188,7 +191,8 @@ class Table:
     def __init__(self, num_shards, num_fields, emb_dim, hidden=0, partition=PART_HASH, optimizer=OPT_SGD,
                  max_rows=1 << 20, max_load=0.5, rows_per_shard=None, seed=0, init_scale=0.01, lr=0.01,
                  eps=1e-8, init_acc=0.0, max_nnz=1 << 20, max_batch=1 << 16, max_uniq=0, lin_optimizer=LIN_SAME,
-                 beta1=0.9, beta2=0.999, ftrl_alpha=0.05, ftrl_beta=1.0, ftrl_l1=0.0, ftrl_l2=0.0):
+                 beta1=0.9, beta2=0.999, ftrl_alpha=0.05, ftrl_beta=1.0, ftrl_l1=0.0, ftrl_l2=0.0, shard_world=0,
+                 shard_rank=0):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_1909_04823_b200 needs a CUDA device; there is no CPU path")
         self.L = load()
@@ -205,18 +209,20 @@ class Table:
         cfg.seed, cfg.init_scale, cfg.lr, cfg.eps, cfg.init_acc = int(seed), init_scale, lr, eps, init_acc
         cfg.lin_optimizer, cfg.beta1, cfg.beta2 = lin_optimizer, beta1, beta2
         cfg.ftrl_alpha, cfg.ftrl_beta, cfg.ftrl_l1, cfg.ftrl_l2 = ftrl_alpha, ftrl_beta, ftrl_l1, ftrl_l2
+        cfg.shard_world, cfg.shard_rank = shard_world, shard_rank
         cfg.max_nnz, cfg.max_batch, cfg.max_uniq = int(max_nnz), int(max_batch), int(max_uniq)
         self.h = C.c_void_p()
         self._check(self.L.des_table_create(C.byref(cfg), C.byref(self.h)), "des_table_create")
 
     @classmethod
-    def for_workload(cls, w, max_rows, max_nnz, max_batch=None, rows_per_shard=None, max_uniq=0, max_load=0.5):
+    def for_workload(cls, w, max_rows, max_nnz, max_batch=None, rows_per_shard=None, max_uniq=0, max_load=0.5,
+                     shard_world=0, shard_rank=0):
         return cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, max_rows=max_rows,
                    max_load=max_load, rows_per_shard=rows_per_shard, seed=w.seed, init_scale=w.init_scale,
                    lr=w.lr, eps=w.eps, init_acc=w.init_acc, lin_optimizer=w.lin_optimizer, beta1=w.beta1,
                    beta2=w.beta2, ftrl_alpha=w.ftrl_alpha, ftrl_beta=w.ftrl_beta, ftrl_l1=w.ftrl_l1,
                    ftrl_l2=w.ftrl_l2, max_nnz=max_nnz,
-                   max_batch=max_batch or w.batch, max_uniq=max_uniq)
+                   max_batch=max_batch or w.batch, max_uniq=max_uniq, shard_world=shard_world, shard_rank=shard_rank)
 
     def _check(self, code, where):
         if code != 0:
@@ -274,6 +280,15 @@ class Table:
         self._check(self.L.des_step_host(self.h, ops, batch_size, nnz, _ptr(h_offsets), _ptr(h_ids),
                                          _ptr(h_vals), C.byref(g), _ptr(d_pooled), _ptr(d_Z),
                                          _ptr(h_out_small), _stream()), "des_step_host")
+
+    # -- (+) across processes -----------------------------------------------------------
+    def rank_partial(self, batch_size: int, part_small: torch.Tensor, rank_part: torch.Tensor):
+        self._check(self.L.des_rank_partial(self.h, batch_size, _ptr(part_small), _ptr(rank_part), _stream()),
+                    "des_rank_partial")
+
+    def aggregate_ranks(self, ops: int, batch_size: int, world: int, rank_parts: torch.Tensor, out_small: torch.Tensor):
+        self._check(self.L.des_aggregate_ranks(self.h, ops, batch_size, world, _ptr(rank_parts), _ptr(out_small),
+                                               _stream()), "des_aggregate_ranks")
 
     def step_host_submit(self, ops, batch_size, nnz, h_offsets, h_ids, h_vals, h_out_small, d_pooled=None, d_Z=None,
                          gL=None, gF=None, gE=None, gZ=None, gE_work=None) -> int:

@@ -414,3 +414,34 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
   }
   return DES_OK;
 }
+
+// ---- two-level (+) for shards spread over several processes -------------------
+extern "C" des_status_t des_rank_partial(des_table_t* t, int32_t batch, const float* d_part_small,
+                                         float* d_rank_part, void* stream) {
+  if (!t || !d_part_small || !d_rank_part || batch <= 0 || batch > t->max_batch) return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
+  reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(d_part_small, (size_t)batch * t->stride, t->S, d_rank_part);
+  DES_LAUNCH_CHECK(t, "reduce_shards_kernel");
+  return DES_OK;
+}
+
+extern "C" des_status_t des_aggregate_ranks(des_table_t* t, uint32_t ops, int32_t batch, int32_t world,
+                                            const float* d_rank_parts, float* d_out_small, void* stream) {
+  if (!t || !d_rank_parts || !d_out_small || batch <= 0 || batch > t->max_batch || world < 1 || (ops & ~15u) ||
+      !(ops & (DES_OP_LR | DES_OP_FM)))
+    return DES_ERR_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)stream;
+  des_api_begin(t, cs);
+  const int G = group_for(t->k);
+  const int grid = (int)(((long long)batch * G + 255) / 256);
+  switch (G) {   // the processes' messages are added like shards' partials: fixed (rank) order, then F
+    case 1: aggregate_small_kernel<1><<<grid, 256, 0, cs>>>(d_rank_parts, batch, world, t->k, ops, d_out_small); break;
+    case 2: aggregate_small_kernel<2><<<grid, 256, 0, cs>>>(d_rank_parts, batch, world, t->k, ops, d_out_small); break;
+    case 4: aggregate_small_kernel<4><<<grid, 256, 0, cs>>>(d_rank_parts, batch, world, t->k, ops, d_out_small); break;
+    case 8: aggregate_small_kernel<8><<<grid, 256, 0, cs>>>(d_rank_parts, batch, world, t->k, ops, d_out_small); break;
+    default: aggregate_small_kernel<16><<<grid, 256, 0, cs>>>(d_rank_parts, batch, world, t->k, ops, d_out_small); break;
+  }
+  DES_LAUNCH_CHECK(t, "aggregate_small_kernel");
+  return DES_OK;
+}

@@ -45,8 +45,9 @@ struct SlotGeom { unsigned long long slot_base[DES_MAX_SHARDS + 1]; };   // kern
 
 __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
-    int S, int F, int partition, int insert, Slot* slots, DevMeta* meta, const __grid_constant__ SlotGeom geom,
-    uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards, uint32_t* __restrict__ rows) {
+    int S, int F, int partition, int insert, uint32_t world, uint32_t rank, Slot* slots, DevMeta* meta,
+    const __grid_constant__ SlotGeom geom, uint32_t* __restrict__ slot_of, uint8_t* __restrict__ shards,
+    uint32_t* __restrict__ rows) {
   // occurrence j = tile * (256 * PROBE_ILP) + q * 256 + thread: every access of a warp is contiguous.
   // Per occurrence the probe keeps its key, the table-global slot it looks at (DES_SLOT_NONE once it
   // is done) and the bounds of the owning shard's slot region: all 32-bit but the key.
@@ -67,6 +68,8 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
       shards[j] = (uint8_t)s;
       if (id[q] == DES_KEY_EMPTY) {
         des_raise(meta, DES_ERR_RESERVED_KEY);
+      } else if (world > 1 && s % world != rank) {
+        // another process holds this shard: the occurrence has no row here
       } else {
         lo[q] = (uint32_t)geom.slot_base[s];
         hi[q] = (uint32_t)geom.slot_base[s + 1];
@@ -322,7 +325,8 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   SlotGeom geom;
   for (uint32_t s = 0; s <= t->S; ++s) geom.slot_base[s] = t->h_slot_base[s];
   probe_claim_kernel<<<(nnz + 256 * PROBE_ILP - 1) / (256 * PROBE_ILP), 256, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
-                                          t->cfg.partition, insert, t->slots, t->meta, geom, t->slot_of, b->shards, b->rows);
+                                          t->cfg.partition, insert, t->cfg.shard_world, t->cfg.shard_rank, t->slots, t->meta, geom,
+                                          t->slot_of, b->shards, b->rows);
   DES_LAUNCH_CHECK(t, "probe_claim_kernel");
   if (!insert) return DES_OK;
   flag_count_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);

@@ -124,6 +124,8 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
       (int64_t)c.max_batch * c.num_fields >= (1ll << 31))
     return DES_ERR_INVALID_ARG;
   if ((c.alloc == nullptr) != (c.dealloc == nullptr)) return DES_ERR_INVALID_ARG;
+  if (c.shard_world > 1 && c.shard_rank >= c.shard_world) return DES_ERR_INVALID_ARG;
+  if (c.shard_world <= 1 && c.shard_rank != 0) return DES_ERR_INVALID_ARG;
   if (c.optimizer == DES_OPT_ADAM && !(c.beta1 >= 0.f && c.beta1 < 1.f && c.beta2 >= 0.f && c.beta2 < 1.f))
     return DES_ERR_INVALID_ARG;
   if (c.lin_optimizer == DES_LIN_FTRL && !(c.ftrl_alpha > 0.f && c.ftrl_beta >= 0.f && c.ftrl_l1 >= 0.f && c.ftrl_l2 >= 0.f))
@@ -140,9 +142,13 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev);
   DevMeta hm; memset(&hm, 0, sizeof(hm));
   uint64_t rows = 0, slots = 0;
+  const uint32_t world = c.shard_world > 1 ? c.shard_world : 1;
+  uint32_t owned = 0;
+  for (uint32_t s = 0; s < t->S; ++s) owned += (s % world == c.shard_rank);
   for (uint32_t s = 0; s < t->S; ++s) {
     uint64_t cap = c.h_rows_per_shard ? c.h_rows_per_shard[s]
-                                      : (uint64_t)((double)(c.max_rows / t->S) * 1.05) + 1024;
+                                      : (uint64_t)((double)(c.max_rows / (owned ? owned : 1)) * 1.05) + 1024;
+    if (s % world != c.shard_rank) cap = 0;            // another process holds this shard
     if (cap == 0) cap = 1;
     uint64_t ns = (uint64_t)((double)cap / (double)c.max_load) + 1;
     if (cap >= 0xFFFFFFF0ull) { delete t; return DES_ERR_INVALID_ARG; }
@@ -314,8 +320,9 @@ __global__ void read_rows_kernel(const uint32_t* __restrict__ grows, long long n
 
 extern "C" des_status_t des_table_read_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n, float* d_emb,
                                             float* d_lin, float* d_acc_emb, float* d_acc_lin, void* stream) {
-  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
-  if (n == 0) return DES_OK;
+  if (!t || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;                 // nothing to do, whatever the pointers
+  if (!d_global_rows) return DES_ERR_INVALID_ARG;
   des_api_begin(t, (cudaStream_t)stream);
   read_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
@@ -346,8 +353,9 @@ __global__ void write_rows_kernel(const uint32_t* __restrict__ grows, long long 
 extern "C" des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
                                              const float* d_emb, const float* d_lin, const float* d_acc_emb,
                                              const float* d_acc_lin, void* stream) {
-  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
-  if (n == 0) return DES_OK;
+  if (!t || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;                 // nothing to do, whatever the pointers
+  if (!d_global_rows) return DES_ERR_INVALID_ARG;
   des_api_begin(t, (cudaStream_t)stream);
   write_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->W, t->A, d_emb, d_lin, d_acc_emb, d_acc_lin);
@@ -374,8 +382,9 @@ __global__ void state2_kernel(const uint32_t* __restrict__ grows, long long n, i
 
 extern "C" des_status_t des_table_read_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
                                               float* d_acc2_emb, float* d_lin2, void* stream) {
-  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
-  if (n == 0) return DES_OK;
+  if (!t || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;                 // nothing to do, whatever the pointers
+  if (!d_global_rows) return DES_ERR_INVALID_ARG;
   des_api_begin(t, (cudaStream_t)stream);
   state2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->A, t->A2, d_acc2_emb, d_lin2, 0);
@@ -385,8 +394,9 @@ extern "C" des_status_t des_table_read_state2(des_table_t* t, const uint32_t* d_
 
 extern "C" des_status_t des_table_write_state2(des_table_t* t, const uint32_t* d_global_rows, int64_t n,
                                                const float* d_acc2_emb, const float* d_lin2, void* stream) {
-  if (!t || !d_global_rows || n < 0) return DES_ERR_INVALID_ARG;
-  if (n == 0) return DES_OK;
+  if (!t || n < 0) return DES_ERR_INVALID_ARG;
+  if (n == 0) return DES_OK;                 // nothing to do, whatever the pointers
+  if (!d_global_rows) return DES_ERR_INVALID_ARG;
   des_api_begin(t, (cudaStream_t)stream);
   state2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       d_global_rows, n, t->k, t->stride, t->total_rows, t->A, t->A2, const_cast<float*>(d_acc2_emb),
