@@ -96,27 +96,37 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
   }
 }
 
-// dest[j] = gradient row of occurrence j: the key's own row, or one of its replicas.
+// dest[j] = gradient row of occurrence j: the key's own row, one of its replicas, or the tag of a
+// register-summed key.  Four occurrences per thread: their look-up chains are in flight together.
 __global__ void __launch_bounds__(256) make_dest_kernel(const uint32_t* __restrict__ uidx, int nnz,
                                                         const uint32_t* __restrict__ hinfo,
                                                         const uint32_t* __restrict__ hot_base,
                                                         const uint32_t* __restrict__ hot_R, long long max_uniq,
                                                         uint32_t* __restrict__ dest) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= nnz) return;
-  const uint32_t u = __ldg(uidx + j);
-  uint32_t d = DES_ROW_NONE;
-  if (u != DES_ROW_NONE && (long long)u < max_uniq) {
-    const uint32_t hv = __ldg(hinfo + u);
-    if (hv == DES_ROW_NONE) {
-      d = u;
-    } else if (hv >> 24) {
-      d = SUPER_TAG | ((hv >> 24) - 1u);
-    } else {
-      d = (uint32_t)max_uniq + __ldg(hot_base + hv) + hash_u32((uint32_t)j) % __ldg(hot_R + hv);
+  const int j0 = blockIdx.x * 1024 + threadIdx.x;
+  uint32_t u[4], hv[4], d[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * 256;
+    u[q] = (j < nnz) ? __ldg(uidx + j) : DES_ROW_NONE;
+    if (u[q] != DES_ROW_NONE && (long long)u[q] >= max_uniq) u[q] = DES_ROW_NONE;
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) hv[q] = (u[q] != DES_ROW_NONE) ? __ldg(hinfo + u[q]) : DES_ROW_NONE;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * 256;
+    d[q] = u[q];                                          // cold key (or no row)
+    if (u[q] != DES_ROW_NONE && hv[q] != DES_ROW_NONE) {
+      if (hv[q] >> 24) d[q] = SUPER_TAG | ((hv[q] >> 24) - 1u);
+      else d[q] = (uint32_t)max_uniq + __ldg(hot_base + hv[q]) + hash_u32((uint32_t)j) % __ldg(hot_R + hv[q]);
     }
   }
-  dest[j] = d;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * 256;
+    if (j < nnz) dest[j] = d[q];
+  }
 }
 
 // Replica reduction, stage 1: one warp per work item = HOT_RCHUNK replica rows
@@ -378,7 +388,9 @@ __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
   }
 }
 
+#ifndef UP_UNROLL
 #define UP_UNROLL 4
+#endif
 
 // Advances Adam's step count and recomputes the bias corrections 1 - beta^t in double.
 __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
@@ -520,7 +532,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
                                                        t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
                                                        t->hot_work, t->work_max, super_min);
     DES_LAUNCH_CHECK(t, "hot_select_kernel");
-    make_dest_kernel<<<(nnz + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
+    make_dest_kernel<<<(nnz + 1023) / 1024, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
                                                         t->dest);
     DES_LAUNCH_CHECK(t, "make_dest_kernel");
   }
@@ -556,7 +568,10 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
                                                      t->hot_acc);
   DES_LAUNCH_CHECK(t, "hot_finish_kernel");
   {
-    const unsigned grid = (unsigned)(t->sm_count * 8);
+#ifndef UP_GRID
+#define UP_GRID 8
+#endif
+    const unsigned grid = (unsigned)(t->sm_count * UP_GRID);
 #define UP(GG) update_rows_kernel<GG><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops,       \
                                                            opt, t->meta, t->Gbuf, t->W, t->A, t->A2, t->hinfo)
     switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }

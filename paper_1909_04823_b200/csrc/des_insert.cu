@@ -122,25 +122,38 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
 }
 
 // flags: bit0 = first occurrence of its key in the batch, bit1 = key is new.
-__global__ void __launch_bounds__(IB) flag_count_kernel(
+__global__ void __launch_bounds__(IB / 4) flag_count_kernel(
     int nnz, int S, const Slot* __restrict__ slots, const uint32_t* __restrict__ slot_of,
     const uint8_t* __restrict__ shards, uint8_t* __restrict__ flags, uint32_t* __restrict__ blk_cnt, int nblk_max) {
+  // IB occurrences per block, IB / 4 threads: a thread's four slot look-ups are in flight together
   __shared__ uint32_t cnt[DES_MAX_SHARDS + 1];
   if (threadIdx.x <= DES_MAX_SHARDS) cnt[threadIdx.x] = 0;
   __syncthreads();
-  int j = blockIdx.x * IB + threadIdx.x;
-  uint8_t fl = 0;
-  if (j < nnz) {
-    uint32_t so = slot_of[j];
-    if (so != DES_SLOT_NONE) {
-      Slot sl = slots[so];
-      if (sl.first_occ == (uint32_t)j) fl = (sl.row == DES_ROW_NONE) ? 3 : 1;
-    }
-    flags[j] = fl;
+  const int j0 = blockIdx.x * IB + threadIdx.x;
+  uint32_t so[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * (IB / 4);
+    so[q] = (j < nnz) ? slot_of[j] : DES_SLOT_NONE;
   }
-  unsigned firsts = __ballot_sync(0xFFFFFFFFu, fl & 1);
-  if ((threadIdx.x & 31) == 0 && firsts) atomicAdd(&cnt[0], __popc(firsts));
-  if (fl & 2) atomicAdd(&cnt[1 + shards[j]], 1u);
+  Slot sl[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    sl[q].row = 0; sl[q].first_occ = DES_ROW_NONE;
+    if (so[q] != DES_SLOT_NONE) sl[q] = slots[so[q]];
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * (IB / 4);
+    uint8_t fl = 0;
+    if (j < nnz) {
+      if (so[q] != DES_SLOT_NONE && sl[q].first_occ == (uint32_t)j) fl = (sl[q].row == DES_ROW_NONE) ? 3 : 1;
+      flags[j] = fl;
+    }
+    const unsigned firsts = __ballot_sync(0xFFFFFFFFu, fl & 1);
+    if ((threadIdx.x & 31) == 0 && firsts) atomicAdd(&cnt[0], __popc(firsts));
+    if (fl & 2) atomicAdd(&cnt[1 + shards[j]], 1u);
+  }
   __syncthreads();
   if (threadIdx.x <= S) blk_cnt[(size_t)threadIdx.x * nblk_max + blockIdx.x] = cnt[threadIdx.x];
 }
@@ -285,16 +298,30 @@ __global__ void __launch_bounds__(256) apply_first_kernel(
   }
 }
 
-__global__ void __launch_bounds__(IB) resolve_kernel(int nnz, const Slot* __restrict__ slots,
-                                                     const uint32_t* __restrict__ slot_of,
-                                                     uint32_t* __restrict__ rows, uint32_t* __restrict__ uidx) {
-  int j = blockIdx.x * IB + threadIdx.x;
-  if (j >= nnz) return;
-  uint32_t so = slot_of[j];
-  uint32_t row = DES_ROW_NONE, u = DES_ROW_NONE;
-  if (so != DES_SLOT_NONE) { Slot sl = slots[so]; row = sl.row; u = sl.first_occ; }
-  rows[j] = row;
-  uidx[j] = (row == DES_ROW_NONE) ? DES_ROW_NONE : u;
+// IB occurrences per block, IB / 4 threads: a thread's four slot look-ups are in flight together.
+__global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const Slot* __restrict__ slots,
+                                                         const uint32_t* __restrict__ slot_of,
+                                                         uint32_t* __restrict__ rows, uint32_t* __restrict__ uidx) {
+  const int j0 = blockIdx.x * IB + threadIdx.x;
+  uint32_t so[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * (IB / 4);
+    so[q] = (j < nnz) ? slot_of[j] : DES_SLOT_NONE;
+  }
+  Slot sl[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    sl[q].row = DES_ROW_NONE; sl[q].first_occ = DES_ROW_NONE;
+    if (so[q] != DES_SLOT_NONE) sl[q] = slots[so[q]];
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * (IB / 4);
+    if (j >= nnz) continue;
+    rows[j] = sl[q].row;
+    uidx[j] = (sl[q].row == DES_ROW_NONE) ? DES_ROW_NONE : sl[q].first_occ;
+  }
 }
 
 __global__ void __launch_bounds__(256) finish_kernel(int S, Slot* slots, const uint32_t* __restrict__ uslot,
@@ -329,7 +356,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
                                           t->slot_of, b->shards, b->rows);
   DES_LAUNCH_CHECK(t, "probe_claim_kernel");
   if (!insert) return DES_OK;
-  flag_count_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);
+  flag_count_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);
   DES_LAUNCH_CHECK(t, "flag_count_kernel");
   scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
   DES_LAUNCH_CHECK(t, "scan_blocks_kernel");
@@ -343,7 +370,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
                                                       (t->cfg.lin_optimizer == DES_LIN_FTRL ||
                                                        t->cfg.optimizer != DES_OPT_ADAGRAD) ? 0.f : t->cfg.init_acc);
   DES_LAUNCH_CHECK(t, "apply_first_kernel");
-  resolve_kernel<<<nblk, IB, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
+  resolve_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
   DES_LAUNCH_CHECK(t, "resolve_kernel");
   finish_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->S, t->slots, t->uslot, t->meta, b->n_uniq);
   DES_LAUNCH_CHECK(t, "finish_kernel");
