@@ -38,19 +38,36 @@ __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
   return x;
 }
 
-// hinfo[u] += 1 for a 1 / 2^shift sample of the occurrences.
-__global__ void __launch_bounds__(256) sample_count_kernel(const uint32_t* __restrict__ uidx, int nnz, int shift,
-                                                           long long max_uniq, uint32_t* hinfo) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+// hinfo[u] += 1 for a 1 / 2^shift sample of the occurrences.  A hot key would draw tens of
+// thousands of atomics on one word, which L2 serialises; so counts are first merged per warp
+// (lanes holding the same key), then per block in a small shared-memory table keyed by a hash of
+// the key (a slot taken by another key sends the count straight to memory), and each block adds
+// its table to hinfo once.
+#define SC_THREADS 1024
+#define SC_SLOTS 1024
+__global__ void __launch_bounds__(SC_THREADS) sample_count_kernel(const uint32_t* __restrict__ uidx, int nnz, int shift,
+                                                                  long long max_uniq, uint32_t* hinfo) {
+  __shared__ uint32_t s_key[SC_SLOTS], s_cnt[SC_SLOTS];
+  for (int i = threadIdx.x; i < SC_SLOTS; i += SC_THREADS) { s_key[i] = DES_ROW_NONE; s_cnt[i] = 0u; }
+  __syncthreads();
+  const int i = blockIdx.x * SC_THREADS + threadIdx.x;
   const long long j = ((long long)i << shift) + (shift ? (hash_u32((uint32_t)i) & ((1u << shift) - 1u)) : 0u);
   uint32_t u = DES_ROW_NONE;
   if (j < nnz) u = __ldg(uidx + j);
   const bool ok = u != DES_ROW_NONE && (long long)u < max_uniq;
-  // one atomic per distinct key of the warp (a hot key fills several lanes)
   const unsigned act = __ballot_sync(0xFFFFFFFFu, ok);
-  if (!ok) return;
-  const unsigned same = __match_any_sync(act, u);
-  if ((threadIdx.x & 31) == __ffs(same) - 1) atomicAdd(hinfo + u, (uint32_t)__popc(same));
+  if (ok) {
+    const unsigned same = __match_any_sync(act, u);
+    if ((threadIdx.x & 31) == __ffs(same) - 1) {
+      const uint32_t c = (uint32_t)__popc(same), slot = hash_u32(u) & (SC_SLOTS - 1);
+      const uint32_t old = atomicCAS(&s_key[slot], DES_ROW_NONE, u);
+      if (old == DES_ROW_NONE || old == u) atomicAdd(&s_cnt[slot], c);
+      else atomicAdd(hinfo + u, c);
+    }
+  }
+  __syncthreads();
+  for (int s = threadIdx.x; s < SC_SLOTS; s += SC_THREADS)
+    if (s_cnt[s]) atomicAdd(hinfo + s_key[s], s_cnt[s]);
 }
 
 // Turns the sampled counts into the hot list: hinfo[u] becomes the key's hot
@@ -526,7 +543,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   const uint32_t super_min = use_super ? (uint32_t)(nnz >> 7) : 0u;
   {
     const int n = (nnz >> shift) + 1;
-    sample_count_kernel<<<(n + 255) / 256, 256, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
+    sample_count_kernel<<<(n + SC_THREADS - 1) / SC_THREADS, SC_THREADS, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
     DES_LAUNCH_CHECK(t, "sample_count_kernel");
     hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
                                                        t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,

@@ -184,7 +184,8 @@ __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, in
     }
     wsum[threadIdx.x] = wi - w;
     if (threadIdx.x == 31) {
-      if (blockIdx.x == 0) meta->n_uniq = wi; else meta->new_total[blockIdx.x - 1] = wi;
+      if (blockIdx.x == 0) meta->n_uniq = wi;
+      else { meta->new_total[blockIdx.x - 1] = wi; if (wi) atomicOr(&meta->any_new, 1u); }
     }
   }
   __syncthreads();
@@ -205,15 +206,18 @@ __global__ void __launch_bounds__(IB) assign_kernel(
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint8_t fl = (j < nnz) ? flags[j] : 0;
   const uint32_t s = (j < nnz) ? shards[j] : 0;
-  for (int i = threadIdx.x; i < 32 * DES_MAX_SHARDS; i += IB) (&wnew[0][0])[i] = 0;
+  // steady state of a populated table: no new key in the whole batch, and the per-shard numbering below
+  // has nothing to do (any_new is settled by scan_blocks_kernel, which ran before this kernel)
+  const bool any_new = meta->any_new != 0u;
+  if (any_new) for (int i = threadIdx.x; i < 32 * DES_MAX_SHARDS; i += IB) (&wnew[0][0])[i] = 0;
   __syncthreads();
   // rank among firsts / among the shard's new keys inside the warp (lane order = CSR order)
   const unsigned fmask = __ballot_sync(0xFFFFFFFFu, fl & 1);
   const unsigned lt = (1u << lane) - 1u;
   uint32_t frank = __popc(fmask & lt);
-  const unsigned nmask_all = __ballot_sync(0xFFFFFFFFu, fl & 2);
+  const unsigned nmask_all = any_new ? __ballot_sync(0xFFFFFFFFu, fl & 2) : 0u;
   uint32_t nrank = 0;
-  if (fl & 2) {
+  if (any_new && (fl & 2)) {
     unsigned same = __match_any_sync(nmask_all, s);
     nrank = __popc(same & lt);
     if ((same >> lane) == 1u) wnew[warp][s] = (uint16_t)__popc(same);   // highest lane of the group
@@ -229,7 +233,7 @@ __global__ void __launch_bounds__(IB) assign_kernel(
       if (threadIdx.x >= d) in += o;
     }
     wfirst[threadIdx.x] = in - v;
-  } else if (threadIdx.x >= 64 && threadIdx.x < 64 + S) {
+  } else if (any_new && threadIdx.x >= 64 && threadIdx.x < 64 + S) {
     const int sh = threadIdx.x - 64;
     uint32_t run = 0;
     for (int w = 0; w < 32; ++w) { uint16_t v = wnew[w][sh]; wnew[w][sh] = (uint16_t)run; run += v; }
@@ -334,7 +338,7 @@ __global__ void __launch_bounds__(256) finish_kernel(int S, Slot* slots, const u
     uint32_t n = meta->n_rows[threadIdx.x] + meta->new_total[threadIdx.x];
     meta->n_rows[threadIdx.x] = min(n, meta->row_cap[threadIdx.x]);
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) *n_uniq_out = U;
+  if (blockIdx.x == 0 && threadIdx.x == 0) { *n_uniq_out = U; meta->any_new = 0u; }
 }
 
 extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b, int insert, void* stream) {

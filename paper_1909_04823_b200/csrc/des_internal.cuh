@@ -31,6 +31,7 @@ struct DevMeta {
   uint32_t new_total[DES_MAX_SHARDS];                // new keys of the running insert call
   uint32_t n_uniq;                                   // unique keys of the running insert call
   uint32_t err;                                      // sticky des_status_t raised on device
+  uint32_t any_new;                                  // the running insert call has at least one new key
   uint32_t field_order[1024];                        // fields sorted by (owning shard, field)
   unsigned long long opt_step;                       // backward calls so far (Adam's t), advanced on device
   float adam_c1, adam_c2;                            // 1 - beta1^t, 1 - beta2^t for the running step
