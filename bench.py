@@ -186,12 +186,13 @@ class ClockSampler:
 # 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
-    ("cfg5", "grad_scatter_kernel"): 1949e6,
-    ("cfg5", "shard_partials_kernel"): 1071e6,
+    ("cfg5", "grad_scatter_kernel"): 1711e6,
+    ("cfg5", "super_dense_kernel"): 482e6,
+    ("cfg5", "shard_partials_kernel"): 941e6,
     ("cfg5", "pool_kernel"): 1207e6,
-    ("cfg5", "update_rows_kernel"): 1936e6,
-    ("cfg5", "probe_claim_kernel"): 599e6,
-    ("cfg5", "route_kernel"): 697e6,
+    ("cfg5", "update_rows_kernel"): 1937e6,
+    ("cfg5", "probe_claim_kernel"): 595e6,
+    ("cfg5", "route_kernel"): 628e6,
 }
 
 
@@ -221,8 +222,13 @@ def kernel_bytes(name, st):
         return 4 * S * B * (k + 4) + 4 * B * (k + 4)
     if name == "make_dest_kernel":
         return 8 * nnz + 4 * U
-    if name == "grad_scatter_kernel":
-        return 4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + 2 * row * (U + R)
+    if name == "grad_scatter_kernel":   # + the per-bag counts of the register-summed keys on skewed batches
+        return (4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + 2 * row * (U + R)
+                + (32 * B * F if st["super"] else 0))
+    if name == "super_dense_kernel":
+        return 32 * B * F + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B
+    if name == "sample_count_kernel":
+        return 4 * (nnz >> st["shift"]) + 4 * U
     if name == "hot_reduce_kernel":
         return 2 * row * R
     if name == "update_rows_kernel":
@@ -230,6 +236,14 @@ def kernel_bytes(name, st):
     if name == "cvt_bf16_kernel":          # three launches per step: pooled (forward), gZ and pooled (backward)
         return 6 * (2 * B * F * k + B * st["H"]) // 3
     return None
+
+
+def shift_of(nnz):
+    """log2 of the sampling stride of the backward's hot-key count (about 2^20 samples)."""
+    shift = 0
+    while shift < 6 and (nnz >> shift) > (1 << 20):
+        shift += 1
+    return shift
 
 
 def kernel_flops(name, st):
@@ -431,7 +445,9 @@ def main():
         a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += ms
     U = int(dbs[0].n_uniq.item())
     stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, H=H, U=U, ops=w.ops,
-                 adagrad=(w.optimizer == synth.OPT_ADAGRAD), rep_rows=0)
+                 adagrad=(w.optimizer == synth.OPT_ADAGRAD), rep_rows=0,
+                 super=(k > 28 and batches[0].nnz >= (1 << 20) and batches[0].vals is None),
+                 shift=shift_of(batches[0].nnz))
     tot_k = sum(v[1] for v in per.values()) or 1.0
     kernels = []
     for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
