@@ -32,6 +32,9 @@
 #define SUPER_T 16u       // keys whose occurrences are summed in registers instead of by atomics
 #define SUPER_R 64u       // replica rows of such a key (they only take one partial sum per lane group)
 #define SUPER_TAG 0xFFFFFF00u   // dest[j] = SUPER_TAG | slot for an occurrence of such a key
+#ifndef SC_BLOCKS_PER_SM
+#define SC_BLOCKS_PER_SM 64     // grid cap of the scatter (it strides over the bags)
+#endif
 
 __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
   x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
@@ -239,45 +242,54 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
     uint16_t* __restrict__ super_cnt) {
   constexpr int LB = G * P;
   const int K4 = k >> 2, stride = k + 4;
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long bag = t / LB;
-  const int sub = (int)(t % LB), c4 = sub % G, p = sub / G;
-  const bool live = bag < nbags, col = c4 < K4, lead = c4 == 0;
-  int lo = 0, hi = 0;
-  if (live) { lo = __ldg(offsets + bag); hi = __ldg(offsets + bag + 1); }
-  float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
-  float gf = 0.f, gl = 0.f;
-  if (lo < hi) {
-    const long long b = bag / F;
-    if (ops & DES_OP_FM) gf = __ldg(gF + b);
-    if (ops & DES_OP_LR) gl = __ldg(gL + b);
-    if (col) {
-      if (ops & DES_OP_FM) {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(out_small + b * stride) + c4);
-        c = make_float4(gf * a.x, gf * a.y, gf * a.z, gf * a.w);
-      }
-      if (gE) {
-        const float4 e = __ldg(reinterpret_cast<const float4*>(gE + bag * k) + c4);
-        c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
-      }
-    }
-  }
+  const int sub = threadIdx.x % LB, c4 = sub % G, p = sub / G;
+  const bool col = c4 < K4, lead = c4 == 0;
   const unsigned rowB = (unsigned)stride * 4u;
   char* gcol = reinterpret_cast<char*>(Gbuf) + c4 * 16;
   char* gtail = reinterpret_cast<char*>(Gbuf + k);
-  uint32_t cnt = 0;
   const uint32_t mine = SUPER_TAG | (uint32_t)c4;
-  int i0 = lo;
+  // grid-stride over bags (every lane of a warp runs the same number of rounds); the next bag's bounds are
+  // fetched while the current bag is scattered, so only the destination loads wait on them
+  const long long slots = (long long)gridDim.x * (256 / LB);
+  const long long rounds = (nbags + slots - 1) / slots;
+  long long bag = (long long)blockIdx.x * (256 / LB) + threadIdx.x / LB;
+  int lo_n = 0, hi_n = 0;
+  if (bag < nbags) { lo_n = __ldg(offsets + bag); hi_n = __ldg(offsets + bag + 1); }
+  for (long long r = 0; r < rounds; ++r, bag += slots) {
+    const bool live = bag < nbags;
+    const int lo = lo_n, hi = hi_n;
+    lo_n = 0; hi_n = 0;
+    if (bag + slots < nbags) { lo_n = __ldg(offsets + bag + slots); hi_n = __ldg(offsets + bag + slots + 1); }
+    float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+    float gf = 0.f, gl = 0.f;
+    if (lo < hi) {
+      const long long b = bag / F;
+      if (ops & DES_OP_FM) gf = __ldg(gF + b);
+      if (ops & DES_OP_LR) gl = __ldg(gL + b);
+      if (col) {
+        if (ops & DES_OP_FM) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(out_small + b * stride) + c4);
+          c = make_float4(gf * a.x, gf * a.y, gf * a.z, gf * a.w);
+        }
+        if (gE) {
+          const float4 e = __ldg(reinterpret_cast<const float4*>(gE + bag * k) + c4);
+          c.x += e.x; c.y += e.y; c.z += e.z; c.w += e.w;
+        }
+      }
+    }
+    uint32_t cnt = 0;
+    int i0 = lo;
 #define SC_STEP(U) scatter_step<U, P, HAS_VALS, SUPER>(dest, vals, i0 + p, gcol, gtail, rowB, col, lead, c, gl, gf, mine, cnt)
-  for (; i0 + 4 * P <= hi; i0 += 4 * P) SC_STEP(4);
-  if (i0 + 2 * P <= hi) { SC_STEP(2); i0 += 2 * P; }
-  if (i0 + P <= hi) { SC_STEP(1); i0 += P; }
-  if (i0 + p < hi) SC_STEP(1);
+    for (; i0 + 4 * P <= hi; i0 += 4 * P) SC_STEP(4);
+    if (i0 + 2 * P <= hi) { SC_STEP(2); i0 += 2 * P; }
+    if (i0 + P <= hi) { SC_STEP(1); i0 += P; }
+    if (i0 + p < hi) SC_STEP(1);
 #undef SC_STEP
-  if (SUPER) {
+    if (SUPER) {
 #pragma unroll
-    for (int d = G; d < LB; d <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
-    if (live && p == 0) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
+      for (int d = G; d < LB; d <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+      if (live && p == 0) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
+    }
   }
 }
 
@@ -557,7 +569,9 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
     // long bags: a whole warp per bag (its sub-groups take alternate occurrences); short bags: G lanes per bag
     const bool wide = (long long)nnz >= 4 * nbags;
     const long long threads = nbags * (wide ? 32 : G);
-    const unsigned grid = (unsigned)((threads + 255) / 256);
+    long long blocks = (threads + 255) / 256;
+    if (blocks > (long long)t->sm_count * SC_BLOCKS_PER_SM) blocks = (long long)t->sm_count * SC_BLOCKS_PER_SM;
+    const unsigned grid = (unsigned)blocks;
 #define SC4(GG, PP, HV, SU) grad_scatter_kernel<GG, PP, HV, SU><<<grid, 256, 0, cs>>>(                                  \
         b->offsets, b->vals, t->dest, nbags, t->F, t->k, ops, out->out_small, gr->gL, gr->gF, gE, t->Gbuf, t->super_cnt)
 #define SC3(GG, HV) do { if (wide) SC4(GG, 32 / GG, HV, false); else SC4(GG, 1, HV, false); } while (0)

@@ -25,6 +25,10 @@
 //                 materialised (with atomics) when the caller asks for it.
 #include "des_internal.cuh"
 
+#ifndef POOL_BLOCKS_PER_SM
+#define POOL_BLOCKS_PER_SM 64   // grid cap of the pooling kernel (it strides over the bags)
+#endif
+
 
 __global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
@@ -226,33 +230,42 @@ __global__ void __launch_bounds__(256) pool_kernel(
     uint32_t null_row, float* __restrict__ pooled, float* __restrict__ part_pooled) {
   constexpr int LB = G * P;                            // lanes per bag
   const int K4 = k >> 2, stride = k + 4;
-  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long bag = t / LB;
-  const int sub = (int)(t % LB), c4 = sub % G, p = sub / G;
-  const bool live = bag < nbags, col = c4 < K4;
-  int lo = 0, hi = 0;
-  if (live) { lo = __ldg(offsets + bag); hi = __ldg(offsets + bag + 1); }
+  const int sub = threadIdx.x % LB, c4 = sub % G, p = sub / G;
+  const bool col = c4 < K4;
   const unsigned rowB = (unsigned)stride * 4u;
   const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  // MATERIALISE: this lane's column of block (shard 0, sample, field) of part_pooled [S][B][F*k]
-  float* part_block = nullptr;
   const size_t shard_pitch = (size_t)B * F * k;
-  if (MATERIALISE && live) part_block = part_pooled + (size_t)bag * k + (col ? c4 : 0) * 4;
-  int i0 = lo;
+  // grid-stride over bags (every lane of a warp runs the same number of rounds); the next bag's bounds are
+  // fetched while the current bag is summed
+  const long long slots = (long long)gridDim.x * (256 / LB);
+  const long long rounds = (nbags + slots - 1) / slots;
+  long long bag = (long long)blockIdx.x * (256 / LB) + threadIdx.x / LB;
+  int lo_n = 0, hi_n = 0;
+  if (bag < nbags) { lo_n = __ldg(offsets + bag); hi_n = __ldg(offsets + bag + 1); }
+  for (long long r = 0; r < rounds; ++r, bag += slots) {
+    const bool live = bag < nbags;
+    const int lo = lo_n, hi = hi_n;
+    lo_n = 0; hi_n = 0;
+    if (bag + slots < nbags) { lo_n = __ldg(offsets + bag + slots); hi_n = __ldg(offsets + bag + slots + 1); }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // MATERIALISE: this lane's column of block (shard 0, sample, field) of part_pooled [S][B][F*k]
+    float* part_block = nullptr;
+    if (MATERIALISE && live) part_block = part_pooled + (size_t)bag * k + (col ? c4 : 0) * 4;
+    int i0 = lo;
 #define POOL_STEP(U) pool_step<U, P, HAS_VALS, MATERIALISE>(grow_csr, vals, shards, i0 + p, Wc, rowB, null_row, part_block, \
                                                            shard_pitch, col, acc)
-  for (; i0 + 4 * P <= hi; i0 += 4 * P) POOL_STEP(4);
-  if (i0 + 2 * P <= hi) { POOL_STEP(2); i0 += 2 * P; }
-  if (i0 + P <= hi) { POOL_STEP(1); i0 += P; }
-  if (i0 + p < hi) POOL_STEP(1);
+    for (; i0 + 4 * P <= hi; i0 += 4 * P) POOL_STEP(4);
+    if (i0 + 2 * P <= hi) { POOL_STEP(2); i0 += 2 * P; }
+    if (i0 + P <= hi) { POOL_STEP(1); i0 += P; }
+    if (i0 + p < hi) POOL_STEP(1);
 #undef POOL_STEP
 #pragma unroll
-  for (int d = G; d < LB; d <<= 1) {                   // combine the bag's sub-groups
-    acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
-    acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
+    for (int d = G; d < LB; d <<= 1) {                 // combine the bag's sub-groups
+      acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
+      acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
+    }
+    if (live && p == 0 && col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
   }
-  if (live && p == 0 && col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
 }
 
 // (+) over shards and F.  G lanes per sample, one float4 column each; lane 0 of
@@ -340,7 +353,9 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
     // long bags: a whole warp per bag (its halves take alternate occurrences); short bags: G lanes per bag
     const bool wide = b->nnz >= 4 * nbags;
     const long long threads = nbags * (wide ? 32 : G);
-    const unsigned grid = (unsigned)((threads + 255) / 256);
+    long long blocks = (threads + 255) / 256;
+    if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
+    const unsigned grid = (unsigned)blocks;
 #define PK4(GG, PP, HV, MT) pool_kernel<GG, PP, HV, MT><<<grid, 256, 0, cs>>>(b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, \
                                                                              t->k, t->W, (uint32_t)t->total_rows, pl, pp)
 #define PK3(GG, HV, MT) do { if (wide) PK4(GG, 32 / GG, HV, MT); else PK4(GG, 1, HV, MT); } while (0)
