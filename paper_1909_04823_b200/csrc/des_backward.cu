@@ -417,6 +417,9 @@ __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
   }
 }
 
+#ifndef UP_MINB
+#define UP_MINB 2
+#endif
 #ifndef UP_UNROLL
 #define UP_UNROLL 4
 #endif
@@ -434,7 +437,7 @@ __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
 // keys at a time so that their gradient rows, row numbers, weights and state
 // are all in flight together: the kernel is a pure stream of 272-byte rows.
 template <int G>
-__global__ void __launch_bounds__(256) update_rows_kernel(
+__global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
     uint32_t ops, const OptParams opt_in, const DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
     float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2, uint32_t* __restrict__ hinfo) {

@@ -55,15 +55,12 @@ __global__ void __launch_bounds__(256) route_kernel(
         const int j = base + lane;
         const uint32_t r = r_n; const int s = s_n;
         if (j + 32 < hi) { r_n = __ldg(rows + j + 32); s_n = __ldg(shards + j + 32); }
-        int key = -1 - lane;
         if (j < hi) {
           grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
-          if (r != DES_ROW_NONE) key = s;
+          if (r != DES_ROW_NONE) atomicAdd(&cur[s], 1);     // counting only: order does not matter here
         }
-        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
-        if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
-        __syncwarp();
       }
+      __syncwarp();
     }
     // exclusive scan over shards -> segment starts (lane 0 walks the <= 64 counters)
     if (lane == 0) {
