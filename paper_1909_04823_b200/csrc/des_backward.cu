@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
     float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
     float gf = 0.f, gl = 0.f;
     if (lo < hi) {
-      const long long b = bag / F;
+      const long long b = (long long)((unsigned)bag / (unsigned)F);   // bags < 2^31: no 64-bit division
       if (ops & DES_OP_FM) gf = __ldg(gF + b);
       if (ops & DES_OP_LR) gl = __ldg(gL + b);
       if (col) {

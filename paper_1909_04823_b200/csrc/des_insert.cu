@@ -41,7 +41,10 @@ __device__ __forceinline__ Slot load_slot(const Slot* p) {
 #define PROBE_MINB 8
 #endif
 
-struct SlotGeom { unsigned long long slot_base[DES_MAX_SHARDS + 1]; };   // kernel parameter: constant-bank reads
+struct SlotGeom {
+  unsigned long long slot_base[DES_MAX_SHARDS + 1];
+  uint32_t mod_M, mod_two32;        // constants of the division-free mod S (des_mod_consts)
+};   // kernel parameter: constant-bank reads
 
 __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     const unsigned long long* __restrict__ ids, const int32_t* __restrict__ offsets, int nnz, int nbags,
@@ -63,7 +66,7 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     if (j < nnz) {
       id[q] = ids[j];
       uint32_t s;
-      if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S);
+      if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S, geom.mod_M, geom.mod_two32);
       else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
       shards[j] = (uint8_t)s;
       if (id[q] == DES_KEY_EMPTY) {
@@ -355,6 +358,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   const int nblk = (nnz + IB - 1) / IB;
   SlotGeom geom;
   for (uint32_t s = 0; s <= t->S; ++s) geom.slot_base[s] = t->h_slot_base[s];
+  des_mod_consts(t->S, &geom.mod_M, &geom.mod_two32);
   probe_claim_kernel<<<(nnz + 256 * PROBE_ILP - 1) / (256 * PROBE_ILP), 256, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
                                           t->cfg.partition, insert, t->cfg.shard_world, t->cfg.shard_rank, t->slots, t->meta, geom,
                                           t->slot_of, b->shards, b->rows);

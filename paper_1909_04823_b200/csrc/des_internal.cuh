@@ -108,12 +108,25 @@ __host__ __device__ __forceinline__ unsigned long long des_mix64(unsigned long l
   return z;
 }
 
-// h mod S for a small S (<= 64), exactly, with 32-bit divisions only:
-// h = hi * 2^32 + lo  =>  h mod S = ((hi mod S) * (2^32 mod S) + lo mod S) mod S.
-__device__ __forceinline__ uint32_t des_mod_small(unsigned long long h, uint32_t S) {
+// x mod S for a 32-bit x and a small S, exactly, without a division: with M = floor(2^32 / S) + 1 the
+// quotient estimate q = floor(x M / 2^32) is floor(x / S) or one more, so x - q S is the remainder or the
+// remainder minus S (x M / 2^32 = x / S + x e / 2^32 with 0 < e <= 1, i.e. less than x / S + 1).
+__device__ __forceinline__ uint32_t des_mod32(uint32_t x, uint32_t S, uint32_t M) {
+  const int r = (int)(x - __umulhi(x, M) * S);
+  return (uint32_t)(r < 0 ? r + (int)S : r);
+}
+
+// h mod S for a small S (<= 64), exactly:
+// h = hi * 2^32 + lo  =>  h mod S = ((hi mod S) * (2^32 mod S) + lo mod S) mod S,
+// with M = floor(2^32 / S) + 1 and two32 = 2^32 mod S computed once on the host (des_mod_consts).
+__device__ __forceinline__ uint32_t des_mod_small(unsigned long long h, uint32_t S, uint32_t M, uint32_t two32) {
+  if (S == 1u) return 0u;                              // (M does not fit 32 bits for S = 1)
   const uint32_t hi = (uint32_t)(h >> 32), lo = (uint32_t)h;
-  const uint32_t two32 = (0xFFFFFFFFu % S + 1u) % S;
-  return ((hi % S) * two32 + lo % S) % S;
+  return des_mod32(des_mod32(hi, S, M) * two32 + des_mod32(lo, S, M), S, M);
+}
+static inline void des_mod_consts(uint32_t S, uint32_t* M, uint32_t* two32) {
+  *M = (uint32_t)((1ull << 32) / S + 1ull);
+  *two32 = (uint32_t)((1ull << 32) % S);
 }
 
 // Philox4x32-10 block function.
