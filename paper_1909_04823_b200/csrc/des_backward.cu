@@ -436,7 +436,7 @@ __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
 // 16-byte column each, lane 0 also the linear weight); it works on UP_UNROLL
 // keys at a time so that their gradient rows, row numbers, weights and state
 // are all in flight together: the kernel is a pure stream of 272-byte rows.
-template <int G>
+template <int G, bool ADAM>
 __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
     uint32_t ops, const OptParams opt_in, const DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
@@ -455,27 +455,36 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
   long long u0 = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
   for (long long it = 0; it < iters; ++it, u0 += gstep * UP_UNROLL) {
     uint32_t r[UP_UNROLL];
-    float4 g[UP_UNROLL], tail[UP_UNROLL], v[UP_UNROLL], s[UP_UNROLL], s2[UP_UNROLL], vt[UP_UNROLL], st[UP_UNROLL];
+    float4 g[UP_UNROLL], v[UP_UNROLL], s[UP_UNROLL], s2[ADAM ? UP_UNROLL : 1];
+    float2 tail[UP_UNROLL], st[UP_UNROLL];   // gradient tail (G_w, sum x^2 gF); linear weight's two state words
+    float lw[UP_UNROLL];                      // linear weight (lead lane)
 #pragma unroll
     for (int q = 0; q < UP_UNROLL; ++q) {
       const long long u = u0 + q * gstep;
       r[q] = (u < U) ? __ldg(uniq_rows + u) : DES_ROW_NONE;
-      g[q] = zero; tail[q] = zero;
+      g[q] = zero; tail[q] = make_float2(0.f, 0.f);
       if (u < U) {
         const float4* grow = reinterpret_cast<const float4*>(Gbuf + (size_t)u * stride);
         if (col) g[q] = grow[c4];
-        tail[q] = grow[K4];
+        tail[q] = *reinterpret_cast<const float2*>(grow + K4);
       }
     }
 #pragma unroll
     for (int q = 0; q < UP_UNROLL; ++q) {
-      v[q] = zero; s[q] = zero; s2[q] = zero; vt[q] = zero; st[q] = zero;
+      v[q] = zero; s[q] = zero; lw[q] = 0.f; st[q] = make_float2(0.f, 0.f);
+      if (ADAM) s2[ADAM ? q : 0] = zero;
       if (r[q] != DES_ROW_NONE) {
         const float4* w = reinterpret_cast<const float4*>(W + (size_t)r[q] * stride);
         const float4* a = A ? reinterpret_cast<const float4*>(A + (size_t)r[q] * stride) : nullptr;
-        const float4* a2 = A2 ? reinterpret_cast<const float4*>(A2 + (size_t)r[q] * stride) : nullptr;
-        if (col) { v[q] = w[c4]; if (a && upd_v) s[q] = a[c4]; if (a2 && upd_v) s2[q] = a2[c4]; }
-        if (lead) { vt[q] = w[K4]; if (a && upd_w) st[q] = a[K4]; }
+        if (col) {
+          v[q] = w[c4];
+          if (a && upd_v) s[q] = a[c4];
+          if (ADAM && upd_v) s2[ADAM ? q : 0] = reinterpret_cast<const float4*>(A2 + (size_t)r[q] * stride)[c4];
+        }
+        if (lead) {
+          lw[q] = *reinterpret_cast<const float*>(w + K4);
+          if (a && upd_w) st[q] = *reinterpret_cast<const float2*>(a + K4);
+        }
       }
     }
     __syncwarp();   // all lanes of a group have read the gradient row before its lead lane clears it
@@ -488,12 +497,13 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
         if (col) grow[c4] = zero;
         if (lead) { grow[K4] = zero; hinfo[u] = 0u; }
       }
+      float4& m2 = s2[ADAM ? q : 0];            // Adam's second moment (unused otherwise)
       if (mapped && col && upd_v) {
         const float t1 = tail[q].y;
-        des_opt_step(opt, v[q].x, s[q].x, s2[q].x, g[q].x - v[q].x * t1);
-        des_opt_step(opt, v[q].y, s[q].y, s2[q].y, g[q].y - v[q].y * t1);
-        des_opt_step(opt, v[q].z, s[q].z, s2[q].z, g[q].z - v[q].z * t1);
-        des_opt_step(opt, v[q].w, s[q].w, s2[q].w, g[q].w - v[q].w * t1);
+        des_opt_step(opt, v[q].x, s[q].x, m2.x, g[q].x - v[q].x * t1);
+        des_opt_step(opt, v[q].y, s[q].y, m2.y, g[q].y - v[q].y * t1);
+        des_opt_step(opt, v[q].z, s[q].z, m2.z, g[q].z - v[q].z * t1);
+        des_opt_step(opt, v[q].w, s[q].w, m2.w, g[q].w - v[q].w * t1);
       }
       // squared norm of the (new) latent vector, kept in the row's tail for the forward's M_2
       float n2 = v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
@@ -505,16 +515,15 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
       if (col && upd_v) {
         w[c4] = v[q];
         if (a) a[c4] = s[q];
-        if (A2) reinterpret_cast<float4*>(A2 + (size_t)r[q] * stride)[c4] = s2[q];
+        if (ADAM) reinterpret_cast<float4*>(A2 + (size_t)r[q] * stride)[c4] = m2;
       }
       if (lead) {
         if (upd_w) {     // linear weight: its two state words sit side by side in the state row's tail
-          if (opt.lin_optimizer == DES_LIN_FTRL) des_ftrl_step(opt, vt[q].x, st[q].x, st[q].y, tail[q].x);
-          else des_opt_step(opt, vt[q].x, st[q].x, st[q].y, tail[q].x);
+          if (opt.lin_optimizer == DES_LIN_FTRL) des_ftrl_step(opt, lw[q], st[q].x, st[q].y, tail[q].x);
+          else des_opt_step(opt, lw[q], st[q].x, st[q].y, tail[q].x);
         }
-        vt[q].y = n2;
-        w[K4] = vt[q];
-        if (a && upd_w) a[K4] = st[q];
+        w[K4] = make_float4(lw[q], n2, 0.f, 0.f);
+        if (a && upd_w) a[K4] = make_float4(st[q].x, st[q].y, 0.f, 0.f);
       }
     }
   }
@@ -606,10 +615,12 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
 #define UP_GRID 8
 #endif
     const unsigned grid = (unsigned)(t->sm_count * UP_GRID);
-#define UP(GG) update_rows_kernel<GG><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops,       \
-                                                           opt, t->meta, t->Gbuf, t->W, t->A, t->A2, t->hinfo)
+#define UP2(GG, AD) update_rows_kernel<GG, AD><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops, \
+                                                                   opt, t->meta, t->Gbuf, t->W, t->A, t->A2, t->hinfo)
+#define UP(GG) do { if (t->A2) UP2(GG, true); else UP2(GG, false); } while (0)
     switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }
 #undef UP
+#undef UP2
     DES_LAUNCH_CHECK(t, "update_rows_kernel");
   }
   return DES_OK;
