@@ -123,5 +123,10 @@ def test_adam_step_count_survives_graph_replay():
             t.close()
     # the forward results fed to the three backward calls are the same stale ones on both sides,
     # so the two runs execute identical arithmetic except for atomic summation order
+    # (a sum that cancels to rounding size can come out with the other sign in another order, and Adam then
+    # moves the weight by lr the other way: allow a handful of such elements)
     for n in ("emb", "lin", "acc_emb"):
-        np.testing.assert_allclose(res[0][n], res[1][n], rtol=2e-4, atol=2e-6, err_msg=n)
+        a, c = res[0][n].astype(np.float64), res[1][n].astype(np.float64)
+        off = np.abs(a - c) > 2e-4 * np.abs(c) + 2e-6
+        assert off.mean() < 1e-3, (n, int(off.sum()), off.size)
+    # (a bias correction frozen at the captured step would shift EVERY weight of steps 2 and 3)

@@ -5,13 +5,17 @@ import pytest
 import torch
 
 from paper_1909_04823_b200 import synth
-from paper_1909_04823_b200.synth import OP_FM, OP_LR, OP_POOL, OPT_ADAGRAD
+from paper_1909_04823_b200.synth import OP_FM, OP_LR, OP_POOL, OPT_SGD
 
 pytestmark = pytest.mark.gpu
 
 
 def _workload():
-    return synth.config(4).scaled(batch=512, prepopulate=2000, init_scale=0.05, optimizer=OPT_ADAGRAD,
+    # SGD: the update is linear in the summed gradient, so two runs that differ only in the order of the
+    # gradient atomics stay within rounding of each other (Adagrad / Adam divide by |G|-sized quantities and
+    # can turn a rounding-sized difference of a cancelling sum into an lr-sized one)
+    # (and a small step: with O(1) upstream gradients a larger one blows the weights up within three steps)
+    return synth.config(4).scaled(batch=512, prepopulate=2000, init_scale=0.05, optimizer=OPT_SGD, lr=1e-5,
                                   ops=OP_LR | OP_FM | OP_POOL)
 
 
@@ -22,6 +26,15 @@ def _batches(w, n):
 
 def _pinned(b):
     return (torch.from_numpy(b.offsets).pin_memory(), torch.from_numpy(b.ids.view(np.int64)).pin_memory())
+
+
+def _close(a, b, what=""):
+    """Equal up to the order of float32 additions: relative to the element, or to the size of the row's
+    largest element where the element itself is a sum that cancels."""
+    a = np.asarray(a, dtype=np.float64); b = np.asarray(b, dtype=np.float64)
+    scale = np.abs(b).reshape(b.shape[0], -1).max(axis=1).reshape((-1,) + (1,) * (b.ndim - 1)) if b.ndim > 1 else np.abs(b).max()
+    bad = np.abs(a - b) > 2e-4 * np.abs(b) + 2e-6 * np.maximum(scale, 1.0)
+    assert not bad.any(), (what, int(bad.sum()), float(np.abs(a - b).max()))
 
 
 def _final_rows(t, keys_batch):
@@ -60,12 +73,12 @@ def test_step_host_equals_device_call_sequence():
             torch.cuda.synchronize()
             assert ta.status() == 0 and tb.status() == 0
             # same kernels on the same table state: equal up to the order of the gradient atomics of earlier steps
-            np.testing.assert_allclose(h_out.numpy(), out.cpu().numpy(), rtol=2e-4, atol=2e-6)
-            np.testing.assert_allclose(pooled_a.cpu().numpy(), pooled_b.cpu().numpy(), rtol=2e-4, atol=2e-6)
+            _close(h_out.numpy(), out.cpu().numpy(), "out_small")
+            _close(pooled_a.cpu().numpy(), pooled_b.cpu().numpy(), "pooled")
         assert ta.size() == tb.size()
         ra, rb = _final_rows(ta, bs[-1]), _final_rows(tb, bs[-1])
         for n in ra:
-            np.testing.assert_allclose(ra[n], rb[n], rtol=2e-4, atol=2e-6, err_msg=n)
+            _close(ra[n], rb[n], n)
     finally:
         ta.close(); tb.close()
 
@@ -105,10 +118,10 @@ def test_pipelined_submit_wait_equals_blocking_steps():
         finally:
             t.close()
     for a, b_ in zip(outs["blocking"][0], outs["pipelined"][0]):
-        np.testing.assert_allclose(a, b_, rtol=2e-4, atol=2e-6)
+        _close(a, b_, "out_small")
     assert outs["blocking"][1] == outs["pipelined"][1]
     for nm in outs["blocking"][2]:
-        np.testing.assert_allclose(outs["blocking"][2][nm], outs["pipelined"][2][nm], rtol=2e-4, atol=2e-6, err_msg=nm)
+        _close(outs["blocking"][2][nm], outs["pipelined"][2][nm], nm)
 
 
 def test_blocking_step_after_submits_waits_for_them():
