@@ -28,7 +28,6 @@
 
 #define HOT_MIN 512u      // estimated occurrences from which a key is treated as hot
 #define HOT_CHAIN 256u    // target number of additions per replica row
-#define HOT_RCHUNK 64u    // replica rows summed by one warp of the reduction
 #define SUPER_T 16u       // keys whose occurrences are summed in registers instead of by atomics
 #define SUPER_R 64u       // replica rows of such a key (they only take one partial sum per lane group)
 #define SUPER_TAG 0xFFFFFF00u   // dest[j] = SUPER_TAG | slot for an occurrence of such a key
@@ -94,7 +93,8 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
       bool sup = false;
       uint32_t ts = 0;
       if (super_min && est >= super_min) { ts = atomicAdd(&ctr[3], 1u); sup = ts < SUPER_T; }
-      const uint32_t R = sup ? SUPER_R : (est + HOT_CHAIN - 1) / HOT_CHAIN;
+      // (capped so that a key's chunk number fits the 18 bits of a work item; longer chains only cost accuracy)
+      const uint32_t R = sup ? SUPER_R : min((est + HOT_CHAIN - 1) / HOT_CHAIN, 0x3FFFFu * HOT_RCHUNK);
       const uint32_t hh = atomicAdd(&ctr[0], 1u);
       if (hh < h_max) {
         const uint32_t base = atomicAdd(&ctr[1], R);
@@ -168,11 +168,29 @@ __global__ void __launch_bounds__(256) hot_reduce_kernel(const uint32_t* __restr
     const uint32_t r_lo = chunk * HOT_RCHUNK, r_hi = min(R, r_lo + HOT_RCHUNK);
     float* rep = Gbuf + ((size_t)max_uniq + hot_base[h]) * stride;
     double a0 = 0.0, a1 = 0.0, a2 = 0.0;
-    for (uint32_t r = r_lo; r < r_hi; ++r) {
+    const bool c0 = lane < stride, c1 = lane + 32 < stride, c2 = lane + 64 < stride;
+    uint32_t r = r_lo;
+    for (; r + 4 <= r_hi; r += 4) {                    // four rows in flight
+      float v0[4], v1[4], v2[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float* row = rep + (size_t)(r + q) * stride;
+        v0[q] = c0 ? row[lane] : 0.f; v1[q] = c1 ? row[lane + 32] : 0.f; v2[q] = c2 ? row[lane + 64] : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float* row = rep + (size_t)(r + q) * stride;
+        a0 += (double)v0[q]; a1 += (double)v1[q]; a2 += (double)v2[q];
+        if (c0) row[lane] = 0.f;
+        if (c1) row[lane + 32] = 0.f;
+        if (c2) row[lane + 64] = 0.f;
+      }
+    }
+    for (; r < r_hi; ++r) {
       float* row = rep + (size_t)r * stride;
-      if (lane < stride) { a0 += (double)row[lane]; row[lane] = 0.f; }
-      if (lane + 32 < stride) { a1 += (double)row[lane + 32]; row[lane + 32] = 0.f; }
-      if (lane + 64 < stride) { a2 += (double)row[lane + 64]; row[lane + 64] = 0.f; }
+      if (c0) { a0 += (double)row[lane]; row[lane] = 0.f; }
+      if (c1) { a1 += (double)row[lane + 32]; row[lane + 32] = 0.f; }
+      if (c2) { a2 += (double)row[lane + 64]; row[lane + 64] = 0.f; }
     }
     double* dst = hot_acc + (size_t)h * stride;
     if (lane < stride) atomicAdd(dst + lane, a0);

@@ -9,6 +9,7 @@
 
 #define DES_MAX_SHARDS 64
 #define DES_SLOT_NONE 0xFFFFFFFFu
+#define HOT_RCHUNK 16u     // replica rows of a hot key summed by one warp of the backward's replica reduction
 
 // One open-addressing slot: 16 bytes, read with a single vector load.
 //   key        DES_KEY_EMPTY until claimed by a 64-bit CAS; never changes after.

@@ -194,7 +194,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->hot_R, (size_t)t->hot_max * 4);
   A(t->hot_u, (size_t)t->hot_max * 4);
   A(t->hot_ctr, 256);
-  t->work_max = t->rep_max / 64 + t->hot_max;
+  t->work_max = t->rep_max / HOT_RCHUNK + t->hot_max;
   A(t->hot_work, (size_t)t->work_max * 4);
   A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);
   if (t->k > 28 && t->max_nnz >= (1 << 20)) A(t->super_cnt, (size_t)t->max_batch * t->F * 16 * 2);
