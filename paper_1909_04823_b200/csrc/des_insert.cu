@@ -2,7 +2,7 @@
 // including shard routing (Section 5, "Large-scale Sparse Features": weights of
 // field f live on node f mod N; Section 4.2: any balanced partition).
 //
-// One call = seven short kernels, none of which waits on another thread:
+// One call = eight short kernels, none of which waits on another thread:
 //   probe_claim   every occurrence finds its key's slot in the owning shard's
 //                 region (linear probing) or claims an empty one with a 64-bit
 //                 CAS; the slot remembers the smallest occurrence index.
@@ -13,7 +13,9 @@
 //   assign        first occurrences get the batch-unique index (rank among
 //                 firsts) and, for new keys, the next shard-local row (rank
 //                 among the shard's new keys): both in CSR order, so the result
-//                 does not depend on thread scheduling.
+//                 does not depend on thread scheduling.  Two kernels: the ranks
+//                 among firsts always, the new-key numbering only when the
+//                 batch has a new key at all.
 //   apply_first   one thread per unique key writes these numbers into the
 //                 key's slot and initialises new rows from the counter-based
 //                 generator.
@@ -210,61 +212,92 @@ __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, in
   for (int i = lo; i < hi; ++i) { uint32_t v = seq[i]; seq[i] = run; run += v; }
 }
 
-// Ranks only: first_j[u] = occurrence index of unique key u (bit 31 set for a new
-// key) and, for a new key, its shard-local row in uniq_rows[u].  The random slot
+// The common case of assign_kernel below — a batch without a single new key — needs the rank among the
+// first occurrences only: IB occurrences per block, four consecutive ones per thread (their flags are one
+// 32-bit load), one block-wide scan.  Runs always; when the batch does have new keys, assign_kernel
+// rewrites first_j with the new-key marks.
+__global__ void __launch_bounds__(IB / 4) assign_firsts_kernel(int nnz, const uint8_t* __restrict__ flags,
+                                                               const uint32_t* __restrict__ blk_cnt,
+                                                               uint32_t* __restrict__ first_j) {
+  __shared__ uint32_t wsum[IB / 128];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int j0 = blockIdx.x * IB + threadIdx.x * 4;
+  uint32_t w = 0;
+  if (j0 + 3 < nnz) w = *reinterpret_cast<const uint32_t*>(flags + j0);
+  else for (int q = 0; q < 4; ++q) if (j0 + q < nnz) w |= (uint32_t)flags[j0 + q] << (8 * q);
+  w &= 0x01010101u;                                           // bit 0 of each flag: first occurrence of its key
+  const uint32_t cnt = __popc(w);
+  uint32_t incl = cnt;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+    if (lane >= d) incl += v;
+  }
+  if (lane == 31) wsum[warp] = incl;
+  __syncthreads();
+  uint32_t before = 0;
+  for (int i = 0; i < warp; ++i) before += wsum[i];
+  uint32_t u = blk_cnt[blockIdx.x] + before + incl - cnt;
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    if ((w >> (8 * q)) & 1u) first_j[u++] = (uint32_t)(j0 + q);
+}
+
+// New keys only: first_j[u] gets bit 31 and uniq_rows[u] the key's shard-local row (rank among the
+// shard's new keys on top of the shard's size).  The random slot
 // accesses are left to apply_first_kernel, which runs one thread per unique key.
 __global__ void __launch_bounds__(IB) assign_kernel(
-    int nnz, int S, DevMeta* meta, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
+    int nnz, int nblk, int S, DevMeta* meta, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
     const uint32_t* __restrict__ blk_cnt, int nblk_max, uint32_t* __restrict__ first_j,
     uint32_t* __restrict__ uniq_rows) {
   __shared__ uint32_t wfirst[32];
   __shared__ uint16_t wnew[32][DES_MAX_SHARDS];
-  const int j = blockIdx.x * IB + threadIdx.x;
+  // steady state of a populated table: no new key in the whole batch (settled by scan_blocks_kernel, which
+  // ran before this kernel), and assign_firsts_kernel has done all there is to do
+  if (meta->any_new == 0u) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint8_t fl = (j < nnz) ? flags[j] : 0;
-  const uint32_t s = (j < nnz) ? shards[j] : 0;
-  // steady state of a populated table: no new key in the whole batch, and the per-shard numbering below
-  // has nothing to do (any_new is settled by scan_blocks_kernel, which ran before this kernel)
-  const bool any_new = meta->any_new != 0u;
-  if (any_new) for (int i = threadIdx.x; i < 32 * DES_MAX_SHARDS; i += IB) (&wnew[0][0])[i] = 0;
-  __syncthreads();
-  // rank among firsts / among the shard's new keys inside the warp (lane order = CSR order)
-  const unsigned fmask = __ballot_sync(0xFFFFFFFFu, fl & 1);
   const unsigned lt = (1u << lane) - 1u;
-  uint32_t frank = __popc(fmask & lt);
-  const unsigned nmask_all = any_new ? __ballot_sync(0xFFFFFFFFu, fl & 2) : 0u;
-  uint32_t nrank = 0;
-  if (any_new && (fl & 2)) {
-    unsigned same = __match_any_sync(nmask_all, s);
-    nrank = __popc(same & lt);
-    if ((same >> lane) == 1u) wnew[warp][s] = (uint16_t)__popc(same);   // highest lane of the group
-  }
-  if (lane == 0) wfirst[warp] = __popc(fmask);
-  __syncthreads();
-  // exclusive prefix over warps
-  if (threadIdx.x < 32) {
-    uint32_t v = wfirst[threadIdx.x], in = v;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      uint32_t o = __shfl_up_sync(0xFFFFFFFFu, in, d);
-      if (threadIdx.x >= d) in += o;
+  for (int tile = blockIdx.x; tile < nblk; tile += gridDim.x) {   // a few resident blocks walk the tiles
+    const int j = tile * IB + threadIdx.x;
+    const uint8_t fl = (j < nnz) ? flags[j] : 0;
+    const uint32_t s = (j < nnz) ? shards[j] : 0;
+    for (int i = threadIdx.x; i < 32 * DES_MAX_SHARDS; i += IB) (&wnew[0][0])[i] = 0;
+    __syncthreads();
+    // rank among firsts / among the shard's new keys inside the warp (lane order = CSR order)
+    const unsigned fmask = __ballot_sync(0xFFFFFFFFu, fl & 1);
+    const uint32_t frank = __popc(fmask & lt);
+    const unsigned nmask_all = __ballot_sync(0xFFFFFFFFu, fl & 2);
+    uint32_t nrank = 0;
+    if (fl & 2) {
+      unsigned same = __match_any_sync(nmask_all, s);
+      nrank = __popc(same & lt);
+      if ((same >> lane) == 1u) wnew[warp][s] = (uint16_t)__popc(same);   // highest lane of the group
     }
-    wfirst[threadIdx.x] = in - v;
-  } else if (any_new && threadIdx.x >= 64 && threadIdx.x < 64 + S) {
-    const int sh = threadIdx.x - 64;
-    uint32_t run = 0;
-    for (int w = 0; w < 32; ++w) { uint16_t v = wnew[w][sh]; wnew[w][sh] = (uint16_t)run; run += v; }
-  }
-  __syncthreads();
-  if (!(fl & 1)) return;
-  const uint32_t u = blk_cnt[blockIdx.x] + wfirst[warp] + frank;
-  if (fl & 2) {
-    uint32_t local = meta->n_rows[s] + blk_cnt[(size_t)(1 + s) * nblk_max + blockIdx.x] + wnew[warp][s] + nrank;
-    if (local >= meta->row_cap[s]) { local = DES_ROW_NONE; des_raise(meta, DES_ERR_CAPACITY); }
-    uniq_rows[u] = local;
-    first_j[u] = (uint32_t)j | 0x80000000u;
-  } else {
-    first_j[u] = (uint32_t)j;
+    if (lane == 0) wfirst[warp] = __popc(fmask);
+    __syncthreads();
+    // exclusive prefix over warps
+    if (threadIdx.x < 32) {
+      uint32_t v = wfirst[threadIdx.x], in = v;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, in, d);
+        if (threadIdx.x >= d) in += o;
+      }
+      wfirst[threadIdx.x] = in - v;
+    } else if (threadIdx.x >= 64 && threadIdx.x < 64 + S) {
+      const int sh = threadIdx.x - 64;
+      uint32_t run = 0;
+      for (int w = 0; w < 32; ++w) { uint16_t v = wnew[w][sh]; wnew[w][sh] = (uint16_t)run; run += v; }
+    }
+    __syncthreads();
+    if (fl & 2) {                                     // (first_j of the other firsts is already in place)
+      const uint32_t u = blk_cnt[tile] + wfirst[warp] + frank;
+      uint32_t local = meta->n_rows[s] + blk_cnt[(size_t)(1 + s) * nblk_max + tile] + wnew[warp][s] + nrank;
+      if (local >= meta->row_cap[s]) { local = DES_ROW_NONE; des_raise(meta, DES_ERR_CAPACITY); }
+      uniq_rows[u] = local;
+      first_j[u] = (uint32_t)j | 0x80000000u;
+    }
+    __syncthreads();                                  // the shared tables are reused by the next tile
   }
 }
 
@@ -382,8 +415,10 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   DES_LAUNCH_CHECK(t, "flag_count_kernel");
   scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
   DES_LAUNCH_CHECK(t, "scan_blocks_kernel");
-  assign_kernel<<<nblk, IB, 0, cs>>>(nnz, t->S, t->meta, b->shards, t->flags, t->blk_cnt, t->nblk_max, t->dest,
-                                     b->uniq_rows);
+  assign_firsts_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->flags, t->blk_cnt, t->dest);
+  DES_LAUNCH_CHECK(t, "assign_firsts_kernel");
+  assign_kernel<<<nblk < t->sm_count * 2 ? nblk : t->sm_count * 2, IB, 0, cs>>>(nnz, nblk, t->S, t->meta, b->shards, t->flags,
+                                                                                t->blk_cnt, t->nblk_max, t->dest, b->uniq_rows);
   DES_LAUNCH_CHECK(t, "assign_kernel");
   apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>((const unsigned long long*)b->ids, t->k, t->stride, t->slots,
                                                       t->meta, t->slot_of, b->shards, t->dest, t->uslot, b->uniq_rows,
