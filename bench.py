@@ -186,13 +186,13 @@ class ClockSampler:
 # 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
-    ("cfg5", "grad_scatter_kernel"): 1711e6,
-    ("cfg5", "super_dense_kernel"): 482e6,
-    ("cfg5", "shard_partials_kernel"): 941e6,
-    ("cfg5", "pool_kernel"): 1207e6,
+    ("cfg5", "grad_scatter_kernel"): 1732e6,
+    ("cfg5", "super_dense_kernel"): 481e6,
+    ("cfg5", "shard_partials_kernel"): 939e6,
+    ("cfg5", "pool_kernel"): 1211e6,
     ("cfg5", "update_rows_kernel"): 1937e6,
-    ("cfg5", "probe_claim_kernel"): 595e6,
-    ("cfg5", "route_kernel"): 628e6,
+    ("cfg5", "probe_claim_kernel"): 596e6,
+    ("cfg5", "route_kernel"): 683e6,
 }
 
 
