@@ -23,30 +23,20 @@
 //   finish        slots' scratch word is reset, shard sizes are advanced.
 #include "des_internal.cuh"
 
-#ifndef PROBE_VOLATILE
-#define PROBE_VOLATILE 0
-#endif
-#define IB 1024  // threads (= occurrences) per block in every kernel of this file
+#define IB 1024  // occurrences per block (tile) in every per-occurrence kernel of this file
 
 // A probe may read a slot through L1 although other SMs claim slots meanwhile: a key never changes once
 // it is set, so a stale line can only show EMPTY where a key now is (the CAS that follows returns the
 // truth) or a too-large scratch word (the atomicMin that follows is then merely redundant).
+// (One 16-byte load; "volatile" keeps the compiler from reusing an earlier read of the same slot.)
 __device__ __forceinline__ Slot load_slot(const Slot* p) {
-#if PROBE_VOLATILE
-  unsigned long long a, b;
-  asm volatile("ld.volatile.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p));
-#else
   unsigned long long a, b;
   asm volatile("ld.global.ca.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p));
-#endif
   Slot s;
   s.key = a; s.row = (uint32_t)b; s.first_occ = (uint32_t)(b >> 32);
   return s;
 }
 
-#ifndef PROBE_VOLATILE
-#define PROBE_VOLATILE 0
-#endif
 // Occurrences per thread and resident blocks per SM: one probe chain per thread at full occupancy
 // measured fastest (more chains per thread cost registers, hence warps in flight; electing one lane
 // per distinct key of a warp costs more in match instructions than the cached slot loads it saves).
