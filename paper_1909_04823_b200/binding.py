@@ -197,6 +197,7 @@ class Table:
             raise RuntimeError("paper_1909_04823_b200 needs a CUDA device; there is no CPU path")
         self.L = load()
         self.S, self.F, self.k, self.H = num_shards, num_fields, emb_dim, hidden
+        self.partition, self.max_nnz, self.max_batch = partition, int(max_nnz), int(max_batch)
         self.stride = emb_dim + 4
         cfg = des_config_t()
         cfg.num_shards, cfg.num_fields, cfg.emb_dim, cfg.hidden = num_shards, num_fields, emb_dim, hidden
@@ -350,6 +351,29 @@ class Table:
         m = min(int(n.value), cap)
         return dict(n=int(n.value), keys=keys[:m], shards=shards[:m], rows=rows[:m], emb=emb[:m], lin=lin[:m],
                     acc_emb=ae[:m], acc_lin=al[:m])
+
+    def import_rows(self, keys: torch.Tensor, shards: torch.Tensor, emb=None, lin=None, acc_emb=None, acc_lin=None):
+        """Restores a dump made by `export` (of this or another table with the same S, partition, k):
+        inserts the keys — their rows get new numbers, a key's contents are what count — and writes
+        weights and state over the freshly initialised rows.  Plumbing over find_or_insert + write_rows:
+        one key per sample, in the bag of field 0 (HASH) or of the field that its shard owns (FIELD)."""
+        n, F = int(keys.numel()), self.F
+        chunk = max(1, min(self.max_batch, self.max_nnz))
+        base = torch.tensor(self.row_base()[:-1], dtype=torch.int64, device="cuda")
+        for lo in range(0, n, chunk):
+            hi = min(n, lo + chunk)
+            m = hi - lo
+            fb = shards[lo:hi].to(torch.int64) if self.partition == PART_FIELD else torch.zeros(m, dtype=torch.int64, device="cuda")
+            f = torch.arange(F, dtype=torch.int64, device="cuda")[None, :]
+            off = (torch.arange(m, dtype=torch.int64, device="cuda")[:, None] + (f > fb[:, None])).reshape(-1)
+            off = torch.cat([off, torch.tensor([m], dtype=torch.int64, device="cuda")]).to(torch.int32)
+            db = DeviceBatch(off, keys[lo:hi].contiguous(), None, m)
+            self.find_or_insert(db, True)
+            grow = (base[db.shards[:m].to(torch.int64)] + db.rows[:m].to(torch.int64)).to(torch.int32)
+            sl = slice(lo, hi)
+            pick = lambda a: None if a is None else a[sl].contiguous()
+            self.write_rows(grow, pick(emb), pick(lin), pick(acc_emb), pick(acc_lin))
+        torch.cuda.current_stream().synchronize()
 
     def read_rows(self, global_rows: torch.Tensor):
         n = int(global_rows.numel())
