@@ -247,3 +247,32 @@ def test_cfg5_multihot_million_occurrences():
     w = synth.config(5).scaled(batch=640, vocab=50000, prepopulate=50000, init_scale=0.05)
     assert synth.Stream(w).next_batch().nnz > (1 << 20)
     _run(w, 2, max_rows=120000, prepop=1)
+
+
+def test_forward_is_run_to_run_identical():
+    # the forward has no atomics on its fast path and a fixed order of additions: same bits every time,
+    # also across two tables built the same way
+    from paper_1909_04823_b200.binding import DeviceBatch, Table
+    w = synth.config(5).scaled(batch=256, vocab=50000, prepopulate=0, init_scale=0.05)
+    b = synth.Stream(w).next_batch()
+    B, F, k, S = b.batch, w.fields, w.emb_dim, w.shards
+    res = []
+    for rep in range(2):
+        t = Table.for_workload(w, max_rows=200000, max_nnz=b.nnz)
+        try:
+            db = DeviceBatch.from_synth(b)
+            t.find_or_insert(db, True)
+            for again in range(2):
+                part = torch.full((S, B, k + 4), float("nan"), device="cuda")
+                out = torch.full((B, k + 4), float("nan"), device="cuda")
+                pooled = torch.full((B, F * k), float("nan"), device="cuda")
+                t.forward_partials(w.ops, db, part, pooled, None, None)
+                t.aggregate(w.ops, db, part, pooled, None, None, out, pooled, None)
+                torch.cuda.synchronize()
+                res.append((part.clone(), out.clone(), pooled.clone()))
+            assert t.status() == 0
+        finally:
+            t.close()
+    for r in res[1:]:
+        for a, c in zip(r, res[0]):
+            assert torch.equal(a.view(torch.int32), c.view(torch.int32))
