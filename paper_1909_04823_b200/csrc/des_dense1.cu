@@ -169,7 +169,7 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
     const int FK = t->F * t->k;
     des_status_t e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
     if (e != DES_OK) return e;
-    const int rc = des_tc_gemm_fwd(B, t->H, FK, t->pooled_b, t->W1b, Z, Z, 0.f, t->gemm_ws, t->gemm_ws_bytes, st);
+    const int rc = des_tc_gemm_fwd(B, t->H, FK, 1, t->pooled_b, t->W1b, Z, Z, 0.f, t->gemm_ws, t->gemm_ws_bytes, st);
     if (rc == 0) { DES_LAUNCH_CHECK(t, "tc_gemm_fwd"); return DES_OK; }
     if (rc != 1) return DES_ERR_CUDA;
   }
@@ -195,15 +195,20 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
     des_status_t e = to_bf16(t, gZ, t->gZ_b, (size_t)B * t->H, st);
     if (e == DES_OK) e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
     if (e != DES_OK) return e;
-    const int rc1 = des_tc_gemm_dgrad(B, FK, t->H, t->gZ_b, t->W1b, gE ? gE : gE_work, gE_work, gE ? 1.f : 0.f,
+    const int rc1 = des_tc_gemm_dgrad(B, FK, t->H, 1, t->gZ_b, t->W1b, gE ? gE : gE_work, gE_work, gE ? 1.f : 0.f,
                                       t->gemm_ws, t->gemm_ws_bytes, st);
     if (rc1 == 0) {
       DES_LAUNCH_CHECK(t, "tc_gemm_dgrad");
-      const int rc2 = des_tc_gemm_wgrad(FK, t->H, B, t->pooled_b, t->gZ_b, t->gW1_part, t->gW1_part, 0.f, t->gemm_ws,
-                                        t->gemm_ws_bytes, st);
+      // The product has few output tiles (F*k x H) and a long contraction (the batch): cut the batch into L
+      // pieces so that every SM gets tiles (L partial products, added in piece order by w1_update_kernel).
+      const int tiles = ((FK + 127) / 128) * ((t->H + 127) / 128);
+      int L = 1;
+      while (L < t->gw1_splits && tiles * L < 2 * t->sm_count && B % (2 * L * 64) == 0) L *= 2;
+      const int rc2 = des_tc_gemm_wgrad(FK, t->H, B / L, L, t->pooled_b, t->gZ_b, t->gW1_part, t->gW1_part, 0.f,
+                                        t->gemm_ws, t->gemm_ws_bytes, st);
       if (rc2 != 0) return DES_ERR_CUDA;           // same alignment rules as the dgrad: cannot differ
       DES_LAUNCH_CHECK(t, "tc_gemm_wgrad");
-      w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, 1, (size_t)FK * t->H, t->W1, t->accW1, t->acc2W1,
+      w1_update_kernel<<<t->sm_count * 2, 256, 0, st>>>(t->gW1_part, L, (size_t)FK * t->H, t->W1, t->accW1, t->acc2W1,
                                                         t->W1b, des_opt_params(t), t->meta);
       DES_LAUNCH_CHECK(t, "w1_update_kernel");
       return DES_OK;

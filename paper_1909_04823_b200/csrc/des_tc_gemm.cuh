@@ -4,8 +4,11 @@
 // ships with the Python environment; nothing of it is copied here).  One
 // translation unit per operand layout, each exporting one plain function:
 //
-//   rc = f(M, N, K, A, B, C, D, beta, workspace, workspace_bytes, stream)
-//        D[M][N] (fp32, row-major) = A * B + beta * C
+//   rc = f(M, N, K, L, A, B, C, D, beta, workspace, workspace_bytes, stream)
+//        D[l][M][N] (fp32, row-major) = A_l * B_l + beta * C[l]   for l < L,
+//        where the K extent of A and B is cut into L consecutive pieces of K each (a batched
+//        GEMM over packed operands: with L > 1 this is a split-K product whose L partial
+//        results the caller adds up; L = 1 is the plain product)
 //   rc: 0 ok; 1 shape / alignment not supported by the TMA path (caller falls
 //       back to the CUDA-core kernel); 2 workspace too small; 3, 4 CUTLASS error.
 #pragma once
@@ -52,14 +55,14 @@
     using StrideB = Gemm::GemmKernel::StrideB;                                                                        \
     using StrideC = Gemm::GemmKernel::StrideC;                                                                        \
     using StrideD = Gemm::GemmKernel::StrideD;                                                                        \
-    static int run(int M, int N, int K, const void* A, const void* B, const float* C, float* D, float beta,           \
+    static int run(int M, int N, int K, int L, const void* A, const void* B, const float* C, float* D, float beta,    \
                    void* workspace, size_t ws_bytes, cudaStream_t stream) {                                           \
-      StrideA sa = cutlass::make_cute_packed_stride(StrideA{}, cute::make_shape(M, K, 1));                            \
-      StrideB sb = cutlass::make_cute_packed_stride(StrideB{}, cute::make_shape(N, K, 1));                            \
-      StrideC sc = cutlass::make_cute_packed_stride(StrideC{}, cute::make_shape(M, N, 1));                            \
-      StrideD sd = cutlass::make_cute_packed_stride(StrideD{}, cute::make_shape(M, N, 1));                            \
+      StrideA sa = cutlass::make_cute_packed_stride(StrideA{}, cute::make_shape(M, K, L));                            \
+      StrideB sb = cutlass::make_cute_packed_stride(StrideB{}, cute::make_shape(N, K, L));                            \
+      StrideC sc = cutlass::make_cute_packed_stride(StrideC{}, cute::make_shape(M, N, L));                            \
+      StrideD sd = cutlass::make_cute_packed_stride(StrideD{}, cute::make_shape(M, N, L));                            \
       Gemm::Arguments args{cutlass::gemm::GemmUniversalMode::kGemm,                                                   \
-                           {M, N, K, 1},                                                                              \
+                           {M, N, K, L},                                                                              \
                            {(const ElementA*)A, sa, (const ElementB*)B, sb},                                          \
                            {{1.0f, beta}, C, sc, D, sd}};                                                             \
       Gemm gemm;                                                                                                      \
@@ -70,18 +73,19 @@
       return 0;                                                                                                       \
     }                                                                                                                 \
   };
-#define DES_TC_GEMM_BODY(NAME) return NAME::run(M, N, K, A, B, C, D, beta, ws, ws_bytes, stream);
+#define DES_TC_GEMM_BODY(NAME) return NAME::run(M, N, K, L, A, B, C, D, beta, ws, ws_bytes, stream);
 #else
 #define DES_DEFINE_TC_GEMM(NAME, LayoutA, LayoutB)
 #define DES_TC_GEMM_BODY(NAME) return 1;   /* built without the CUTLASS headers: CUDA-core fallback only */
 #endif
 
 // Z = V W: A = pooled bf16 [B][F*k] (K contiguous), B = W1 bf16 [F*k][H] (N contiguous)
-int des_tc_gemm_fwd(int M, int N, int K, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
+int des_tc_gemm_fwd(int M, int N, int K, int L, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
                     size_t ws_bytes, cudaStream_t stream);
 // gE = gZ W1^T: A = gZ bf16 [B][H] (K contiguous), B = W1 bf16 [F*k][H] read as (N = F*k, K = H), K contiguous
-int des_tc_gemm_dgrad(int M, int N, int K, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
+int des_tc_gemm_dgrad(int M, int N, int K, int L, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
                       size_t ws_bytes, cudaStream_t stream);
-// gW1 = V^T gZ: A = pooled bf16 [B][F*k] read as (M = F*k, K = B), M contiguous; B = gZ bf16 [B][H] (N contiguous)
-int des_tc_gemm_wgrad(int M, int N, int K, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
+// gW1 = V^T gZ: A = pooled bf16 [B][F*k] read as (M = F*k, K = B), M contiguous; B = gZ bf16 [B][H] (N contiguous);
+// L > 1 cuts the batch into L pieces (K = B / L samples each) whose partial products the caller adds
+int des_tc_gemm_wgrad(int M, int N, int K, int L, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
                       size_t ws_bytes, cudaStream_t stream);

@@ -1,7 +1,7 @@
 // tcgen05 GEMM, operand layout "wgrad" (see des_tc_gemm.cuh).
 #include "des_tc_gemm.cuh"
 DES_DEFINE_TC_GEMM(TcGemm_wgrad, cutlass::layout::ColumnMajor, cutlass::layout::RowMajor)
-int des_tc_gemm_wgrad(int M, int N, int K, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
+int des_tc_gemm_wgrad(int M, int N, int K, int L, const void* A, const void* B, const float* C, float* D, float beta, void* ws,
                    size_t ws_bytes, cudaStream_t stream) {
   DES_TC_GEMM_BODY(TcGemm_wgrad)
 }
