@@ -473,6 +473,10 @@ def main():
                         "share": top["share"]}
             break
     step_bytes = sum((kernel_bytes(kk["kernel"], stats) or 0) * kk["launches"] for kk in kernels) / args.steps
+    row_b = 4 * k + 16
+    extra = max(0, batches[0].nnz - U)                   # occurrences beyond the first of their key
+    occ_bytes = step_bytes + extra * ((row_b if (w.ops & (OP_LR | OP_FM)) else 0)
+                                      + (4 * k if (w.ops & (OP_POOL | OP_DENSE1)) else 0) + row_b)
 
     # ---- end to end from pinned host buffers
     e2e = None
@@ -545,7 +549,11 @@ def main():
                 "roofline": roofline,
                 "hbm": {"alg_bytes_per_step": int(step_bytes), "alg_gbs": round(step_bytes / ms_step / 1e6, 1),
                         "frac_of_measured_copy": round(step_bytes / ms_step / 1e6 / hbm_peak, 4),
-                        "frac_of_nominal_8000": round(step_bytes / ms_step / 1e6 / 8000.0, 4)},
+                        "frac_of_nominal_8000": round(step_bytes / ms_step / 1e6 / 8000.0, 4),
+                        # occurrence-level accounting: what the load / store units move when every occurrence
+                        # gathers (twice: per-shard partials and pooling) and scatters its own row; these are
+                        # mostly L1 / L2 hits in a skewed batch, so this is not an HBM figure
+                        "occ_bytes_per_step": int(occ_bytes), "occ_gbs": round(occ_bytes / ms_step / 1e6, 1)},
                 "kernels": kernels, "cpu_baseline": cpu}
         print(json.dumps(line), flush=True)
     if world > 1:
