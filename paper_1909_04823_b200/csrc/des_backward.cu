@@ -597,7 +597,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   }
   {
     // long bags: a whole warp per bag (its sub-groups take alternate occurrences); short bags: G lanes per bag
-    const bool wide = (long long)nnz >= 4 * nbags;
+    const bool wide = (long long)nnz >= 8 * nbags;   // (at 4 ids per bag the narrow form measured faster)
     const long long threads = nbags * (wide ? 32 : G);
     long long blocks = (threads + 255) / 256;
     if (blocks > (long long)t->sm_count * SC_BLOCKS_PER_SM) blocks = (long long)t->sm_count * SC_BLOCKS_PER_SM;

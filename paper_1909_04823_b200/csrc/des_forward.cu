@@ -348,7 +348,7 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   if (pl) {
     const long long nbags = (long long)B * t->F;
     // long bags: a whole warp per bag (its halves take alternate occurrences); short bags: G lanes per bag
-    const bool wide = b->nnz >= 4 * nbags;
+    const bool wide = b->nnz >= 8 * nbags;            // (at 4 ids per bag the narrow form measured faster)
     const long long threads = nbags * (wide ? 32 : G);
     long long blocks = (threads + 255) / 256;
     if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;

@@ -2,7 +2,7 @@
 // including shard routing (Section 5, "Large-scale Sparse Features": weights of
 // field f live on node f mod N; Section 4.2: any balanced partition).
 //
-// One call = eight short kernels, none of which waits on another thread:
+// One call = nine short kernels, none of which waits on another thread:
 //   probe_claim   every occurrence finds its key's slot in the owning shard's
 //                 region (linear probing) or claims an empty one with a 64-bit
 //                 CAS; the slot remembers the smallest occurrence index.
@@ -17,8 +17,8 @@
 //                 among firsts always, the new-key numbering only when the
 //                 batch has a new key at all.
 //   apply_first   one thread per unique key writes these numbers into the
-//                 key's slot and initialises new rows from the counter-based
-//                 generator.
+//                 key's slot; init_new_rows then fills the new keys' rows from
+//                 the counter-based generator (a lane group per row).
 //   resolve       every occurrence reads row and unique index from its slot.
 //   finish        slots' scratch word is reset, shard sizes are advanced.
 #include "des_internal.cuh"
@@ -295,10 +295,9 @@ __global__ void __launch_bounds__(IB) assign_kernel(
 // their rows, publish the key's batch-unique index in its slot (read back by
 // every occurrence in resolve_kernel), record slot and table-global row.
 __global__ void __launch_bounds__(256) apply_first_kernel(
-    const unsigned long long* __restrict__ ids, int k, int stride, Slot* slots, const DevMeta* __restrict__ meta,
+    Slot* slots, const DevMeta* __restrict__ meta,
     const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint32_t* __restrict__ first_j,
-    uint32_t* __restrict__ uslot, uint32_t* __restrict__ uniq_rows, float* __restrict__ W, float* __restrict__ A,
-    float* __restrict__ A2, unsigned long long seed, float init_scale, float state_init, float lin_state_init) {
+    uint32_t* __restrict__ uslot, uint32_t* __restrict__ uniq_rows) {
   const uint32_t U = meta->n_uniq;
   for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
     const uint32_t fj = first_j[u];
@@ -317,27 +316,47 @@ __global__ void __launch_bounds__(256) apply_first_kernel(
     uslot[u] = so;
     const unsigned long long g = meta->row_base[s] + local;
     uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
-    if (is_new && local != DES_ROW_NONE) {
-      const unsigned long long id = ids[j];
-      float4* w = reinterpret_cast<float4*>(W + g * stride);
-      const int q4 = k >> 2;
-      float n2 = 0.f;
-      for (int q = 0; q < q4; ++q) {
-        const float4 v = des_init4(seed, id, q, init_scale);
-        n2 += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        w[q] = v;
-      }
-      w[q4] = make_float4(0.f, n2, 0.f, 0.f);   // linear weight, squared norm of the latent vector
-      if (A) {
-        float4* a = reinterpret_cast<float4*>(A + g * stride);
-        const float4 ia = make_float4(state_init, state_init, state_init, state_init);
-        for (int q = 0; q < q4; ++q) a[q] = ia;
-        a[q4] = make_float4(lin_state_init, 0.f, 0.f, 0.f);
-      }
-      if (A2) {
-        float4* a2 = reinterpret_cast<float4*>(A2 + g * stride);
-        for (int q = 0; q <= q4; ++q) a2[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
+  }
+}
+
+// Rows of the batch's new keys: weights from the counter-based generator keyed on the id, optimizer state
+// at its start value.  G lanes per unique key (one 16-byte column each); keys that are not new cost one
+// load.  uniq_rows[u] already holds the table-global row (apply_first_kernel).
+template <int G>
+__global__ void __launch_bounds__(256) init_new_rows_kernel(
+    const unsigned long long* __restrict__ ids, int k, int stride, const DevMeta* __restrict__ meta,
+    const uint32_t* __restrict__ first_j, const uint32_t* __restrict__ uniq_rows, float* __restrict__ W,
+    float* __restrict__ A, float* __restrict__ A2, unsigned long long seed, float init_scale, float state_init,
+    float lin_state_init) {
+  if (meta->any_new == 0u) return;                     // steady state of a populated table: nothing to initialise
+  const uint32_t U = meta->n_uniq;
+  const int K4 = k >> 2, c4 = threadIdx.x % G;
+  const long long gstep = (long long)gridDim.x * (256 / G);
+  // every lane of a warp runs the same number of rounds (the squared norm is a warp-level sum)
+  const long long rounds = ((long long)U + gstep - 1) / gstep;
+  long long u = (long long)blockIdx.x * (256 / G) + threadIdx.x / G;
+  for (long long r = 0; r < rounds; ++r, u += gstep) {
+    uint32_t fj = 0, grow = DES_ROW_NONE;
+    if (u < U) { fj = first_j[u]; if (fj >> 31) grow = uniq_rows[u]; }
+    const bool init = grow != DES_ROW_NONE;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (init && c4 < K4) v = des_init4(seed, ids[fj & 0x7FFFFFFFu], (uint32_t)c4, init_scale);
+    float n2 = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+    for (int d = 1; d < G; d <<= 1) n2 += __shfl_xor_sync(0xFFFFFFFFu, n2, d);
+    if (!init) continue;
+    float4* w = reinterpret_cast<float4*>(W + (size_t)grow * stride);
+    if (c4 < K4) w[c4] = v;
+    if (c4 == 0) w[K4] = make_float4(0.f, n2, 0.f, 0.f);      // linear weight, squared norm of the latent vector
+    if (A) {
+      float4* a = reinterpret_cast<float4*>(A + (size_t)grow * stride);
+      if (c4 < K4) a[c4] = make_float4(state_init, state_init, state_init, state_init);
+      if (c4 == 0) a[K4] = make_float4(lin_state_init, 0.f, 0.f, 0.f);
+    }
+    if (A2) {
+      float4* a2 = reinterpret_cast<float4*>(A2 + (size_t)grow * stride);
+      if (c4 < K4) a2[c4] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c4 == 0) a2[K4] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
 }
@@ -410,13 +429,22 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   assign_kernel<<<nblk < t->sm_count * 2 ? nblk : t->sm_count * 2, IB, 0, cs>>>(nnz, nblk, t->S, t->meta, b->shards, t->flags,
                                                                                 t->blk_cnt, t->nblk_max, t->dest, b->uniq_rows);
   DES_LAUNCH_CHECK(t, "assign_kernel");
-  apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>((const unsigned long long*)b->ids, t->k, t->stride, t->slots,
-                                                      t->meta, t->slot_of, b->shards, t->dest, t->uslot, b->uniq_rows,
-                                                      t->W, t->A, t->A2, t->cfg.seed, t->cfg.init_scale,
-                                                      t->cfg.optimizer == DES_OPT_ADAGRAD ? t->cfg.init_acc : 0.f,
-                                                      (t->cfg.lin_optimizer == DES_LIN_FTRL ||
-                                                       t->cfg.optimizer != DES_OPT_ADAGRAD) ? 0.f : t->cfg.init_acc);
+  apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->meta, t->slot_of, b->shards, t->dest, t->uslot,
+                                                      b->uniq_rows);
   DES_LAUNCH_CHECK(t, "apply_first_kernel");
+  {
+    const float state_init = t->cfg.optimizer == DES_OPT_ADAGRAD ? t->cfg.init_acc : 0.f;
+    const float lin_state_init =
+        (t->cfg.lin_optimizer == DES_LIN_FTRL || t->cfg.optimizer != DES_OPT_ADAGRAD) ? 0.f : t->cfg.init_acc;
+    int G = 1;
+    while (G < (int)t->k / 4) G <<= 1;
+#define INIT(GG) init_new_rows_kernel<GG><<<t->sm_count * 8, 256, 0, cs>>>(                                            \
+        (const unsigned long long*)b->ids, t->k, t->stride, t->meta, t->dest, b->uniq_rows, t->W, t->A, t->A2,         \
+        t->cfg.seed, t->cfg.init_scale, state_init, lin_state_init)
+    switch (G) { case 1: INIT(1); break; case 2: INIT(2); break; case 4: INIT(4); break; case 8: INIT(8); break; default: INIT(16); }
+#undef INIT
+    DES_LAUNCH_CHECK(t, "init_new_rows_kernel");
+  }
   resolve_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
   DES_LAUNCH_CHECK(t, "resolve_kernel");
   finish_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->S, t->slots, t->uslot, t->meta, b->n_uniq);
