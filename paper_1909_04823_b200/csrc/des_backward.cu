@@ -659,7 +659,8 @@ static void* st_alloc(des_table* t, size_t bytes) {
 // kernels of the step before; everything the kernels produce is single (kernels of consecutive steps run
 // in order on the caller's stream).
 static des_status_t st_prepare(des_table* t) {
-  if (t->st_ids[0]) return DES_OK;
+  if (t->st_ready) return DES_OK;
+  if (t->st_ids[0]) return DES_ERR_CUDA;               // an earlier attempt ran out of memory half-way
   const size_t nb = (size_t)t->max_batch * t->F + 1;
   for (int s = 0; s < 2; ++s) {
     t->st_offsets[s] = (int32_t*)st_alloc(t, nb * 4);
@@ -683,6 +684,7 @@ static des_status_t st_prepare(des_table* t) {
     if (cudaEventCreateWithFlags(&t->st_done[s], cudaEventDisableTiming) != cudaSuccess) return DES_ERR_CUDA;
     t->st_busy[s] = 0;
   }
+  t->st_ready = 1;
   return DES_OK;
 }
 
@@ -764,7 +766,7 @@ extern "C" des_status_t des_step_host_submit(des_table_t* t, uint32_t ops, int32
 
 extern "C" des_status_t des_step_host_wait(des_table_t* t, int32_t ticket) {
   if (!t || ticket < 0 || ticket > 1) return DES_ERR_INVALID_ARG;
-  if (!t->st_ids[0] || !t->st_busy[ticket]) return DES_OK;
+  if (!t->st_ready || !t->st_busy[ticket]) return DES_OK;
   DES_CUDA(cudaEventSynchronize(t->st_done[ticket]));
   t->st_busy[ticket] = 0;
   return DES_OK;

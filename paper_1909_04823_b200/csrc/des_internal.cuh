@@ -80,6 +80,7 @@ struct des_table {
   // host-step staging
   int32_t* st_offsets[2]; unsigned long long* st_ids[2]; float* st_vals[2];   // two input slots (pipelined submit)
   cudaStream_t st_copy_stream; cudaEvent_t st_copied[2], st_done[2]; int st_busy[2]; uint64_t st_next;
+  int st_ready;                      // staging, copy stream and events all exist
   uint32_t* st_rows; uint8_t* st_shards; uint32_t* st_uidx; uint32_t* st_uniq_rows; uint32_t* st_n_uniq;
   float* st_part_small; float* st_out_small;
   uint64_t launches;
