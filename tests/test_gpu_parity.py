@@ -276,3 +276,17 @@ def test_forward_is_run_to_run_identical():
     for r in res[1:]:
         for a, c in zip(r, res[0]):
             assert torch.equal(a.view(torch.int32), c.view(torch.int32))
+
+
+@pytest.mark.parametrize("k", [8, 32, 64])
+def test_long_bags_with_feature_values(k):
+    # bags of about 20 ids (a whole warp per bag in pooling and scatter, 32 / (k/4) sub-groups taking alternate
+    # occurrences) together with real feature values and materialised per-shard partials
+    w = synth.config(5).scaled(batch=48, vocab=20000, prepopulate=0, emb_dim=k, shards=7, init_scale=0.05)
+    _run(w, 2, max_rows=120000, materialise=True, with_vals=True)
+
+
+def test_long_bags_field_partition():
+    w = synth.config(5).scaled(batch=48, vocab=3000, prepopulate=0, emb_dim=16, shards=6, fields=40, partition=PART_FIELD,
+                               shared_vocab=False, init_scale=0.05)
+    _run(w, 2, max_rows=150000, materialise=False)
