@@ -290,3 +290,11 @@ def test_long_bags_field_partition():
     w = synth.config(5).scaled(batch=48, vocab=3000, prepopulate=0, emb_dim=16, shards=6, fields=40, partition=PART_FIELD,
                                shared_vocab=False, init_scale=0.05)
     _run(w, 2, max_rows=150000, materialise=False)
+
+
+@pytest.mark.parametrize("partition", [PART_HASH, PART_FIELD])
+def test_maximum_fields_and_shards(partition):
+    # the largest field count and shard count the library accepts (1024 fields, 64 shards)
+    w = synth.Workload("max_fields", 6, 1024, 4, 64, partition, OPT_ADAGRAD, OP_LR | OP_FM | OP_POOL, zipf_s=1.1, vocab=500,
+                       shared_vocab=(partition == PART_HASH), len_law="uniform", len_a=0, len_b=2, seed=31, init_scale=0.05)
+    _run(w, 2, max_rows=80000, materialise=True)
