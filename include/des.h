@@ -71,14 +71,15 @@ typedef enum {
 
 /* operator kind bitmask */
 enum { DES_OP_LR = 1, DES_OP_FM = 2, DES_OP_POOL = 4, DES_OP_DENSE1 = 8 };
-/* weight placement: HASH = mix64(id) mod S ("any partition policy that
- * balances", Section 4.2); FIELD = field mod S (Section 5, "Large-scale
- * Sparse Features"; required for a weight-disjoint row split, Section 4.3). */
+/* weight placement: HASH = mix64(id) mod S (Section 4.2 allows any partition
+ * that keeps the shards balanced); FIELD = field mod S (the rule of Section 5,
+ * paragraph on large-scale sparse features; required for a weight-disjoint row
+ * split, Section 4.3). */
 enum { DES_PART_HASH = 0, DES_PART_FIELD = 1 };
 /* optimizer of the latent vectors and of the first dense layer; the order-1
  * (linear) weights follow it unless lin_optimizer says FTRL (Section 6,
- * "Parameter Settings": FTRL for order-1 components, AdaGrad or Adam for the
- * embedding and DNN components). */
+ * parameter settings: the paper trains the order-1 parts with FTRL and the
+ * embeddings and dense layers with Adagrad or Adam). */
 enum { DES_OPT_SGD = 0, DES_OPT_ADAGRAD = 1, DES_OPT_ADAM = 2 };
 enum { DES_LIN_SAME = 0, DES_LIN_FTRL = 1 };
 

@@ -8,7 +8,7 @@
 // substitution operator F = 1/2 <(+)M_1,(+)M_1> - 1/2 (+)M_2 (Eq. 8).
 //
 // Kernels.
-//  route_kernel   "each shard looks up its own ids": one warp per sample buckets
+//  route_kernel   every shard gets the ids it owns: one warp per sample buckets
 //                 the sample's occurrences by owning shard with a stable counting
 //                 sort (warp match + running cursors), writing the table-global
 //                 row of every occurrence in shard-major order, the segment
