@@ -170,19 +170,20 @@ __global__ void __launch_bounds__(IB / 4) flag_count_kernel(
 // One block per sequence (sequence 0 = firsts, 1 + s = new keys of shard s):
 // in-place exclusive scan over the blocks of the batch, total to meta.
 __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, int nblk, int nblk_max, DevMeta* meta) {
+  // Warp w owns the contiguous chunk [w * per, (w + 1) * per) of the sequence and walks it 32 entries at a
+  // time (coalesced loads and stores, a warp scan per row, a running carry); the 32 warp totals are scanned
+  // in between, and sequences that are all zero (new keys of a shard in a populated table) are not rewritten.
   __shared__ uint32_t wsum[32];
+  __shared__ uint32_t s_total;
   uint32_t* seq = blk_cnt + (size_t)blockIdx.x * nblk_max;
-  const int per = (nblk + 1023) / 1024;
-  const int lo = threadIdx.x * per, hi = min(nblk, lo + per);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int per = ((nblk + 31) / 32 + 31) / 32 * 32;          // entries per warp, a multiple of 32
+  const int lo = warp * per, hi = min(nblk, lo + per);
   uint32_t sum = 0;
-  for (int i = lo; i < hi; ++i) sum += seq[i];
-  uint32_t incl = sum;
+  for (int i = lo + lane; i < hi; i += 32) sum += seq[i];
 #pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-    if ((threadIdx.x & 31) >= d) incl += v;
-  }
-  if ((threadIdx.x & 31) == 31) wsum[threadIdx.x >> 5] = incl;
+  for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+  if (lane == 0) wsum[warp] = sum;
   __syncthreads();
   if (threadIdx.x < 32) {
     uint32_t w = wsum[threadIdx.x], wi = w;
@@ -193,13 +194,26 @@ __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint32_t* blk_cnt, in
     }
     wsum[threadIdx.x] = wi - w;
     if (threadIdx.x == 31) {
+      s_total = wi;
       if (blockIdx.x == 0) meta->n_uniq = wi;
       else { meta->new_total[blockIdx.x - 1] = wi; if (wi) atomicOr(&meta->any_new, 1u); }
     }
   }
   __syncthreads();
-  uint32_t run = wsum[threadIdx.x >> 5] + incl - sum;
-  for (int i = lo; i < hi; ++i) { uint32_t v = seq[i]; seq[i] = run; run += v; }
+  if (s_total == 0u) return;                                  // an all-zero sequence is its own exclusive scan
+  uint32_t carry = wsum[warp];
+  for (int base = lo; base < hi; base += 32) {
+    const int i = base + lane;
+    const uint32_t v = (i < hi) ? seq[i] : 0u;
+    uint32_t incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+      if (lane >= d) incl += o;
+    }
+    if (i < hi) seq[i] = carry + incl - v;
+    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+  }
 }
 
 // The common case of assign_kernel below — a batch without a single new key — needs the rank among the
