@@ -298,3 +298,9 @@ def test_maximum_fields_and_shards(partition):
     w = synth.Workload("max_fields", 6, 1024, 4, 64, partition, OPT_ADAGRAD, OP_LR | OP_FM | OP_POOL, zipf_s=1.1, vocab=500,
                        shared_vocab=(partition == PART_HASH), len_law="uniform", len_a=0, len_b=2, seed=31, init_scale=0.05)
     _run(w, 2, max_rows=80000, materialise=True)
+
+
+@pytest.mark.parametrize("ops", [OP_LR, OP_FM, OP_POOL, OP_LR | OP_POOL, OP_FM | OP_POOL])
+def test_long_bags_operator_subsets(ops):
+    w = synth.config(5).scaled(batch=40, vocab=20000, prepopulate=0, shards=9, init_scale=0.05, ops=ops)
+    _run(w, 2, max_rows=120000, ops=ops)
