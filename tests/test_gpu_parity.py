@@ -249,6 +249,15 @@ def test_cfg5_multihot_million_occurrences():
     _run(w, 2, max_rows=120000, prepop=1)
 
 
+@pytest.mark.parametrize("ops", [OP_LR | OP_FM, OP_POOL])
+def test_million_occurrences_operator_subsets(ops):
+    # the counted-and-multiplied path of the keys that own the batch, without the pooling gradient (LR + FM
+    # only) and without the per-sample gradients (pooling only)
+    w = synth.config(5).scaled(batch=640, vocab=50000, prepopulate=0, init_scale=0.05, ops=ops)
+    assert synth.Stream(w).next_batch().nnz > (1 << 20)
+    _run(w, 1, max_rows=120000, ops=ops)
+
+
 def test_forward_is_run_to_run_identical():
     # the forward has no atomics on its fast path and a fixed order of additions: same bits every time,
     # also across two tables built the same way
