@@ -186,8 +186,8 @@ class ClockSampler:
 # 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
-    ("cfg5", "grad_scatter_kernel"): 1732e6,
-    ("cfg5", "super_dense_kernel"): 481e6,
+    ("cfg5", "grad_scatter_kernel"): 1801e6,
+    ("cfg5", "super_dense_kernel"): 533e6,
     ("cfg5", "shard_partials_kernel"): 939e6,
     ("cfg5", "pool_kernel"): 1211e6,
     ("cfg5", "update_rows_kernel"): 1937e6,
@@ -224,9 +224,9 @@ def kernel_bytes(name, st):
         return 8 * nnz + 4 * U
     if name == "grad_scatter_kernel":   # + the per-bag counts of the register-summed keys on skewed batches
         return (4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + 2 * row * (U + R)
-                + (32 * B * F if st["super"] else 0))
+                + (64 * B * F if st["super"] else 0))
     if name == "super_dense_kernel":
-        return 32 * B * F + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B
+        return 64 * B * F + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B
     if name == "sample_count_kernel":
         return 4 * (nnz >> st["shift"]) + 4 * U
     if name == "hot_reduce_kernel":

@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ dest,
     long long nbags, int F, int k, uint32_t ops, const float* __restrict__ out_small,
     const float* __restrict__ gL, const float* __restrict__ gF, const float* __restrict__ gE, float* Gbuf,
-    uint16_t* __restrict__ super_cnt) {
+    float* __restrict__ super_cnt) {
   constexpr int LB = G * P;
   const int K4 = k >> 2, stride = k + 4;
   const int sub = threadIdx.x % LB, c4 = sub % G, p = sub / G;
@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
     if (SUPER) {
 #pragma unroll
       for (int d = G; d < LB; d <<= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
-      if (live && p == 0) super_cnt[bag * 16 + c4] = (uint16_t)min(cnt, 65535u);
+      if (live && p == 0) super_cnt[bag * 16 + c4] = (float)cnt;
     }
   }
 }
@@ -318,100 +318,117 @@ __global__ void __launch_bounds__(256) grad_scatter_kernel(
 // accumulator of key t, 16-byte column c4.  Each CTA adds its sums to one replica row per key
 // (summed in double by hot_reduce).  All feature values are 1 on this path.
 #define SD_TILE 32
+#define SD_STAGES 4
 #define SD_THREADS 288   // 256 column threads + one warp for the linear-weight tails
+
+__device__ __forceinline__ void sd_cp_async16(void* smem, const void* gmem) {
+  const unsigned sa = (unsigned)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gmem));
+}
+__device__ __forceinline__ void sd_cp_async4(void* smem, const void* gmem) {
+  const unsigned sa = (unsigned)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sa), "l"(gmem));
+}
+__device__ __forceinline__ void sd_cp_commit() { asm volatile("cp.async.commit_group;"); }
+template <int N>
+__device__ __forceinline__ void sd_cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N)); }
+
+// The kernel is one stream over gE.  Per tile of SD_TILE bags a ring of SD_STAGES shared-memory stages takes,
+// by asynchronous copies, the bags' rows of gE, their samples' rows of A and (gL, gF), and the counts; thread
+// (c4, kg, sub) multiplies column c4 of c_bag = gE row + gF A by the counts of keys 8 kg .. 8 kg + 7 for
+// bags sub, sub + 8, ... of the tile; the extra warp sums the linear-weight tails.  One barrier per tile:
+// behind it every thread has finished the previous tile, whose stage the next copies overwrite.
 __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
-    const uint16_t* __restrict__ super_cnt, int nbags, int F, int k, uint32_t ops,
+    const float* __restrict__ super_cnt, int nbags, int F, int k, uint32_t ops,
     const float* __restrict__ out_small, const float* __restrict__ gL, const float* __restrict__ gF,
     const float* __restrict__ gE, float* Gbuf, const uint32_t* __restrict__ ctr,
     const uint32_t* __restrict__ hot_base, const uint32_t* __restrict__ hot_R, long long max_uniq) {
   uint32_t ns = __ldg(ctr + 3);
   if (ns == 0) return;
   if (ns > SUPER_T) ns = SUPER_T;
-  __shared__ float4 s_c[SD_TILE][16];
-  __shared__ __align__(16) float s_n[SD_TILE][16];
-  __shared__ float2 s_g[SD_TILE];
+  extern __shared__ __align__(16) unsigned char sd_smem[];
+  typedef float4 (*tile_t)[SD_TILE][16];
+  tile_t s_c = reinterpret_cast<tile_t>(sd_smem);                                      // gE rows
+  tile_t s_a = s_c + SD_STAGES;                                                        // A rows
+  float (*s_n)[SD_TILE][16] = reinterpret_cast<float (*)[SD_TILE][16]>(s_a + SD_STAGES);   // counts
+  float2 (*s_g)[SD_TILE] = reinterpret_cast<float2 (*)[SD_TILE]>(s_n + SD_STAGES);     // (gL, gF) per bag
   const int K4 = k >> 2, stride = k + 4;
   const int tid = threadIdx.x;
   const bool tailw = tid >= 256;                       // the extra warp
-  // staging role (threads < 256): thread (tk, c4) fetches column c4 of bags tk and tk + 16 of a tile
-  const int c4 = tid & 15, tk = (tid >> 4) & 15;
-  // multiply role (threads < 256): column c4, keys 4 kg .. 4 kg + 3, bags sub, sub + 4, ...
-  const int kg = (tid >> 4) & 3, sub = (tid >> 6) & 3;
-  // tail role (extra warp): key tt, bags th, th + 2, ...
-  const int tt = tid & 15, th = (tid >> 4) & 1;
+  const int c4 = tid & 15, tk = (tid >> 4) & 15;       // copy role: column c4 of bags tk and tk + 16 of a tile
+  const int kg = (tid >> 4) & 1, sub = (tid >> 5) & 7; // multiply role
+  const int tt = tid & 15, th = (tid >> 4) & 1;        // tail role: key tt, bags th, th + 2, ...
   const bool col = c4 < K4, fm = ops & DES_OP_FM, lr = ops & DES_OP_LR;
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-  float4 acc[4] = {zero, zero, zero, zero};
+  float4 acc[8] = {zero, zero, zero, zero, zero, zero, zero, zero};
   float tw = 0.f, tq = 0.f;
-  float4 e[2], a[2];
-  float gfv[2], nv[2];
-  float2 g2;
-  auto fetch = [&](int base) {
-    if (tailw) {
-      g2 = make_float2(0.f, 0.f);
-      const int i = tid - 256;
-      if (base + i < nbags) {
-        const int b = (base + i) / F;
-        g2.x = lr ? __ldg(gL + b) : 0.f;
-        g2.y = fm ? __ldg(gF + b) : 0.f;
-      }
-      return;
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      const int bag = base + r * 16 + tk;
-      e[r] = zero; a[r] = zero; gfv[r] = 0.f; nv[r] = 0.f;
-      if (bag < nbags) {
-        const int b = bag / F;
-        nv[r] = (float)__ldg(super_cnt + (size_t)bag * 16 + c4);
-        if (col && gE) e[r] = __ldg(reinterpret_cast<const float4*>(gE + (size_t)bag * k) + c4);
-        if (col && fm) { a[r] = __ldg(reinterpret_cast<const float4*>(out_small + (size_t)b * stride) + c4); gfv[r] = __ldg(gF + b); }
-      }
-    }
-  };
   const int tstep = gridDim.x * SD_TILE;
-  int base = blockIdx.x * SD_TILE;
-  if (base < nbags) fetch(base);
-  for (; base < nbags; base += tstep) {
-    __syncthreads();                                   // previous tile fully consumed
-    if (tailw) {
-      s_g[tid - 256] = g2;
-    } else {
+  const int base0 = blockIdx.x * SD_TILE;
+  // one group of asynchronous copies per tile and thread (an empty one past the end)
+  auto issue = [&](int base, int stage) {
+    if (base < nbags) {
+      if (!tailw) {
 #pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int i = r * 16 + tk;
-        s_c[i][c4] = make_float4(fmaf(gfv[r], a[r].x, e[r].x), fmaf(gfv[r], a[r].y, e[r].y),
-                                 fmaf(gfv[r], a[r].z, e[r].z), fmaf(gfv[r], a[r].w, e[r].w));
-        s_n[i][c4] = nv[r];
+        for (int r = 0; r < 2; ++r) {
+          const int i = r * 16 + tk, bag = base + i;
+          const bool in = bag < nbags && col;
+          if (in && gE) sd_cp_async16(&s_c[stage][i][c4], gE + (size_t)bag * k + c4 * 4);
+          else s_c[stage][i][c4] = zero;
+          if (in && fm) sd_cp_async16(&s_a[stage][i][c4], out_small + (size_t)(bag / F) * stride + c4 * 4);
+          else s_a[stage][i][c4] = zero;
+        }
+        if (tid < 128) {                               // 32 bags x 16 counts: 128 copies of 16 bytes
+          const int i = tid >> 2, q = tid & 3, bag = base + i;
+          if (bag < nbags) sd_cp_async16(&s_n[stage][i][q * 4], super_cnt + (size_t)bag * 16 + q * 4);
+          else *reinterpret_cast<float4*>(&s_n[stage][i][q * 4]) = zero;
+        }
+      } else {
+        const int i = tid - 256, bag = base + i;
+        const int b = bag / F;                         // (a plain store and a copy never target the same word)
+        if (bag < nbags && lr) sd_cp_async4(&s_g[stage][i].x, gL + b); else s_g[stage][i].x = 0.f;
+        if (bag < nbags && fm) sd_cp_async4(&s_g[stage][i].y, gF + b); else s_g[stage][i].y = 0.f;
       }
     }
-    __syncthreads();
-    if (base + tstep < nbags) fetch(base + tstep);     // in flight while this tile is multiplied
+    sd_cp_commit();
+  };
+#pragma unroll
+  for (int p = 0; p < SD_STAGES - 1; ++p) issue(base0 + p * tstep, p);
+  int it = 0;
+  for (int base = base0; base < nbags; base += tstep, ++it) {
+    const int stage = it % SD_STAGES;
+    sd_cp_wait<SD_STAGES - 2>();                       // this thread's copies of the tile have landed
+    __syncthreads();                                   // ... and everybody's; the previous tile is consumed
+    issue(base + (SD_STAGES - 1) * tstep, (it + SD_STAGES - 1) % SD_STAGES);
     if (tailw) {
 #pragma unroll 4
       for (int i = th; i < SD_TILE; i += 2) {
-        const float f = s_n[i][tt];
-        const float2 gg = s_g[i];
-        tw = fmaf(f, gg.x, tw); tq = fmaf(f, gg.y, tq);
+        const float f = s_n[stage][i][tt];
+        const float2 gg = s_g[stage][i];
+        tw = fmaf(f, gg.x, tw);
+        tq = fmaf(f, gg.y, tq);
       }
     } else {
 #pragma unroll
-      for (int i = sub; i < SD_TILE; i += 4) {
-        const float4 f = *reinterpret_cast<const float4*>(&s_n[i][kg * 4]);
-        const float4 c = s_c[i][c4];
-        acc[0].x = fmaf(f.x, c.x, acc[0].x); acc[0].y = fmaf(f.x, c.y, acc[0].y);
-        acc[0].z = fmaf(f.x, c.z, acc[0].z); acc[0].w = fmaf(f.x, c.w, acc[0].w);
-        acc[1].x = fmaf(f.y, c.x, acc[1].x); acc[1].y = fmaf(f.y, c.y, acc[1].y);
-        acc[1].z = fmaf(f.y, c.z, acc[1].z); acc[1].w = fmaf(f.y, c.w, acc[1].w);
-        acc[2].x = fmaf(f.z, c.x, acc[2].x); acc[2].y = fmaf(f.z, c.y, acc[2].y);
-        acc[2].z = fmaf(f.z, c.z, acc[2].z); acc[2].w = fmaf(f.z, c.w, acc[2].w);
-        acc[3].x = fmaf(f.w, c.x, acc[3].x); acc[3].y = fmaf(f.w, c.y, acc[3].y);
-        acc[3].z = fmaf(f.w, c.z, acc[3].z); acc[3].w = fmaf(f.w, c.w, acc[3].w);
+      for (int i = sub; i < SD_TILE; i += 8) {
+        const float4 f0 = *reinterpret_cast<const float4*>(&s_n[stage][i][kg * 8]);
+        const float4 f1 = *reinterpret_cast<const float4*>(&s_n[stage][i][kg * 8 + 4]);
+        float4 c = s_c[stage][i][c4];
+        if (fm) {
+          const float4 a = s_a[stage][i][c4];
+          const float gf = s_g[stage][i].y;
+          c.x = fmaf(gf, a.x, c.x); c.y = fmaf(gf, a.y, c.y); c.z = fmaf(gf, a.z, c.z); c.w = fmaf(gf, a.w, c.w);
+        }
+#define SD_FMA(q, f) acc[q].x = fmaf(f, c.x, acc[q].x); acc[q].y = fmaf(f, c.y, acc[q].y); \
+                     acc[q].z = fmaf(f, c.z, acc[q].z); acc[q].w = fmaf(f, c.w, acc[q].w)
+        SD_FMA(0, f0.x); SD_FMA(1, f0.y); SD_FMA(2, f0.z); SD_FMA(3, f0.w);
+        SD_FMA(4, f1.x); SD_FMA(5, f1.y); SD_FMA(6, f1.z); SD_FMA(7, f1.w);
+#undef SD_FMA
       }
     }
   }
+  sd_cp_wait<0>();
   // each (CTA, bag subset) hands its sums to one replica row per key
-  const uint32_t salt = hash_u32(blockIdx.x * 4u + (uint32_t)(tailw ? th : sub));
+  const uint32_t salt = hash_u32(blockIdx.x * 8u + (uint32_t)(tailw ? th : sub));
   if (tailw) {
     if ((uint32_t)tt >= ns) return;
     const uint32_t hh = __ldg(ctr + 4 + tt);
@@ -423,8 +440,8 @@ __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
     return;
   }
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const uint32_t key = (uint32_t)(kg * 4 + q);
+  for (int q = 0; q < 8; ++q) {
+    const uint32_t key = (uint32_t)(kg * 8 + q);
     if (key >= ns || !col) continue;
     const uint32_t hh = __ldg(ctr + 4 + key);
     if (hh == DES_ROW_NONE) continue;
@@ -619,7 +636,11 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
     DES_LAUNCH_CHECK(t, "grad_scatter_kernel");
   }
   if (use_super) {
-    super_dense_kernel<<<t->sm_count * 3, SD_THREADS, 0, cs>>>(t->super_cnt, (int)nbags, t->F, t->k, ops, out->out_small,
+    const int sd_smem = SD_STAGES * SD_TILE * (2 * 16 * (int)sizeof(float4) + 16 * (int)sizeof(float) + (int)sizeof(float2));
+    // (an attribute of the function on the current device, not a stream operation: legal under capture)
+    if (cudaFuncSetAttribute(super_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sd_smem) != cudaSuccess)
+      return DES_ERR_CUDA;
+    super_dense_kernel<<<t->sm_count * 3, SD_THREADS, sd_smem, cs>>>(t->super_cnt, (int)nbags, t->F, t->k, ops, out->out_small,
                                                                gr->gL, gr->gF, gE, t->Gbuf, t->hot_ctr, t->hot_base,
                                                                t->hot_R, t->max_uniq);
     DES_LAUNCH_CHECK(t, "super_dense_kernel");

@@ -67,7 +67,7 @@ struct des_table {
   uint32_t *hot_base, *hot_R, *hot_u, *hot_ctr;   // hot list [hot_max] and its two counters
   uint32_t* hot_work;                // [work_max] (hot index << 18 | chunk) items of the replica reduction
   double* hot_acc;                   // [hot_max][stride] double sums of the replicas; zero between calls
-  uint16_t* super_cnt;               // [max_batch * F][16] per-bag counts of the register-summed keys (k > 28 only)
+  float* super_cnt;                  // [max_batch * F][16] per-bag counts of the register-summed keys (k > 28 only)
   uint32_t hot_max, rep_max, work_max;
   // first dense layer
   float* W1; float* accW1;           // [F*k][H] fp32 master and state

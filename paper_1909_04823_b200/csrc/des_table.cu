@@ -197,7 +197,7 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   t->work_max = t->rep_max / HOT_RCHUNK + t->hot_max;
   A(t->hot_work, (size_t)t->work_max * 4);
   A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);
-  if (t->k > 28 && t->max_nnz >= (1 << 20)) A(t->super_cnt, (size_t)t->max_batch * t->F * 16 * 2);
+  if (t->k > 28 && t->max_nnz >= (1 << 20)) A(t->super_cnt, (size_t)t->max_batch * t->F * 16 * sizeof(float));
   if (t->H) {
     A(t->W1, FKH * 4); A(t->accW1, FKH * 4); A(t->W1b, FKH * 2);
     if (c.optimizer == DES_OPT_ADAM) A(t->acc2W1, FKH * 4);
