@@ -297,8 +297,9 @@ des_status_t des_table_size(des_table_t* t, uint64_t* h_rows_per_shard);
 /* First table-global row of each shard and the grand total, host array [S+1]. */
 des_status_t des_table_row_base(des_table_t* t, uint64_t* h_row_base);
 /* Dumps up to `cap` keys (device arrays, any order): key, shard, shard-local
- * row, latent vector [k], linear weight and their optimizer state.  *h_n_out =
- * number of keys in the table (may exceed cap; then only cap are written). */
+ * row, latent vector [k], linear weight and their optimizer state (each of the
+ * four float arrays may be NULL: not written).  *h_n_out = number of keys in
+ * the table (may exceed cap; then only cap are written). */
 des_status_t des_table_export(des_table_t* t, uint64_t* d_keys, uint8_t* d_shards, uint32_t* d_rows,
                               float* d_emb, float* d_lin, float* d_acc_emb, float* d_acc_lin,
                               uint64_t cap, uint64_t* h_n_out);

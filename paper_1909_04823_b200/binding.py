@@ -335,22 +335,26 @@ class Table:
     def launch_count(self) -> int:
         return int(self.L.des_table_launch_count(self.h))
 
-    def export(self, cap: int):
+    def export(self, cap: int, weights: bool = True):
+        """Dump of up to `cap` keys with their shard and shard-local row; with `weights`, also the
+        rows' weights and first optimizer state (several times the size of the keys)."""
         dev = "cuda"
         keys = torch.empty(cap, dtype=torch.int64, device=dev)
         shards = torch.empty(cap, dtype=torch.uint8, device=dev)
         rows = torch.empty(cap, dtype=torch.int32, device=dev)
-        emb = torch.empty((cap, self.k), dtype=torch.float32, device=dev)
-        lin = torch.empty(cap, dtype=torch.float32, device=dev)
-        ae = torch.empty((cap, self.k), dtype=torch.float32, device=dev)
-        al = torch.empty(cap, dtype=torch.float32, device=dev)
+        emb = torch.empty((cap, self.k), dtype=torch.float32, device=dev) if weights else None
+        lin = torch.empty(cap, dtype=torch.float32, device=dev) if weights else None
+        ae = torch.empty((cap, self.k), dtype=torch.float32, device=dev) if weights else None
+        al = torch.empty(cap, dtype=torch.float32, device=dev) if weights else None
         n = C.c_uint64(0)
         torch.cuda.synchronize()
         self._check(self.L.des_table_export(self.h, _ptr(keys), _ptr(shards), _ptr(rows), _ptr(emb), _ptr(lin),
                                             _ptr(ae), _ptr(al), cap, C.byref(n)), "des_table_export")
         m = min(int(n.value), cap)
-        return dict(n=int(n.value), keys=keys[:m], shards=shards[:m], rows=rows[:m], emb=emb[:m], lin=lin[:m],
-                    acc_emb=ae[:m], acc_lin=al[:m])
+        out = dict(n=int(n.value), keys=keys[:m], shards=shards[:m], rows=rows[:m])
+        if weights:
+            out.update(emb=emb[:m], lin=lin[:m], acc_emb=ae[:m], acc_lin=al[:m])
+        return out
 
     def import_rows(self, keys: torch.Tensor, shards: torch.Tensor, emb=None, lin=None, acc_emb=None, acc_lin=None):
         """Restores a dump made by `export` (of this or another table with the same S, partition, k):

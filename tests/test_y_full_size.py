@@ -97,3 +97,85 @@ def test_full_size_step_matches_oracle():
         assert np.array_equal(rows, want)
     finally:
         p.close()
+
+
+# ------------------------------------------------------------------ streaming workload at full size
+def _prepopulate_both(p, st, w):
+    per_call = w.batch * w.fields
+    for ids in st.prepopulation_ids(chunk=1 << 20):
+        for lo in range(0, ids.size, per_call):
+            p.insert_only(synth.prepopulation_batch(ids[lo:lo + per_call], w.fields))
+
+
+def test_streaming_full_size_first_steps_match_oracle():
+    """The streaming workload (batch 65536 x 30 fields, 7.9 M occurrences, half a million new keys
+    per step) at full size from its 1e6-key table: three steps, every stage against the oracle,
+    row numbers included (the oracle holds the whole table here)."""
+    from harness import Pair
+    w = synth.config(4)
+    st = synth.Stream(w)
+    b = st.next_batch()
+    p = Pair(w, max_rows=4_000_000, max_nnz=int(b.nnz * 1.1))
+    try:
+        _prepopulate_both(p, st, w)
+        sel = np.sort(np.random.default_rng(2).choice(w.batch, 64, replace=False))
+        for s in range(3):
+            before = sum(p.t.size())
+            p.step(b, synth.upstream_grads(w, b.batch, s), pooled_samples=sel)
+            assert sum(p.t.size()) == st.n_seen > before          # the table grew by exactly the fresh ids
+            b = st.next_batch() if s < 2 else None
+    finally:
+        p.close()
+
+
+def test_streaming_full_size_growth_invariants():
+    """Many full-size steps of the streaming workload on the CUDA path alone, checked by what needs
+    no oracle: after every step the table holds exactly the ids the generator has emitted so far,
+    and at the end the exported key set is that set, every key sits in the shard the partition rule
+    gives it, and the rows of a shard are 0 .. n_s - 1, each once."""
+    import os
+    from paper_1909_04823_b200.binding import DeviceBatch, Table
+    steps = int(os.environ.get("DES_TEST_STREAMING_STEPS", "20"))
+    w = synth.config(4)
+    st = synth.Stream(w)
+    B, F, k = w.batch, w.fields, w.emb_dim
+    cap = int(w.prepopulate + steps * w.p_new * B * F * 4.2 * 1.05) + 1_000_000
+    first = st.next_batch()
+    t = Table.for_workload(w, max_rows=cap, max_nnz=int(first.nnz * 1.1))
+    try:
+        per_call = B * F
+        for ids in st.prepopulation_ids(chunk=1 << 20):
+            for lo in range(0, ids.size, per_call):
+                t.find_or_insert(DeviceBatch.from_synth(synth.prepopulation_batch(ids[lo:lo + per_call], F)), True)
+        assert sum(t.size()) == w.prepopulate
+        out_small = torch.empty((B, k + 4), device="cuda")
+        pooled = torch.empty((B, F * k), device="cuda")
+        b = first
+        for s in range(steps):
+            g = {n: torch.from_numpy(v).cuda() for n, v in synth.upstream_grads(w, B, s % 4).items()}
+            db = DeviceBatch.from_synth(b)
+            t.find_or_insert(db, True)
+            t.forward_fused(w.ops, db, None, pooled, out_small, None)
+            t.backward_update(w.ops, db, out_small, pooled, None, g["gL"], g["gF"], g["gE"], None, None)
+            assert t.status() == 0
+            assert sum(t.size()) == st.n_seen, (s, sum(t.size()), st.n_seen)
+            assert bool(torch.isfinite(out_small[:, :k + 3]).all())
+            if s + 1 < steps:
+                b = st.next_batch()
+        n = st.n_seen
+        assert n > w.prepopulate + steps * 400_000
+        d = t.export(n + 16, weights=False)
+        assert d["n"] == n
+        keys = d["keys"].cpu().numpy().view(np.uint64)
+        shards = d["shards"].cpu().numpy()
+        rows = d["rows"].cpu().numpy().view(np.uint32)
+        # the key set: ids are fmix64(rank) for ranks 0 .. n - 1 (pre-populated ranks, then fresh ones in order)
+        ranks = np.sort(fmix64_inverse(keys))
+        assert np.array_equal(ranks, np.arange(n, dtype=np.uint64))
+        assert np.array_equal(shards, oracle.shard_of_many(keys, w.shards))
+        sizes = t.size()
+        for s in range(w.shards):
+            r = np.sort(rows[shards == s])
+            assert r.size == sizes[s] and np.array_equal(r, np.arange(r.size, dtype=np.uint32)), s
+    finally:
+        t.close()
