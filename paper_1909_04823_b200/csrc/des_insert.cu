@@ -60,6 +60,11 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
   // occurrence j = tile * (256 * PROBE_ILP) + q * 256 + thread: every access of a warp is contiguous.
   // Per occurrence the probe keeps its key, the table-global slot it looks at (DES_SLOT_NONE once it
   // is done) and the bounds of the owning shard's slot region: all 32-bit but the key.
+  // the bounds of the shards' slot regions, staged once per block: indexing the kernel parameter by a
+  // per-lane shard would replay the constant-bank read once per distinct shard of the warp
+  __shared__ uint32_t s_base[DES_MAX_SHARDS + 1];
+  if (threadIdx.x <= (unsigned)S) s_base[threadIdx.x] = (uint32_t)geom.slot_base[threadIdx.x];
+  __syncthreads();
   const int j0 = blockIdx.x * (256 * PROBE_ILP) + threadIdx.x;
   unsigned long long id[PROBE_ILP];
   uint32_t cur[PROBE_ILP], lo[PROBE_ILP], hi[PROBE_ILP], found[PROBE_ILP], row[PROBE_ILP], seen_fo[PROBE_ILP];
@@ -80,8 +85,8 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
       } else if (world > 1 && s % world != rank) {
         // another process holds this shard: the occurrence has no row here
       } else {
-        lo[q] = (uint32_t)geom.slot_base[s];
-        hi[q] = (uint32_t)geom.slot_base[s + 1];
+        lo[q] = s_base[s];
+        hi[q] = s_base[s + 1];
         const uint32_t n = hi[q] - lo[q];
         cur[q] = lo[q] + (uint32_t)__umul64hi(des_mix64(id[q] ^ 0x9E3779B97F4A7C15ull), (unsigned long long)n);
         nmax = max(nmax, n);
