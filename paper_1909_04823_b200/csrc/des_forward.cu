@@ -30,6 +30,9 @@
 #endif
 
 
+#ifndef ROUTE_PF
+#define ROUTE_PF 8    // batches of 32 occurrences whose loads a warp keeps in flight
+#endif
 __global__ void __launch_bounds__(256) route_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
     const uint8_t* __restrict__ shards, int B, int F, int S, const DevMeta* __restrict__ meta, uint32_t null_row,
@@ -47,54 +50,86 @@ __global__ void __launch_bounds__(256) route_kernel(
     for (int s = lane; s < S; s += 32) cur[s] = 0;
     __syncwarp();
     // pass 1: occurrences per shard (mapped rows only); CSR-order rows for the pooling kernel.
-    // Both passes load the next 32 occurrences before they work on the current ones.
+    // Both passes keep the loads of the next ROUTE_PF x 32 occurrences in flight while they work on the
+    // current ones (a warp is one dependent chain per sample; what it waits for is memory latency).
     {
-      uint32_t r_n = DES_ROW_NONE; int s_n = 0;
-      if (lo + lane < hi) { r_n = __ldg(rows + lo + lane); s_n = __ldg(shards + lo + lane); }
-      for (int base = lo; base < hi; base += 32) {
-        const int j = base + lane;
-        const uint32_t r = r_n; const int s = s_n;
-        if (j + 32 < hi) { r_n = __ldg(rows + j + 32); s_n = __ldg(shards + j + 32); }
-        if (j < hi) {
-          grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
-          if (r != DES_ROW_NONE) atomicAdd(&cur[s], 1);     // counting only: order does not matter here
+      uint32_t rq[ROUTE_PF]; int sq[ROUTE_PF];
+#pragma unroll
+      for (int q = 0; q < ROUTE_PF; ++q) {
+        const int j = lo + q * 32 + lane;
+        rq[q] = DES_ROW_NONE; sq[q] = 0;
+        if (j < hi) { rq[q] = __ldg(rows + j); sq[q] = __ldg(shards + j); }
+      }
+      for (int base = lo; base < hi; base += 32 * ROUTE_PF) {
+#pragma unroll
+        for (int q = 0; q < ROUTE_PF; ++q) {
+          const int j = base + q * 32 + lane;
+          const uint32_t r = rq[q]; const int s = sq[q];
+          if (j + 32 * ROUTE_PF < hi) { rq[q] = __ldg(rows + j + 32 * ROUTE_PF); sq[q] = __ldg(shards + j + 32 * ROUTE_PF); }
+          if (j < hi) {
+            grow_csr[j] = (r == DES_ROW_NONE) ? null_row : row_base[s] + r;
+            if (r != DES_ROW_NONE) atomicAdd(&cur[s], 1);   // counting only: order does not matter here
+          }
         }
       }
       __syncwarp();
     }
-    // exclusive scan over shards -> segment starts (lane 0 walks the <= 64 counters)
-    if (lane == 0) {
-      int run = lo;
+    // exclusive scan over shards -> segment starts (two counters per lane, S <= 64, warp scans)
+    {
+      static_assert(DES_MAX_SHARDS <= 64, "two counters per lane");
+      const int c0 = lane < S ? cur[lane] : 0, c1 = lane + 32 < S ? cur[lane + 32] : 0;
+      int i0 = c0, i1 = c1;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int v0 = __shfl_up_sync(0xFFFFFFFFu, i0, d), v1 = __shfl_up_sync(0xFFFFFFFFu, i1, d);
+        if (lane >= d) { i0 += v0; i1 += v1; }
+      }
+      const int t0 = __shfl_sync(0xFFFFFFFFu, i0, 31), t1 = __shfl_sync(0xFFFFFFFFu, i1, 31);
       int32_t* so = seg_off + (size_t)b * (S + 1);
-      for (int s = 0; s < S; ++s) { const int c = cur[s]; cur[s] = run; so[s] = run; run += c; }
-      so[S] = run;
+      __syncwarp();
+      if (lane < S) { cur[lane] = lo + i0 - c0; so[lane] = lo + i0 - c0; }
+      if (lane + 32 < S) { cur[lane + 32] = lo + t0 + i1 - c1; so[lane + 32] = lo + t0 + i1 - c1; }
+      if (lane == 0) so[S] = lo + t0 + t1;
     }
     __syncwarp();
     // pass 2: stable placement
     {
-      uint32_t r_n = DES_ROW_NONE; int s_n = 0; float x_n = 1.f;
-      if (lo + lane < hi) {
-        r_n = __ldg(rows + lo + lane); s_n = __ldg(shards + lo + lane);
-        if (vals) x_n = __ldg(vals + lo + lane);
+      uint32_t rq[ROUTE_PF]; int sq[ROUTE_PF]; float xq[ROUTE_PF];
+#pragma unroll
+      for (int q = 0; q < ROUTE_PF; ++q) {
+        const int j = lo + q * 32 + lane;
+        rq[q] = DES_ROW_NONE; sq[q] = 0; xq[q] = 1.f;
+        if (j < hi) {
+          rq[q] = __ldg(rows + j); sq[q] = __ldg(shards + j);
+          if (vals) xq[q] = __ldg(vals + j);
+        }
       }
-      for (int base = lo; base < hi; base += 32) {
-        const int j = base + lane;
-        const uint32_t r = r_n; const int s = s_n; const float x = x_n;
-        if (j + 32 < hi) {
-          r_n = __ldg(rows + j + 32); s_n = __ldg(shards + j + 32);
-          if (vals) x_n = __ldg(vals + j + 32);
+      for (int base = lo; base < hi; base += 32 * ROUTE_PF) {
+#pragma unroll
+        for (int q = 0; q < ROUTE_PF; ++q) {
+          if (base + q * 32 >= hi) break;                  // whole warp
+          const int j = base + q * 32 + lane;
+          const uint32_t r = rq[q]; const int s = sq[q]; const float x = xq[q];
+          if (j + 32 * ROUTE_PF < hi) {
+            rq[q] = __ldg(rows + j + 32 * ROUTE_PF); sq[q] = __ldg(shards + j + 32 * ROUTE_PF);
+            if (vals) xq[q] = __ldg(vals + j + 32 * ROUTE_PF);
+          }
+          int key = -1 - lane; uint32_t gr = 0;
+          if (j < hi && r != DES_ROW_NONE) { key = s; gr = row_base[s] + r; }
+          // the first lane of every group of equal shards advances the shard's cursor (a warp's
+          // shared-memory atomics execute in program order, so successive batches stay ordered) and
+          // hands the old value to its group
+          const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
+          const int leader = __ffs(same) - 1;
+          int first = 0;
+          if (key >= 0 && lane == leader) first = atomicAdd(&cur[key], __popc(same));
+          first = __shfl_sync(0xFFFFFFFFu, first, leader);
+          if (key >= 0) {
+            const int pos = first + __popc(same & lt);
+            grow_sorted[pos] = gr;
+            if (vals) x_sorted[pos] = x;
+          }
         }
-        int key = -1 - lane; uint32_t gr = 0;
-        if (j < hi && r != DES_ROW_NONE) { key = s; gr = row_base[s] + r; }
-        const unsigned same = __match_any_sync(0xFFFFFFFFu, key);
-        if (key >= 0) {
-          const int pos = cur[key] + __popc(same & lt);
-          grow_sorted[pos] = gr;
-          if (vals) x_sorted[pos] = x;
-        }
-        __syncwarp();
-        if (key >= 0 && (same & lt) == 0) cur[key] += __popc(same);
-        __syncwarp();
       }
     }
   }
