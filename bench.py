@@ -186,13 +186,13 @@ class ClockSampler:
 # 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
-    ("cfg5", "grad_scatter_kernel"): 1801e6,
+    ("cfg5", "grad_scatter_kernel"): 1806e6,
     ("cfg5", "super_dense_kernel"): 533e6,
     ("cfg5", "shard_partials_kernel"): 939e6,
     ("cfg5", "pool_kernel"): 1211e6,
     ("cfg5", "update_rows_kernel"): 1937e6,
     ("cfg5", "probe_claim_kernel"): 596e6,
-    ("cfg5", "route_kernel"): 683e6,
+    ("cfg5", "route_kernel"): 454e6,
 }
 
 
@@ -206,12 +206,12 @@ def kernel_bytes(name, st):
     pool = bool(st["ops"] & (OP_POOL | OP_DENSE1))
     if name == "probe_claim_kernel":
         return 8 * nnz + 16 * U + 4 * nnz + nnz
-    if name == "flag_count_kernel":
-        return 4 * nnz + 16 * U + nnz + nnz
+    if name == "flag_count_kernel":      # slot index and shard in; the slot's (row, scratch); flag, row, first occurrence out
+        return 4 * nnz + nnz + 8 * U + nnz + 4 * nnz + 4 * nnz
     if name == "assign_kernel":
         return nnz + nnz + 4 * U + 8 * U + 4 * U
-    if name == "resolve_kernel":
-        return 4 * nnz + 16 * U + 8 * nnz
+    if name == "resolve_kernel":         # first occurrence and row in, the firsts' unique index, row and unique index out
+        return 8 * nnz + 4 * U + 8 * nnz
     if name == "route_kernel":
         return 8 * B + 2 * 5 * nnz + 8 * nnz + 4 * B * (S + 1)
     if name == "shard_partials_kernel":

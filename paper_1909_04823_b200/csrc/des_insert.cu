@@ -2,13 +2,16 @@
 // including shard routing (Section 5, "Large-scale Sparse Features": weights of
 // field f live on node f mod N; Section 4.2: any balanced partition).
 //
-// One call = nine short kernels, none of which waits on another thread:
+// One call = ten short kernels, none of which waits on another thread; the table's slots are read
+// once per occurrence by the probe and once more by flag_count, and written only for new keys:
+//   reset_scratch exits at once unless the scratch range of the slots ran out (see Slot::first_occ).
 //   probe_claim   every occurrence finds its key's slot in the owning shard's
 //                 region (linear probing) or claims an empty one with a 64-bit
 //                 CAS; the slot remembers the smallest occurrence index.
-//   flag_count    occurrence j is the FIRST of its key iff slot.first_occ == j,
+//   flag_count    occurrence j is the FIRST of its key iff the slot remembers j,
 //                 and the key is NEW iff its slot has no row yet; per-block
-//                 counts of firsts and of new keys per shard.
+//                 counts of firsts and of new keys per shard.  Leaves the
+//                 slot's row and the first occurrence's index per occurrence.
 //   scan          exclusive scan of those counts over blocks.
 //   assign        first occurrences get the batch-unique index (rank among
 //                 firsts) and, for new keys, the next shard-local row (rank
@@ -16,11 +19,13 @@
 //                 does not depend on thread scheduling.  Two kernels: the ranks
 //                 among firsts always, the new-key numbering only when the
 //                 batch has a new key at all.
-//   apply_first   one thread per unique key writes these numbers into the
-//                 key's slot; init_new_rows then fills the new keys' rows from
-//                 the counter-based generator (a lane group per row).
-//   resolve       every occurrence reads row and unique index from its slot.
-//   finish        slots' scratch word is reset, shard sizes are advanced.
+//   apply_first   one thread per unique key: the key's unique index (and a new
+//                 key's row) at its first occurrence, a new key's row into its
+//                 slot; init_new_rows then fills the new keys' rows from the
+//                 counter-based generator (a lane group per row).
+//   resolve       every other occurrence takes row and unique index from its
+//                 key's first occurrence.
+//   finish        shard sizes advance, the call's scratch range is retired.
 #include "des_internal.cuh"
 
 #define IB 1024  // occurrences per block (tile) in every per-occurrence kernel of this file
@@ -65,6 +70,7 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
   __shared__ uint32_t s_base[DES_MAX_SHARDS + 1];
   if (threadIdx.x <= (unsigned)S) s_base[threadIdx.x] = (uint32_t)geom.slot_base[threadIdx.x];
   __syncthreads();
+  const uint32_t base = meta->scratch_base - (uint32_t)nnz;   // this call's scratch range (Slot::first_occ)
   const int j0 = blockIdx.x * (256 * PROBE_ILP) + threadIdx.x;
   unsigned long long id[PROBE_ILP];
   uint32_t cur[PROBE_ILP], lo[PROBE_ILP], hi[PROBE_ILP], found[PROBE_ILP], row[PROBE_ILP], seen_fo[PROBE_ILP];
@@ -126,23 +132,28 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
   for (int q = 0; q < PROBE_ILP; ++q) {
     const int j = j0 + q * 256;
     if (j >= nnz) continue;
-    // the slot's scratch word as seen by the probe may be stale, but only ever too LARGE:
-    // skipping the atomic when it is already smaller than j is safe
-    if (found[q] != DES_SLOT_NONE && insert && seen_fo[q] > (uint32_t)j)
-      atomicMin(&slots[found[q]].first_occ, (uint32_t)j);
+    // the slot's scratch word as seen by the probe may be stale (or an earlier call's), but only ever
+    // too LARGE: skipping the atomic when it is already smaller than this occurrence's is safe
+    if (found[q] != DES_SLOT_NONE && insert && seen_fo[q] > base + (uint32_t)j)
+      atomicMin(&slots[found[q]].first_occ, base + (uint32_t)j);
     if (insert) slot_of[j] = found[q];
     else rows[j] = row[q];
   }
 }
 
-// flags: bit0 = first occurrence of its key in the batch, bit1 = key is new.
+// flags: bit0 = first occurrence of its key in the batch, bit1 = key is new.  This is the only pass
+// that reads every occurrence's slot after the claims: it also leaves the slot's row (DES_ROW_NONE for a
+// new key) in rows[] and the index of the key's first occurrence in first_of[], which is all that the
+// later passes need.
 __global__ void __launch_bounds__(IB / 4) flag_count_kernel(
-    int nnz, int S, const Slot* __restrict__ slots, const uint32_t* __restrict__ slot_of,
-    const uint8_t* __restrict__ shards, uint8_t* __restrict__ flags, uint32_t* __restrict__ blk_cnt, int nblk_max) {
+    int nnz, int S, const Slot* __restrict__ slots, const DevMeta* __restrict__ meta,
+    const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, uint8_t* __restrict__ flags,
+    uint32_t* __restrict__ rows, uint32_t* __restrict__ first_of, uint32_t* __restrict__ blk_cnt, int nblk_max) {
   // IB occurrences per block, IB / 4 threads: a thread's four slot look-ups are in flight together
   __shared__ uint32_t cnt[DES_MAX_SHARDS + 1];
   if (threadIdx.x <= DES_MAX_SHARDS) cnt[threadIdx.x] = 0;
   __syncthreads();
+  const uint32_t base = meta->scratch_base - (uint32_t)nnz;
   const int j0 = blockIdx.x * IB + threadIdx.x;
   uint32_t so[4];
 #pragma unroll
@@ -150,19 +161,22 @@ __global__ void __launch_bounds__(IB / 4) flag_count_kernel(
     const int j = j0 + q * (IB / 4);
     so[q] = (j < nnz) ? slot_of[j] : DES_SLOT_NONE;
   }
-  Slot sl[4];
+  uint2 rf[4];                                         // (row, first_occ): the slot's second half
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    sl[q].row = 0; sl[q].first_occ = DES_ROW_NONE;
-    if (so[q] != DES_SLOT_NONE) sl[q] = slots[so[q]];
+    rf[q] = make_uint2(DES_ROW_NONE, DES_ROW_NONE);
+    if (so[q] != DES_SLOT_NONE) rf[q] = reinterpret_cast<const uint2*>(slots + so[q])[1];
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
     uint8_t fl = 0;
     if (j < nnz) {
-      if (so[q] != DES_SLOT_NONE && sl[q].first_occ == (uint32_t)j) fl = (sl[q].row == DES_ROW_NONE) ? 3 : 1;
+      const bool mapped = so[q] != DES_SLOT_NONE;
+      if (mapped && rf[q].y == base + (uint32_t)j) fl = (rf[q].x == DES_ROW_NONE) ? 3 : 1;
       flags[j] = fl;
+      rows[j] = rf[q].x;
+      first_of[j] = mapped ? rf[q].y - base : DES_ROW_NONE;
     }
     const unsigned firsts = __ballot_sync(0xFFFFFFFFu, fl & 1);
     if ((threadIdx.x & 31) == 0 && firsts) atomicAdd(&cnt[0], __popc(firsts));
@@ -310,29 +324,28 @@ __global__ void __launch_bounds__(IB) assign_kernel(
   }
 }
 
-// One thread per unique key of the batch: number new keys' slots and initialise
-// their rows, publish the key's batch-unique index in its slot (read back by
-// every occurrence in resolve_kernel), record slot and table-global row.
+// One thread per unique key of the batch: a new key's row number goes into its slot (the only slot
+// access) and into rows[] at its first occurrence; the first occurrence also takes the key's batch-unique
+// index (resolve_kernel hands both on to the key's other occurrences); uniq_rows gets the table-global row.
 __global__ void __launch_bounds__(256) apply_first_kernel(
-    Slot* slots, const DevMeta* __restrict__ meta,
-    const uint32_t* __restrict__ slot_of, const uint8_t* __restrict__ shards, const uint32_t* __restrict__ first_j,
-    uint32_t* __restrict__ uslot, uint32_t* __restrict__ uniq_rows) {
+    Slot* slots, const DevMeta* __restrict__ meta, const uint32_t* __restrict__ slot_of,
+    const uint8_t* __restrict__ shards, const uint32_t* __restrict__ first_j, uint32_t* __restrict__ rows,
+    uint32_t* __restrict__ uidx, uint32_t* __restrict__ uniq_rows) {
   const uint32_t U = meta->n_uniq;
   for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
     const uint32_t fj = first_j[u];
     const bool is_new = fj >> 31;
     const uint32_t j = fj & 0x7FFFFFFFu;
-    const uint32_t so = slot_of[j];
     const uint32_t s = shards[j];
     uint32_t local;
     if (is_new) {
-      local = uniq_rows[u];
-      if (local != DES_ROW_NONE) slots[so].row = local;
+      local = uniq_rows[u];                            // DES_ROW_NONE: the shard is full
+      if (local != DES_ROW_NONE) slots[slot_of[j]].row = local;
+      rows[j] = local;
     } else {
-      local = slots[so].row;
+      local = rows[j];
     }
-    slots[so].first_occ = u;
-    uslot[u] = so;
+    uidx[j] = (local == DES_ROW_NONE) ? DES_ROW_NONE : u;
     const unsigned long long g = meta->row_base[s] + local;
     uniq_rows[u] = (local == DES_ROW_NONE) ? DES_ROW_NONE : (uint32_t)g;
   }
@@ -380,43 +393,65 @@ __global__ void __launch_bounds__(256) init_new_rows_kernel(
   }
 }
 
-// IB occurrences per block, IB / 4 threads: a thread's four slot look-ups are in flight together.
-__global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const Slot* __restrict__ slots,
-                                                         const uint32_t* __restrict__ slot_of,
-                                                         uint32_t* __restrict__ rows, uint32_t* __restrict__ uidx) {
+// Every occurrence that is not its key's first one takes the unique index — and, for a key that was new,
+// the row — from the first one (a look-up in the batch's own arrays, not in the table).  IB occurrences per
+// block, IB / 4 threads: a thread's four look-ups are in flight together.  First occurrences are only read
+// here (apply_first_kernel wrote them), the others only written.
+__global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const uint32_t* __restrict__ first_of,
+                                                         uint32_t* rows, uint32_t* uidx, DevMeta* meta) {
   const int j0 = blockIdx.x * IB + threadIdx.x;
-  uint32_t so[4];
+  uint32_t f[4], r[4], u[4];
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
-    so[q] = (j < nnz) ? slot_of[j] : DES_SLOT_NONE;
-  }
-  Slot sl[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    sl[q].row = DES_ROW_NONE; sl[q].first_occ = DES_ROW_NONE;
-    if (so[q] != DES_SLOT_NONE) sl[q] = slots[so[q]];
+    f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE;
+    if (j < nnz) { f[q] = first_of[j]; r[q] = rows[j]; }
+    // (a first-occurrence index is an index into this batch; anything else would be a broken scratch word)
+    if (f[q] != DES_ROW_NONE && f[q] >= (uint32_t)nnz) { f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE; des_raise(meta, DES_ERR_CUDA); }
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
-    if (j >= nnz) continue;
-    rows[j] = sl[q].row;
-    uidx[j] = (sl[q].row == DES_ROW_NONE) ? DES_ROW_NONE : sl[q].first_occ;
+    u[q] = DES_ROW_NONE;
+    if (f[q] != DES_ROW_NONE && f[q] != (uint32_t)j) {
+      u[q] = uidx[f[q]];
+      if (r[q] == DES_ROW_NONE) r[q] = rows[f[q]];
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int j = j0 + q * (IB / 4);
+    if (j >= nnz || f[q] == (uint32_t)j) continue;
+    rows[j] = r[q];
+    uidx[j] = u[q];
   }
 }
 
-__global__ void __launch_bounds__(256) finish_kernel(int S, Slot* slots, const uint32_t* __restrict__ uslot,
-                                                     DevMeta* meta, uint32_t* n_uniq_out) {
-  const uint32_t U = meta->n_uniq;
-  for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x)
-    slots[uslot[u]].first_occ = DES_ROW_NONE;
-  if (blockIdx.x == 0 && threadIdx.x < S) {
-    // block 0 is the only writer of n_rows; no other block of this kernel reads it
+// Clears the scratch word of every slot when the call before ran out of scratch range (see Slot::first_occ);
+// launched by every insert call, exits at once otherwise.
+__global__ void __launch_bounds__(256) reset_scratch_kernel(Slot* slots, unsigned long long total_slots,
+                                                            const DevMeta* __restrict__ meta) {
+  if (meta->scratch_reset == 0u) return;
+  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_slots;
+       i += (unsigned long long)gridDim.x * blockDim.x)
+    slots[i].first_occ = DES_ROW_NONE;
+}
+
+// One block: shard sizes advance, the call's scratch range is retired.
+__global__ void __launch_bounds__(DES_MAX_SHARDS) finish_kernel(int S, int nnz, uint32_t max_nnz, DevMeta* meta,
+                                                                uint32_t* n_uniq_out) {
+  if ((int)threadIdx.x < S) {
     uint32_t n = meta->n_rows[threadIdx.x] + meta->new_total[threadIdx.x];
     meta->n_rows[threadIdx.x] = min(n, meta->row_cap[threadIdx.x]);
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) { *n_uniq_out = U; meta->any_new = 0u; }
+  if (threadIdx.x == 0) {
+    *n_uniq_out = meta->n_uniq;
+    meta->any_new = 0u;
+    const uint32_t base = meta->scratch_base - (uint32_t)nnz;
+    const bool out = base < max_nnz;                   // the next call may need up to max_nnz below the base
+    meta->scratch_base = out ? 0xFFFFFFFFu : base;
+    meta->scratch_reset = out ? 1u : 0u;
+  }
 }
 
 extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b, int insert, void* stream) {
@@ -434,12 +469,18 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   SlotGeom geom;
   for (uint32_t s = 0; s <= t->S; ++s) geom.slot_base[s] = t->h_slot_base[s];
   des_mod_consts(t->S, &geom.mod_M, &geom.mod_two32);
+  if (insert) {
+    reset_scratch_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->total_slots, t->meta);
+    DES_LAUNCH_CHECK(t, "reset_scratch_kernel");
+  }
   probe_claim_kernel<<<(nnz + 256 * PROBE_ILP - 1) / (256 * PROBE_ILP), 256, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
                                           t->cfg.partition, insert, t->cfg.shard_world, t->cfg.shard_rank, t->slots, t->meta, geom,
                                           t->slot_of, b->shards, b->rows);
   DES_LAUNCH_CHECK(t, "probe_claim_kernel");
   if (!insert) return DES_OK;
-  flag_count_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->S, t->slots, t->slot_of, b->shards, t->flags, t->blk_cnt, t->nblk_max);
+  uint32_t* first_of = t->uslot;
+  flag_count_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->S, t->slots, t->meta, t->slot_of, b->shards, t->flags, b->rows,
+                                             first_of, t->blk_cnt, t->nblk_max);
   DES_LAUNCH_CHECK(t, "flag_count_kernel");
   scan_blocks_kernel<<<t->S + 1, 1024, 0, cs>>>(t->blk_cnt, nblk, t->nblk_max, t->meta);
   DES_LAUNCH_CHECK(t, "scan_blocks_kernel");
@@ -448,8 +489,8 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   assign_kernel<<<nblk < t->sm_count * 2 ? nblk : t->sm_count * 2, IB, 0, cs>>>(nnz, nblk, t->S, t->meta, b->shards, t->flags,
                                                                                 t->blk_cnt, t->nblk_max, t->dest, b->uniq_rows);
   DES_LAUNCH_CHECK(t, "assign_kernel");
-  apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->meta, t->slot_of, b->shards, t->dest, t->uslot,
-                                                      b->uniq_rows);
+  apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->meta, t->slot_of, b->shards, t->dest, b->rows,
+                                                      b->uidx, b->uniq_rows);
   DES_LAUNCH_CHECK(t, "apply_first_kernel");
   {
     const float state_init = t->cfg.optimizer == DES_OPT_ADAGRAD ? t->cfg.init_acc : 0.f;
@@ -464,9 +505,9 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
 #undef INIT
     DES_LAUNCH_CHECK(t, "init_new_rows_kernel");
   }
-  resolve_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->slots, t->slot_of, b->rows, b->uidx);
+  resolve_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, first_of, b->rows, b->uidx, t->meta);
   DES_LAUNCH_CHECK(t, "resolve_kernel");
-  finish_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->S, t->slots, t->uslot, t->meta, b->n_uniq);
+  finish_kernel<<<1, DES_MAX_SHARDS, 0, cs>>>(t->S, nnz, (uint32_t)t->max_nnz, t->meta, b->n_uniq);
   DES_LAUNCH_CHECK(t, "finish_kernel");
   return DES_OK;
 }

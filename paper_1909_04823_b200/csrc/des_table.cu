@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include "des_internal.cuh"
+#include <cstdlib>
 
 static void* dalloc(const des_config_t& c, size_t bytes) {
   if (bytes == 0) bytes = 256;
@@ -141,6 +142,11 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   if (t->max_uniq > t->max_nnz) t->max_uniq = t->max_nnz;
   cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev);
   DevMeta hm; memset(&hm, 0, sizeof(hm));
+  hm.scratch_base = 0xFFFFFFFFu;                      // top of the insert calls' scratch range (Slot::first_occ)
+  if (const char* e = getenv("DES_DEBUG_SCRATCH_BASE")) {   // tests: start near the end of the range, so that
+    const unsigned long long v = strtoull(e, nullptr, 0);   // the rare reset pass runs within a few calls
+    if (v >= t->max_nnz && v <= 0xFFFFFFFFull) hm.scratch_base = (uint32_t)v;
+  }
   uint64_t rows = 0, slots = 0;
   const uint32_t world = c.shard_world > 1 ? c.shard_world : 1;
   uint32_t owned = 0;

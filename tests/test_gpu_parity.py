@@ -313,3 +313,23 @@ def test_maximum_fields_and_shards(partition):
 def test_long_bags_operator_subsets(ops):
     w = synth.config(5).scaled(batch=40, vocab=20000, prepopulate=0, shards=9, init_scale=0.05, ops=ops)
     _run(w, 2, max_rows=120000, ops=ops)
+
+
+def test_insert_scratch_range_wraps(monkeypatch):
+    """The slots' scratch word works in a range that moves down with every insert call and is reset by
+    one pass over the table when it runs out (every few billion occurrences).  Started three calls
+    before the end of the range, the reset must happen unnoticed: every step matches the oracle."""
+    w = synth.config(1).scaled(batch=256, ops=OP_LR | OP_FM | OP_POOL, init_scale=0.05, optimizer=OPT_ADAGRAD)
+    st = synth.Stream(w)
+    first = st.next_batch()
+    max_nnz = int(first.nnz * 1.5) + 1024
+    monkeypatch.setenv("DES_DEBUG_SCRATCH_BASE", str(max_nnz + 3 * first.nnz))
+    p = _pair(w, 60000, max_nnz=max_nnz)
+    monkeypatch.delenv("DES_DEBUG_SCRATCH_BASE")
+    try:
+        b = first
+        for s in range(8):
+            p.step(b, synth.upstream_grads(w, b.batch, s), check_init=(s == 0))
+            b = st.next_batch()
+    finally:
+        p.close()
