@@ -2,9 +2,8 @@
 // including shard routing (Section 5, "Large-scale Sparse Features": weights of
 // field f live on node f mod N; Section 4.2: any balanced partition).
 //
-// One call = ten short kernels, none of which waits on another thread; the table's slots are read
+// One call = nine short kernels, none of which waits on another thread; the table's slots are read
 // once per occurrence by the probe and once more by flag_count, and written only for new keys:
-//   reset_scratch exits at once unless the scratch range of the slots ran out (see Slot::first_occ).
 //   probe_claim   every occurrence finds its key's slot in the owning shard's
 //                 region (linear probing) or claims an empty one with a 64-bit
 //                 CAS; the slot remembers the smallest occurrence index.
@@ -18,7 +17,8 @@
 //                 among the shard's new keys): both in CSR order, so the result
 //                 does not depend on thread scheduling.  Two kernels: the ranks
 //                 among firsts always, the new-key numbering only when the
-//                 batch has a new key at all.
+//                 batch has a new key at all (that kernel also clears the slots'
+//                 scratch words when their range runs out, see Slot::first_occ).
 //   apply_first   one thread per unique key: the key's unique index (and a new
 //                 key's row) at its first occurrence, a new key's row into its
 //                 slot; init_new_rows then fills the new keys' rows from the
@@ -272,9 +272,16 @@ __global__ void __launch_bounds__(IB / 4) assign_firsts_kernel(int nnz, const ui
 __global__ void __launch_bounds__(IB) assign_kernel(
     int nnz, int nblk, int S, DevMeta* meta, const uint8_t* __restrict__ shards, const uint8_t* __restrict__ flags,
     const uint32_t* __restrict__ blk_cnt, int nblk_max, uint32_t* __restrict__ first_j,
-    uint32_t* __restrict__ uniq_rows) {
+    uint32_t* __restrict__ uniq_rows, Slot* slots, unsigned long long total_slots, uint32_t max_nnz) {
   __shared__ uint32_t wfirst[32];
   __shared__ uint16_t wnew[32][DES_MAX_SHARDS];
+  // The slots' scratch range ends with this call (see Slot::first_occ; finish_kernel then starts a new one):
+  // nothing reads the scratch words after flag_count_kernel, so this kernel — a few blocks that are idle
+  // in the steady state — clears them all, once every few billion occurrences.
+  if (meta->scratch_base - (uint32_t)nnz < max_nnz)
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_slots;
+         i += (unsigned long long)gridDim.x * blockDim.x)
+      slots[i].first_occ = DES_ROW_NONE;
   // steady state of a populated table: no new key in the whole batch (settled by scan_blocks_kernel, which
   // ran before this kernel), and assign_firsts_kernel has done all there is to do
   if (meta->any_new == 0u) return;
@@ -427,16 +434,6 @@ __global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const uint32_t
   }
 }
 
-// Clears the scratch word of every slot when the call before ran out of scratch range (see Slot::first_occ);
-// launched by every insert call, exits at once otherwise.
-__global__ void __launch_bounds__(256) reset_scratch_kernel(Slot* slots, unsigned long long total_slots,
-                                                            const DevMeta* __restrict__ meta) {
-  if (meta->scratch_reset == 0u) return;
-  for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total_slots;
-       i += (unsigned long long)gridDim.x * blockDim.x)
-    slots[i].first_occ = DES_ROW_NONE;
-}
-
 // One block: shard sizes advance, the call's scratch range is retired.
 __global__ void __launch_bounds__(DES_MAX_SHARDS) finish_kernel(int S, int nnz, uint32_t max_nnz, DevMeta* meta,
                                                                 uint32_t* n_uniq_out) {
@@ -448,9 +445,9 @@ __global__ void __launch_bounds__(DES_MAX_SHARDS) finish_kernel(int S, int nnz, 
     *n_uniq_out = meta->n_uniq;
     meta->any_new = 0u;
     const uint32_t base = meta->scratch_base - (uint32_t)nnz;
-    const bool out = base < max_nnz;                   // the next call may need up to max_nnz below the base
-    meta->scratch_base = out ? 0xFFFFFFFFu : base;
-    meta->scratch_reset = out ? 1u : 0u;
+    // the next call may need up to max_nnz below the base; if that is not left, assign_kernel has
+    // cleared every slot's scratch word in this call and the range starts again at the top
+    meta->scratch_base = base < max_nnz ? 0xFFFFFFFFu : base;
   }
 }
 
@@ -469,10 +466,6 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   SlotGeom geom;
   for (uint32_t s = 0; s <= t->S; ++s) geom.slot_base[s] = t->h_slot_base[s];
   des_mod_consts(t->S, &geom.mod_M, &geom.mod_two32);
-  if (insert) {
-    reset_scratch_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->total_slots, t->meta);
-    DES_LAUNCH_CHECK(t, "reset_scratch_kernel");
-  }
   probe_claim_kernel<<<(nnz + 256 * PROBE_ILP - 1) / (256 * PROBE_ILP), 256, 0, cs>>>((const unsigned long long*)b->ids, b->offsets, nnz, nbags, t->S, t->F,
                                           t->cfg.partition, insert, t->cfg.shard_world, t->cfg.shard_rank, t->slots, t->meta, geom,
                                           t->slot_of, b->shards, b->rows);
@@ -487,7 +480,8 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   assign_firsts_kernel<<<nblk, IB / 4, 0, cs>>>(nnz, t->flags, t->blk_cnt, t->dest);
   DES_LAUNCH_CHECK(t, "assign_firsts_kernel");
   assign_kernel<<<nblk < t->sm_count * 2 ? nblk : t->sm_count * 2, IB, 0, cs>>>(nnz, nblk, t->S, t->meta, b->shards, t->flags,
-                                                                                t->blk_cnt, t->nblk_max, t->dest, b->uniq_rows);
+                                                                                t->blk_cnt, t->nblk_max, t->dest, b->uniq_rows,
+                                                                                t->slots, t->total_slots, (uint32_t)t->max_nnz);
   DES_LAUNCH_CHECK(t, "assign_kernel");
   apply_first_kernel<<<t->sm_count * 8, 256, 0, cs>>>(t->slots, t->meta, t->slot_of, b->shards, t->dest, b->rows,
                                                       b->uidx, b->uniq_rows);

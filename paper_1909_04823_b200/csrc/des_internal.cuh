@@ -18,8 +18,9 @@
 //              the key in the call's batch).  Every call works scratch_base - nnz below the
 //              call before it, so what earlier calls left behind is larger than anything
 //              the running call writes and never needs to be cleared; when the base runs
-//              out (every few billion occurrences) one pass resets all slots to
-//              DES_ROW_NONE, the value of a slot that was never touched.
+//              out (every few billion occurrences) the call that used its last part resets
+//              all slots to DES_ROW_NONE, the value of a slot that was never touched, once
+//              it has read them.
 struct __align__(16) Slot {
   unsigned long long key;
   uint32_t row;
@@ -37,7 +38,6 @@ struct DevMeta {
   uint32_t err;                                      // sticky des_status_t raised on device
   uint32_t any_new;                                  // the running insert call has at least one new key
   uint32_t scratch_base;                             // see Slot::first_occ: the last insert call's base
-  uint32_t scratch_reset;                            // the next insert call must clear every slot's scratch first
   uint32_t field_order[1024];                        // fields sorted by (owning shard, field)
   unsigned long long opt_step;                       // backward calls so far (Adam's t), advanced on device
   float adam_c1, adam_c2;                            // 1 - beta1^t, 1 - beta2^t for the running step
