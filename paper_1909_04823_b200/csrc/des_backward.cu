@@ -47,24 +47,35 @@ __device__ __forceinline__ uint32_t hash_u32(uint32_t x) {
 // its table to hinfo once.
 #define SC_THREADS 1024
 #define SC_SLOTS 1024
+#ifndef SC_PER
+#define SC_PER 4
+#endif
 __global__ void __launch_bounds__(SC_THREADS) sample_count_kernel(const uint32_t* __restrict__ uidx, int nnz, int shift,
                                                                   long long max_uniq, uint32_t* hinfo) {
   __shared__ uint32_t s_key[SC_SLOTS], s_cnt[SC_SLOTS];
   for (int i = threadIdx.x; i < SC_SLOTS; i += SC_THREADS) { s_key[i] = DES_ROW_NONE; s_cnt[i] = 0u; }
   __syncthreads();
-  const int i = blockIdx.x * SC_THREADS + threadIdx.x;
-  const long long j = ((long long)i << shift) + (shift ? (hash_u32((uint32_t)i) & ((1u << shift) - 1u)) : 0u);
-  uint32_t u = DES_ROW_NONE;
-  if (j < nnz) u = __ldg(uidx + j);
-  const bool ok = u != DES_ROW_NONE && (long long)u < max_uniq;
-  const unsigned act = __ballot_sync(0xFFFFFFFFu, ok);
-  if (ok) {
-    const unsigned same = __match_any_sync(act, u);
-    if ((threadIdx.x & 31) == __ffs(same) - 1) {
-      const uint32_t c = (uint32_t)__popc(same), slot = hash_u32(u) & (SC_SLOTS - 1);
-      const uint32_t old = atomicCAS(&s_key[slot], DES_ROW_NONE, u);
-      if (old == DES_ROW_NONE || old == u) atomicAdd(&s_cnt[slot], c);
-      else atomicAdd(hinfo + u, c);
+  // SC_PER samples per thread, their loads in flight together
+  uint32_t u[SC_PER];
+#pragma unroll
+  for (int q = 0; q < SC_PER; ++q) {
+    const long long i = ((long long)blockIdx.x * SC_PER + q) * SC_THREADS + threadIdx.x;
+    const long long j = (i << shift) + (shift ? (hash_u32((uint32_t)i) & ((1u << shift) - 1u)) : 0u);
+    u[q] = DES_ROW_NONE;
+    if (j < nnz) u[q] = __ldg(uidx + j);
+  }
+#pragma unroll
+  for (int q = 0; q < SC_PER; ++q) {
+    const bool ok = u[q] != DES_ROW_NONE && (long long)u[q] < max_uniq;
+    const unsigned act = __ballot_sync(0xFFFFFFFFu, ok);
+    if (ok) {
+      const unsigned same = __match_any_sync(act, u[q]);
+      if ((threadIdx.x & 31) == __ffs(same) - 1) {
+        const uint32_t c = (uint32_t)__popc(same), slot = hash_u32(u[q]) & (SC_SLOTS - 1);
+        const uint32_t old = atomicCAS(&s_key[slot], DES_ROW_NONE, u[q]);
+        if (old == DES_ROW_NONE || old == u[q]) atomicAdd(&s_cnt[slot], c);
+        else atomicAdd(hinfo + u[q], c);
+      }
     }
   }
   __syncthreads();
@@ -139,7 +150,8 @@ __global__ void __launch_bounds__(256) make_dest_kernel(const uint32_t* __restri
     d[q] = u[q];                                          // cold key (or no row)
     if (u[q] != DES_ROW_NONE && hv[q] != DES_ROW_NONE) {
       if (hv[q] >> 24) d[q] = SUPER_TAG | ((hv[q] >> 24) - 1u);
-      else d[q] = (uint32_t)max_uniq + __ldg(hot_base + hv[q]) + hash_u32((uint32_t)j) % __ldg(hot_R + hv[q]);
+      else   // replica floor(hash * R / 2^32): uniform over the R replicas without a division
+        d[q] = (uint32_t)max_uniq + __ldg(hot_base + hv[q]) + __umulhi(hash_u32((uint32_t)j), __ldg(hot_R + hv[q]));
     }
   }
 #pragma unroll
@@ -604,7 +616,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   const uint32_t super_min = use_super ? (uint32_t)(nnz >> 7) : 0u;
   {
     const int n = (nnz >> shift) + 1;
-    sample_count_kernel<<<(n + SC_THREADS - 1) / SC_THREADS, SC_THREADS, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
+    sample_count_kernel<<<(n + SC_THREADS * SC_PER - 1) / (SC_THREADS * SC_PER), SC_THREADS, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
     DES_LAUNCH_CHECK(t, "sample_count_kernel");
     hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
                                                        t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
