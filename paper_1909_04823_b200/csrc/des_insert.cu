@@ -408,13 +408,16 @@ __global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const uint32_t
                                                          uint32_t* rows, uint32_t* uidx, DevMeta* meta) {
   const int j0 = blockIdx.x * IB + threadIdx.x;
   uint32_t f[4], r[4], u[4];
+  bool newrow[4];                                      // the occurrence's row comes from the first occurrence
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
-    f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE;
+    f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE; newrow[q] = false;
     if (j < nnz) { f[q] = first_of[j]; r[q] = rows[j]; }
     // (a first-occurrence index is an index into this batch; anything else would be a broken scratch word)
-    if (f[q] != DES_ROW_NONE && f[q] >= (uint32_t)nnz) { f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE; des_raise(meta, DES_ERR_CUDA); }
+    if (f[q] != DES_ROW_NONE && f[q] >= (uint32_t)nnz) {
+      f[q] = DES_ROW_NONE; r[q] = DES_ROW_NONE; newrow[q] = true; des_raise(meta, DES_ERR_CUDA);
+    }
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
@@ -422,14 +425,14 @@ __global__ void __launch_bounds__(IB / 4) resolve_kernel(int nnz, const uint32_t
     u[q] = DES_ROW_NONE;
     if (f[q] != DES_ROW_NONE && f[q] != (uint32_t)j) {
       u[q] = uidx[f[q]];
-      if (r[q] == DES_ROW_NONE) r[q] = rows[f[q]];
+      if (r[q] == DES_ROW_NONE) { r[q] = rows[f[q]]; newrow[q] = true; }
     }
   }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
     if (j >= nnz || f[q] == (uint32_t)j) continue;
-    rows[j] = r[q];
+    if (newrow[q]) rows[j] = r[q];                     // (every other row is in place since flag_count_kernel)
     uidx[j] = u[q];
   }
 }
