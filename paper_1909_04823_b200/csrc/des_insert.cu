@@ -83,7 +83,8 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     if (j < nnz) {
       id[q] = ids[j];
       uint32_t s;
-      if (partition == DES_PART_HASH) s = des_mod_small(des_mix64(id[q]), (uint32_t)S, geom.mod_M, geom.mod_two32);
+      const unsigned long long h = des_mix64(id[q]);
+      if (partition == DES_PART_HASH) s = des_mod_small(h, (uint32_t)S, geom.mod_M, geom.mod_two32);
       else s = (uint32_t)(des_bag_of(offsets, nbags, j) % F) % (unsigned)S;
       shards[j] = (uint8_t)s;
       if (id[q] == DES_KEY_EMPTY) {
@@ -94,7 +95,9 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
         lo[q] = s_base[s];
         hi[q] = s_base[s + 1];
         const uint32_t n = hi[q] - lo[q];
-        cur[q] = lo[q] + (uint32_t)__umul64hi(des_mix64(id[q] ^ 0x9E3779B97F4A7C15ull), (unsigned long long)n);
+        // position inside the region: the top bits of an odd multiple of the same mixed word (the shard is its
+        // residue mod S; a second full mixing round bought nothing measurable in probe lengths)
+        cur[q] = lo[q] + (uint32_t)__umul64hi(h * 0x9E3779B97F4A7C15ull, (unsigned long long)n);
         nmax = max(nmax, n);
       }
     }
