@@ -208,8 +208,8 @@ def kernel_bytes(name, st):
         return 8 * nnz + 16 * U + 4 * nnz + nnz
     if name == "flag_count_kernel":      # slot index and shard in; the slot's (row, scratch); flag, row, first occurrence out
         return 4 * nnz + nnz + 8 * U + nnz + 4 * nnz + 4 * nnz
-    if name == "assign_kernel":
-        return nnz + nnz + 4 * U + 8 * U + 4 * U
+    if name == "assign_kernel":          # exits at once when the batch has no new key (a populated table)
+        return (nnz + nnz + 4 * U + 8 * U + 4 * U) if st.get("new_keys", True) else None
     if name == "resolve_kernel":         # first occurrence and row in, the firsts' unique index, row and unique index out
         return 8 * nnz + 4 * U + 8 * nnz
     if name == "route_kernel":
@@ -447,7 +447,7 @@ def main():
     stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, H=H, U=U, ops=w.ops,
                  adagrad=(w.optimizer == synth.OPT_ADAGRAD), rep_rows=0,
                  super=(k > 28 and batches[0].nnz >= (1 << 20) and batches[0].vals is None),
-                 shift=shift_of(batches[0].nnz))
+                 shift=shift_of(batches[0].nnz), new_keys=(w.p_new > 0 or not w.prepopulate))
     tot_k = sum(v[1] for v in per.values()) or 1.0
     kernels = []
     for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
