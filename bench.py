@@ -181,9 +181,8 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-# profiles/memory_counters_cfg5_batch_small_table.md: the benchmark's own batch on a 4e6-key table (the
-# 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from an ncu capture of the benchmark's
+# own batch on a 4e6-key table (the 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
     ("cfg5", "grad_scatter_kernel"): 1806e6,
@@ -198,7 +197,7 @@ NCU_DRAM_TRAFFIC = {
 
 def kernel_bytes(name, st):
     """Algorithmic bytes one launch of `name` must move (what the method needs,
-    each datum once; see the design notes for the derivation)."""
+    each datum once: ids, offsets and index arrays per occurrence, table rows per unique key)."""
     nnz, B, F, k, S, U, R = st["nnz"], st["B"], st["F"], st["k"], st["S"], st["U"], st["rep_rows"]
     row = 4 * k + 16
     state = 1 if st["adagrad"] else 0

@@ -12,16 +12,21 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "des_oracle.cpp")
 _LIB = os.path.join(_HERE, "libdes_oracle.so")
+_LIB_OMP = os.path.join(_HERE, "libdes_oracle_omp.so")   # the same source with -fopenmp (all host cores)
 _lib = None
+_lib_omp = None
 
 ROW_NONE = 0xFFFFFFFF
 
 
-def build(force: bool = False) -> str:
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared",
-                               "-o", _LIB, _SRC])
-    return _LIB
+def build(force: bool = False, omp: bool = False) -> str:
+    """Compiles the oracle: the plain sequential build (the parity oracle) or, with omp=True, the same
+    source with -fopenmp (used only to time the oracle on all host cores)."""
+    out = _LIB_OMP if omp else _LIB
+    if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(_SRC):
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared"]
+                              + (["-fopenmp"] if omp else []) + ["-o", out, _SRC])
+    return out
 
 
 def _p(a, t):
@@ -30,28 +35,40 @@ def _p(a, t):
     return a.ctypes.data_as(C.POINTER(t))
 
 
-def lib():
-    global _lib
+def lib(omp: bool = False):
+    global _lib, _lib_omp
+    if omp:
+        if _lib_omp is None:
+            _lib_omp = _declare(C.CDLL(build(omp=True)))
+        return _lib_omp
     if _lib is None:
-        _lib = C.CDLL(build())
-        L = _lib
-        L.orc_mix64.restype = C.c_uint64
-        L.orc_mix64.argtypes = [C.c_uint64]
-        L.orc_init_value.restype = C.c_float
-        L.orc_init_value.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_float]
-        L.orc_bf16_round.restype = C.c_float
-        L.orc_bf16_round.argtypes = [C.c_float]
-        L.orc_create.restype = C.c_void_p
-        L.orc_create.argtypes = [C.c_uint32] * 6 + [C.c_uint64] + [C.c_float] * 4
-        L.orc_destroy.argtypes = [C.c_void_p]
-        L.orc_find_or_insert.restype = C.c_int64
-        for name in ("orc_dense1_set", "orc_dense1_get", "orc_size", "orc_find_or_insert",
-                     "orc_forward_original", "orc_fm_pairs", "orc_forward_partials", "orc_aggregate",
-                     "orc_backward_update", "orc_read_rows", "orc_poke", "orc_philox4x32_10",
-                     "orc_shard_of_many", "orc_comm_saving", "orc_set_opt", "orc_read_state2",
-                     "orc_dense1_get_state2"):
-            getattr(L, name).argtypes = None
+        _lib = _declare(C.CDLL(build()))
     return _lib
+
+
+def _declare(L):
+    L.orc_mix64.restype = C.c_uint64
+    L.orc_mix64.argtypes = [C.c_uint64]
+    L.orc_init_value.restype = C.c_float
+    L.orc_init_value.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_float]
+    L.orc_bf16_round.restype = C.c_float
+    L.orc_bf16_round.argtypes = [C.c_float]
+    L.orc_create.restype = C.c_void_p
+    L.orc_create.argtypes = [C.c_uint32] * 6 + [C.c_uint64] + [C.c_float] * 4
+    L.orc_destroy.argtypes = [C.c_void_p]
+    L.orc_find_or_insert.restype = C.c_int64
+    for name in ("orc_dense1_set", "orc_dense1_get", "orc_size", "orc_find_or_insert",
+                 "orc_forward_original", "orc_fm_pairs", "orc_forward_partials", "orc_aggregate",
+                 "orc_backward_update", "orc_read_rows", "orc_poke", "orc_philox4x32_10",
+                 "orc_shard_of_many", "orc_comm_saving", "orc_set_opt", "orc_read_state2",
+                 "orc_dense1_get_state2"):
+        getattr(L, name).argtypes = None
+    return L
+
+
+def num_threads(omp: bool = False) -> int:
+    """Threads the oracle's parallel loops use: 1 for the plain build, the OpenMP default for the other."""
+    return int(lib(omp).orc_num_threads())
 
 
 def mix64(x: int) -> int:
@@ -115,9 +132,9 @@ def cross_backward(x0, x, w, P, gY):
 
 class Oracle:
     def __init__(self, S, F, k, H=0, partition=0, optimizer=0, seed=0, init_scale=0.01,
-                 lr=0.01, eps=1e-8, init_acc=0.0):
+                 lr=0.01, eps=1e-8, init_acc=0.0, omp=False):
         self.S, self.F, self.k, self.H = S, F, k, H
-        self.L = lib()
+        self.L = lib(omp)
         self.h = C.c_void_p(self.L.orc_create(S, F, k, H, partition, optimizer, C.c_uint64(seed),
                                               C.c_float(init_scale), C.c_float(lr), C.c_float(eps),
                                               C.c_float(init_acc)))
@@ -129,9 +146,9 @@ class Oracle:
                            C.c_float(ftrl_alpha), C.c_float(ftrl_beta), C.c_float(ftrl_l1), C.c_float(ftrl_l2))
 
     @classmethod
-    def for_workload(cls, w):
+    def for_workload(cls, w, omp=False):
         o = cls(w.shards, w.fields, w.emb_dim, w.hidden, w.partition, w.optimizer, w.seed,
-                w.init_scale, w.lr, w.eps, w.init_acc)
+                w.init_scale, w.lr, w.eps, w.init_acc, omp=omp)
         o.set_opt(getattr(w, "lin_optimizer", 0), getattr(w, "beta1", 0.9), getattr(w, "beta2", 0.999),
                   getattr(w, "ftrl_alpha", 0.05), getattr(w, "ftrl_beta", 1.0), getattr(w, "ftrl_l1", 0.0),
                   getattr(w, "ftrl_l2", 0.0))

@@ -19,8 +19,15 @@
 //     gradient, state local to the shard (Section 4.3, closing paragraph);
 //   * the dynamic hash table's lookup / insert / update (Section 5).
 // Where the paper is silent (which hash, how a new weight is initialised, how
-// rows are numbered, Adagrad's exact form) it follows the readings listed in
-// the design notes; each is marked "reading" below.
+// rows are numbered, Adagrad's exact form) it takes one fixed reading; each is
+// marked "reading" below.
+//
+// All-cores build: compiled a second time with -fopenmp, the per-sample loops of
+// the forward, the per-element loops of the first layer's backward and the
+// per-unique-key loops of the update run as `omp parallel for`; every sum keeps
+// the order of the sequential build (a key's occurrences are added in CSR order
+// either way), so both builds return the same bits.  Without -fopenmp the
+// pragmas and the grouped form of the gradient sum below are compiled out.
 //
 // Arithmetic: weights and optimizer state are float32 (the paper's storage
 // type, Section 4.1); every sum is accumulated in double and rounded once.
@@ -31,6 +38,9 @@
 // dedup/Adagrad special cases; row-split GEMM == one dense matmul; canonical
 // row numbering vs a dictionary walk.  The hash/shard rule itself is fixed by
 // no passage: "parity unpinned" beyond bijectivity and balance.
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -169,6 +179,15 @@ inline void apply_opt(const Table& t, float& theta, float& acc, float& acc2, dou
 
 extern "C" {
 
+// threads the parallel loops of this build use (1 without -fopenmp)
+int orc_num_threads() {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
 uint64_t orc_mix64(uint64_t x) { return mix64(x); }
 void orc_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) { philox4x32_10(ctr, key, out); }
 float orc_init_value(uint64_t seed, uint64_t id, uint32_t c, float scale) { return init_value(seed, id, c, scale); }
@@ -276,11 +295,10 @@ void orc_forward_original(void* p, uint32_t ops, const int32_t* offsets, const u
                           double* fm2, double* pooled0, double* Z0, double* Sabs) {
   Table* t = (Table*)p;
   const uint32_t F = t->F, k = t->k, H = t->H;
-  std::vector<double> A(k), pool((size_t)F * k);
+#pragma omp parallel for schedule(dynamic, 16)
   for (int32_t b = 0; b < B; ++b) {
+    std::vector<double> A(k, 0.0), pool((size_t)F * k, 0.0);
     double lr = 0, Q = 0;
-    std::fill(A.begin(), A.end(), 0.0);
-    std::fill(pool.begin(), pool.end(), 0.0);
     for (uint32_t f = 0; f < F; ++f) {
       int64_t bag = (int64_t)b * F + f;
       for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
@@ -357,13 +375,13 @@ void orc_forward_partials(void* p, uint32_t ops, const int32_t* offsets, const f
   Table* t = (Table*)p;
   const uint32_t S = t->S, F = t->F, k = t->k, H = t->H;
   const size_t FK = (size_t)F * k;
-  std::vector<double> pool(FK);
   for (uint32_t s = 0; s < S; ++s) {
     const Shard& h = t->sh[s];
+#pragma omp parallel for schedule(dynamic, 16)
     for (int32_t b = 0; b < B; ++b) {
+      std::vector<double> pool(FK, 0.0);
       double* ps = part_small ? part_small + ((size_t)s * B + b) * (k + 2) : nullptr;
       if (ps) for (uint32_t c = 0; c < k + 2; ++c) ps[c] = 0;
-      std::fill(pool.begin(), pool.end(), 0.0);
       for (uint32_t f = 0; f < F; ++f) {
         int64_t bag = (int64_t)b * F + f;
         for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
@@ -398,6 +416,7 @@ void orc_aggregate(void* p, int32_t B, const double* part_small, const double* p
   Table* t = (Table*)p;
   const uint32_t S = t->S, F = t->F, k = t->k, H = t->H;
   const size_t FK = (size_t)F * k;
+#pragma omp parallel for schedule(static)
   for (int32_t b = 0; b < B; ++b) {
     if (part_small && out_small) {
       double* o = out_small + (size_t)b * (k + 3);
@@ -452,7 +471,8 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
   const bool use_pool = (ops & (OP_POOL | OP_DENSE1)) != 0;
   if (use_pool) {
     gEt.assign((size_t)B * FK, 0.0f);
-    for (size_t i = 0; i < (size_t)B * FK; ++i) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)((size_t)B * FK); ++i) {
       double a = ((ops & OP_POOL) && gE) ? (double)gE[i] : 0.0;
       if ((ops & OP_DENSE1) && gZ) {
         size_t b = i / FK, col = i % FK;
@@ -467,25 +487,48 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
   std::vector<double> Gw((size_t)U, 0.0), Gv((size_t)U * k, 0.0);
   std::vector<double> Sw((size_t)U, 0.0), Sv((size_t)U * k, 0.0);
   std::vector<uint8_t> us((size_t)U); std::vector<uint32_t> ur((size_t)U);
+  // the per-occurrence terms of one key, added in CSR order
+  auto add_occurrence = [&](int32_t b, uint32_t f, int32_t j) {
+    uint32_t u = uidx[j], s = shards[j], row = rows[j];
+    us[u] = (uint8_t)s; ur[u] = row;
+    const Shard& h = t->sh[s];
+    double x = vals ? (double)vals[j] : 1.0;
+    if (ops & OP_LR) { Gw[u] += x * (double)gL[b]; Sw[u] += std::fabs(x * (double)gL[b]); }
+    for (uint32_t c = 0; c < k; ++c) {
+      double g = 0;
+      if (ops & OP_FM) g += (double)gF[b] * ((double)A[(size_t)b * k + c] - (double)h.emb[(size_t)row * k + c] * x);
+      if (use_pool) g += (double)gEt[(size_t)b * FK + (size_t)f * k + c];
+      Gv[(size_t)u * k + c] += x * g;
+      Sv[(size_t)u * k + c] += std::fabs(x * g);
+    }
+  };
+#ifndef _OPENMP
   for (int32_t b = 0; b < B; ++b)
     for (uint32_t f = 0; f < F; ++f) {
       int64_t bag = (int64_t)b * F + f;
-      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j) {
-        if (rows[j] == ROW_NONE) continue;
-        uint32_t u = uidx[j], s = shards[j], row = rows[j];
-        us[u] = (uint8_t)s; ur[u] = row;
-        const Shard& h = t->sh[s];
-        double x = vals ? (double)vals[j] : 1.0;
-        if (ops & OP_LR) { Gw[u] += x * (double)gL[b]; Sw[u] += std::fabs(x * (double)gL[b]); }
-        for (uint32_t c = 0; c < k; ++c) {
-          double g = 0;
-          if (ops & OP_FM) g += (double)gF[b] * ((double)A[(size_t)b * k + c] - (double)h.emb[(size_t)row * k + c] * x);
-          if (use_pool) g += (double)gEt[(size_t)b * FK + (size_t)f * k + c];
-          Gv[(size_t)u * k + c] += x * g;
-          Sv[(size_t)u * k + c] += std::fabs(x * g);
-        }
-      }
+      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j)
+        if (rows[j] != ROW_NONE) add_occurrence(b, f, j);
     }
+#else
+  {
+    // all-cores build: the same sums grouped by key first (a counting sort of the occurrences by
+    // unique index that keeps CSR order inside a key), then one thread per key
+    std::vector<int64_t> start((size_t)U + 1, 0);
+    const int64_t nnz = offsets[(int64_t)B * F];
+    for (int64_t j = 0; j < nnz; ++j) if (rows[j] != ROW_NONE) start[uidx[j] + 1]++;
+    for (int64_t u = 0; u < U; ++u) start[u + 1] += start[u];
+    std::vector<int32_t> occ((size_t)start[U]), bag_of((size_t)start[U]);
+    std::vector<int64_t> fill(start.begin(), start.end() - 1);
+    for (int64_t bag = 0; bag < (int64_t)B * F; ++bag)
+      for (int32_t j = offsets[bag]; j < offsets[bag + 1]; ++j)
+        if (rows[j] != ROW_NONE) { int64_t p_ = fill[uidx[j]]++; occ[p_] = j; bag_of[p_] = (int32_t)bag; }
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t u = 0; u < U; ++u)
+      for (int64_t p_ = start[u]; p_ < start[u + 1]; ++p_)
+        add_occurrence((int32_t)(bag_of[p_] / F), (uint32_t)(bag_of[p_] % F), occ[p_]);
+  }
+#endif
+#pragma omp parallel for schedule(dynamic, 64)
   for (int64_t u = 0; u < U; ++u) {
     Shard& h = t->sh[us[u]];
     uint32_t row = ur[u];
@@ -503,7 +546,8 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
     if (Gv_out) for (uint32_t c = 0; c < k; ++c) Gv_out[(size_t)u * k + c] = (float)Gv[(size_t)u * k + c];
   }
   if ((ops & OP_DENSE1) && gZ && pooled) {
-    for (size_t i = 0; i < FK; ++i)
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)FK; ++i)
       for (uint32_t h2 = 0; h2 < H; ++h2) {
         double g = 0;
         for (int32_t b = 0; b < B; ++b)

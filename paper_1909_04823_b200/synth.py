@@ -123,7 +123,7 @@ class Workload:
 
 
 def config(i: int) -> Workload:
-    """The five benchmark workloads, 1-based as in the design notes."""
+    """The five benchmark workloads, numbered from 1."""
     if i == 1:
         return Workload("cfg1_tiny_lr_fm", 512, 8, 8, 4, PART_HASH, OPT_SGD, OP_LR | OP_FM,
                         zipf_s=1.1, vocab=100_000, shared_vocab=True,

@@ -37,13 +37,29 @@ from paper_1909_04823_b200.synth import OP_DENSE1, OP_FM, OP_LR, OP_POOL, PART_F
 RTOL, ATOL, SUMTOL, SUMTOL_FWD = 1e-5, 1e-6, 2e-7, 2e-6
 
 
-def close32(got, ref, what, rtol=RTOL, atol=ATOL, extra=None):
+# Per output: how many compared elements were outside the STATED bound rtol |ref| + atol (before the
+# condition-aware term), out of how many, the worst condition number sum|t| / |sum t| among those, and their
+# worst error in units of the stated bound.  Filled by close32 whenever it is given the extra term; the
+# full-size tests assert caps on it and conftest writes it out when DES_TOL_REPORT names a file.
+TOL_STATS = {}
+TOL_CONTEXT = [""]          # label of the workload being compared (set by Pair.step)
+
+
+def close32(got, ref, what, rtol=RTOL, atol=ATOL, extra=None, sumabs=None):
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
     err = np.abs(got - ref)
     tol = rtol * np.abs(ref) + atol
     if extra is not None:
+        out = err > tol
+        st = TOL_STATS.setdefault(f"{TOL_CONTEXT[0]}: {what}", dict(outside_stated=0, total=0, worst_cond=0.0, worst_over=0.0))
+        st["outside_stated"] += int(out.sum()); st["total"] += int(err.size)
+        if out.any():
+            st["worst_over"] = max(st["worst_over"], float((err[out] / tol[out]).max()))
+            if sumabs is not None:
+                sa = np.broadcast_to(np.asarray(sumabs, dtype=np.float64), err.shape)
+                st["worst_cond"] = max(st["worst_cond"], float((sa[out] / np.maximum(np.abs(ref[out]), 1e-300)).max()))
         tol = tol + extra
     if not np.all(err <= tol):
         i = np.unravel_index(np.argmax(err - tol), err.shape)
@@ -51,9 +67,10 @@ def close32(got, ref, what, rtol=RTOL, atol=ATOL, extra=None):
                              f"{int((err > tol).sum())} of {err.size} out of tolerance")
 
 
-def close_gemm(got, ref, what, extra=None):
+def close_gemm(got, ref, what, extra=None, sumabs=None):
     ref = np.asarray(ref, dtype=np.float64)
-    close32(got, ref, what, rtol=2e-2, atol=1e-3 * max(float(np.abs(ref).max()), 1e-30), extra=extra)
+    close32(got, ref, "[gemm] " + what, rtol=2e-2, atol=1e-3 * max(float(np.abs(ref).max()), 1e-30), extra=extra,
+            sumabs=sumabs)
 
 
 def u32(t: torch.Tensor) -> np.ndarray:
@@ -205,16 +222,21 @@ class Pair:
 
     # ------------------------------------------------------------------
     def step(self, batch, grads, ops=None, materialise=False, check_init=False, by_key=False,
-             pooled_samples=None):
+             pooled_samples=None, dense_samples=None):
         """One full step on both sides with every intermediate compared.
         pooled_samples: compare `pooled` only on these sample indices (the dense
-        per-shard pooled partial of the oracle is too large at full size)."""
+        per-shard pooled partial of the oracle is too large at full size).
+        dense_samples: full-size first-layer workloads — the oracle's per-shard partial
+        products P_s (S x B x H x F k multiply-adds) are skipped; `pooled` is compared in
+        full against the unsubstituted operator, Z on these sample indices against the
+        unsubstituted operator on the sub-batch; the backward is compared in full."""
         from paper_1909_04823_b200.binding import DeviceBatch
         w = self.w
         ops = w.ops if ops is None else ops
         B, F, k, S, H = batch.batch, w.fields, w.emb_dim, w.shards, w.hidden
         dev = "cuda"
         cmp = close_gemm if self.drifted else close32
+        TOL_CONTEXT[0] = f"{w.name} B={B} S={S} k={k}"
         # ---- index
         fi = self.o.find_or_insert(batch)
         db = DeviceBatch.from_synth(batch)
@@ -223,10 +245,13 @@ class Pair:
         if check_init:
             self.compare_rows(fi, db, exact=True, what="initial rows")
         # ---- forward
-        op = self.o.forward_partials(ops, batch, fi, want_pooled=pooled_samples is None,
-                                     want_dense=bool(ops & OP_DENSE1))
+        op = self.o.forward_partials(ops, batch, fi, want_pooled=pooled_samples is None and dense_samples is None,
+                                     want_dense=bool(ops & OP_DENSE1) and dense_samples is None)
         oa = self.o.aggregate(B, op)
-        sabs = self.o.forward_original(ops & ~OP_DENSE1, batch)["Sabs"]
+        fo = self.o.forward_original(ops & ~OP_DENSE1, batch)
+        sabs = fo["Sabs"]
+        if dense_samples is not None and (ops & (OP_POOL | OP_DENSE1)):
+            oa["pooled"] = fo["pooled"]
         xa, xl = SUMTOL_FWD * sabs[:, :k], SUMTOL_FWD * sabs[:, k]
         part_small = torch.full((S, B, k + 4), float("nan"), device=dev)
         pooled = torch.full((B, F * k), float("nan"), device=dev)
@@ -255,18 +280,18 @@ class Pair:
         ps = part_small.cpu().numpy()
         osm = out_small.cpu().numpy()
         if ops & OP_FM:
-            cmp(ps[:, :, :k], op["part_small"][:, :, :k], "part_small.M1_fm", extra=xa[None])
+            cmp(ps[:, :, :k], op["part_small"][:, :, :k], "part_small.M1_fm", extra=xa[None], sumabs=sabs[None, :, :k])
             cmp(ps[:, :, k + 1], op["part_small"][:, :, k + 1], "part_small.M2_fm",
                 extra=SUMTOL_FWD * op["part_small"][:, :, k + 1])
-            cmp(osm[:, :k], oa["A"], "A", extra=xa)
+            cmp(osm[:, :k], oa["A"], "A", extra=xa, sumabs=sabs[:, :k])
             cmp(osm[:, k + 2], oa["Q"], "Q", extra=SUMTOL_FWD * oa["Q"])
             # fm2 = (<A,A> - Q)/2 subtracts two float32-rounded inputs of size <A,A>/2 and Q/2
             AA = np.sum(oa["A"] ** 2, axis=1)
             cmp(osm[:, k + 1], oa["fm2"], "fm2",
                 extra=SUMTOL_FWD * (AA + np.abs(oa["Q"])) + np.sum(np.abs(oa["A"]) * xa, axis=1))
         if ops & OP_LR:
-            cmp(ps[:, :, k], op["part_small"][:, :, k], "part_small.M1_lr", extra=xl[None])
-            cmp(osm[:, k], oa["lr"], "R_lr", extra=xl)
+            cmp(ps[:, :, k], op["part_small"][:, :, k], "part_small.M1_lr", extra=xl[None], sumabs=sabs[None, :, k])
+            cmp(osm[:, k], oa["lr"], "R_lr", extra=xl, sumabs=sabs[:, k])
         if ops & (OP_LR | OP_FM):
             assert not np.any(ps[:, :, k + 2:]) and not np.any(osm[:, k + 3]), "padding must be zero"
         if (ops & (OP_POOL | OP_DENSE1)) and pooled_samples is not None:
@@ -278,7 +303,11 @@ class Pair:
             cmp(pooled.cpu().numpy(), oa["pooled"], "pooled")
             if materialise:
                 cmp(part_pooled.cpu().numpy(), op["part_pooled"], "part_pooled")
-        if ops & OP_DENSE1:
+        if (ops & OP_DENSE1) and dense_samples is not None:
+            sel = np.asarray(dense_samples)
+            ref_Z = self.o.forward_original(ops, select_samples(batch, sel))["Z"]
+            close_gemm(Z[torch.from_numpy(sel).to(dev)].cpu().numpy(), ref_Z, "Z (sampled)")
+        elif ops & OP_DENSE1:
             close_gemm(Z.cpu().numpy(), oa["Z"], "Z")
             if materialise:
                 close_gemm(part_dense.cpu().numpy(), op["part_dense"], "part_dense")

@@ -56,9 +56,12 @@ def test_cfg2_wide_deep_scaled_materialised():
     _run(w, 3, max_rows=400000, materialise=True)
 
 
-def test_cfg2_wide_deep_full_shape():
-    w = synth.config(2)
-    _run(w, 2, max_rows=2_000_000)
+def test_adagrad_nonzero_initial_accumulator():
+    # accumulators that start at init_acc = 0.1 (rows, linear weights and the first layer), three steps
+    w = synth.config(2).scaled(batch=512, vocab=3000, hidden=64, init_scale=0.05, init_acc=0.1)
+    _run(w, 3, max_rows=200000)
+    w = synth.config(4).scaled(batch=256, prepopulate=2000, init_scale=0.05, init_acc=0.1)
+    _run(w, 3, max_rows=200000, prepop=1)
 
 
 # ------------------------------------------------------------------ config 3 (DeepFM)

@@ -458,6 +458,121 @@ def test_ftrl_l1_keeps_small_weights_at_exact_zero():
     np.testing.assert_allclose(o.read_state2(f["uniq_shard"], f["uniq_row"])["lin2"], tot, rtol=1e-5, atol=1e-6)
 
 
+# --------------------------------------------------------------------------- Adagrad over several steps
+@pytest.mark.parametrize("init_acc", [0.0, 0.1])
+def test_adagrad_equals_library_adagrad_over_several_steps(init_acc):
+    # Section 6 ("Parameter Settings") names AdaGrad for the embedding and DNN parts; the form used here
+    # (accumulator starts at init_acc and keeps growing, eps outside the root) is the library's
+    # torch.optim.Adagrad without decay.  Every key is in every batch, so lazy == dense; latent vectors,
+    # linear weights and the first layer's W1 are followed for six steps in float64.
+    n, k, H, lr, eps = 7, 4, 5, 0.05, 1e-8
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    b = _one_key_per_sample(keys)
+    o = Oracle(3, 1, k, H, PART_HASH, OPT_ADAGRAD, seed=5, init_scale=0.5, lr=lr, eps=eps, init_acc=init_acc)
+    rng = np.random.default_rng(8)
+    W1 = rng.standard_normal((k, H)).astype(np.float32)
+    o.dense1_set(W1)
+    f = o.find_or_insert(b)
+    assert f["U"] == n and np.array_equal(f["uidx"], np.arange(n))
+    r0 = o.read_rows(f["uniq_shard"], f["uniq_row"])
+    np.testing.assert_array_equal(r0["acc_emb"], np.full((n, k), np.float32(init_acc)))
+    np.testing.assert_array_equal(r0["acc_lin"], np.full(n, np.float32(init_acc)))
+    np.testing.assert_array_equal(o.dense1_get()[1], np.full((k, H), np.float32(init_acc)))
+    P = torch.tensor(r0["emb"], dtype=torch.float64, requires_grad=True)
+    Pl = torch.zeros(n, dtype=torch.float64, requires_grad=True)
+    PW = torch.tensor(W1, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adagrad([P, Pl, PW], lr=lr, eps=eps, initial_accumulator_value=init_acc, lr_decay=0.0)
+    bf = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).to(torch.float64)
+    for step in range(6):
+        gE = rng.standard_normal((n, k)).astype(np.float32)
+        gL = rng.standard_normal(n).astype(np.float32)
+        gZ = rng.standard_normal((n, H)).astype(np.float32)
+        pooled = o.read_rows(f["uniq_shard"], f["uniq_row"])["emb"]        # one key per sample, x = 1
+        W1_now = o.dense1_get()[0]
+        o.backward_update(OP_LR | OP_POOL | OP_DENSE1, b, f, np.zeros((n, k)), pooled, gL, None, gE, gZ)
+        gZ64 = torch.from_numpy(gZ.astype(np.float64))
+        P.grad = torch.from_numpy(gE.astype(np.float64)) + gZ64 @ bf(W1_now).T
+        Pl.grad = torch.from_numpy(gL.astype(np.float64))
+        PW.grad = bf(pooled).T @ gZ64
+        opt.step()
+        r = o.read_rows(f["uniq_shard"], f["uniq_row"])
+        W1n, accW1 = o.dense1_get()
+        np.testing.assert_allclose(r["emb"], P.detach().numpy(), rtol=2e-5, atol=2e-7)
+        np.testing.assert_allclose(r["lin"], Pl.detach().numpy(), rtol=2e-5, atol=2e-7)
+        np.testing.assert_allclose(W1n, PW.detach().numpy(), rtol=2e-5, atol=2e-7)
+        np.testing.assert_allclose(r["acc_emb"], opt.state[P]["sum"].numpy(), rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(r["acc_lin"], opt.state[Pl]["sum"].numpy(), rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(accW1, opt.state[PW]["sum"].numpy(), rtol=2e-5, atol=1e-9)
+
+
+@pytest.mark.parametrize("init_acc", [0.0, 0.1])
+def test_adagrad_is_lazy(init_acc):
+    # A key that is absent from a step keeps its weight and its accumulator; the keys of the step follow
+    # per-key Adagrad with their own history (closed form written out: a_t = init_acc + sum of G^2 so far).
+    n, k, lr, eps = 9, 4, 0.03, 1e-8
+    keys = synth.fmix64(np.arange(n, dtype=np.uint64))
+    o = Oracle(2, 1, k, 0, PART_HASH, OPT_ADAGRAD, seed=6, init_scale=0.5, lr=lr, eps=eps, init_acc=init_acc)
+    fall = o.find_or_insert(_one_key_per_sample(keys))
+    theta = o.read_rows(fall["uniq_shard"], fall["uniq_row"])["emb"].astype(np.float64)
+    acc = np.full((n, k), np.float64(np.float32(init_acc)))
+    rng = np.random.default_rng(4)
+    for step in range(8):
+        sub = np.sort(rng.choice(n, size=rng.integers(1, n), replace=False))
+        b = _one_key_per_sample(keys[sub])
+        f = o.find_or_insert(b)
+        gE = rng.standard_normal((len(sub), k)).astype(np.float32)
+        before = o.read_rows(fall["uniq_shard"], fall["uniq_row"])
+        o.backward_update(OP_POOL, b, f, np.zeros((len(sub), k)), None, None, None, gE)
+        after = o.read_rows(fall["uniq_shard"], fall["uniq_row"])
+        rest = np.setdiff1d(np.arange(n), sub)
+        for name in ("emb", "lin", "acc_emb", "acc_lin"):
+            assert np.array_equal(before[name][rest], after[name][rest]), name
+        G = gE.astype(np.float64)
+        acc[sub] += G * G
+        theta[sub] -= lr * G / (np.sqrt(acc[sub]) + eps)
+        np.testing.assert_allclose(after["emb"], theta, rtol=2e-5, atol=2e-7)
+        np.testing.assert_allclose(after["acc_emb"], acc, rtol=2e-5, atol=1e-9)
+
+
+# --------------------------------------------------------------------------- all-cores build
+@pytest.mark.parametrize("cfg", [2, 5])
+def test_openmp_build_equals_the_sequential_oracle(cfg):
+    # The oracle compiled with -fopenmp (timed by the benchmark on all host cores) must return what the
+    # sequential parity oracle returns: every output of two steps, to 1e-12 relative.
+    if cfg == 2:
+        w = synth.config(2).scaled(batch=96, vocab=300, hidden=24, init_scale=0.5)
+    else:
+        w = synth.config(5).scaled(batch=12, vocab=500, prepopulate=0, shards=7, init_scale=0.5)
+    outs = []
+    for omp in (False, True):
+        assert (oracle.num_threads(omp) >= 1) and (omp or oracle.num_threads(False) == 1)
+        o = Oracle.for_workload(w, omp=omp)
+        if w.hidden:
+            o.dense1_set(synth.dense1_weights(w))
+        st = synth.Stream(w, with_vals=(cfg == 5))
+        rec = []
+        for step in range(2):
+            b = st.next_batch()
+            g = synth.upstream_grads(w, b.batch, step)
+            fi = o.find_or_insert(b)
+            part = o.forward_partials(w.ops, b, fi, want_pooled=True, want_dense=bool(w.hidden))
+            agg = o.aggregate(b.batch, part)
+            org = o.forward_original(w.ops, b)
+            pooled32 = agg["pooled"].astype(np.float32)
+            res = o.backward_update(w.ops, b, fi, agg["A"].astype(np.float32), pooled32, g["gL"], g["gF"],
+                                    g["gE"] if (w.ops & OP_POOL) else None, g.get("gZ") if w.hidden else None)
+            rows = o.read_rows(fi["uniq_shard"], fi["uniq_row"])
+            rec += [fi["rows"], fi["uidx"], part["part_small"], part["part_pooled"], agg["out_small"], agg["pooled"],
+                    org["A"], org["fm2"], org["pooled"], org["Sabs"], res["Gv"], res["Gw"], res["Sv"], res["gE_total"],
+                    rows["emb"], rows["lin"], rows["acc_emb"], rows["acc_lin"]]
+            if w.hidden:
+                rec += [part["part_dense"], agg["Z"], org["Z"], res["gW1"], *o.dense1_get()]
+        outs.append(rec)
+        o.close()
+    for a, c in zip(*outs):
+        np.testing.assert_allclose(np.asarray(c, dtype=np.float64), np.asarray(a, dtype=np.float64), rtol=1e-12, atol=0)
+
+
 # --------------------------------------------------------------------------- DCN cross layer
 @pytest.mark.parametrize("S", [1, 3, 4, 16])
 def test_cross_layer_matches_the_unsplit_layer_and_autograd(S):
