@@ -104,9 +104,10 @@ def oracle_step(o, w, b, g):
                       g.get("gE") if (w.ops & OP_POOL) else None, g.get("gZ") if (w.ops & OP_DENSE1) else None)
 
 
-def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0):
+def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0, omp=False):
     """Times the CPU oracle on the first Bs samples of `batch`, Bs sized so that
-    one step takes about budget_s seconds.  Returns (samples/s, Bs, seconds per step)."""
+    one step takes about budget_s seconds.  omp: the same source compiled with
+    -fopenmp, on all host cores.  Returns (samples/s, Bs, seconds per step)."""
     from oracle import Oracle
     if w.hidden:
         W1 = synth.dense1_weights(w)
@@ -114,7 +115,7 @@ def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0):
     def run(bs, n):
         sb = sub_batch(batch, bs)
         g = {k_: v[:bs] for k_, v in grads.items()}
-        o = Oracle.for_workload(w)
+        o = Oracle.for_workload(w, omp=omp)
         if w.hidden:
             o.dense1_set(W1)
         ts = []
@@ -125,7 +126,7 @@ def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0):
         o.close()
         return ts
 
-    probe = max(1, min(batch.batch, 8))
+    probe = max(1, min(batch.batch, 64 if omp else 8))
     t = run(probe, 1)[0]
     per_sample = max(t / probe, 1e-7)
     bs = int(max(1, min(batch.batch, budget_s / per_sample)))
@@ -136,48 +137,72 @@ def time_oracle(w, batch, grads, budget_s=15.0, steps=1, warmup=0):
 
 # ---------------------------------------------------------------------------
 class ClockSampler:
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """SM clock, power and throttle reasons of one GPU, sampled every 20 ms by a thread (NVML, read-only
+    queries) with host time stamps, so that every timed window gets its own median clock."""
+    REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"), (0x4, "sw_power_cap"))
 
-    def __init__(self, gpu_index):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
+    def __init__(self, torch_index):
+        import threading
+        self.samples = []           # (time, sm MHz, reasons bitmask, watts)
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "50"],
-                                      stdout=self.f, stderr=subprocess.DEVNULL)
-        except Exception:
-            self.p = None
-
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.p is None:
-            return out
-        self.p.terminate()
-        try:
-            self.p.wait(timeout=5)
-        except Exception:
-            self.p.kill()
-        self.f.flush()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in open(self.f.name):
-            c = [x.strip() for x in line.split(",")]
-            if len(c) < 9:
-                continue
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            h = None
             try:
-                sm.append(float(c[1])); mx.append(float(c[2]))
-            except ValueError:
-                continue
-            for n_, v in zip(names, c[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(n_)
-        os.unlink(self.f.name)
-        if sm:
-            out = {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)), "reasons": sorted(reasons),
-                   "samples": len(sm)}
-        return out
+                uuid = str(torch.cuda.get_device_properties(torch_index).uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            except Exception:
+                h = pynvml.nvmlDeviceGetHandleByIndex(torch_index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            reasons_fn = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(pynvml, "nvmlDeviceGetCurrentClocksThrottleReasons")
+
+            def loop():
+                while not self._stop.is_set():
+                    try:
+                        self.samples.append((time.perf_counter(), float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)),
+                                             int(reasons_fn(h)), pynvml.nvmlDeviceGetPowerUsage(h) / 1e3))
+                    except Exception:
+                        pass
+                    self._stop.wait(0.02)
+            self._thread = threading.Thread(target=loop, daemon=True)
+            self._thread.start()
+        except Exception as ex:
+            log(f"[bench] clock sampling unavailable: {ex!r}")
+
+    def window(self, t0, t1):
+        """Median SM MHz and the throttle reasons seen between two host time stamps."""
+        sel = [s for s in self.samples if t0 <= s[0] <= t1]
+        if not sel:   # a window shorter than the sampling period: the nearest sample
+            sel = sorted(self.samples, key=lambda s_: abs(s_[0] - 0.5 * (t0 + t1)))[:1]
+        if not sel:
+            return {"sm_mhz": None, "reasons": [], "samples": 0}
+        bits = 0
+        for s_ in sel:
+            bits |= s_[2]
+        return {"sm_mhz": float(np.median([s_[1] for s_ in sel])), "samples": len(sel),
+                "reasons": sorted(n for b, n in self.REASONS if bits & b)}
+
+    def stop(self, windows=None):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        sel = self.samples
+        if windows:
+            inw = [s_ for s_ in self.samples if any(a <= s_[0] <= b for a, b in windows)]
+            sel = inw or sel
+        bits = 0
+        for s_ in sel:
+            bits |= s_[2]
+        return {"sm_mhz": float(np.median([s_[1] for s_ in sel])), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(n for b, n in self.REASONS if bits & b), "samples": len(sel),
+                "power_w_max": round(max(s_[3] for s_ in sel), 1), "scope": "timed windows only" if windows else "whole run"}
 
 
 # ---------------------------------------------------------------------------
@@ -252,76 +277,63 @@ def kernel_flops(name, st):
     return None
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=5, help="workload 1..5 (default: 5, the large multi-hot one)")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--vocab", type=int, default=0, help="override the number of pre-populated keys (config 5)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--graph", action="store_true",
-                    help="replay the step from a CUDA graph (launch-bound small workloads); per-kernel times then "
-                         "come from a separate, untimed eager pass")
-    ap.add_argument("--fused", action="store_true",
-                    help="use des_forward_fused (per-shard partials kept on chip) instead of partials + aggregate")
-    ap.add_argument("--cpu-budget", type=float, default=15.0)
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 0)
+TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on the benchmark's own batch with a "
+                  "4e6-key table (the 2e8-key table cannot be captured under multi-pass replay); constant, not measured "
+                  "in this run")
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    w = synth.config(args.config)
-    w = per_rank_workload(w, rank, world)           # every replica has its own data stream
 
-    # ------------------------------------------------------------------ reference arm: the CPU oracle
-    if args.impl == "reference":
-        if rank != 0:
-            return 0
-        ww = w
-        if ww.vocab > 20_000_000 or ww.prepopulate > 20_000_000:
-            # the sample touches a few thousand keys; their rows are a pure function of the id, so the
-            # oracle needs no pre-populated table to reproduce the first step of the full workload
-            pass
-        st = synth.Stream(ww)
-        b = st.next_batch()
-        g = synth.upstream_grads(ww, b.batch, 0)
-        budget = min(args.cpu_budget, 120.0 / max(1, args.steps + args.warmup))
-        v, bs, sec = time_oracle(ww, b, g, budget_s=budget, steps=max(1, args.steps), warmup=args.warmup)
-        cores = 1
-        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
-                "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                "config": {"workload": ww.name, "batch": ww.batch, "fields": ww.fields, "emb_dim": ww.emb_dim,
-                           "shards": ww.shards, "sample": f"first {bs} of {ww.batch} samples per step"},
-                "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                 "sample": f"first {bs} of {ww.batch} samples of one batch, table holding the keys it touches"},
-                "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-                "gpu_launches": 0}
-        print(json.dumps(line), flush=True)
-        return 0
+def build_table(w, cfg_index, batches, steps_total, prepop, dev):
+    """Table sized for the workload and the number of steps that will run on it; pre-populated (untimed)."""
+    import torch
+    from paper_1909_04823_b200.binding import DeviceBatch, Table
+    max_nnz = int(max(b.nnz for b in batches) * 1.02) + 1024
+    if cfg_index == 4:
+        max_rows = int(prepop + (steps_total + 2) * batches[0].nnz * w.p_new * 1.3) + 100000
+    elif cfg_index == 5:
+        max_rows = prepop
+    else:
+        max_rows = int(sum(len(np.unique(b.ids)) for b in batches) * (3 + steps_total)) + 100000
+        max_rows = min(max_rows, 40_000_000)
+    uniq0 = int(len(np.unique(batches[0].ids)))
+    max_uniq = min(max_nnz, int(uniq0 * 1.5) + 4096)
+    t = Table.for_workload(w, max_rows=max_rows, max_nnz=max(max_nnz, w.batch * w.fields), max_batch=w.batch,
+                           rows_per_shard=rows_per_shard(w, max_rows), max_uniq=max_uniq)
+    if w.hidden:
+        t.dense1_set(torch.from_numpy(synth.dense1_weights(w)).to(dev))
+    if prepop:
+        t0 = time.time()
+        per_call = w.batch * w.fields
+        stream = synth.Stream(w)
+        for ids in stream.prepopulation_ids(chunk=per_call * 8):
+            d_all = torch.from_numpy(ids.view(np.int64)).to(dev)
+            for lo in range(0, ids.size, per_call):
+                n = min(per_call, ids.size - lo)
+                pb = synth.prepopulation_batch(ids[lo:lo + n], w.fields)
+                t.find_or_insert(DeviceBatch(pb.offsets, d_all[lo:lo + n], None, pb.batch, dev), True)
+        t.check_status()
+        log(f"[bench] pre-populated {sum(t.size())} keys in {time.time() - t0:.1f}s")
+    return t
 
-    # ------------------------------------------------------------------ our arm
+
+def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want_e2e, want_cpu, profile_in_timed):
+    """Measures one workload.  modes: "eager" and / or "graph".  Returns a dict with one entry per mode
+    (step times of every repeat, per-kernel shares, dominant-kernel roofline) plus e2e / cpu_baseline."""
     import torch
     import torch.distributed as dist
-    from paper_1909_04823_b200.binding import DeviceBatch, Table
+    from paper_1909_04823_b200.binding import DeviceBatch
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the DES path has no CPU fallback")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dev = torch.device("cuda", local)
-    hbm_peak, tc_peak, peak_kind = measured_peaks()
+    rank, world, dev, sampler = ctx["rank"], ctx["world"], ctx["dev"], ctx["sampler"]
+    hbm_peak, tc_peak, peak_kind = ctx["peaks"]
 
-    # ---- size the table for the memory that is actually free
-    free_b, total_b = torch.cuda.mem_get_info()
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
     prepop = w.prepopulate
-    vocab = w.vocab
-    if args.config == 5:
+    if cfg_index == 5:
+        free_b, _ = torch.cuda.mem_get_info()
+        vocab = w.vocab
         if args.vocab:
             prepop = vocab = args.vocab
         per_key = 2 * (4 * w.emb_dim + 16) * 1.06 + 16 * 2.2      # rows + state + slots at load 0.5
@@ -331,38 +343,12 @@ def main():
             log(f"[bench] only {free_b / 1e9:.0f} GB free: table scaled to {prepop} keys")
         w = w.scaled(vocab=vocab, prepopulate=prepop)
     stream = synth.Stream(w)
-    n_batches = 2 if args.config != 4 else min(args.steps + args.warmup, 12)
+    steps_total = (steps * repeats + warmup + 3) * len(modes) + (steps if "graph" in modes else 0) + 16
+    n_batches = 2 if cfg_index != 4 else min(steps + warmup, 12)
     t0 = time.time()
     batches = [stream.next_batch() for _ in range(n_batches)]
     log(f"[bench] generated {n_batches} batches of {w.name}: nnz {batches[0].nnz} in {time.time() - t0:.1f}s")
-    max_nnz = int(max(b.nnz for b in batches) * 1.02) + 1024
-    if args.config == 4:
-        max_rows = int(prepop + (args.steps + args.warmup + 2) * batches[0].nnz * w.p_new * 1.3) + 100000
-    elif args.config == 5:
-        max_rows = prepop
-    else:
-        max_rows = int(sum(len(np.unique(b.ids)) for b in batches) * (3 + args.steps)) + 100000
-        max_rows = min(max_rows, 40_000_000)
-    uniq0 = int(len(np.unique(batches[0].ids)))
-    max_uniq = min(max_nnz, int(uniq0 * 1.5) + 4096)
-    t = Table.for_workload(w, max_rows=max_rows, max_nnz=max(max_nnz, w.batch * w.fields), max_batch=w.batch,
-                           rows_per_shard=rows_per_shard(w, max_rows), max_uniq=max_uniq)
-    if w.hidden:
-        t.dense1_set(torch.from_numpy(synth.dense1_weights(w)).to(dev))
-
-    # ---- pre-population (not timed)
-    if prepop:
-        t0 = time.time()
-        per_call = w.batch * w.fields
-        for ids in stream.prepopulation_ids(chunk=per_call * 8):
-            d_all = torch.from_numpy(ids.view(np.int64)).to(dev)
-            for lo in range(0, ids.size, per_call):
-                n = min(per_call, ids.size - lo)
-                pb = synth.prepopulation_batch(ids[lo:lo + n], w.fields)
-                db = DeviceBatch(pb.offsets, d_all[lo:lo + n], None, pb.batch, dev)
-                t.find_or_insert(db, True)
-        t.check_status()
-        log(f"[bench] pre-populated {sum(t.size())} keys in {time.time() - t0:.1f}s")
+    t = build_table(w, cfg_index, batches, steps_total, prepop, dev)
 
     B, F, k, S, H = w.batch, w.fields, w.emb_dim, w.shards, w.hidden
     dbs = [DeviceBatch.from_synth(b, dev) for b in batches]
@@ -387,165 +373,305 @@ def main():
             t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
         t.backward_update(w.ops, db, out_small, pooled, Z, gd.get("gL"), gd.get("gF"), gE, gZ, gE_work)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+    U = None
+    stats = None
 
-    sampler = ClockSampler(local) if rank == 0 else None     # sampling from the warm-up on, every 50 ms
-    for i in range(args.warmup):
+    def kernel_table(prof, n_steps):
+        per = {}
+        for name, ms in prof:
+            a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += ms
+        tot_k = sum(v[1] for v in per.values()) or 1.0
+        kernels = []
+        for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
+            by = kernel_bytes(name, stats)
+            fl = kernel_flops(name, stats)
+            avg = ms / n_
+            kernels.append({"kernel": name, "launches": n_, "ms_per_launch": round(avg, 4), "share": round(ms / tot_k, 4),
+                            "alg_gbs": None if by is None else round(by / avg / 1e6, 1),
+                            "tflops": None if fl is None else round(fl / avg / 1e9, 1)})
+        roofline = None
+        for top in kernels:      # the kernel with the largest share of the timed region that has a byte / flop model
+            if top["alg_gbs"] is not None:
+                tr = NCU_DRAM_TRAFFIC.get((w.name.split("_")[0], top["kernel"]))
+                roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
+                            "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4), "traffic": tr,
+                            "traffic_source": TRAFFIC_SOURCE if tr is not None else None,
+                            "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
+                break
+            if top["tflops"] is not None:
+                roofline = {"bound": "tensor", "kernel": top["kernel"], "achieved": top["tflops"], "peak": tc_peak,
+                            "unit": "TFLOP/s", "frac": round(top["tflops"] / tc_peak, 4), "traffic": None,
+                            "peak_kind": f"of {peak_kind} (sustained bf16)", "ms_per_launch": top["ms_per_launch"],
+                            "share": top["share"]}
+                break
+        step_bytes = sum((kernel_bytes(kk["kernel"], stats) or 0) * kk["launches"] for kk in kernels) / max(1, n_steps)
+        return kernels, roofline, step_bytes
+
+    results = {}
+    windows = []
+    done_steps = 0
+    for i in range(warmup):
         step(i)
+    done_steps += warmup
     t.check_status()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    graphs = None
-    if args.graph:
-        # one graph per batch; the step has no host synchronisation and allocates nothing
-        graphs = []
-        for i in range(len(dbs)):
-            gph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gph):
-                step(i)
-            graphs.append(gph)
-        for i in range(max(args.warmup, 3)):
-            graphs[i % len(graphs)].replay()
-        barrier()
-    launches0 = t.launch_count()
-    if graphs is None:
-        t.profile_enable(True)
-    e0.record()
-    for i in range(args.steps):
-        if graphs is None:
-            step(args.warmup + i)
-        else:
-            graphs[(args.warmup + i) % len(graphs)].replay()
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else None
-    if graphs is not None:
-        # kernel shares from an eager pass outside the timed region; launches per step counted there too
-        t.profile_enable(True)
-        launches0 = t.launch_count()
-        for i in range(args.steps):
-            step(args.warmup + i)
-        barrier()
-    prof = t.profile_read()
-    t.profile_enable(False)
-    launches = t.launch_count() - launches0
-    t.check_status()
-    ms_total = max_over_ranks(ms_total, world, dev)
-    ms_step = ms_total / args.steps
-    value = job_throughput(B, world, ms_step)
-
-    # ---- per-kernel shares and the roofline of the dominant kernel
-    per = {}
-    for name, ms in prof:
-        a = per.setdefault(name, [0, 0.0]); a[0] += 1; a[1] += ms
     U = int(dbs[0].n_uniq.item())
     stats = dict(nnz=batches[0].nnz, B=B, F=F, k=k, S=S, H=H, U=U, ops=w.ops,
                  adagrad=(w.optimizer == synth.OPT_ADAGRAD), rep_rows=0,
                  super=(k > 28 and batches[0].nnz >= (1 << 20) and batches[0].vals is None),
                  shift=shift_of(batches[0].nnz), new_keys=(w.p_new > 0 or not w.prepopulate))
-    tot_k = sum(v[1] for v in per.values()) or 1.0
-    kernels = []
-    for name, (n_, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
-        by = kernel_bytes(name, stats)
-        fl = kernel_flops(name, stats)
-        avg = ms / n_
-        kernels.append({"kernel": name, "launches": n_, "ms_per_launch": round(avg, 4), "share": round(ms / tot_k, 4),
-                        "alg_gbs": None if by is None else round(by / avg / 1e6, 1),
-                        "tflops": None if fl is None else round(fl / avg / 1e9, 1)})
-    # the kernel with the largest share of the timed region that has a byte / flop model
-    roofline = None
-    for top in kernels:
-        if top["alg_gbs"] is not None:
-            roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
-                        "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4),
-                        "traffic": NCU_DRAM_TRAFFIC.get((w.name.split("_")[0], top["kernel"])),
-                        "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
-            break
-        if top["tflops"] is not None:
-            roofline = {"bound": "tensor", "kernel": top["kernel"], "achieved": top["tflops"], "peak": tc_peak,
-                        "unit": "TFLOP/s", "frac": round(top["tflops"] / tc_peak, 4), "traffic": None,
-                        "peak_kind": f"of {peak_kind} (sustained bf16)", "ms_per_launch": top["ms_per_launch"],
-                        "share": top["share"]}
-            break
-    step_bytes = sum((kernel_bytes(kk["kernel"], stats) or 0) * kk["launches"] for kk in kernels) / args.steps
-    row_b = 4 * k + 16
-    extra = max(0, batches[0].nnz - U)                   # occurrences beyond the first of their key
-    occ_bytes = step_bytes + extra * ((row_b if (w.ops & (OP_LR | OP_FM)) else 0)
-                                      + (4 * k if (w.ops & (OP_POOL | OP_DENSE1)) else 0) + row_b)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for mode in modes:
+        graphs = None
+        if mode == "graph":
+            graphs = []                       # one graph per batch; the step has no host synchronisation and allocates nothing
+            for i in range(len(dbs)):
+                gph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gph):
+                    step(i)
+                graphs.append(gph)
+            for i in range(max(warmup, 3)):
+                graphs[i % len(graphs)].replay()
+            barrier()
+        prof_live = graphs is None and profile_in_timed
+        launches0 = t.launch_count()
+        if prof_live:
+            t.profile_enable(True)
+        rep_ms, rep_clk, prof = [], [], []
+        for r in range(repeats):
+            barrier()
+            h0 = time.perf_counter()
+            e0.record()
+            for i in range(steps):
+                if graphs is None:
+                    step(done_steps + i)
+                else:
+                    graphs[(done_steps + i) % len(graphs)].replay()
+            e1.record()
+            barrier()
+            h1 = time.perf_counter()
+            done_steps += steps
+            rep_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev) / steps)
+            windows.append((h0, h1))
+            if sampler:
+                rep_clk.append(sampler.window(h0, h1))
+            if prof_live:
+                prof += t.profile_read()
+        n_prof_steps = steps * repeats
+        if not prof_live:
+            # kernel shares from an eager pass outside the timed region; launches per step counted there too
+            t.profile_enable(True)
+            launches0 = t.launch_count()
+            for i in range(steps):
+                step(done_steps + i)
+            done_steps += steps
+            barrier()
+            prof = t.profile_read()
+            n_prof_steps = steps
+        t.profile_enable(False)
+        launches = (t.launch_count() - launches0) // max(1, (repeats if prof_live else 1))
+        t.check_status()
+        kernels, roofline, step_bytes = kernel_table(prof, n_prof_steps)
+        ms_step = float(np.median(rep_ms))
+        results[mode] = {"ms_per_step": ms_step, "value": job_throughput(B, world, ms_step),
+                         "repeats": {"n": repeats, "steps_each": steps, "ms_per_step": [round(v, 4) for v in rep_ms],
+                                     "min": round(min(rep_ms), 4), "max": round(max(rep_ms), 4),
+                                     "sm_mhz": [c["sm_mhz"] for c in rep_clk],
+                                     "reasons": sorted({r_ for c in rep_clk for r_ in c["reasons"]})},
+                         "kernels": kernels, "roofline": roofline, "step_bytes": step_bytes, "gpu_launches": int(launches)}
 
     # ---- end to end from pinned host buffers
     e2e = None
-    try:
-        if args.no_e2e:
-            raise RuntimeError("skipped by --no-e2e")
-        hb = batches[0]
-        h_off = torch.from_numpy(hb.offsets).pin_memory()
-        h_ids = torch.from_numpy(hb.ids.view(np.int64)).pin_memory()
-        h_out = [torch.empty((B, k + 4), dtype=torch.float32).pin_memory() for _ in range(2)]
-        kw = dict(d_pooled=pooled, d_Z=Z, gL=gd.get("gL"), gF=gd.get("gF"), gE=gE, gZ=gZ, gE_work=gE_work)
-
-        def run_blocking(n):
-            for i in range(n):
-                t.step_host(w.ops, B, hb.nnz, h_off, h_ids, None, h_out[i & 1], **kw)
-
-        def run_pipelined(n):          # the copy of step i+1 overlaps the kernels of step i
-            prev = None
-            for i in range(n):
-                tk = t.step_host_submit(w.ops, B, hb.nnz, h_off, h_ids, None, h_out[i & 1], **kw)
-                if prev is not None:
-                    t.step_host_wait(prev)
-                prev = tk
-            t.step_host_wait(prev)
-
-        n_e2e = max(3, min(args.steps, 10))
-        ms_mode = {}
-        for name, fn in (("blocking", run_blocking), ("pipelined", run_pipelined)):
-            fn(max(1, min(args.warmup, 3)))
-            barrier()
-            e0.record()
-            fn(n_e2e)
-            e1.record()
-            barrier()
-            ms_mode[name] = max_over_ranks(e0.elapsed_time(e1) / n_e2e, world, dev)
-        ms_e = ms_mode["pipelined"]
-        e2e = {"value": job_throughput(B, world, ms_e), "unit": UNIT, "ms_per_step": ms_e,
-               "mode": "des_step_host_submit / des_step_host_wait, two steps in flight",
-               "blocking_ms_per_step": ms_mode["blocking"],
-               "h2d_bytes_per_step": int(h_off.numel() * 4 + h_ids.numel() * 8),
-               "d2h_bytes_per_step": int(h_out[0].numel() * 4)}
-    except Exception as ex:  # keep the device-resident number even if the host path fails
-        log(f"[bench] e2e failed: {ex!r}")
-    t.check_status()
-
-    # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only)
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if want_e2e:
         try:
-            v, bs, sec = time_oracle(w, batches[0], g_host, budget_s=args.cpu_budget)
+            hb = batches[0]
+            h_off = torch.from_numpy(hb.offsets).pin_memory()
+            h_ids = torch.from_numpy(hb.ids.view(np.int64)).pin_memory()
+            h_out = [torch.empty((B, k + 4), dtype=torch.float32).pin_memory() for _ in range(2)]
+            kw = dict(d_pooled=pooled, d_Z=Z, gL=gd.get("gL"), gF=gd.get("gF"), gE=gE, gZ=gZ, gE_work=gE_work)
+
+            def run_blocking(n):
+                for i in range(n):
+                    t.step_host(w.ops, B, hb.nnz, h_off, h_ids, None, h_out[i & 1], **kw)
+
+            def run_pipelined(n):          # the copy of step i+1 overlaps the kernels of step i
+                prev = None
+                for i in range(n):
+                    tk = t.step_host_submit(w.ops, B, hb.nnz, h_off, h_ids, None, h_out[i & 1], **kw)
+                    if prev is not None:
+                        t.step_host_wait(prev)
+                    prev = tk
+                t.step_host_wait(prev)
+
+            n_e2e = max(3, min(steps, 10))
+            ms_mode = {}
+            for name, fn in (("blocking", run_blocking), ("pipelined", run_pipelined)):
+                fn(max(1, min(warmup, 3)))
+                barrier()
+                e0.record()
+                fn(n_e2e)
+                e1.record()
+                barrier()
+                ms_mode[name] = max_over_ranks(e0.elapsed_time(e1) / n_e2e, world, dev)
+            ms_e = ms_mode["pipelined"]
+            e2e = {"value": job_throughput(B, world, ms_e), "unit": UNIT, "ms_per_step": ms_e,
+                   "mode": "des_step_host_submit / des_step_host_wait from pinned host buffers, two steps in flight; "
+                           "copied every step: offsets + ids host to device, out_small [B][k+4] back; resident on the "
+                           "device: the upstream gradients gL / gF / gE (they come from the rest of the model) and the "
+                           "pooled output (its consumer)",
+                   "blocking_ms_per_step": ms_mode["blocking"],
+                   "h2d_bytes_per_step": int(h_off.numel() * 4 + h_ids.numel() * 8),
+                   "d2h_bytes_per_step": int(h_out[0].numel() * 4)}
+        except Exception as ex:  # keep the device-resident number even if the host path fails
+            log(f"[bench] e2e failed: {ex!r}")
+        t.check_status()
+
+    # ---- CPU oracle on a bounded sample (rank 0, single GPU runs only): one core, then all cores
+    cpu = None
+    if want_cpu:
+        try:
+            import oracle
+            v, bs, sec = time_oracle(w, batches[0], g_host, budget_s=args.cpu_budget * 0.6)
             cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": f"first {bs} of {B} samples of one batch ({sec:.1f} s), table holding the keys it touches"}
+            try:
+                n_thr = oracle.num_threads(True)
+                v2, bs2, sec2 = time_oracle(w, batches[0], g_host, budget_s=args.cpu_budget * 0.4, omp=True)
+                cpu["all_cores"] = {"value": v2, "unit": UNIT, "cores": n_thr, "host_cpus": os.cpu_count(),
+                                    "kind": "oracle, same source built with -fopenmp",
+                                    "sample": f"first {bs2} of {B} samples of one batch ({sec2:.1f} s)"}
+            except Exception as ex:
+                log(f"[bench] all-cores cpu baseline failed: {ex!r}")
         except Exception as ex:
             log(f"[bench] cpu baseline failed: {ex!r}")
 
+    table_keys = sum(t.size())
+    t.close()
+    del t
+    torch.cuda.empty_cache()
+    return dict(w=w, results=results, e2e=e2e, cpu=cpu, windows=windows, nnz=batches[0].nnz, U=U, table_keys=table_keys,
+                l2_note="inputs larger than L2 (no flush)" if batches[0].nnz * 8 > 126e6 else
+                        "small workload: inputs fit in L2, two batches alternate, no flush")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=5, help="the --steps region is timed this many times back to back")
+    ap.add_argument("--config", type=int, default=5, help="workload 1..5 (default: 5, the large multi-hot one)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--vocab", type=int, default=0, help="override the number of pre-populated keys (config 5)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-side-configs", action="store_true",
+                    help="skip the short eager / graph-replay runs of the other four workloads")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the step from a CUDA graph (launch-bound small workloads); per-kernel times then "
+                         "come from a separate, untimed eager pass")
+    ap.add_argument("--fused", action="store_true",
+                    help="use des_forward_fused (per-shard partials kept on chip) instead of partials + aggregate")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    args.repeats = max(args.repeats, 1)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = synth.config(args.config)
+    w = per_rank_workload(w, rank, world)           # every replica has its own data stream
+
+    # ------------------------------------------------------------------ reference arm: the CPU oracle
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        # the sample touches a few thousand keys; their rows are a pure function of the id, so the oracle
+        # needs no pre-populated table to reproduce the first step of the full workload
+        st = synth.Stream(w)
+        b = st.next_batch()
+        g = synth.upstream_grads(w, b.batch, 0)
+        budget = min(args.cpu_budget, 120.0 / max(1, args.steps + args.warmup))
+        v, bs, sec = time_oracle(w, b, g, budget_s=budget, steps=max(1, args.steps), warmup=args.warmup)
+        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": {"workload": w.name, "batch": w.batch, "fields": w.fields, "emb_dim": w.emb_dim,
+                           "shards": w.shards, "sample": f"first {bs} of {w.batch} samples per step"},
+                "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "host_cpus": os.cpu_count(), "kind": "oracle",
+                                 "sample": f"first {bs} of {w.batch} samples of one batch, table holding the keys it touches"},
+                "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line), flush=True)
+        return 0
+
+    # ------------------------------------------------------------------ our arm
+    import torch
+    import torch.distributed as dist
+    from paper_1909_04823_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DES path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    sampler = ClockSampler(local) if rank == 0 else None     # every 20 ms, from here to the end of the timed regions
+    ctx = dict(rank=rank, world=world, dev=dev, sampler=sampler, peaks=measured_peaks())
+    hbm_peak = ctx["peaks"][0]
+
+    # ---- the other workloads, short (single-GPU default run only): eager and CUDA-graph replay
+    side = []
+    if world == 1 and not args.no_side_configs and args.config == 5 and not args.graph:
+        for ci in (1, 2, 3, 4):
+            try:
+                r = run_workload(args, ci, synth.config(ci), ctx, steps=20 if ci < 4 else 6, warmup=3, repeats=3,
+                                 modes=["eager", "graph"], want_e2e=False, want_cpu=False, profile_in_timed=False)
+                for mode in ("eager", "graph"):
+                    m = r["results"][mode]
+                    rf = m["roofline"] or {}
+                    side.append({"workload": r["w"].name, "launch": mode, "ms_per_step": round(m["ms_per_step"], 4),
+                                 "value": round(m["value"], 1), "unit": UNIT, "repeats_ms": m["repeats"]["ms_per_step"],
+                                 "nnz_per_step": r["nnz"], "unique_keys_per_step": r["U"],
+                                 "dominant_kernel": rf.get("kernel"), "dominant_share": rf.get("share"),
+                                 "dominant_achieved": rf.get("achieved"), "dominant_unit": rf.get("unit"),
+                                 "dominant_frac": rf.get("frac"), "gpu_launches_per_step": m["gpu_launches"] // max(1, 20 if ci < 4 else 6)})
+            except Exception as ex:
+                log(f"[bench] side run of config {ci} failed: {ex!r}")
+                side.append({"workload": f"config {ci}", "error": repr(ex)})
+
+    mode = "graph" if args.graph else "eager"
+    r = run_workload(args, args.config, w, ctx, steps=args.steps, warmup=args.warmup, repeats=args.repeats, modes=[mode],
+                     want_e2e=not args.no_e2e, want_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline),
+                     profile_in_timed=True)
+    clocks = sampler.stop(r["windows"]) if sampler else None
+    m = r["results"][mode]
+    w = r["w"]
+    ms_step = m["ms_per_step"]
+    B, F, k, S = w.batch, w.fields, w.emb_dim, w.shards
+    step_bytes = m["step_bytes"]
+    row_b = 4 * k + 16
+    extra = max(0, r["nnz"] - r["U"])                    # occurrences beyond the first of their key
+    occ_bytes = step_bytes + extra * ((row_b if (w.ops & (OP_LR | OP_FM)) else 0)
+                                      + (4 * k if (w.ops & (OP_POOL | OP_DENSE1)) else 0) + row_b)
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": w.name, "batch": B, "fields": F, "emb_dim": k, "shards": S,
-                           "nnz_per_step": batches[0].nnz, "unique_keys_per_step": U, "table_keys": sum(t.size()),
+                           "nnz_per_step": r["nnz"], "unique_keys_per_step": r["U"], "table_keys": r["table_keys"],
                            "ops": w.ops, "optimizer": "adagrad" if w.optimizer else "sgd",
                            "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
                            "launch": "CUDA graph replay" if args.graph else "eager",
                            "forward": "fused (per-shard partials on chip)" if args.fused else
                                       "per-shard partials materialised, then aggregated",
-                           "l2": "inputs larger than L2 (no flush)" if batches[0].nnz * 8 > 126e6 else
-                                 "small workload: inputs fit in L2, two batches alternate, no flush"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline,
+                           "tensor_core_gemm": bool(binding.uses_tensor_cores()),
+                           "l2": r["l2_note"]},
+                "timing": "ms_per_step = median over `repeats.n` back-to-back timings of --steps steps each",
+                "repeats": m["repeats"],
+                "clocks": clocks, "e2e": r["e2e"], "gpu_launches": int(m["gpu_launches"]),
+                "roofline": m["roofline"],
                 "hbm": {"alg_bytes_per_step": int(step_bytes), "alg_gbs": round(step_bytes / ms_step / 1e6, 1),
                         "frac_of_measured_copy": round(step_bytes / ms_step / 1e6 / hbm_peak, 4),
                         "frac_of_nominal_8000": round(step_bytes / ms_step / 1e6 / 8000.0, 4),
@@ -553,11 +679,10 @@ def main():
                         # gathers (twice: per-shard partials and pooling) and scatters its own row; these are
                         # mostly L1 / L2 hits in a skewed batch, so this is not an HBM figure
                         "occ_bytes_per_step": int(occ_bytes), "occ_gbs": round(occ_bytes / ms_step / 1e6, 1)},
-                "kernels": kernels, "cpu_baseline": cpu}
+                "kernels": m["kernels"], "cpu_baseline": r["cpu"], "configs": side}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
-    t.close()
     return 0
 
 

@@ -38,6 +38,18 @@
  *   as void*; NULL = the legacy default stream).  Only des_table_status,
  *   des_table_size, des_table_export, des_dense1_get/set on host pointers,
  *   des_step_host and des_step_host_wait synchronise.
+ * - One table, one order: every call on a table reuses workspace that the table
+ *   owns (routing arrays, the gradient buffer, hot-key lists), so all calls on
+ *   one table must be ordered — the same stream, or streams ordered by events.
+ *   Two calls on one table that overlap on the GPU race.  Different tables are
+ *   independent.  A table belongs to the device that was current when it was
+ *   created; calls with another device current return DES_ERR_INVALID_ARG where
+ *   the library can tell, and are undefined otherwise.
+ * - Reproducibility: the integer outputs (shards, rows, unique indices, the key
+ *   set) and the forward's floating-point results are identical from run to
+ *   run.  The backward sums a key's gradient terms with floating-point atomics
+ *   in an order that changes from run to run: updated weights agree between
+ *   runs within rounding (the tolerance of the parity tests), not bit for bit.
  * - Device-side problems (reserved key, full shard) never fault: the
  *   offending occurrences get row DES_ROW_NONE, are skipped by every later
  *   kernel, and a sticky error word is raised that des_table_status returns.
@@ -66,7 +78,9 @@ typedef enum {
   DES_ERR_UNSUPPORTED = 4,
   DES_ERR_CUDA = 5,          /* a CUDA runtime call failed, or no device                */
   DES_ERR_NOT_FOUND = 6,
-  DES_ERR_TOO_LARGE = 7      /* problem exceeds the fixed scratch of a no-allocation entry point */
+  DES_ERR_TOO_LARGE = 7,     /* problem exceeds the fixed scratch of a no-allocation entry point */
+  DES_ERR_RANGE = 8          /* checking build only (libdes_debug.so): a kernel met an index outside the
+                                table's bounds, skipped the access and raised this (sticky, device-side) */
 } des_status_t;
 
 /* operator kind bitmask */
@@ -207,8 +221,11 @@ des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_
 
 /* Aggregation (+) over shards in the fixed order s = 0..S-1 (Eq. 1) and the
  * substitution operator F (Algorithm 1, R = F(f_1..f_m)): out_small from
- * part_small; Z from pooled and W1 (K loop in shard order) or, when
- * part->part_dense is given, P_s materialised first and Z = sum_s P_s. */
+ * part_small; Z from pooled and W1 in one product on the tensor cores (its K loop
+ * runs over the columns of pooled in field order; under the FIELD partition that
+ * visits every shard's block once, not shard by shard — inside the 2e-2 bound of
+ * bf16 operands) or, when part->part_dense is given, P_s materialised first (K
+ * slices in shard order, CUDA-core kernel) and Z = sum_s P_s. */
 des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* batch,
                            const des_partials_t* part, const des_outputs_t* out, void* stream);
 
@@ -413,6 +430,15 @@ des_status_t des_profile_read(des_table_t* t, const char** h_names, float* h_ms,
 
 /* Number of kernel launches the library has issued for this table so far. */
 uint64_t des_table_launch_count(des_table_t* t);
+
+/* 1 when the library was built with the tcgen05 tensor-core GEMMs of the first dense
+ * layer (Section 4.3), 0 when the header tree they need was missing at build time and
+ * only the CUDA-core kernel exists.  des_table_uses_tensor_cores: 1 when this table's
+ * first layer runs on them (built in, and F*k and H multiples of 8), else 0. */
+int des_build_has_tensor_cores(void);
+int des_table_uses_tensor_cores(des_table_t* t);
+/* 1 in the checking build (libdes_debug.so), 0 in the product library. */
+int des_build_is_debug(void);
 
 const char* des_status_string(des_status_t s);
 

@@ -22,14 +22,15 @@ KEY_EMPTY = 0xFFFFFFFFFFFFFFFF
 
 STATUS = {0: "DES_OK", 1: "DES_ERR_INVALID_ARG", 2: "DES_ERR_RESERVED_KEY", 3: "DES_ERR_CAPACITY",
           4: "DES_ERR_UNSUPPORTED", 5: "DES_ERR_CUDA", 6: "DES_ERR_NOT_FOUND",
-          7: "DES_ERR_TOO_LARGE"}
+          7: "DES_ERR_TOO_LARGE", 8: "DES_ERR_RANGE"}
 
 EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_forward_partials",
            "des_aggregate", "des_rank_partial", "des_aggregate_ranks", "des_forward_fused", "des_backward_update", "des_dense1_set", "des_dense1_get", "des_dense1_get_state", "des_dense1_set_state", "des_dense1_forward_noalloc", "des_table_status",
            "des_table_size", "des_table_row_base", "des_table_export", "des_table_read_rows", "des_table_write_rows",
            "des_table_read_state2", "des_table_write_state2",
            "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_cross_forward", "des_cross_backward",
-           "des_cross_workspace_floats", "des_comm_volume", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string"]
+           "des_cross_workspace_floats", "des_comm_volume", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string",
+           "des_build_has_tensor_cores", "des_table_uses_tensor_cores", "des_build_is_debug"]
 
 
 class des_comm_model_t(C.Structure):
@@ -83,66 +84,90 @@ class des_grads_t(C.Structure):
 
 
 _lib = None
+_lib_debug = None
+_use_debug = False
 
 
 def lib_path() -> str:
-    return _build.LIB
+    return _build.LIB_DEBUG if _use_debug else _build.LIB
+
+
+def use_debug_library(on: bool = True) -> bool:
+    """Tables created from now on use the checking build (libdes_debug.so: index range checks in every
+    gather / scatter / probe, test hooks) instead of the product library.  Returns the previous setting."""
+    global _use_debug
+    prev, _use_debug = _use_debug, bool(on)
+    return prev
+
+
+def uses_tensor_cores() -> bool:
+    """True when the loaded library carries the tcgen05 GEMMs of the first dense layer."""
+    return bool(load().des_build_has_tensor_cores())
 
 
 def load():
     """Loads (building first if the sources are newer) the CUDA library."""
-    global _lib
+    global _lib, _lib_debug
+    if _use_debug:
+        if _lib_debug is None:
+            _lib_debug = _declare(C.CDLL(_build.build(debug=True)))
+        return _lib_debug
     if _lib is None:
-        path = _build.build()
-        L = C.CDLL(path)
-        for name in EXPORTS:
-            getattr(L, name)  # fail loudly on a missing symbol
-        L.des_table_create.argtypes = [C.POINTER(des_config_t), C.POINTER(C.c_void_p)]
-        L.des_table_destroy.argtypes = [C.c_void_p]
-        L.des_find_or_insert.argtypes = [C.c_void_p, C.POINTER(des_batch_t), C.c_int, C.c_void_p]
-        L.des_forward_partials.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
-                                           C.POINTER(des_partials_t), C.c_void_p]
-        L.des_aggregate.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
-                                    C.POINTER(des_outputs_t), C.c_void_p]
-        L.des_forward_fused.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
-                                        C.POINTER(des_outputs_t), C.c_void_p]
-        L.des_backward_update.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
-                                          C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
-        L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_dense1_get.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_dense1_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_dense1_set_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_dense1_forward_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
-        L.des_table_status.argtypes = [C.c_void_p]
-        L.des_table_size.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
-        L.des_table_row_base.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
-        L.des_table_export.argtypes = [C.c_void_p] + [C.c_void_p] * 7 + [C.c_uint64, C.POINTER(C.c_uint64)]
-        L.des_table_read_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
-        L.des_table_write_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
-        L.des_table_read_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_table_write_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_step_host.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
-                                    C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
-                                    C.c_void_p]
-        L.des_step_host_submit.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
-                                           C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
-                                           C.c_void_p, C.POINTER(C.c_int32)]
-        L.des_step_host_wait.argtypes = [C.c_void_p, C.c_int32]
-        L.des_rank_partial.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_aggregate_ranks.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
-        L.des_cross_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 8
-        L.des_cross_backward.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 11
-        L.des_cross_workspace_floats.argtypes = [C.c_int32, C.c_int32]
-        L.des_cross_workspace_floats.restype = C.c_int64
-        L.des_comm_volume.argtypes = [C.POINTER(des_comm_model_t), C.POINTER(des_comm_volume_t)]
-        L.des_table_launch_count.argtypes = [C.c_void_p]
-        L.des_profile_enable.argtypes = [C.c_void_p, C.c_int]
-        L.des_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int,
-                                       C.POINTER(C.c_int)]
-        L.des_table_launch_count.restype = C.c_uint64
-        L.des_status_string.restype = C.c_char_p
-        _lib = L
+        _lib = _declare(C.CDLL(_build.build()))
     return _lib
+
+
+def _declare(L):
+    for name in EXPORTS:
+        getattr(L, name)  # fail loudly on a missing symbol
+    L.des_table_create.argtypes = [C.POINTER(des_config_t), C.POINTER(C.c_void_p)]
+    L.des_table_destroy.argtypes = [C.c_void_p]
+    L.des_find_or_insert.argtypes = [C.c_void_p, C.POINTER(des_batch_t), C.c_int, C.c_void_p]
+    L.des_forward_partials.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
+                                       C.POINTER(des_partials_t), C.c_void_p]
+    L.des_aggregate.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
+                                C.POINTER(des_outputs_t), C.c_void_p]
+    L.des_forward_fused.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t), C.POINTER(des_partials_t),
+                                    C.POINTER(des_outputs_t), C.c_void_p]
+    L.des_backward_update.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(des_batch_t),
+                                      C.POINTER(des_outputs_t), C.POINTER(des_grads_t), C.c_void_p]
+    L.des_dense1_set.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_dense1_get.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_dense1_get_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_dense1_set_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_dense1_forward_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    L.des_table_status.argtypes = [C.c_void_p]
+    L.des_table_size.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    L.des_table_row_base.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    L.des_table_export.argtypes = [C.c_void_p] + [C.c_void_p] * 7 + [C.c_uint64, C.POINTER(C.c_uint64)]
+    L.des_table_read_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
+    L.des_table_write_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int64] + [C.c_void_p] * 4 + [C.c_void_p]
+    L.des_table_read_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_table_write_state2.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_step_host.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
+                                C.c_void_p]
+    L.des_step_host_submit.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int64, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.POINTER(des_grads_t), C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.POINTER(C.c_int32)]
+    L.des_step_host_wait.argtypes = [C.c_void_p, C.c_int32]
+    L.des_rank_partial.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_aggregate_ranks.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.des_cross_forward.argtypes = [C.c_int32, C.c_int32, C.c_int32] + [C.c_void_p] * 8
+    L.des_cross_backward.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 11
+    L.des_cross_workspace_floats.argtypes = [C.c_int32, C.c_int32]
+    L.des_cross_workspace_floats.restype = C.c_int64
+    L.des_comm_volume.argtypes = [C.POINTER(des_comm_model_t), C.POINTER(des_comm_volume_t)]
+    L.des_table_launch_count.argtypes = [C.c_void_p]
+    L.des_profile_enable.argtypes = [C.c_void_p, C.c_int]
+    L.des_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_char_p), C.POINTER(C.c_float), C.c_int,
+                                   C.POINTER(C.c_int)]
+    L.des_table_launch_count.restype = C.c_uint64
+    L.des_status_string.restype = C.c_char_p
+    L.des_build_has_tensor_cores.argtypes = []
+    L.des_table_uses_tensor_cores.argtypes = [C.c_void_p]
+    L.des_build_is_debug.argtypes = []
+    return L
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -331,6 +356,9 @@ class Table:
         out = (C.c_uint64 * (self.S + 1))()
         self._check(self.L.des_table_row_base(self.h, out), "des_table_row_base")
         return [int(v) for v in out]
+
+    def uses_tensor_cores(self) -> bool:
+        return bool(self.L.des_table_uses_tensor_cores(self.h))
 
     def launch_count(self) -> int:
         return int(self.L.des_table_launch_count(self.h))

@@ -263,6 +263,10 @@ extern "C" des_status_t des_dense1_forward_noalloc(des_table_t* t, const float* 
   int dev = 0;
   DES_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return DES_ERR_UNSUPPORTED;
+  // the scratch array is this device's copy; the table's weights must live on the same device
+  if (dev != t->device) return DES_ERR_INVALID_ARG;
+  // (two host threads making the first call on a device at the same time both store the same address:
+  // the unlocked write below is benign)
   if (!g_noalloc_ptr[dev]) {          // set-up, once per device, with that device current
     float* p = nullptr;
     if (cudaGetSymbolAddress((void**)&p, g_noalloc_partials) != cudaSuccess || !p) { cudaGetLastError(); return DES_ERR_CUDA; }

@@ -90,12 +90,15 @@ extern "C" const char* des_status_string(des_status_t s) {
     case DES_ERR_CUDA: return "CUDA runtime error or no device";
     case DES_ERR_NOT_FOUND: return "not found";
     case DES_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
+    case DES_ERR_RANGE: return "checking build: an index outside the table's bounds was met and skipped";
   }
   return "?";
 }
 
 extern "C" des_status_t des_table_destroy(des_table_t* t) {
   if (!t) return DES_OK;
+  int caller_dev = -1;                                   // the caller's current device is put back at the end
+  if (cudaGetDevice(&caller_dev) != cudaSuccess) { cudaGetLastError(); caller_dev = -1; }
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->A2, t->acc2W1, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
@@ -109,7 +112,9 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   }
   if (t->prof_ev) { for (int i = 0; i < DES_PROF_MAX; ++i) cudaEventDestroy(t->prof_ev[i]); delete[] t->prof_ev; }
   delete[] t->prof_name;
+  const int own_dev = t->device;
   delete t;
+  if (caller_dev >= 0 && caller_dev != own_dev) cudaSetDevice(caller_dev);
   return DES_OK;
 }
 
@@ -143,10 +148,12 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   cudaDeviceGetAttribute(&t->sm_count, cudaDevAttrMultiProcessorCount, dev);
   DevMeta hm; memset(&hm, 0, sizeof(hm));
   hm.scratch_base = 0xFFFFFFFFu;                      // top of the insert calls' scratch range (Slot::first_occ)
-  if (const char* e = getenv("DES_DEBUG_SCRATCH_BASE")) {   // tests: start near the end of the range, so that
-    const unsigned long long v = strtoull(e, nullptr, 0);   // the rare reset pass runs within a few calls
-    if (v >= t->max_nnz && v <= 0xFFFFFFFFull) hm.scratch_base = (uint32_t)v;
+#ifdef DES_DEBUG
+  if (const char* e = getenv("DES_DEBUG_SCRATCH_BASE")) {   // checking build only — tests start near the end of the
+    const unsigned long long v = strtoull(e, nullptr, 0);   // range, so that the rare reset pass runs within a few calls
+    if (v >= (unsigned long long)t->max_nnz && v <= 0xFFFFFFFFull) hm.scratch_base = (uint32_t)v;
   }
+#endif
   uint64_t rows = 0, slots = 0;
   const uint32_t world = c.shard_world > 1 ? c.shard_world : 1;
   uint32_t owned = 0;
@@ -261,6 +268,22 @@ extern "C" des_status_t des_table_row_base(des_table_t* t, uint64_t* h) {
 }
 
 extern "C" uint64_t des_table_launch_count(des_table_t* t) { return t ? t->launches : 0; }
+
+extern "C" int des_build_has_tensor_cores(void) {
+#ifdef DES_NO_CUTLASS
+  return 0;
+#else
+  return 1;
+#endif
+}
+extern "C" int des_table_uses_tensor_cores(des_table_t* t) { return (t && t->H && t->use_tc && des_build_has_tensor_cores()) ? 1 : 0; }
+extern "C" int des_build_is_debug(void) {
+#ifdef DES_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 __global__ void export_kernel(const Slot* __restrict__ slots, unsigned long long nslots, const DevMeta* __restrict__ meta,
                               int S, int k, int stride, const float* __restrict__ W, const float* __restrict__ A,

@@ -326,8 +326,15 @@ def test_insert_scratch_range_wraps(monkeypatch):
     st = synth.Stream(w)
     first = st.next_batch()
     max_nnz = int(first.nnz * 1.5) + 1024
+    # the starting point of the range can only be moved in the checking build of the library
+    from paper_1909_04823_b200 import binding
     monkeypatch.setenv("DES_DEBUG_SCRATCH_BASE", str(max_nnz + 3 * first.nnz))
-    p = _pair(w, 60000, max_nnz=max_nnz)
+    prev = binding.use_debug_library(True)
+    try:
+        p = _pair(w, 60000, max_nnz=max_nnz)
+        assert p.t.L.des_build_is_debug() == 1
+    finally:
+        binding.use_debug_library(prev)
     monkeypatch.delenv("DES_DEBUG_SCRATCH_BASE")
     try:
         b = first
