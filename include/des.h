@@ -230,11 +230,19 @@ des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* batc
                            const des_partials_t* part, const des_outputs_t* out, void* stream);
 
 /* des_forward_partials + des_aggregate in one call, with the per-shard partial
- * results of LR / FM kept on chip: every sample's partials are formed shard by
- * shard in registers, aggregated in the same fixed shard order and passed
- * through F without ever being written (Algorithm 1 with the aggregation made
- * an on-chip reduction).  Results are bit-identical to the two-call path.
- * part->part_small may be NULL (or given, to receive the partials as well);
+ * results of LR / FM kept on chip (Algorithm 1 with the aggregation made an
+ * on-chip reduction).  Two forms:
+ *  - `ops` holds LR / FM only, or part->part_small is given (to receive the
+ *    partials as well): every sample's partials are formed shard by shard in
+ *    registers, aggregated in the same fixed shard order and passed through F
+ *    without being written; results are bit-identical to the two-call path.
+ *  - `ops` holds LR / FM together with POOL / DENSE1 and part->part_small is
+ *    NULL: every occurrence's row is gathered once; the pass that pools a bag
+ *    also sums its linear weights and squared norms, and (+)M_1, (+)M_1^lr,
+ *    (+)M_2 are the sums over a sample's bags, taken in double in field order.
+ *    The per-shard partials are never formed — Eq. 1's sum over a sample's
+ *    occurrences grouped by field instead of by shard — so the results agree
+ *    with the two-call path within the float32 tolerance, not bit for bit.
  * part->part_pooled and part->part_dense must be NULL. */
 des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* batch,
                                const des_partials_t* part, const des_outputs_t* out, void* stream);

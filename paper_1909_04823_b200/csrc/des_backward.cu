@@ -28,9 +28,7 @@
 
 #define HOT_MIN 512u      // estimated occurrences from which a key is treated as hot
 #define HOT_CHAIN 256u    // target number of additions per replica row
-#define SUPER_T 16u       // keys whose occurrences are summed in registers instead of by atomics
-#define SUPER_R 64u       // replica rows of such a key (they only take one partial sum per lane group)
-#define SUPER_TAG 0xFFFFFF00u   // dest[j] = SUPER_TAG | slot for an occurrence of such a key
+#define SUPER_R 64u       // replica rows of a super key (they only take one partial sum per lane group)
 #ifndef SC_BLOCKS_PER_SM
 #define SC_BLOCKS_PER_SM 64     // grid cap of the scatter (it strides over the bags)
 #endif
@@ -121,7 +119,7 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
           hot_R[hh] = 0;
         }
       }
-      if (sup) ctr[4 + ts] = (h == DES_ROW_NONE) ? DES_ROW_NONE : (h & 0xFFFFFFu);
+      if (sup) ctr[HOT_CTR_SLOT + ts] = (h == DES_ROW_NONE) ? DES_ROW_NONE : (h & 0xFFFFFFu);
     }
     hinfo[u] = h;
   }
@@ -443,7 +441,7 @@ __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
   const uint32_t salt = hash_u32(blockIdx.x * 8u + (uint32_t)(tailw ? th : sub));
   if (tailw) {
     if ((uint32_t)tt >= ns) return;
-    const uint32_t hh = __ldg(ctr + 4 + tt);
+    const uint32_t hh = __ldg(ctr + HOT_CTR_SLOT + tt);
     if (hh == DES_ROW_NONE) return;
     const uint32_t R = __ldg(hot_R + hh);
     if (R == 0) return;
@@ -455,7 +453,7 @@ __global__ void __launch_bounds__(SD_THREADS) super_dense_kernel(
   for (int q = 0; q < 8; ++q) {
     const uint32_t key = (uint32_t)(kg * 8 + q);
     if (key >= ns || !col) continue;
-    const uint32_t hh = __ldg(ctr + 4 + key);
+    const uint32_t hh = __ldg(ctr + HOT_CTR_SLOT + key);
     if (hh == DES_ROW_NONE) continue;
     const uint32_t R = __ldg(hot_R + hh);
     if (R == 0) continue;
@@ -487,7 +485,7 @@ template <int G, bool ADAM>
 __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
     uint32_t ops, const OptParams opt_in, const DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
-    float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2, uint32_t* __restrict__ hinfo) {
+    float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2) {
   const int K4 = k >> 2, stride = k + 4;
   const OptParams opt = des_opt_load(opt_in, meta);
   long long U = *n_uniq;
@@ -542,7 +540,7 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
       if (live) {
         float4* grow = reinterpret_cast<float4*>(Gbuf + (size_t)u * stride);
         if (col) grow[c4] = zero;
-        if (lead) { grow[K4] = zero; hinfo[u] = 0u; }
+        if (lead) grow[K4] = zero;
       }
       float4& m2 = s2[ADAM ? q : 0];            // Adam's second moment (unused otherwise)
       if (mapped && col && upd_v) {
@@ -578,6 +576,39 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
 
 static int group_for(int k) { int K4 = k / 4, G = 1; while (G < K4) G <<= 1; return G; }
 
+// Skewed-batch path: 16-lane groups, unit feature values, batches large enough to fill a persistent grid.
+// The dense product of the backward costs time per BAG, the atomics it replaces per OCCURRENCE: it pays from
+// about ten ids per bag on (measured: 20 ids per bag 1.50 -> 0.85 + 0.25 ms; 4 ids per bag 0.43 -> 0.39 + 0.29 ms).
+static bool super_path(const des_table* t, const des_batch_t* b) {
+  const long long nbags = (long long)b->batch * t->F;
+  return group_for(t->k) == 16 && !b->vals && b->nnz >= (1 << 20) && t->super_cnt && b->nnz >= 8 * nbags;
+}
+
+des_status_t des_tags_ensure(des_table* t, const des_batch_t* b, cudaStream_t cs) {
+  if (t->tag_valid && t->tag_uidx == (const void*)b->uidx && t->tag_nnz == (long long)b->nnz) return DES_OK;
+  t->tag_valid = 0;
+  if (b->nnz == 0) return DES_OK;
+  const int nnz = (int)b->nnz;
+  int shift = 0;
+  while (shift < 6 && ((long long)nnz >> shift) > (1ll << 20)) ++shift;
+  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, HOT_CTR_WORDS * 4, cs));
+  DES_CUDA(cudaMemsetAsync(t->hinfo, 0, (size_t)t->max_uniq * 4, cs));
+  const bool use_super = super_path(t, b);
+  const uint32_t super_min = use_super ? (uint32_t)(nnz >> 7) : 0u;
+  const int n = (nnz >> shift) + 1;
+  sample_count_kernel<<<(n + SC_THREADS * SC_PER - 1) / (SC_THREADS * SC_PER), SC_THREADS, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
+  DES_LAUNCH_CHECK(t, "sample_count_kernel");
+  hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
+                                                     t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
+                                                     t->hot_work, t->work_max, super_min);
+  DES_LAUNCH_CHECK(t, "hot_select_kernel");
+  make_dest_kernel<<<(nnz + 1023) / 1024, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
+                                                      t->dest);
+  DES_LAUNCH_CHECK(t, "make_dest_kernel");
+  t->tag_uidx = b->uidx; t->tag_nnz = (long long)b->nnz; t->tag_super = use_super ? 1 : 0; t->tag_valid = 1;
+  return DES_OK;
+}
+
 extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const des_batch_t* b,
                                             const des_outputs_t* out, const des_grads_t* gr, void* stream) {
   des_status_t st = des_check_batch(t, b, 1);
@@ -605,27 +636,10 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   const int G = group_for(t->k);
   const int nnz = (int)b->nnz;
   const long long nbags = (long long)B * t->F;
-  // hot-key detection on a sample, replica assignment, per-occurrence destination row
-  int shift = 0;
-  while (shift < 6 && ((long long)nnz >> shift) > (1ll << 20)) ++shift;
-  DES_CUDA(cudaMemsetAsync(t->hot_ctr, 0, 128, cs));
-  // skewed-batch scatter: 16-lane groups, unit feature values, batches large enough to fill a persistent grid
-  // the dense product costs time per BAG, the atomics it replaces per OCCURRENCE: it pays from about ten ids
-  // per bag on (measured: 20 ids per bag 1.50 -> 0.85 + 0.25 ms; 4 ids per bag 0.43 -> 0.39 + 0.29 ms)
-  const bool use_super = G == 16 && !b->vals && nnz >= (1 << 20) && t->super_cnt && (long long)nnz >= 8 * nbags;
-  const uint32_t super_min = use_super ? (uint32_t)(nnz >> 7) : 0u;
-  {
-    const int n = (nnz >> shift) + 1;
-    sample_count_kernel<<<(n + SC_THREADS * SC_PER - 1) / (SC_THREADS * SC_PER), SC_THREADS, 0, cs>>>(b->uidx, nnz, shift, t->max_uniq, t->hinfo);
-    DES_LAUNCH_CHECK(t, "sample_count_kernel");
-    hot_select_kernel<<<t->sm_count * 4, 256, 0, cs>>>(t->hinfo, b->n_uniq, t->max_uniq, shift, t->hot_base, t->hot_R,
-                                                       t->hot_u, t->hot_ctr, t->hot_max, t->rep_max, t->meta,
-                                                       t->hot_work, t->work_max, super_min);
-    DES_LAUNCH_CHECK(t, "hot_select_kernel");
-    make_dest_kernel<<<(nnz + 1023) / 1024, 256, 0, cs>>>(b->uidx, nnz, t->hinfo, t->hot_base, t->hot_R, t->max_uniq,
-                                                        t->dest);
-    DES_LAUNCH_CHECK(t, "make_dest_kernel");
-  }
+  // hot-key detection on a sample, replica assignment, per-occurrence destination row: normally done when
+  // find_or_insert closed (the forward uses the same tags); rebuilt here if another batch came in between
+  if ((st = des_tags_ensure(t, b, cs)) != DES_OK) return st;
+  const bool use_super = t->tag_super;
   {
     // long bags: a whole warp per bag (its sub-groups take alternate occurrences); short bags: G lanes per bag
     const bool wide = (long long)nnz >= 8 * nbags;   // (at 4 ids per bag the narrow form measured faster)
@@ -669,7 +683,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
 #endif
     const unsigned grid = (unsigned)(t->sm_count * UP_GRID);
 #define UP2(GG, AD) update_rows_kernel<GG, AD><<<grid, 256, 0, cs>>>(b->uniq_rows, b->n_uniq, t->max_uniq, t->k, ops, \
-                                                                   opt, t->meta, t->Gbuf, t->W, t->A, t->A2, t->hinfo)
+                                                                   opt, t->meta, t->Gbuf, t->W, t->A, t->A2)
 #define UP(GG) do { if (t->A2) UP2(GG, true); else UP2(GG, false); } while (0)
     switch (G) { case 1: UP(1); break; case 2: UP(2); break; case 4: UP(4); break; case 8: UP(8); break; default: UP(16); }
 #undef UP

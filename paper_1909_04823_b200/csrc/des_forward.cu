@@ -23,6 +23,11 @@
 //  pool_kernel    one group per bag: sum pooling of the latent vectors in
 //                 registers.  The per-shard pooled partial [S][B][F*k] is only
 //                 materialised (with atomics) when the caller asks for it.
+//
+// Accuracy.  A lane never adds more than a few dozen terms into one float32 accumulator (long
+// segments are summed in two levels), and the sum over shards is taken in double and rounded once, so
+// every per-sample sum keeps the stated float32 tolerance even when one key contributes
+// hundreds of equal terms that the other terms cancel.
 #include "des_internal.cuh"
 
 #ifndef POOL_BLOCKS_PER_SM
@@ -193,13 +198,18 @@ __device__ __forceinline__ void pool_step(const uint32_t* __restrict__ grow_csr,
 // occurrences).  The loop body is kept to the loads and adds: whole iterations
 // carry no bound checks, row addresses are one multiply-add from a per-lane base,
 // and lanes without a column of their own (k not a multiple of 4 G) re-read
-// column 0 instead of branching.  part_small (optional) receives each segment's
-// partial sums as soon as the segment ends; with FUSED the aggregation (+) over
-// shards and the substitution operator F are applied on chip, in the same shard
-// order and with the same arithmetic as aggregate_small_kernel, and out_small is
-// written directly — the per-shard partials then never touch memory.
+// column 0 instead of branching.  In a long segment a lane's float32 sums move on
+// into a second set of accumulators every SP_FLUSH iterations; the sum over shards
+// runs in double.  part_small
+// (optional) receives each segment's partial sums, rounded to float32, as soon as
+// the segment ends; with FUSED the aggregation (+) over shards and the substitution
+// operator F are applied on chip, in the same shard order and with the same
+// arithmetic as aggregate_small_kernel (the sum of the float32-rounded partials in
+// double), and out_small is written directly — the per-shard partials then never
+// touch memory.
+#define SP_FLUSH 8
 template <int G, bool HAS_VALS, bool FUSED>
-__global__ void __launch_bounds__(256) shard_partials_kernel(
+__global__ void __launch_bounds__(256, FUSED ? 4 : 8) shard_partials_kernel(
     const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted, const int32_t* __restrict__ seg_off,
     int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small,
     float* __restrict__ out_small) {
@@ -215,7 +225,7 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
   const unsigned rowB = (unsigned)stride * 4u;         // bytes per row
   const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
   const char* Wt = reinterpret_cast<const char*>(W + k);                       // (w, |v|^2)
-  float4 A = zero4; float R = 0.f, Q = 0.f;            // FUSED: (+)M_1, (+)M_1^lr, (+)M_2
+  double Ax = 0.0, Ay = 0.0, Az = 0.0, Aw = 0.0, R = 0.0, Q = 0.0;   // FUSED: (+)M_1, (+)M_1^lr, (+)M_2
   const int32_t* so = seg_off + (size_t)b * (S + 1);
   int hi = __ldg(so);
   for (int s = 0; s < S; ++s) {
@@ -223,13 +233,26 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
     hi = __ldg(so + s + 1);
     float4 acc = zero4;
     float m1lr = 0.f, m2 = 0.f;
+    int i0 = lo;
+    // a long segment (one hot id occurring hundreds of times in the sample): the sums move on into a second
+    // set of accumulators every SP_FLUSH iterations, so that no float32 accumulator takes more than a few
+    // dozen additions (a single chain of hundreds of equal terms would lose the 1e-5 the sum must keep)
+    float4 up = zero4;
+    float up_l = 0.f, up_q = 0.f;
+    while (hi - i0 > 4 * P * SP_FLUSH) {
+#pragma unroll 1
+      for (int it = 0; it < SP_FLUSH; ++it, i0 += 2 * P)
+        sp_step<2, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
+      up.x += acc.x; up.y += acc.y; up.z += acc.z; up.w += acc.w; up_l += m1lr; up_q += m2;
+      acc = zero4; m1lr = 0.f; m2 = 0.f;
+    }
     // whole blocks of 2 and 1 occurrences per lane (no bound checks), then one checked step; segments are
     // short (a sample's occurrences spread over S shards), so deeper unrolling only adds ragged steps
-    int i0 = lo;
     for (; i0 + 2 * P <= hi; i0 += 2 * P)
       sp_step<2, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
     if (i0 + P <= hi) { sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2); i0 += P; }
     if (i0 + p < hi) sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
+    acc.x += up.x; acc.y += up.y; acc.z += up.z; acc.w += up.w; m1lr += up_l; m2 += up_q;
 #pragma unroll
     for (int d = G; d < 32; d <<= 1) {                 // combine the sub-groups (same result in every lane)
       acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
@@ -243,15 +266,18 @@ __global__ void __launch_bounds__(256) shard_partials_kernel(
       if (col) dst[c4] = acc;
       if (c4 == 0) dst[K4] = make_float4(m1lr, m2, 0.f, 0.f);
     }
-    if (FUSED) { A.x += acc.x; A.y += acc.y; A.z += acc.z; A.w += acc.w; R += m1lr; Q += m2; }
+    if (FUSED) {
+      Ax += (double)acc.x; Ay += (double)acc.y; Az += (double)acc.z; Aw += (double)acc.w;
+      R += (double)m1lr; Q += (double)m2;
+    }
   }
   if (FUSED) {
-    double aa = col ? (double)A.x * A.x + (double)A.y * A.y + (double)A.z * A.z + (double)A.w * A.w : 0.0;
+    double aa = col ? Ax * Ax + Ay * Ay + Az * Az + Aw * Aw : 0.0;
 #pragma unroll
     for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
     float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
-    if (p == 0 && col) o[c4] = A;
-    if (lane == 0) o[K4] = make_float4(R, fm ? (float)(0.5 * aa - 0.5 * (double)Q) : 0.f, Q, 0.f);
+    if (p == 0 && col) o[c4] = make_float4((float)Ax, (float)Ay, (float)Az, (float)Aw);
+    if (lane == 0) o[K4] = make_float4((float)R, fm ? (float)(0.5 * aa - 0.5 * Q) : 0.f, (float)Q, 0.f);
   }
 }
 
@@ -301,7 +327,8 @@ __global__ void __launch_bounds__(256) pool_kernel(
 }
 
 // (+) over shards and F.  G lanes per sample, one float4 column each; lane 0 of
-// the group also carries the tail (R_lr, Q).  <A, A> is taken in double.
+// the group also carries the tail (R_lr, Q).  The float32 partials are added in
+// double in shard order and rounded once; <A, A> is taken on the double sums.
 template <int G>
 __global__ void __launch_bounds__(256) aggregate_small_kernel(const float* __restrict__ part_small, int B, int S, int k,
                                                               uint32_t ops, float* __restrict__ out_small) {
@@ -309,24 +336,149 @@ __global__ void __launch_bounds__(256) aggregate_small_kernel(const float* __res
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int b = t / G, c4 = t % G;
   const bool live = b < B;
-  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), tail = a;
+  double ax = 0.0, ay = 0.0, az = 0.0, aw = 0.0, tr = 0.0, tq = 0.0;
   if (live) {
     for (int s = 0; s < S; ++s) {
       const float4* p = reinterpret_cast<const float4*>(part_small + ((size_t)s * B + b) * stride);
-      if (c4 < K4) { float4 v = __ldg(p + c4); a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w; }
-      if (c4 == 0) { float4 v = __ldg(p + K4); tail.x += v.x; tail.y += v.y; }
+      if (c4 < K4) { float4 v = __ldg(p + c4); ax += (double)v.x; ay += (double)v.y; az += (double)v.z; aw += (double)v.w; }
+      if (c4 == 0) { float4 v = __ldg(p + K4); tr += (double)v.x; tq += (double)v.y; }
     }
   }
-  double aa = (double)a.x * a.x + (double)a.y * a.y + (double)a.z * a.z + (double)a.w * a.w;
+  double aa = ax * ax + ay * ay + az * az + aw * aw;
 #pragma unroll
   for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
   if (!live) return;
   float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
-  if (c4 < K4) o[c4] = a;
+  if (c4 < K4) o[c4] = make_float4((float)ax, (float)ay, (float)az, (float)aw);
   if (c4 == 0) {
-    const float fm2 = (ops & DES_OP_FM) ? (float)(0.5 * aa - 0.5 * (double)tail.y) : 0.f;
-    o[K4] = make_float4(tail.x, fm2, tail.y, 0.f);
+    const float fm2 = (ops & DES_OP_FM) ? (float)(0.5 * aa - 0.5 * tq) : 0.f;
+    o[K4] = make_float4((float)tr, fm2, (float)tq, 0.f);
   }
+}
+
+// ---- single-gather forward (des_forward_fused with pooling in `ops`) -----------------------------------
+// Every occurrence's row is read ONCE: the group that pools a bag also sums the bag's linear weights and
+// cached squared norms, and a second, small kernel adds a sample's bags up in double: A = sum over fields of
+// the pooled vectors, R_lr and Q = the sums of the bag tails.  The per-shard partials are never formed (the
+// sum over a sample's occurrences is taken field by field instead of shard by shard — Eq. 1 with (+) = +
+// allows any grouping), so the results agree with the two-call path within the float32 tolerance, not bit
+// for bit.  Reads the batch as find_or_insert left it (shard-local rows + shards): no routing pass.
+template <int U, int P, bool HAS_VALS>
+__device__ __forceinline__ void sg_step(const uint32_t* __restrict__ rows, const uint8_t* __restrict__ shards,
+                                        const float* __restrict__ vals, const uint32_t* __restrict__ s_base, int i,
+                                        const char* __restrict__ Wc, const char* __restrict__ Wt, unsigned rowB,
+                                        uint32_t null_row, float4& acc, float& bl, float& bq) {
+  float4 v[U]; float2 tl[U]; float x[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const uint32_t r = __ldg(rows + i + u * P);
+    const uint32_t g = (r == DES_ROW_NONE) ? null_row : s_base[__ldg(shards + i + u * P)] + r;
+    const size_t off = (size_t)g * rowB;
+    if (HAS_VALS) x[u] = __ldg(vals + i + u * P);
+    v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
+    tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    if (HAS_VALS) {
+      acc.x += v[u].x * x[u]; acc.y += v[u].y * x[u]; acc.z += v[u].z * x[u]; acc.w += v[u].w * x[u];
+      bl += tl[u].x * x[u]; bq += tl[u].y * x[u] * x[u];
+    } else {
+      acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w;
+      bl += tl[u].x; bq += tl[u].y;
+    }
+  }
+}
+
+template <int G, int P, bool HAS_VALS>
+__global__ void __launch_bounds__(256) single_gather_kernel(
+    const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
+    const uint8_t* __restrict__ shards, long long nbags, int S, int k, const float* __restrict__ W,
+    const DevMeta* __restrict__ meta, uint32_t null_row, float* __restrict__ pooled, float2* __restrict__ bag_tail) {
+  constexpr int LB = G * P;                            // lanes per bag
+  __shared__ uint32_t s_base[DES_MAX_SHARDS];
+  if (threadIdx.x < S) s_base[threadIdx.x] = (uint32_t)meta->row_base[threadIdx.x];
+  __syncthreads();
+  const int K4 = k >> 2, stride = k + 4;
+  const int sub = threadIdx.x % LB, c4 = sub % G, p = sub / G;
+  const bool col = c4 < K4;
+  const unsigned rowB = (unsigned)stride * 4u;
+  const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
+  const char* Wt = reinterpret_cast<const char*>(W + k);
+  const long long slots = (long long)gridDim.x * (256 / LB);
+  const long long rounds = (nbags + slots - 1) / slots;
+  long long bag = (long long)blockIdx.x * (256 / LB) + threadIdx.x / LB;
+  int lo_n = 0, hi_n = 0;
+  if (bag < nbags) { lo_n = __ldg(offsets + bag); hi_n = __ldg(offsets + bag + 1); }
+  for (long long r = 0; r < rounds; ++r, bag += slots) {
+    const bool live = bag < nbags;
+    const int lo = lo_n, hi = hi_n;
+    lo_n = 0; hi_n = 0;
+    if (bag + slots < nbags) { lo_n = __ldg(offsets + bag + slots); hi_n = __ldg(offsets + bag + slots + 1); }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float bl = 0.f, bq = 0.f;
+    int i0 = lo;
+#define SG_STEP(U) sg_step<U, P, HAS_VALS>(rows, shards, vals, s_base, i0 + p, Wc, Wt, rowB, null_row, acc, bl, bq)
+    for (; i0 + 4 * P <= hi; i0 += 4 * P) SG_STEP(4);
+    if (i0 + 2 * P <= hi) { SG_STEP(2); i0 += 2 * P; }
+    if (i0 + P <= hi) { SG_STEP(1); i0 += P; }
+    if (i0 + p < hi) SG_STEP(1);
+#undef SG_STEP
+#pragma unroll
+    for (int d = G; d < LB; d <<= 1) {                 // combine the bag's sub-groups
+      acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
+      acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
+      bl += __shfl_xor_sync(0xFFFFFFFFu, bl, d); bq += __shfl_xor_sync(0xFFFFFFFFu, bq, d);
+    }
+    if (live && p == 0) {
+      if (col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+      if (c4 == 0) bag_tail[bag] = make_float2(bl, bq);
+    }
+  }
+}
+
+// A, R_lr, Q and F per sample from the pooled vectors and bag tails of its F bags, added in double in field
+// order.  G lanes per sample, one float4 column each; lane 0 of the group carries the tails.
+template <int G>
+__global__ void __launch_bounds__(256) fused_finish_kernel(const float* __restrict__ pooled, const float2* __restrict__ bag_tail,
+                                                           int B, int F, int k, uint32_t ops, float* __restrict__ out_small) {
+  const int K4 = k >> 2, stride = k + 4;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = t / G, c4 = t % G;
+  const bool live = b < B;
+  const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
+  double ax = 0.0, ay = 0.0, az = 0.0, aw = 0.0, tr = 0.0, tq = 0.0;
+  if (live) {
+    const float4* pb = reinterpret_cast<const float4*>(pooled + (size_t)b * F * k) + c4;
+    const float2* tb = bag_tail + (size_t)b * F;
+    int f = 0;
+    for (; f + 4 <= F; f += 4) {                       // four bags in flight
+      float4 v[4]; float2 tl[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        v[q] = (c4 < K4 && fm) ? __ldg(pb + (size_t)(f + q) * K4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        tl[q] = (c4 == 0) ? __ldg(tb + f + q) : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        ax += (double)v[q].x; ay += (double)v[q].y; az += (double)v[q].z; aw += (double)v[q].w;
+        tr += (double)tl[q].x; tq += (double)tl[q].y;
+      }
+    }
+    for (; f < F; ++f) {
+      if (c4 < K4 && fm) { const float4 v = __ldg(pb + (size_t)f * K4); ax += (double)v.x; ay += (double)v.y; az += (double)v.z; aw += (double)v.w; }
+      if (c4 == 0) { const float2 tl = __ldg(tb + f); tr += (double)tl.x; tq += (double)tl.y; }
+    }
+  }
+  if (!lr) tr = 0.0;
+  if (!fm) tq = 0.0;
+  double aa = ax * ax + ay * ay + az * az + aw * aw;
+#pragma unroll
+  for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
+  if (!live) return;
+  float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
+  if (c4 < K4) o[c4] = make_float4((float)ax, (float)ay, (float)az, (float)aw);
+  if (c4 == 0) o[K4] = make_float4((float)tr, fm ? (float)(0.5 * aa - 0.5 * tq) : 0.f, (float)tq, 0.f);
 }
 
 // sum over shards of a dense [S][B][n] tensor (materialised pooled / dense partials)
@@ -364,7 +516,7 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   // which has finished with it by the time a forward can run on the same stream)
   uint32_t* grow_csr = t->uslot;
   uint32_t* grow_sorted = t->slot_of;
-  float* x_sorted = reinterpret_cast<float*>(t->dest);
+  float* x_sorted = t->x_sorted;
   route_kernel<<<(B + 7) / 8 < t->sm_count * 8 ? (B + 7) / 8 : t->sm_count * 8, 256, 0, cs>>>(
       b->offsets, b->vals, b->rows, b->shards, B, t->F, t->S, t->meta, (uint32_t)t->total_rows, grow_csr, grow_sorted,
       x_sorted, t->seg_off);
@@ -406,15 +558,57 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   return forward_impl(t, ops, b, part, nullptr, stream);
 }
 
+// des_forward_fused with pooling among the operators: one gather pass for everything.
+static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const des_batch_t* b, float* pooled,
+                                          float* out_small, cudaStream_t cs) {
+  const int B = b->batch, G = group_for(t->k);
+  const long long nbags = (long long)B * t->F;
+  {
+    const bool wide = b->nnz >= 8 * nbags;
+    const long long threads = nbags * (wide ? 32 : G);
+    long long blocks = (threads + 255) / 256;
+    if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
+    const unsigned grid = (unsigned)blocks;
+#define SG3(GG, PP, HV) single_gather_kernel<GG, PP, HV><<<grid, 256, 0, cs>>>(b->offsets, b->vals, b->rows, b->shards, nbags,   \
+                                                                              (int)t->S, t->k, t->W, t->meta,                 \
+                                                                              (uint32_t)t->total_rows, pooled, t->bag_tail)
+#define SG2(GG, HV) do { if (wide) SG3(GG, 32 / GG, HV); else SG3(GG, 1, HV); } while (0)
+#define SG(GG) do { if (b->vals) SG2(GG, true); else SG2(GG, false); } while (0)
+    switch (G) { case 1: SG(1); break; case 2: SG(2); break; case 4: SG(4); break; case 8: SG(8); break; default: SG(16); }
+#undef SG
+#undef SG2
+#undef SG3
+    DES_LAUNCH_CHECK(t, "single_gather_kernel");
+  }
+  {
+    const int grid = (int)(((long long)B * G + 255) / 256);
+#define FF(GG) fused_finish_kernel<GG><<<grid, 256, 0, cs>>>(pooled, t->bag_tail, B, (int)t->F, t->k, ops, out_small)
+    switch (G) { case 1: FF(1); break; case 2: FF(2); break; case 4: FF(4); break; case 8: FF(8); break; default: FF(16); }
+#undef FF
+    DES_LAUNCH_CHECK(t, "fused_finish_kernel");
+  }
+  return DES_OK;
+}
+
 extern "C" des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* b,
                                           const des_partials_t* part, const des_outputs_t* out, void* stream) {
   if (!t || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
   if ((ops & (DES_OP_LR | DES_OP_FM)) && !out->out_small) return DES_ERR_INVALID_ARG;
   if (part->part_pooled || part->part_dense) return DES_ERR_INVALID_ARG;      // materialised partials: use the two-call path
-  des_status_t st = forward_impl(t, ops, b, part, out->out_small, stream);
+  const uint32_t rest = ops & ~(uint32_t)(DES_OP_LR | DES_OP_FM);
+  des_status_t st;
+  if ((ops & (DES_OP_LR | DES_OP_FM)) && rest && !part->part_small) {
+    // LR / FM together with pooling and no request for the per-shard partials: one gather pass
+    st = des_check_batch(t, b, 0);
+    if (st != DES_OK) return st;
+    if (!part->pooled || ((ops & DES_OP_DENSE1) && !t->H)) return DES_ERR_INVALID_ARG;
+    des_api_begin(t, (cudaStream_t)stream);
+    st = forward_single_gather(t, ops, b, part->pooled, out->out_small, (cudaStream_t)stream);
+  } else {
+    st = forward_impl(t, ops, b, part, out->out_small, stream);
+  }
   if (st != DES_OK) return st;
   // what is left of the aggregation: hand the pooled block over and run the first layer
-  const uint32_t rest = ops & ~(uint32_t)(DES_OP_LR | DES_OP_FM);
   return rest ? des_aggregate(t, rest, b, part, out, stream) : DES_OK;
 }
 

@@ -11,6 +11,16 @@
 #define DES_SLOT_NONE 0xFFFFFFFFu
 #define HOT_RCHUNK 16u     // replica rows of a hot key summed by one warp of the backward's replica reduction
 
+// The few keys that own a large share of a skewed batch ("super" keys) are counted instead of scattered in the
+// backward: a tagged occurrence carries SUPER_TAG | slot where other occurrences carry a gradient row number.
+#define SUPER_T 16u             // slots
+#define SUPER_TAG 0xFFFFFF00u   // tag | slot; DES_ROW_NONE (low byte 0xFF) is not a tag
+// Layout of the hot-key counter block (des_table::hot_ctr, 64 words):
+//   [0] hot keys  [1] replica rows  [2] work items  [3] super slots claimed
+//   [4 + t]   hot index of super slot t (DES_ROW_NONE: slot unused)
+#define HOT_CTR_WORDS 64
+#define HOT_CTR_SLOT 4
+
 // One open-addressing slot: 16 bytes, read with a single vector load.
 //   key        DES_KEY_EMPTY until claimed by a 64-bit CAS; never changes after.
 //   row        shard-local row, DES_ROW_NONE until the key's insert call numbers it.
@@ -68,7 +78,13 @@ struct des_table {
   float* Gbuf;                       // [max_uniq + rep_max][stride]: per-unique gradient rows, then
                                      // hot-key replica rows; all zero between calls
   uint32_t* hinfo;                   // [max_uniq] sampled count, then hot index; zero between calls
-  uint32_t* dest;                    // [max_nnz] gradient row of each occurrence
+  uint32_t* dest;                    // [max_nnz] gradient row of each occurrence (or SUPER_TAG | slot); made by the
+                                     // hot-key pass that closes find_or_insert; the forward reads "hot or not" from
+                                     // it, the backward scatters by it
+  float* x_sorted;                   // [max_nnz] forward routing: feature values in shard-major order
+  float2* bag_tail;                  // [max_batch * F] single-gather forward: per-bag sums of (w x, |v|^2 x^2)
+  // which batch the tags in dest[] / the hot lists belong to (they are rebuilt when another batch comes)
+  const void* tag_uidx; long long tag_nnz; int tag_valid; int tag_super;
   uint32_t *hot_base, *hot_R, *hot_u, *hot_ctr;   // hot list [hot_max] and its two counters
   uint32_t* hot_work;                // [work_max] (hot index << 18 | chunk) items of the replica reduction
   double* hot_acc;                   // [hot_max][stride] double sums of the replicas; zero between calls
@@ -225,3 +241,6 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
                                 const float* part_pooled, cudaStream_t st);
 des_status_t des_dense1_backward(des_table* t, const float* pooled, const float* gE, const float* gZ,
                                  float* gE_work, int B, cudaStream_t st);
+// Hot-key pass over a batch's unique indices (sampled counts, hot list, replica assignment, dest[] with
+// the super-key tags); a no-op when dest[] already belongs to this batch.
+des_status_t des_tags_ensure(des_table* t, const des_batch_t* b, cudaStream_t st);

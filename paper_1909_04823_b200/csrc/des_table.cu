@@ -102,7 +102,7 @@ extern "C" des_status_t des_table_destroy(des_table_t* t) {
   cudaSetDevice(t->device);
   cudaDeviceSynchronize();
   void* ptrs[] = {t->slots, t->W, t->A, t->A2, t->acc2W1, t->meta, t->slot_of, t->flags, t->uslot, t->blk_cnt, t->seg_off, t->Gbuf, t->hinfo, t->dest, t->hot_base,
-                  t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc, t->super_cnt,
+                  t->hot_R, t->hot_u, t->hot_ctr, t->hot_work, t->hot_acc, t->super_cnt, t->x_sorted, t->bag_tail,
                   t->W1, t->accW1, t->W1b, t->gW1_part, t->pooled_b, t->gZ_b, t->gemm_ws, t->st_offsets[0], t->st_ids[0], t->st_vals[0], t->st_offsets[1], t->st_ids[1], t->st_vals[1], t->st_rows,
                   t->st_shards, t->st_uidx, t->st_uniq_rows, t->st_n_uniq, t->st_part_small, t->st_out_small};
   for (void* p : ptrs) dfree(t->cfg, p);
@@ -203,10 +203,12 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
   A(t->Gbuf, ((size_t)t->max_uniq + t->rep_max) * rowbytes);
   A(t->hinfo, (size_t)t->max_uniq * 4);
   A(t->dest, (size_t)t->max_nnz * 4);
+  A(t->x_sorted, (size_t)t->max_nnz * 4);
+  A(t->bag_tail, (size_t)t->max_batch * t->F * sizeof(float2));
   A(t->hot_base, (size_t)t->hot_max * 4);
   A(t->hot_R, (size_t)t->hot_max * 4);
   A(t->hot_u, (size_t)t->hot_max * 4);
-  A(t->hot_ctr, 256);
+  A(t->hot_ctr, HOT_CTR_WORDS * 4);
   t->work_max = t->rep_max / HOT_RCHUNK + t->hot_max;
   A(t->hot_work, (size_t)t->work_max * 4);
   A(t->hot_acc, (size_t)t->hot_max * t->stride * 8);

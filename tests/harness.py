@@ -263,15 +263,20 @@ class Pair:
         self.t.aggregate(ops, db, part_small, pooled, part_pooled, part_dense, out_small, pooled, Z)
         torch.cuda.synchronize()
         assert self.t.status() == 0
+        fused_osm = None
         if not materialise:
-            # the fused call (partials kept on chip) must reproduce the two-call path bit for bit
+            # the fused call (partials kept on chip) must reproduce the two-call path: bit for bit, except that
+            # with pooling among the operators its aggregates come from one gather pass in another (field-wise)
+            # order of addition and are held to the oracle's tolerance below
             f_small = torch.full((B, k + 4), float("nan"), device=dev)
             f_pooled = torch.full((B, F * k), float("nan"), device=dev)
             f_Z = torch.full((B, max(H, 1)), float("nan"), device=dev)
             self.t.forward_fused(ops, db, None, f_pooled, f_small, f_Z)
             torch.cuda.synchronize()
             assert self.t.status() == 0
-            if ops & (OP_LR | OP_FM):
+            if (ops & (OP_LR | OP_FM)) and (ops & (OP_POOL | OP_DENSE1)):
+                fused_osm = f_small.cpu().numpy()
+            elif ops & (OP_LR | OP_FM):
                 assert torch.equal(f_small.view(torch.int32), out_small.view(torch.int32)), "fused out_small"
             if ops & (OP_POOL | OP_DENSE1):
                 assert torch.equal(f_pooled.view(torch.int32), pooled.view(torch.int32)), "fused pooled"
@@ -279,21 +284,31 @@ class Pair:
                 assert torch.equal(f_Z.view(torch.int32), Z.view(torch.int32)), "fused Z"
         ps = part_small.cpu().numpy()
         osm = out_small.cpu().numpy()
+        AA = np.sum(oa["A"] ** 2, axis=1)
+        for o_, tag in ((osm, ""), (fused_osm, "fused ")):
+            if o_ is None or not (ops & (OP_LR | OP_FM)):
+                continue
+            if ops & OP_FM:
+                cmp(o_[:, :k], oa["A"], tag + "A", extra=xa, sumabs=sabs[:, :k])
+                cmp(o_[:, k + 2], oa["Q"], tag + "Q", extra=SUMTOL_FWD * oa["Q"])
+                # fm2 = (<A,A> - Q)/2 subtracts two float32-rounded inputs of size <A,A>/2 and Q/2
+                cmp(o_[:, k + 1], oa["fm2"], tag + "fm2",
+                    extra=SUMTOL_FWD * (AA + np.abs(oa["Q"])) + np.sum(np.abs(oa["A"]) * xa, axis=1))
+            else:
+                assert not np.any(o_[:, :k]) and not np.any(o_[:, k + 1:k + 3]), tag + "FM outputs must be zero without FM"
+            if ops & OP_LR:
+                cmp(o_[:, k], oa["lr"], tag + "R_lr", extra=xl, sumabs=sabs[:, k])
+            else:
+                assert not np.any(o_[:, k]), tag + "R_lr must be zero without LR"
+            assert not np.any(o_[:, k + 3]), "padding must be zero"
         if ops & OP_FM:
             cmp(ps[:, :, :k], op["part_small"][:, :, :k], "part_small.M1_fm", extra=xa[None], sumabs=sabs[None, :, :k])
             cmp(ps[:, :, k + 1], op["part_small"][:, :, k + 1], "part_small.M2_fm",
                 extra=SUMTOL_FWD * op["part_small"][:, :, k + 1])
-            cmp(osm[:, :k], oa["A"], "A", extra=xa, sumabs=sabs[:, :k])
-            cmp(osm[:, k + 2], oa["Q"], "Q", extra=SUMTOL_FWD * oa["Q"])
-            # fm2 = (<A,A> - Q)/2 subtracts two float32-rounded inputs of size <A,A>/2 and Q/2
-            AA = np.sum(oa["A"] ** 2, axis=1)
-            cmp(osm[:, k + 1], oa["fm2"], "fm2",
-                extra=SUMTOL_FWD * (AA + np.abs(oa["Q"])) + np.sum(np.abs(oa["A"]) * xa, axis=1))
         if ops & OP_LR:
             cmp(ps[:, :, k], op["part_small"][:, :, k], "part_small.M1_lr", extra=xl[None], sumabs=sabs[None, :, k])
-            cmp(osm[:, k], oa["lr"], "R_lr", extra=xl, sumabs=sabs[:, k])
         if ops & (OP_LR | OP_FM):
-            assert not np.any(ps[:, :, k + 2:]) and not np.any(osm[:, k + 3]), "padding must be zero"
+            assert not np.any(ps[:, :, k + 2:]), "padding must be zero"
         if (ops & (OP_POOL | OP_DENSE1)) and pooled_samples is not None:
             sel = np.asarray(pooled_samples)
             sb = select_samples(batch, sel)
