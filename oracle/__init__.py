@@ -57,6 +57,9 @@ def _declare(L):
     L.orc_create.argtypes = [C.c_uint32] * 6 + [C.c_uint64] + [C.c_float] * 4
     L.orc_destroy.argtypes = [C.c_void_p]
     L.orc_find_or_insert.restype = C.c_int64
+    L.orc_evict_keys.restype = C.c_int64
+    L.orc_evict_stale.restype = C.c_int64
+    L.orc_clock.restype = C.c_uint64
     for name in ("orc_dense1_set", "orc_dense1_get", "orc_size", "orc_find_or_insert",
                  "orc_forward_original", "orc_fm_pairs", "orc_forward_partials", "orc_aggregate",
                  "orc_backward_update", "orc_read_rows", "orc_poke", "orc_philox4x32_10",
@@ -170,6 +173,17 @@ class Oracle:
         out = np.zeros(self.S, dtype=np.uint64)
         self.L.orc_size(self.h, _p(out, C.c_uint64))
         return out
+
+    # -- eviction --------------------------------------------------------------
+    def evict_keys(self, keys) -> int:
+        keys = np.ascontiguousarray(keys, dtype=np.uint64)
+        return int(self.L.orc_evict_keys(self.h, _p(keys, C.c_uint64), C.c_int64(keys.shape[0])))
+
+    def evict_stale(self, min_clock: int) -> int:
+        return int(self.L.orc_evict_stale(self.h, C.c_uint64(min_clock)))
+
+    def clock(self) -> int:
+        return int(self.L.orc_clock(self.h))
 
     def dense1_set(self, W1):
         W1 = np.ascontiguousarray(W1, dtype=np.float32)

@@ -112,6 +112,7 @@ struct Shard {
   std::vector<uint64_t> keys;                   // row -> key
   std::vector<float> emb, lin, acc_emb, acc_lin;
   std::vector<float> acc2_emb, lin2;            // second state word: Adam's v; linear weight: Adam's v / FTRL's z
+  std::vector<uint64_t> stamp;                  // table clock when the row was inserted or last updated
 };
 
 struct Table {
@@ -122,6 +123,7 @@ struct Table {
   uint32_t lin_optimizer = LIN_SAME;
   float beta1 = 0.9f, beta2 = 0.999f, ftrl_alpha = 0.05f, ftrl_beta = 1.0f, ftrl_l1 = 0.f, ftrl_l2 = 0.f;
   int64_t step = 0;                             // backward calls so far (Adam's t)
+  uint64_t clock = 0;                           // inserting find_or_insert calls so far (the age clock of eviction)
   float state_init() const { return optimizer == OPT_ADAGRAD ? init_acc : 0.0f; }
   float lin_state_init() const { return (lin_optimizer == LIN_FTRL || optimizer != OPT_ADAGRAD) ? 0.0f : init_acc; }
   uint32_t shard_of(uint64_t id, uint32_t field) const {
@@ -137,6 +139,7 @@ struct Table {
     for (uint32_t c = 0; c < k; ++c) { h.acc_emb.push_back(state_init()); h.acc2_emb.push_back(0.0f); }
     h.acc_lin.push_back(lin_state_init());
     h.lin2.push_back(0.0f);
+    h.stamp.push_back(clock);
     return row;
   }
 };
@@ -253,6 +256,7 @@ int64_t orc_find_or_insert(void* p, const int32_t* offsets, const uint64_t* ids,
                            uint32_t* rows, uint8_t* shards, uint32_t* uidx,
                            uint8_t* uniq_shard, uint32_t* uniq_row) {
   Table* t = (Table*)p;
+  if (insert) t->clock += 1;                     // reading: the table's age clock counts inserting calls
   std::unordered_map<uint64_t, uint32_t> seen;   // (shard<<32 | row) -> u
   int64_t U = 0;
   for (int64_t bag = 0; bag < (int64_t)B * t->F; ++bag) {
@@ -532,6 +536,7 @@ void orc_backward_update(void* p, uint32_t ops, const int32_t* offsets, const fl
   for (int64_t u = 0; u < U; ++u) {
     Shard& h = t->sh[us[u]];
     uint32_t row = ur[u];
+    h.stamp[row] = t->clock;                     // updated in the step of the current batch
     if (ops & OP_LR) {
       if (t->lin_optimizer == LIN_FTRL) apply_ftrl(*t, h.lin[row], h.acc_lin[row], h.lin2[row], Gw[u]);
       else apply_opt(*t, h.lin[row], h.acc_lin[row], h.lin2[row], Gw[u]);
@@ -590,6 +595,71 @@ void orc_dense1_get_state2(void* p, float* acc2) {
   Table* t = (Table*)p;
   std::memcpy(acc2, t->acc2W1.data(), t->acc2W1.size() * 4);
 }
+
+// Eviction for streaming tables (Section 1, "Dynamic Features": under an endless stream the set of live
+// features changes with time, so a table that can only grow would not fit any memory).  The paper's three
+// table operations (Section 5) do not include a delete; reading: a key is removed from its shard, its row is
+// freed, and the shard's rows stay the numbers 0 .. n-1 by moving the surviving rows that lie beyond the
+// shard's new size into the freed rows below it — the i-th freed row (ascending) takes the i-th such survivor
+// (ascending).  Rows that are not moved keep their numbers.  A removed key looks up as "no row"; inserting
+// it again makes a new key of it (fresh initial weights).
+static int64_t evict_rows(Table* t, uint32_t s, const std::vector<uint8_t>& dead) {
+  Shard& h = t->sh[s];
+  const uint32_t n = (uint32_t)h.keys.size(), k = t->k;
+  uint32_t e = 0;
+  for (uint32_t r = 0; r < n; ++r) e += dead[r];
+  if (!e) return 0;
+  const uint32_t m = n - e;
+  std::vector<uint32_t> holes, movers;
+  for (uint32_t r = 0; r < m; ++r) if (dead[r]) holes.push_back(r);
+  for (uint32_t r = m; r < n; ++r) if (!dead[r]) movers.push_back(r);
+  for (uint32_t r = 0; r < n; ++r) if (dead[r]) h.map.erase(h.keys[r]);
+  for (size_t i = 0; i < holes.size(); ++i) {
+    const uint32_t to = holes[i], from = movers[i];
+    h.keys[to] = h.keys[from];
+    h.map[h.keys[to]] = to;
+    std::memcpy(&h.emb[(size_t)to * k], &h.emb[(size_t)from * k], k * 4);
+    std::memcpy(&h.acc_emb[(size_t)to * k], &h.acc_emb[(size_t)from * k], k * 4);
+    std::memcpy(&h.acc2_emb[(size_t)to * k], &h.acc2_emb[(size_t)from * k], k * 4);
+    h.lin[to] = h.lin[from]; h.acc_lin[to] = h.acc_lin[from]; h.lin2[to] = h.lin2[from]; h.stamp[to] = h.stamp[from];
+  }
+  h.keys.resize(m); h.lin.resize(m); h.acc_lin.resize(m); h.lin2.resize(m); h.stamp.resize(m);
+  h.emb.resize((size_t)m * k); h.acc_emb.resize((size_t)m * k); h.acc2_emb.resize((size_t)m * k);
+  return e;
+}
+
+// Removes the listed keys (keys that are not in the table, or listed twice, count once or not at all).
+// Under the FIELD partition a key may live in several shards (one per field that uses it): all go.
+int64_t orc_evict_keys(void* p, const uint64_t* keys, int64_t n) {
+  Table* t = (Table*)p;
+  int64_t total = 0;
+  for (uint32_t s = 0; s < t->S; ++s) {
+    Shard& h = t->sh[s];
+    std::vector<uint8_t> dead(h.keys.size(), 0);
+    for (int64_t i = 0; i < n; ++i) {
+      if (t->partition == PART_HASH && (uint32_t)(mix64(keys[i]) % t->S) != s) continue;
+      auto it = h.map.find(keys[i]);
+      if (it != h.map.end()) dead[it->second] = 1;
+    }
+    total += evict_rows(t, s, dead);
+  }
+  return total;
+}
+
+// Removes every key that was neither inserted nor updated since the table's clock showed min_clock.
+int64_t orc_evict_stale(void* p, uint64_t min_clock) {
+  Table* t = (Table*)p;
+  int64_t total = 0;
+  for (uint32_t s = 0; s < t->S; ++s) {
+    Shard& h = t->sh[s];
+    std::vector<uint8_t> dead(h.keys.size(), 0);
+    for (size_t r = 0; r < h.keys.size(); ++r) dead[r] = h.stamp[r] < min_clock;
+    total += evict_rows(t, s, dead);
+  }
+  return total;
+}
+
+uint64_t orc_clock(void* p) { return ((Table*)p)->clock; }
 
 // Test hook: add delta to one stored weight (col < k: latent component,
 // col == k: linear weight).  Used by the finite-difference pins.

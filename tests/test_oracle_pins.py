@@ -534,6 +534,107 @@ def test_adagrad_is_lazy(init_acc):
         np.testing.assert_allclose(after["acc_emb"], acc, rtol=2e-5, atol=1e-9)
 
 
+# --------------------------------------------------------------------------- eviction
+def _table_by_key(o, w):
+    """{(shard, key): (row, emb bits, lin, acc_emb bits, acc_lin)} of everything in the oracle's table."""
+    out = {}
+    for s, n in enumerate(o.size()):
+        n = int(n)
+        if not n:
+            continue
+        r = o.read_rows(np.full(n, s, np.uint8), np.arange(n, dtype=np.uint32))
+        for i in range(n):
+            out[(s, int(r["keys"][i]))] = (i, r["emb"][i].tobytes(), float(r["lin"][i]), r["acc_emb"][i].tobytes(),
+                                          float(r["acc_lin"][i]))
+    return out
+
+
+@pytest.mark.parametrize("partition", [PART_HASH, PART_FIELD])
+def test_eviction_by_key_list(partition):
+    # Section 1 ("Dynamic Features"): the live feature set changes over time.  After removing keys: they look
+    # up as "no row"; every other key keeps its contents; a shard's rows are 0 .. n-1, the freed rows below
+    # the new size taken by the survivors from beyond it in ascending order (brute-force model below); and a
+    # removed key that comes back is a new key: fresh initial weights, zero linear weight, initial state.
+    w, b = tiny(S=3, partition=partition, optimizer=OPT_ADAGRAD, vocab=200, B=40)
+    w = w.scaled(init_acc=0.1)
+    o = Oracle.for_workload(w)
+    fi = o.find_or_insert(b)
+    g = synth.upstream_grads(w, b.batch, 0)
+    part = o.forward_partials(w.ops, b, fi)
+    agg = o.aggregate(b.batch, part)
+    o.backward_update(w.ops, b, fi, agg["A"].astype(np.float32), None, g["gL"], g["gF"], g["gE"])   # rows differ from init now
+    before = _table_by_key(o, w)
+    sizes0 = [int(v) for v in o.size()]
+    rng = np.random.default_rng(9)
+    uniq = np.unique(b.ids)
+    gone = rng.choice(uniq, size=uniq.size // 3, replace=False)
+    ghost = synth.fmix64(np.arange(10_000, 10_005, dtype=np.uint64))                 # never inserted
+    n_ev = o.evict_keys(np.concatenate([gone, gone[:3], ghost]))
+    gone_set = set(int(x) for x in gone)
+    assert n_ev == sum(1 for (s, key) in before if key in gone_set)
+    after = _table_by_key(o, w)
+    assert set(after) == {sk for sk in before if sk[1] not in gone_set}
+    for sk, v in after.items():
+        assert v[1:] == before[sk][1:], "contents of a surviving key changed"
+    # row numbers: brute-force model of the compaction rule
+    for s in range(w.shards):
+        old = sorted((v[0], key) for (ss, key), v in before.items() if ss == s)
+        dead = [key in gone_set for _, key in old]
+        m = len(old) - sum(dead)
+        rows = {key: r for r, key in old if key not in gone_set}
+        holes = [r for r in range(m) if dead[r]]
+        movers = [old[r][1] for r in range(m, len(old)) if not dead[r]]
+        assert len(holes) == len(movers)
+        for r, key in zip(holes, movers):
+            rows[key] = r
+        assert sorted(rows.values()) == list(range(m))
+        for key, r in rows.items():
+            assert after[(s, key)][0] == r
+        assert int(o.size()[s]) == m
+    # lookups
+    look = o.find_or_insert(b, insert=False)
+    is_gone = np.isin(b.ids, gone)
+    assert np.all(look["rows"][is_gone] == 0xFFFFFFFF) and np.all(look["rows"][~is_gone] != 0xFFFFFFFF)
+    assert sum(int(v) for v in o.size()) == sum(sizes0) - n_ev
+    # the removed keys come back as new keys
+    fi2 = o.find_or_insert(b)
+    fresh = Oracle.for_workload(w)
+    ff = fresh.find_or_insert(b)
+    back = _table_by_key(o, w)
+    init = _table_by_key(fresh, w)
+    for (s, key), v in back.items():
+        if key in gone_set:
+            assert v[1:] == init[(s, key)][1:], "a re-inserted key must start from its initial row"
+        else:
+            assert v[1:] == before[(s, key)][1:]
+    assert np.array_equal(fi2["shards"], ff["shards"])
+
+
+def test_eviction_of_stale_keys():
+    # keys that were neither inserted nor updated since a given reading of the table's clock go; the rest stay
+    w, _ = tiny(S=4, optimizer=OPT_ADAGRAD, vocab=500, B=30)
+    o = Oracle.for_workload(w)
+    st = synth.Stream(w)
+    seen_at = {}
+    for step in range(4):
+        b = st.next_batch()
+        fi = o.find_or_insert(b)
+        assert o.clock() == step + 1
+        g = synth.upstream_grads(w, b.batch, step)
+        agg = o.aggregate(b.batch, o.forward_partials(w.ops, b, fi))
+        o.backward_update(w.ops, b, fi, agg["A"].astype(np.float32), None, g["gL"], g["gF"], g["gE"])
+        for key in np.unique(b.ids):
+            seen_at[int(key)] = step + 1
+    n0 = sum(int(v) for v in o.size())
+    assert n0 == len(seen_at)
+    n_ev = o.evict_stale(3)                       # last touched at clock 1 or 2
+    stale = {key for key, c in seen_at.items() if c < 3}
+    assert n_ev == len(stale) and 0 < n_ev < n0
+    left = {key for (_, key) in _table_by_key(o, w)}
+    assert left == set(seen_at) - stale
+    assert o.evict_stale(3) == 0
+
+
 # --------------------------------------------------------------------------- all-cores build
 @pytest.mark.parametrize("cfg", [2, 5])
 def test_openmp_build_equals_the_sequential_oracle(cfg):
