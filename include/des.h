@@ -342,6 +342,31 @@ des_status_t des_table_write_rows(des_table_t* t, const uint32_t* d_global_rows,
                                   const float* d_emb, const float* d_lin, const float* d_acc_emb,
                                   const float* d_acc_lin, void* stream);
 
+/* ---- eviction (Section 1, "Dynamic Features": the live feature set of a streaming model
+ * changes over time; the paper's table — Section 5 — has no delete, this is the reading) --- */
+
+/* Removes keys from the table.  A removed key looks up as DES_ROW_NONE; inserting it again
+ * makes a new key of it (fresh initial weights and state).  Every other key keeps its
+ * contents.  Row numbers: a shard's rows stay 0 .. n-1 — the rows freed below the shard's
+ * new size are taken, in ascending order, by the surviving rows from beyond it, in
+ * ascending order; all other rows keep their numbers.  Row numbers, unique indices and
+ * anything else derived from a batch before the call are stale afterwards: run
+ * des_find_or_insert again.
+ *   des_table_evict_keys   the n keys of the device array d_keys (unknown or repeated keys
+ *                          are ignored; under DES_PART_FIELD a key is removed from every
+ *                          shard that holds it);
+ *   des_table_evict_stale  every key whose row was neither inserted nor updated by
+ *                          des_backward_update since the table's clock read min_clock.  The
+ *                          clock (des_table_clock) counts the inserting des_find_or_insert
+ *                          calls that had at least one occurrence.
+ * *h_n_evicted (optional) = number of rows removed.  Maintenance calls: they synchronise the
+ * device, allocate temporaries with cudaMalloc (4 bytes per table row, 16 bytes per surviving
+ * key of the shards that lose a key) and free them before returning; not for use inside a
+ * stream capture.  Errors: DES_ERR_INVALID_ARG, DES_ERR_CUDA (also: out of memory). */
+des_status_t des_table_evict_keys(des_table_t* t, const uint64_t* d_keys, int64_t n, uint64_t* h_n_evicted);
+des_status_t des_table_evict_stale(des_table_t* t, uint64_t min_clock, uint64_t* h_n_evicted);
+des_status_t des_table_clock(des_table_t* t, uint64_t* h_clock);
+
 /* Second optimizer-state slot of the same rows (what des_table_read_rows /
  * write_rows do for the first): Adam's v of the latent vectors [n][k] and the
  * second state word of the linear weight [n] (Adam's v, FTRL's z; the first

@@ -256,7 +256,7 @@ int64_t orc_find_or_insert(void* p, const int32_t* offsets, const uint64_t* ids,
                            uint32_t* rows, uint8_t* shards, uint32_t* uidx,
                            uint8_t* uniq_shard, uint32_t* uniq_row) {
   Table* t = (Table*)p;
-  if (insert) t->clock += 1;                     // reading: the table's age clock counts inserting calls
+  if (insert && offsets[(int64_t)B * t->F] > 0) t->clock += 1;   // reading: the table's age clock counts the inserting calls (with at least one occurrence)
   std::unordered_map<uint64_t, uint32_t> seen;   // (shard<<32 | row) -> u
   int64_t U = 0;
   for (int64_t bag = 0; bag < (int64_t)B * t->F; ++bag) {

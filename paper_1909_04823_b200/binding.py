@@ -30,7 +30,8 @@ EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_f
            "des_table_read_state2", "des_table_write_state2",
            "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_cross_forward", "des_cross_backward",
            "des_cross_workspace_floats", "des_comm_volume", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string",
-           "des_build_has_tensor_cores", "des_table_uses_tensor_cores", "des_build_is_debug"]
+           "des_build_has_tensor_cores", "des_table_uses_tensor_cores", "des_build_is_debug",
+           "des_table_evict_keys", "des_table_evict_stale", "des_table_clock"]
 
 
 class des_comm_model_t(C.Structure):
@@ -167,6 +168,9 @@ def _declare(L):
     L.des_build_has_tensor_cores.argtypes = []
     L.des_table_uses_tensor_cores.argtypes = [C.c_void_p]
     L.des_build_is_debug.argtypes = []
+    L.des_table_evict_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_uint64)]
+    L.des_table_evict_stale.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
+    L.des_table_clock.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
     return L
 
 
@@ -356,6 +360,22 @@ class Table:
         out = (C.c_uint64 * (self.S + 1))()
         self._check(self.L.des_table_row_base(self.h, out), "des_table_row_base")
         return [int(v) for v in out]
+
+    def evict_keys(self, keys: torch.Tensor) -> int:
+        """keys: int64 / uint64 device tensor of ids to remove.  Returns the number of rows removed."""
+        n = C.c_uint64(0)
+        self._check(self.L.des_table_evict_keys(self.h, _ptr(keys), int(keys.numel()), C.byref(n)), "des_table_evict_keys")
+        return int(n.value)
+
+    def evict_stale(self, min_clock: int) -> int:
+        n = C.c_uint64(0)
+        self._check(self.L.des_table_evict_stale(self.h, int(min_clock), C.byref(n)), "des_table_evict_stale")
+        return int(n.value)
+
+    def clock(self) -> int:
+        c = C.c_uint64(0)
+        self._check(self.L.des_table_clock(self.h, C.byref(c)), "des_table_clock")
+        return int(c.value)
 
     def uses_tensor_cores(self) -> bool:
         return bool(self.L.des_table_uses_tensor_cores(self.h))

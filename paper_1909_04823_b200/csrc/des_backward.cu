@@ -488,6 +488,7 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2) {
   const int K4 = k >> 2, stride = k + 4;
   const OptParams opt = des_opt_load(opt_in, meta);
+  const float stamp = des_stamp_bits(meta->clock);     // "updated in the step of the current batch" (eviction by age)
   long long U = *n_uniq;
   if (U > max_uniq) U = max_uniq;
   const int c4 = (int)(threadIdx.x % G);
@@ -567,7 +568,7 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
           if (opt.lin_optimizer == DES_LIN_FTRL) des_ftrl_step(opt, lw[q], st[q].x, st[q].y, tail[q].x);
           else des_opt_step(opt, lw[q], st[q].x, st[q].y, tail[q].x);
         }
-        w[K4] = make_float4(lw[q], n2, 0.f, 0.f);
+        w[K4] = make_float4(lw[q], n2, stamp, 0.f);
         if (a && upd_w) a[K4] = make_float4(st[q].x, st[q].y, 0.f, 0.f);
       }
     }

@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
         const uint32_t n = hi[q] - lo[q];
         // position inside the region: the top bits of an odd multiple of the same mixed word (the shard is its
         // residue mod S; a second full mixing round bought nothing measurable in probe lengths)
-        cur[q] = lo[q] + (uint32_t)__umul64hi(h * 0x9E3779B97F4A7C15ull, (unsigned long long)n);
+        cur[q] = des_slot_home(h, lo[q], n);
         nmax = max(nmax, n);
       }
     }
@@ -389,7 +389,8 @@ __global__ void __launch_bounds__(256) init_new_rows_kernel(
     if (!init) continue;
     float4* w = reinterpret_cast<float4*>(W + (size_t)grow * stride);
     if (c4 < K4) w[c4] = v;
-    if (c4 == 0) w[K4] = make_float4(0.f, n2, 0.f, 0.f);      // linear weight, squared norm of the latent vector
+    // linear weight, squared norm of the latent vector, age stamp (the clock value this call ends with)
+    if (c4 == 0) w[K4] = make_float4(0.f, n2, des_stamp_bits(meta->clock + 1ull), 0.f);
     if (A) {
       float4* a = reinterpret_cast<float4*>(A + (size_t)grow * stride);
       if (c4 < K4) a[c4] = make_float4(state_init, state_init, state_init, state_init);
@@ -450,6 +451,7 @@ __global__ void __launch_bounds__(DES_MAX_SHARDS) finish_kernel(int S, int nnz, 
   if (threadIdx.x == 0) {
     *n_uniq_out = meta->n_uniq;
     meta->any_new = 0u;
+    meta->clock += 1ull;
     const uint32_t base = meta->scratch_base - (uint32_t)nnz;
     // the next call may need up to max_nnz below the base; if that is not left, assign_kernel has
     // cleared every slot's scratch word in this call and the range starts again at the top

@@ -49,6 +49,8 @@ struct DevMeta {
   uint32_t any_new;                                  // the running insert call has at least one new key
   uint32_t scratch_base;                             // see Slot::first_occ: the last insert call's base
   uint32_t field_order[1024];                        // fields sorted by (owning shard, field)
+  unsigned long long clock;                          // inserting find_or_insert calls so far: the age clock that
+                                                     // stamps a row when it is inserted or updated (eviction by age)
   unsigned long long opt_step;                       // backward calls so far (Adam's t), advanced on device
   float adam_c1, adam_c2;                            // 1 - beta1^t, 1 - beta2^t for the running step
 };
@@ -189,6 +191,14 @@ __device__ __forceinline__ int des_bag_of(const int32_t* __restrict__ offsets, i
 }
 
 __device__ __forceinline__ void des_raise(DevMeta* meta, uint32_t code) { atomicCAS(&meta->err, 0u, code); }
+
+// First slot a key is looked for in, inside its shard's region of n slots starting at lo: the top bits of an odd
+// multiple of the mixed key (the shard is the same word's residue mod S, so the two are independent).
+__device__ __forceinline__ uint32_t des_slot_home(unsigned long long mixed, uint32_t lo, uint32_t n) {
+  return lo + (uint32_t)__umul64hi(mixed * 0x9E3779B97F4A7C15ull, (unsigned long long)n);
+}
+// The age stamp lives in the third word of a row's 16-byte tail, stored as raw bits.
+__device__ __forceinline__ float des_stamp_bits(unsigned long long clock) { return __uint_as_float((uint32_t)clock); }
 
 // Optimizer parameters handed to the update kernels by value.
 struct OptParams {
