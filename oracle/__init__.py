@@ -133,6 +133,32 @@ def cross_backward(x0, x, w, P, gY):
     return dict(gx0=gx0, gx=gx, gw=gw, gb=gb, t=t)
 
 
+def head(hc, R_lr=None, fm2=None, Z=None, pooled=None, xdense=None, y=None):
+    """The fixed read-out (see des_oracle.cpp: orc_head).  hc: dict(b0, c_lr, c_fm, u, b1, q, d) of float32
+    constants; inputs float64 (the oracle's aggregates) except xdense / y (float32).  Terms whose input is
+    None are left out.  -> dict(logit, loss [B], gL, gF, gZ, gE) in float64 (None where not applicable)."""
+    B = int(y.shape[0])
+    f64 = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.float64)
+    f32 = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+    R_lr, fm2, Z, pooled = map(f64, (R_lr, fm2, Z, pooled))
+    xdense, y = f32(xdense), f32(y)
+    u, b1, q, d = f32(hc.get("u")), f32(hc.get("b1")), f32(hc.get("q")), f32(hc.get("d"))
+    H = 0 if Z is None else Z.shape[1]
+    FK = 0 if pooled is None else pooled.shape[1]
+    nd = 0 if xdense is None else xdense.shape[1]
+    logit = np.zeros(B); loss = np.zeros(B)
+    gL = np.zeros(B) if R_lr is not None else None
+    gF = np.zeros(B) if fm2 is not None else None
+    gZ = np.zeros((B, H)) if Z is not None else None
+    gE = np.zeros((B, FK)) if pooled is not None else None
+    lib().orc_head(C.c_int64(B), C.c_int64(H), C.c_int64(FK), C.c_int64(nd), C.c_double(float(hc["b0"])),
+                   C.c_double(float(hc["c_lr"])), C.c_double(float(hc["c_fm"])), _p(u, C.c_float), _p(b1, C.c_float),
+                   _p(q, C.c_float), _p(d, C.c_float), _p(R_lr, C.c_double), _p(fm2, C.c_double), _p(Z, C.c_double),
+                   _p(pooled, C.c_double), _p(xdense, C.c_float), _p(y, C.c_float), _p(logit, C.c_double),
+                   _p(loss, C.c_double), _p(gL, C.c_double), _p(gF, C.c_double), _p(gZ, C.c_double), _p(gE, C.c_double))
+    return dict(logit=logit, loss=loss, gL=gL, gF=gF, gZ=gZ, gE=gE)
+
+
 class Oracle:
     def __init__(self, S, F, k, H=0, partition=0, optimizer=0, seed=0, init_scale=0.01,
                  lr=0.01, eps=1e-8, init_acc=0.0, omp=False):

@@ -661,6 +661,41 @@ int64_t orc_evict_stale(void* p, uint64_t min_clock) {
 
 uint64_t orc_clock(void* p) { return ((Table*)p)->clock; }
 
+// A fixed read-out that stands for the rest of the model (the layers above the first FC layer in Section
+// 4.3 / Fig. 4, which the sparse path does not contain): it turns the aggregated results into one logit
+// per sample and the log loss into upstream gradients, so that multi-step runs are closed loops.  Nothing
+// in it is trained; b0, c_lr, c_fm, u[H], b1[H], q[F*k], d[n_dense] are seeded constants.
+//   logit = b0 + c_lr R_lr + c_fm fm2 + <u, relu(Z + b1)> + <q, pooled> + <d, xdense>
+//           (each term only when its input pointer is given)
+//   p = 1 / (1 + exp(-logit));  loss_b = -(y log p + (1 - y) log(1 - p));  L = mean_b loss_b
+//   g = dL/dlogit = (p - y) / B;  gL = c_lr g;  gF = c_fm g;  gZ = g u (Z + b1 > 0);  gE = g q
+// The paper fixes none of this: parity unpinned by the paper; pinned against the library's
+// binary_cross_entropy_with_logits and autograd in the tests.
+void orc_head(int64_t B, int64_t H, int64_t FK, int64_t nd, double b0, double c_lr, double c_fm,
+              const float* u, const float* b1, const float* q, const float* d,
+              const double* R_lr, const double* fm2, const double* Z, const double* pooled, const float* xdense,
+              const float* y, double* logit, double* loss, double* gL, double* gF, double* gZ, double* gE) {
+  for (int64_t b = 0; b < B; ++b) {
+    double z = b0;
+    if (R_lr) z += c_lr * R_lr[b];
+    if (fm2) z += c_fm * fm2[b];
+    if (Z) for (int64_t h = 0; h < H; ++h) { double a = Z[b * H + h] + (double)b1[h]; if (a > 0) z += (double)u[h] * a; }
+    if (pooled) for (int64_t i = 0; i < FK; ++i) z += (double)q[i] * pooled[b * FK + i];
+    if (xdense) for (int64_t i = 0; i < nd; ++i) z += (double)d[i] * (double)xdense[b * nd + i];
+    // log(1 + exp(-|z|)) + max(-z, 0) = -log sigmoid(z), without overflow
+    const double sp_neg = std::log1p(std::exp(-std::fabs(z))) + (z < 0 ? -z : 0.0);   // -log p
+    const double sp_pos = sp_neg + z;                                                   // -log (1 - p)
+    const double yy = (double)y[b], p = 1.0 / (1.0 + std::exp(-z));
+    logit[b] = z;
+    loss[b] = yy * sp_neg + (1.0 - yy) * sp_pos;
+    const double g = (p - yy) / (double)B;
+    if (gL) gL[b] = c_lr * g;
+    if (gF) gF[b] = c_fm * g;
+    if (gZ) for (int64_t h = 0; h < H; ++h) gZ[b * H + h] = (Z[b * H + h] + (double)b1[h] > 0) ? g * (double)u[h] : 0.0;
+    if (gE) for (int64_t i = 0; i < FK; ++i) gE[b * FK + i] = g * (double)q[i];
+  }
+}
+
 // Test hook: add delta to one stored weight (col < k: latent component,
 // col == k: linear weight).  Used by the finite-difference pins.
 void orc_poke(void* p, uint32_t shard, uint32_t row, uint32_t col, float value, int set) {

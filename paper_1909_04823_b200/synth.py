@@ -257,3 +257,38 @@ def dense1_weights(w: Workload) -> np.ndarray:
     rng = np.random.default_rng([w.seed, 104729])
     K = w.fields * w.emb_dim
     return (rng.standard_normal((K, w.hidden)) / np.sqrt(K)).astype(np.float32)
+
+
+def head_constants(w: Workload, n_dense: int = 0):
+    """Seeded constants of the fixed read-out that closes the loop in multi-step runs (not trained):
+    b0, c_lr, c_fm, u [H], b1 [H], q [F*k], d [n_dense], float32.  Scales are chosen from the workload's shape
+    so that the logit of the first step is of order one (c_fm shrinks with the square of the number of ids
+    per sample, which is how the order-2 term grows when a hot id repeats)."""
+    rng = np.random.default_rng([w.seed, 15485863])
+    K = w.fields * w.emb_dim
+    mean_len = {"onehot": 1.0, "uniform": 0.5 * (w.len_a + w.len_b), "poisson1": w.len_a + 1.0,
+                "geometric": min(1.0 / max(w.len_a, 1e-9), w.len_b)}[w.len_law]
+    n_occ = w.fields * mean_len
+    hc = {"b0": np.float32(-1.0), "c_lr": np.float32(1.0),
+          "c_fm": np.float32(1.0 / (1.0 + 0.01 * n_occ * n_occ * w.emb_dim * w.init_scale ** 2)),
+          "u": None, "b1": None, "q": None, "d": None}
+    if w.hidden:
+        hc["u"] = (rng.standard_normal(w.hidden) / np.sqrt(w.hidden)).astype(np.float32)
+        hc["b1"] = (0.1 * rng.standard_normal(w.hidden)).astype(np.float32)
+    elif w.ops & OP_POOL:
+        hc["q"] = (rng.standard_normal(K) / (np.sqrt(K) * max(w.init_scale * np.sqrt(mean_len), 1e-6))).astype(np.float32)
+    if n_dense:
+        hc["d"] = (rng.standard_normal(n_dense) / np.sqrt(n_dense)).astype(np.float32)
+    return hc
+
+
+def labels(w: Workload, batch: int, step: int, p: float = 0.25) -> np.ndarray:
+    """Seeded Bernoulli(p) click labels, float32 [B]."""
+    rng = np.random.default_rng([w.seed, 32452843, step])
+    return (rng.random(batch) < p).astype(np.float32)
+
+
+def dense_features(w: Workload, batch: int, step: int, n_dense: int) -> np.ndarray:
+    """Seeded N(0, 1) continuous features [B][n_dense], float32 (the 13 continuous Criteo columns)."""
+    rng = np.random.default_rng([w.seed, 49979687, step])
+    return rng.standard_normal((batch, n_dense)).astype(np.float32)

@@ -635,6 +635,50 @@ def test_eviction_of_stale_keys():
     assert o.evict_stale(3) == 0
 
 
+# --------------------------------------------------------------------------- read-out head
+@pytest.mark.parametrize("with_dense1", [True, False])
+def test_head_matches_library_log_loss_and_autograd(with_dense1):
+    # The fixed read-out that closes the loop in multi-step runs: its loss is the library's
+    # binary_cross_entropy_with_logits (mean over the batch) of the logit written out below, and its four
+    # upstream gradients are autograd's.
+    import torch.nn.functional as Fn
+    rng = np.random.default_rng(12)
+    B, H, FK, nd = 9, 7, 10, 3
+    hc = dict(b0=np.float32(-0.3), c_lr=np.float32(0.7), c_fm=np.float32(0.2),
+              u=rng.standard_normal(H).astype(np.float32), b1=rng.standard_normal(H).astype(np.float32),
+              q=rng.standard_normal(FK).astype(np.float32), d=rng.standard_normal(nd).astype(np.float32))
+    R = torch.tensor(rng.standard_normal(B), requires_grad=True)
+    Fm = torch.tensor(rng.standard_normal(B), requires_grad=True)
+    Z = torch.tensor(rng.standard_normal((B, H)), requires_grad=True)
+    Pl = torch.tensor(rng.standard_normal((B, FK)), requires_grad=True)
+    xd = rng.standard_normal((B, nd)).astype(np.float32)
+    y = (rng.random(B) < 0.4).astype(np.float32)
+    y[0] = 0.25                                            # soft labels work too
+    t64 = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
+    logit = float(hc["b0"]) + float(hc["c_lr"]) * R + float(hc["c_fm"]) * Fm + t64(xd) @ t64(hc["d"])
+    if with_dense1:
+        logit = logit + torch.relu(Z + t64(hc["b1"])) @ t64(hc["u"])
+    else:
+        logit = logit + Pl @ t64(hc["q"])
+    per = Fn.binary_cross_entropy_with_logits(logit, t64(y), reduction="none")
+    per.mean().backward()
+    got = oracle.head(hc, R.detach().numpy(), Fm.detach().numpy(), Z.detach().numpy() if with_dense1 else None,
+                      None if with_dense1 else Pl.detach().numpy(), xd, y)
+    np.testing.assert_allclose(got["logit"], logit.detach().numpy(), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(got["loss"], per.detach().numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(got["gL"], R.grad.numpy(), rtol=1e-10, atol=1e-15)
+    np.testing.assert_allclose(got["gF"], Fm.grad.numpy(), rtol=1e-10, atol=1e-15)
+    if with_dense1:
+        np.testing.assert_allclose(got["gZ"], Z.grad.numpy(), rtol=1e-10, atol=1e-15)
+        assert got["gE"] is None
+    else:
+        np.testing.assert_allclose(got["gE"], Pl.grad.numpy(), rtol=1e-10, atol=1e-15)
+    # extreme logits neither overflow nor lose the loss
+    big = oracle.head(dict(hc, c_lr=np.float32(1.0), c_fm=np.float32(0.0), b0=np.float32(0.0), d=None),
+                      np.array([800.0, -800.0]), np.zeros(2), None, None, None, np.array([0.0, 1.0], np.float32))
+    np.testing.assert_allclose(big["loss"], [800.0, 800.0], rtol=1e-12)
+
+
 # --------------------------------------------------------------------------- all-cores build
 @pytest.mark.parametrize("cfg", [2, 5])
 def test_openmp_build_equals_the_sequential_oracle(cfg):
