@@ -363,6 +363,20 @@ def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want
     gE = gd.get("gE") if (w.ops & OP_POOL) else None
     gZ = gd.get("gZ") if (w.ops & OP_DENSE1) else None
 
+    # closed loop: the upstream gradients of every step come from the fixed read-out applied to that step's own
+    # forward results (labels and continuous features are seeded and resident on the device)
+    closed = None
+    if args.closed_loop:
+        n_dense = 13 if cfg_index == 2 else 0          # the Criteo shape: 13 continuous columns beside the 26 categorical
+        hc = synth.head_constants(w, n_dense)
+        closed = dict(hc={n_: (torch.from_numpy(v).to(dev) if isinstance(v, np.ndarray) and v.ndim else v) for n_, v in hc.items()},
+                      y=torch.from_numpy(synth.labels(w, B, 0)).to(dev),
+                      xd=torch.from_numpy(synth.dense_features(w, B, 0, n_dense)).to(dev) if n_dense else None,
+                      logit=torch.zeros(B, device=dev), loss=torch.zeros(B, device=dev),
+                      gL=torch.zeros(B, device=dev), gF=torch.zeros(B, device=dev),
+                      gE=torch.zeros((B, F * k), device=dev) if (pool and not (w.ops & OP_DENSE1)) else None,
+                      gZ=torch.zeros((B, H), device=dev) if (w.ops & OP_DENSE1) else None)
+
     def step(i):
         db = dbs[i % len(dbs)]
         t.find_or_insert(db, True)
@@ -371,7 +385,13 @@ def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want
         else:
             t.forward_partials(w.ops, db, part_small, pooled)
             t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
-        t.backward_update(w.ops, db, out_small, pooled, Z, gd.get("gL"), gd.get("gF"), gE, gZ, gE_work)
+        if closed is None:
+            t.backward_update(w.ops, db, out_small, pooled, Z, gd.get("gL"), gd.get("gF"), gE, gZ, gE_work)
+        else:
+            c = closed
+            t.head(w.ops, B, c["hc"], out_small, pooled, Z, c["xd"], c["y"], c["logit"], c["loss"], c["gL"], c["gF"],
+                   c["gE"], c["gZ"])
+            t.backward_update(w.ops, db, out_small, pooled, Z, c["gL"], c["gF"], c["gE"], c["gZ"], gE_work)
 
     U = None
     stats = None
@@ -572,6 +592,10 @@ def main():
                          "come from a separate, untimed eager pass")
     ap.add_argument("--fused", action="store_true",
                     help="use des_forward_fused (per-shard partials kept on chip) instead of partials + aggregate")
+    ap.add_argument("--closed-loop", action="store_true",
+                    help="gradients from the fixed read-out (des_head) on the step's own forward instead of seeded "
+                         "upstream gradients: the whole Criteo-shaped Wide&Deep / DeepFM step with --config 2 / 3 "
+                         "(throughput only: the dataset is not available here)")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -643,7 +667,7 @@ def main():
 
     mode = "graph" if args.graph else "eager"
     r = run_workload(args, args.config, w, ctx, steps=args.steps, warmup=args.warmup, repeats=args.repeats, modes=[mode],
-                     want_e2e=not args.no_e2e, want_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline),
+                     want_e2e=not (args.no_e2e or args.closed_loop), want_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline),
                      profile_in_timed=True)
     clocks = sampler.stop(r["windows"]) if sampler else None
     m = r["results"][mode]
@@ -667,6 +691,9 @@ def main():
                            "forward": "fused (per-shard partials on chip)" if args.fused else
                                       "per-shard partials materialised, then aggregated",
                            "tensor_core_gemm": bool(binding.uses_tensor_cores()),
+                           "gradients": "closed loop: fixed read-out + log loss on the step's own forward (synthetic labels; "
+                                        "the paper's datasets are not available here)" if args.closed_loop else
+                                        "seeded upstream gradients, resident on the device",
                            "l2": r["l2_note"]},
                 "timing": "ms_per_step = median over `repeats.n` back-to-back timings of --steps steps each",
                 "repeats": m["repeats"],

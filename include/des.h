@@ -410,6 +410,30 @@ des_status_t des_step_host_submit(des_table_t* t, uint32_t ops, int32_t batch, i
                                   float* h_out_small, void* stream, int32_t* ticket);
 des_status_t des_step_host_wait(des_table_t* t, int32_t ticket);
 
+/* ---- a fixed read-out in place of the rest of the model ---------------------- */
+
+/* The sparse path ends at the aggregated results (R_lr, fm2, pooled, Z); the layers above them (Section 4.3,
+ * Fig. 4: the rest of the DNN, the output unit, the loss) are not part of it.  So that multi-step runs and
+ * closed-loop measurements need no gradients from outside, des_head stands in for them with a read-out
+ * whose constants are given and never trained (the paper has no counterpart for its particular form):
+ *   logit = b0 + c_lr R_lr + c_fm fm2 + <u, relu(Z + b1)> + <q, pooled> + <d, xdense>
+ *   p = sigmoid(logit);  loss_b = -(y_b log p + (1 - y_b) log(1 - p));  g = (p - y_b) / batch
+ *   gL = c_lr g;  gF = c_fm g;  gZ = g u [Z + b1 > 0];  gE = g q
+ * Terms follow `ops`: R_lr with DES_OP_LR, fm2 with DES_OP_FM, the Z term with DES_OP_DENSE1 (then there
+ * is no pooled term: pooled feeds the first layer), the pooled term with DES_OP_POOL alone, the xdense term
+ * when d and d_xdense [batch][n_dense] are given.  All pointers are device pointers; u, b1 [H]; q [F*k];
+ * d [n_dense]; d_y [batch] labels in [0, 1]; d_logit, d_loss [batch] outputs; the gradient arrays are what
+ * des_grads_t expects (gL, gF [batch]; gE [batch][F*k]; gZ [batch][H]).  Enqueued on `stream`. */
+typedef struct {
+  float b0, c_lr, c_fm;
+  const float* u; const float* b1; const float* q; const float* d;
+  int32_t n_dense;
+} des_head_t;
+typedef struct { float* gL; float* gF; float* gE; float* gZ; } des_head_grads_t;
+des_status_t des_head(des_table_t* t, uint32_t ops, int32_t batch, const des_head_t* head, const des_outputs_t* out,
+                      const float* d_xdense, const float* d_y, float* d_logit, float* d_loss,
+                      const des_head_grads_t* g, void* stream);
+
 /* ---- DCN cross layer under DES (Section 4.4, paragraph on DCN) --------------- */
 
 /* y = x0 * (+)_s <x[slice s], w[slice s]> + b + x  for x0, x, y [B][d] and w, b [d]

@@ -31,7 +31,7 @@ EXPORTS = ["des_table_create", "des_table_destroy", "des_find_or_insert", "des_f
            "des_step_host", "des_step_host_submit", "des_step_host_wait", "des_cross_forward", "des_cross_backward",
            "des_cross_workspace_floats", "des_comm_volume", "des_profile_enable", "des_profile_read", "des_table_launch_count", "des_status_string",
            "des_build_has_tensor_cores", "des_table_uses_tensor_cores", "des_build_is_debug",
-           "des_table_evict_keys", "des_table_evict_stale", "des_table_clock"]
+           "des_table_evict_keys", "des_table_evict_stale", "des_table_clock", "des_head"]
 
 
 class des_comm_model_t(C.Structure):
@@ -77,6 +77,15 @@ class des_partials_t(C.Structure):
 
 class des_outputs_t(C.Structure):
     _fields_ = [("out_small", C.c_void_p), ("pooled", C.c_void_p), ("Z", C.c_void_p)]
+
+
+class des_head_t(C.Structure):
+    _fields_ = [("b0", C.c_float), ("c_lr", C.c_float), ("c_fm", C.c_float), ("u", C.c_void_p), ("b1", C.c_void_p),
+                ("q", C.c_void_p), ("d", C.c_void_p), ("n_dense", C.c_int32)]
+
+
+class des_head_grads_t(C.Structure):
+    _fields_ = [("gL", C.c_void_p), ("gF", C.c_void_p), ("gE", C.c_void_p), ("gZ", C.c_void_p)]
 
 
 class des_grads_t(C.Structure):
@@ -171,6 +180,8 @@ def _declare(L):
     L.des_table_evict_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.POINTER(C.c_uint64)]
     L.des_table_evict_stale.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
     L.des_table_clock.argtypes = [C.c_void_p, C.POINTER(C.c_uint64)]
+    L.des_head.argtypes = [C.c_void_p, C.c_uint32, C.c_int32, C.POINTER(des_head_t), C.POINTER(des_outputs_t),
+                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(des_head_grads_t), C.c_void_p]
     return L
 
 
@@ -360,6 +371,16 @@ class Table:
         out = (C.c_uint64 * (self.S + 1))()
         self._check(self.L.des_table_row_base(self.h, out), "des_table_row_base")
         return [int(v) for v in out]
+
+    def head(self, ops, batch_size, hc, out_small=None, pooled=None, Z=None, xdense=None, y=None, logit=None, loss=None,
+             gL=None, gF=None, gE=None, gZ=None):
+        """hc: dict(b0, c_lr, c_fm, u, b1, q, d) with device tensors (or None) for the vectors."""
+        h = des_head_t(float(hc["b0"]), float(hc["c_lr"]), float(hc["c_fm"]), _ptr(hc.get("u")), _ptr(hc.get("b1")),
+                       _ptr(hc.get("q")), _ptr(hc.get("d")), 0 if hc.get("d") is None else int(hc["d"].numel()))
+        o = des_outputs_t(_ptr(out_small), _ptr(pooled), _ptr(Z))
+        g = des_head_grads_t(_ptr(gL), _ptr(gF), _ptr(gE), _ptr(gZ))
+        self._check(self.L.des_head(self.h, ops, int(batch_size), C.byref(h), C.byref(o), _ptr(xdense), _ptr(y),
+                                    _ptr(logit), _ptr(loss), C.byref(g), _stream()), "des_head")
 
     def evict_keys(self, keys: torch.Tensor) -> int:
         """keys: int64 / uint64 device tensor of ids to remove.  Returns the number of rows removed."""

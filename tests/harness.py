@@ -222,14 +222,17 @@ class Pair:
 
     # ------------------------------------------------------------------
     def step(self, batch, grads, ops=None, materialise=False, check_init=False, by_key=False,
-             pooled_samples=None, dense_samples=None):
+             pooled_samples=None, dense_samples=None, head=None):
         """One full step on both sides with every intermediate compared.
         pooled_samples: compare `pooled` only on these sample indices (the dense
         per-shard pooled partial of the oracle is too large at full size).
         dense_samples: full-size first-layer workloads — the oracle's per-shard partial
         products P_s (S x B x H x F k multiply-adds) are skipped; `pooled` is compared in
         full against the unsubstituted operator, Z on these sample indices against the
-        unsubstituted operator on the sub-batch; the backward is compared in full."""
+        unsubstituted operator on the sub-batch; the backward is compared in full.
+        head: dict(hc=constants of the fixed read-out, y=labels [B], xdense=[B][n] or None) — the upstream
+        gradients are then not `grads` but what the read-out makes of each side's own forward (a closed
+        loop); with resync the CUDA backward is still fed the oracle's gradients, without it its own."""
         from paper_1909_04823_b200.binding import DeviceBatch
         w = self.w
         ops = w.ops if ops is None else ops
@@ -326,12 +329,59 @@ class Pair:
             close_gemm(Z.cpu().numpy(), oa["Z"], "Z")
             if materialise:
                 close_gemm(part_dense.cpu().numpy(), op["part_dense"], "part_dense")
+        # ---- the read-out in place of the rest of the model: each side's gradients from its own forward
+        head_out = None
+        if head is not None:
+            import oracle as _orc
+            hc, yv, xd = head["hc"], head["y"], head.get("xdense")
+            pool_term = bool(ops & OP_POOL) and not (ops & OP_DENSE1)
+            oh = _orc.head(hc, oa["lr"] if ops & OP_LR else None, oa["fm2"] if ops & OP_FM else None,
+                           oa["Z"] if ops & OP_DENSE1 else None, oa["pooled"] if pool_term else None, xd, yv)
+            td_ = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+            hcd = {n: (td_(v) if isinstance(v, np.ndarray) and v.ndim else v) for n, v in hc.items()}
+            h_logit = torch.full((B,), float("nan"), device=dev); h_loss = torch.full((B,), float("nan"), device=dev)
+            h_gL = torch.zeros(B, device=dev); h_gF = torch.zeros(B, device=dev)
+            h_gE = torch.full((B, F * k), float("nan"), device=dev) if pool_term else None
+            h_gZ = torch.full((B, H), float("nan"), device=dev) if (ops & OP_DENSE1) else None
+            self.t.head(ops, B, hcd, out_small, pooled, Z if (ops & OP_DENSE1) else None, td_(xd), td_(yv), h_logit, h_loss,
+                        h_gL, h_gF, h_gE, h_gZ)
+            torch.cuda.synchronize()
+            assert self.t.status() == 0
+            # the read-out sums hundreds of float32 forward results: a looser bound than the path's own
+            hcmp = close_gemm if ((ops & OP_DENSE1) or self.drifted) else (lambda a, r, wh: close32(a, r, wh, rtol=1e-4, atol=1e-5))
+            hcmp(h_logit.cpu().numpy(), oh["logit"], "head.logit")
+            hcmp(h_loss.cpu().numpy(), oh["loss"], "head.loss")
+            if ops & OP_LR:
+                hcmp(h_gL.cpu().numpy() * B, oh["gL"] * B, "head.gL")
+            if ops & OP_FM:
+                hcmp(h_gF.cpu().numpy() * B, oh["gF"] * B, "head.gF")
+            if pool_term:
+                hcmp(h_gE.cpu().numpy() * B, oh["gE"] * B, "head.gE")
+            if ops & OP_DENSE1:
+                # a unit whose pre-activation is within rounding of zero may switch on one side only
+                gz_g, gz_o = h_gZ.cpu().numpy() * B, oh["gZ"] * B
+                flip = (gz_g == 0) != (gz_o == 0)
+                pre = np.abs(oa["Z"] + hc["b1"][None, :].astype(np.float64))
+                assert np.all(pre[flip] <= 2e-2 * np.abs(oa["Z"][flip]) + 1e-3 * np.abs(oa["Z"]).max()), "relu gate"
+                hcmp(np.where(flip, gz_o, gz_g), gz_o, "head.gZ")
+            f32 = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+            grads = {n: f32(oh[n]) for n in ("gL", "gF", "gE", "gZ") if oh[n] is not None}
+            for n in ("gL", "gF"):
+                grads.setdefault(n, np.zeros(B, np.float32))
+            head_out = dict(oracle=oh, loss=float(oh["loss"].mean()), gpu_loss=float(h_loss.mean().item()))
         # ---- backward + update
         g = grads
         gdev = {n: torch.from_numpy(v).to(dev) for n, v in g.items()}
+        if head is not None and not self.resync:
+            gdev = {"gL": h_gL, "gF": h_gF}
+            if h_gE is not None:
+                gdev["gE"] = h_gE
+            if h_gZ is not None:
+                gdev["gZ"] = h_gZ
         gE_work = torch.empty((B, F * k), device=dev) if (ops & OP_DENSE1) else None
         before = self.o.read_rows(fi["uniq_shard"], fi["uniq_row"]) if w.lin_optimizer == synth.LIN_FTRL else None
         self.nstep += 1
+        W1_pre = self.o.dense1_get()[0].astype(np.float64) if (ops & OP_DENSE1) else None
         ob = self.o.backward_update(ops, batch, fi, oa["A"].astype(np.float32),
                                     oa["pooled"].astype(np.float32) if oa["pooled"] is not None else None,
                                     g.get("gL"), g.get("gF"), g.get("gE") if (ops & OP_POOL) else None,
@@ -353,7 +403,15 @@ class Pair:
         gemm = bool(ops & OP_DENSE1) or self.drifted
         W1o = None
         if ops & OP_DENSE1:
-            close_gemm(gE_work.cpu().numpy(), ob["gE_total"], "gE_total")
+            # the CUDA path rounds gZ to bfloat16 before the product (2^-9 relative per term), the oracle does not:
+            # where the terms of a row-times-column sum cancel, the bound is taken against their magnitudes
+            extra_gE = 2.0 ** -8 * (np.abs(g["gZ"].astype(np.float64)) @ np.abs(W1_pre).T)
+            if head is not None and not self.resync:
+                # free-running loop: the CUDA backward was fed its own read-out gradients; where they differ from
+                # the oracle's (compared above; a unit at the edge of its threshold is on on one side only) the
+                # difference goes through the same product
+                extra_gE = extra_gE + np.abs(gdev["gZ"].cpu().numpy().astype(np.float64) - g["gZ"].astype(np.float64)) @ np.abs(W1_pre).T
+            close_gemm(gE_work.cpu().numpy(), ob["gE_total"], "gE_total", extra=extra_gE)
             W1o, accW1o = self.o.dense1_get()
             acc2W1o = self.o.dense1_get_state2() if w.optimizer == synth.OPT_ADAM else None
             # same reasoning as for the rows: a 2e-2-relative error of the weight gradient, pushed
@@ -389,4 +447,4 @@ class Pair:
             torch.cuda.synchronize()
         else:
             self.drifted = True
-        return dict(fi=fi, db=db, oracle_agg=oa, out_small=osm, oracle_bwd=ob)
+        return dict(fi=fi, db=db, oracle_agg=oa, out_small=osm, oracle_bwd=ob, head=head_out)

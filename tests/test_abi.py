@@ -36,9 +36,9 @@ def test_struct_layouts_match_header_sizes():
     prog = r'''
 #include <stdio.h>
 #include "des.h"
-int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(des_config_t), sizeof(des_batch_t),
+int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu\n", sizeof(des_config_t), sizeof(des_batch_t),
   sizeof(des_partials_t), sizeof(des_outputs_t), sizeof(des_grads_t), sizeof(des_comm_model_t),
-  sizeof(des_comm_volume_t)); return 0; }
+  sizeof(des_comm_volume_t), sizeof(des_head_t), sizeof(des_head_grads_t)); return 0; }
 '''
     with tempfile.TemporaryDirectory() as d:
         open(os.path.join(d, "a.c"), "w").write(prog)
@@ -46,7 +46,7 @@ int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu\n", sizeof(des_config_t), s
         out = subprocess.check_output([os.path.join(d, "a")]).split()
     want = [C.sizeof(binding.des_config_t), C.sizeof(binding.des_batch_t), C.sizeof(binding.des_partials_t),
             C.sizeof(binding.des_outputs_t), C.sizeof(binding.des_grads_t), C.sizeof(binding.des_comm_model_t),
-            C.sizeof(binding.des_comm_volume_t)]
+            C.sizeof(binding.des_comm_volume_t), C.sizeof(binding.des_head_t), C.sizeof(binding.des_head_grads_t)]
     assert [int(v) for v in out] == want
 
 
