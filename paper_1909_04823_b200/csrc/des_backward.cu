@@ -242,7 +242,8 @@ __device__ __forceinline__ void scatter_step(const uint32_t* __restrict__ dest, 
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     if (SUPER) cnt += (d[u] == mine);
-    const bool ok = SUPER ? d[u] < SUPER_TAG : d[u] != DES_ROW_NONE;   // SUPER_TAG.. also covers "no row"
+    bool ok = SUPER ? d[u] < SUPER_TAG : d[u] != DES_ROW_NONE;   // SUPER_TAG.. also covers "no row"
+    if (ok && !DES_DBG_GRAD_OK(d[u])) ok = false;                     // (checking build)
     if (ok) {
       const size_t off = (size_t)d[u] * rowB;
       if (HAS_VALS) {
@@ -508,6 +509,7 @@ __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     for (int q = 0; q < UP_UNROLL; ++q) {
       const long long u = u0 + q * gstep;
       r[q] = (u < U) ? __ldg(uniq_rows + u) : DES_ROW_NONE;
+      if (r[q] != DES_ROW_NONE && DES_DBG_ROW(r[q]) != r[q]) r[q] = DES_ROW_NONE;   // (checking build)
       g[q] = zero; tail[q] = make_float2(0.f, 0.f);
       if (u < U) {
         const float4* grow = reinterpret_cast<const float4*>(Gbuf + (size_t)u * stride);
@@ -621,6 +623,7 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   if ((ops & DES_OP_DENSE1) && (!t->H || !gr->gZ || !gr->gE_work || !out->pooled)) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
   des_api_begin(t, cs);
+  DES_DBG_ARM(t, cs);
   const int B = b->batch;
   const OptParams opt = des_opt_params(t);
   if (opt.optimizer == DES_OPT_ADAM) {               // one optimizer step per backward call (Adam's t)

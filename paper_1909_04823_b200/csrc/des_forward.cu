@@ -148,7 +148,7 @@ __device__ __forceinline__ void sp_step(const uint32_t* __restrict__ grow_sorted
   float4 v[U]; float2 tl[U]; float x[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    const size_t off = (size_t)__ldg(grow_sorted + i + u * P) * rowB;
+    const size_t off = (size_t)DES_DBG_ROW(__ldg(grow_sorted + i + u * P)) * rowB;
     if (HAS_VALS) x[u] = __ldg(x_sorted + i + u * P);
     v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
     tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
@@ -175,7 +175,7 @@ __device__ __forceinline__ void pool_step(const uint32_t* __restrict__ grow_csr,
   float4 v[U]; float x[U]; uint32_t gr[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    gr[u] = __ldg(grow_csr + i + u * P);
+    gr[u] = DES_DBG_ROW(__ldg(grow_csr + i + u * P));
     if (HAS_VALS) x[u] = __ldg(vals + i + u * P);
     v[u] = __ldg(reinterpret_cast<const float4*>(Wc + (size_t)gr[u] * rowB));
   }
@@ -373,7 +373,7 @@ __device__ __forceinline__ void sg_step(const uint32_t* __restrict__ rows, const
   for (int u = 0; u < U; ++u) {
     const uint32_t r = __ldg(rows + i + u * P);
     const uint32_t g = (r == DES_ROW_NONE) ? null_row : s_base[__ldg(shards + i + u * P)] + r;
-    const size_t off = (size_t)g * rowB;
+    const size_t off = (size_t)DES_DBG_ROW(g) * rowB;
     if (HAS_VALS) x[u] = __ldg(vals + i + u * P);
     v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
     tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
@@ -506,6 +506,7 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   if ((ops & DES_OP_DENSE1) && !t->H) return DES_ERR_INVALID_ARG;
   cudaStream_t cs = (cudaStream_t)stream;
   des_api_begin(t, cs);
+  DES_DBG_ARM(t, cs);
   const int B = b->batch;
   float* ps = small ? part->part_small : nullptr;
   float* pl = pool ? part->pooled : nullptr;
@@ -603,6 +604,7 @@ extern "C" des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const de
     if (st != DES_OK) return st;
     if (!part->pooled || ((ops & DES_OP_DENSE1) && !t->H)) return DES_ERR_INVALID_ARG;
     des_api_begin(t, (cudaStream_t)stream);
+    DES_DBG_ARM(t, (cudaStream_t)stream);
     st = forward_single_gather(t, ops, b, part->pooled, out->out_small, (cudaStream_t)stream);
   } else {
     st = forward_impl(t, ops, b, part, out->out_small, stream);

@@ -106,8 +106,10 @@ __global__ void __launch_bounds__(256, PROBE_MINB) probe_claim_kernel(
     Slot sl[PROBE_ILP];
     bool any = false;
 #pragma unroll
-    for (int q = 0; q < PROBE_ILP; ++q)
+    for (int q = 0; q < PROBE_ILP; ++q) {
+      if (cur[q] != DES_SLOT_NONE && !DES_DBG_SLOT_OK(cur[q])) cur[q] = DES_SLOT_NONE;   // (checking build)
       if (cur[q] != DES_SLOT_NONE) { sl[q] = load_slot(slots + cur[q]); any = true; }
+    }
     if (!any) break;
 #pragma unroll
     for (int q = 0; q < PROBE_ILP; ++q) {
@@ -163,6 +165,7 @@ __global__ void __launch_bounds__(IB / 4) flag_count_kernel(
   for (int q = 0; q < 4; ++q) {
     const int j = j0 + q * (IB / 4);
     so[q] = (j < nnz) ? slot_of[j] : DES_SLOT_NONE;
+    if (so[q] != DES_SLOT_NONE && !DES_DBG_SLOT_OK(so[q])) so[q] = DES_SLOT_NONE;              // (checking build)
   }
   uint2 rf[4];                                         // (row, first_occ): the slot's second half
 #pragma unroll
@@ -346,11 +349,12 @@ __global__ void __launch_bounds__(256) apply_first_kernel(
     const uint32_t fj = first_j[u];
     const bool is_new = fj >> 31;
     const uint32_t j = fj & 0x7FFFFFFFu;
+    if (!DES_DBG_OCC_OK(j)) continue;                  // (checking build)
     const uint32_t s = shards[j];
     uint32_t local;
     if (is_new) {
       local = uniq_rows[u];                            // DES_ROW_NONE: the shard is full
-      if (local != DES_ROW_NONE) slots[slot_of[j]].row = local;
+      if (local != DES_ROW_NONE && DES_DBG_SLOT_OK(slot_of[j])) slots[slot_of[j]].row = local;
       rows[j] = local;
     } else {
       local = rows[j];
@@ -386,7 +390,7 @@ __global__ void __launch_bounds__(256) init_new_rows_kernel(
     float n2 = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
 #pragma unroll
     for (int d = 1; d < G; d <<= 1) n2 += __shfl_xor_sync(0xFFFFFFFFu, n2, d);
-    if (!init) continue;
+    if (!init || DES_DBG_ROW(grow) != grow) continue;
     float4* w = reinterpret_cast<float4*>(W + (size_t)grow * stride);
     if (c4 < K4) w[c4] = v;
     // linear weight, squared norm of the latent vector, age stamp (the clock value this call ends with)
@@ -464,6 +468,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   if (st != DES_OK) return st;
   cudaStream_t cs = (cudaStream_t)stream;
   des_api_begin(t, cs);
+  DES_DBG_ARM(t, cs);
   t->tag_valid = 0;                                    // dest[] is scratch of this call; its tags are rebuilt at the end
   const int nnz = (int)b->nnz;
   const int nbags = b->batch * (int)t->F;

@@ -55,8 +55,18 @@ struct DevMeta {
   float adam_c1, adam_c2;                            // 1 - beta1^t, 1 - beta2^t for the running step
 };
 
+// Checking build (-DDES_DEBUG, libdes_debug.so): the bounds every gather, scatter and probe is held to.
+struct DbgBounds {
+  unsigned long long rows;        // table rows + 1 (the all-zero row behind the table is a legal gather target)
+  unsigned long long slots;       // slots of all shards
+  unsigned long long grad_rows;   // gradient rows: unique keys + replica rows
+  unsigned long long nnz;         // occurrences the workspace holds
+  DevMeta* meta;                  // where DES_ERR_RANGE is raised
+};
+
 struct des_table {
   des_config_t cfg;
+  DbgBounds dbg;
   int device;
   uint32_t S, F, k, H, stride;       // stride = k + 4 floats per row
   uint64_t total_rows, total_slots;
@@ -244,6 +254,35 @@ __device__ __forceinline__ OptParams des_opt_load(const OptParams& o, const DevM
   if (o.optimizer == DES_OPT_ADAM) { r.c1 = meta->adam_c1; r.c2 = meta->adam_c2; }
   return r;
 }
+
+// ---- checking build -----------------------------------------------------------
+// In the product library these macros cost nothing.  In the checking build every translation unit keeps a
+// copy of the running table's bounds in device memory (armed at the entry of every call that launches
+// gathers or scatters); an index outside them raises the table's sticky status word and the access is
+// skipped or redirected to the all-zero row — never performed.
+#ifdef DES_DEBUG
+static __device__ DbgBounds g_dbg;
+__device__ __forceinline__ bool des_dbg_in(unsigned long long i, unsigned long long n) {
+  if (i < n) return true;
+  if (g_dbg.meta) atomicCAS(&g_dbg.meta->err, 0u, (uint32_t)DES_ERR_RANGE);
+  return false;
+}
+#define DES_DBG_ROW(g) (des_dbg_in((unsigned long long)(g), g_dbg.rows) ? (g) : (uint32_t)(g_dbg.rows - 1ull))
+#define DES_DBG_SLOT_OK(i) des_dbg_in((unsigned long long)(i), g_dbg.slots)
+#define DES_DBG_GRAD_OK(d) des_dbg_in((unsigned long long)(d), g_dbg.grad_rows)
+#define DES_DBG_OCC_OK(j) des_dbg_in((unsigned long long)(j), g_dbg.nnz)
+#define DES_DBG_ARM(t, cs)                                                                                            \
+  do {                                                                                                                \
+    if (cudaMemcpyToSymbolAsync(g_dbg, &(t)->dbg, sizeof(DbgBounds), 0, cudaMemcpyHostToDevice, (cs)) != cudaSuccess) \
+      return DES_ERR_CUDA;                                                                                            \
+  } while (0)
+#else
+#define DES_DBG_ROW(g) (g)
+#define DES_DBG_SLOT_OK(i) true
+#define DES_DBG_GRAD_OK(d) true
+#define DES_DBG_OCC_OK(j) true
+#define DES_DBG_ARM(t, cs) do { } while (0)
+#endif
 
 // shared declarations across translation units
 des_status_t des_check_batch(const des_table* t, const des_batch_t* b, int need_dedup);

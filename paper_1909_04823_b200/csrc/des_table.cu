@@ -226,6 +226,8 @@ extern "C" des_status_t des_table_create(const des_config_t* cfg, des_table_t** 
     A(t->gemm_ws, t->gemm_ws_bytes);
   }
   if (!ok) { des_table_destroy(t); return DES_ERR_CUDA; }
+  t->dbg.rows = rows + 1; t->dbg.slots = slots; t->dbg.grad_rows = (unsigned long long)t->max_uniq + t->rep_max;
+  t->dbg.nnz = (unsigned long long)t->max_nnz; t->dbg.meta = t->meta;
   bool cu = true;
   cu &= cudaMemset(t->slots, 0xFF, slots * sizeof(Slot)) == cudaSuccess;
   cu &= cudaMemset(t->W + rows * t->stride, 0, rowbytes) == cudaSuccess;
