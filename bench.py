@@ -257,8 +257,8 @@ def kernel_bytes(name, st):
         return 2 * row * R
     if name == "update_rows_kernel":
         return U * (2 * row + 2 * row * (1 + state) + 8)
-    if name == "cvt_bf16_kernel":          # three launches per step: pooled (forward), gZ and pooled (backward)
-        return 6 * (2 * B * F * k + B * st["H"]) // 3
+    if name == "cvt_bf16_kernel":          # one launch per step: gZ and pooled of the backward (the forward's copy of
+        return 6 * (B * F * k + B * st["H"])   # pooled comes out of the pooling kernel)
     return None
 
 

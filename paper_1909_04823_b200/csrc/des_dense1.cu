@@ -157,6 +157,20 @@ __global__ void cvt_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __
   }
 }
 
+// two arrays in one launch (the backward's two operands)
+__global__ void cvt_bf16_pair_kernel(const float* __restrict__ s1, __nv_bfloat16* __restrict__ d1, size_t n1,
+                                     const float* __restrict__ s2, __nv_bfloat16* __restrict__ d2, size_t n2) {
+  size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  const size_t st = (size_t)gridDim.x * blockDim.x * 4;
+  for (; i + 3 < n1 + n2; i += st) {                   // n1 and n2 are multiples of 4
+    const float* src = i < n1 ? s1 + i : s2 + (i - n1);
+    __nv_bfloat16* dst = i < n1 ? d1 + i : d2 + (i - n1);
+    const float4 v = *reinterpret_cast<const float4*>(src);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+  }
+}
+
 static des_status_t to_bf16(des_table* t, const float* src, __nv_bfloat16* dst, size_t n, cudaStream_t st) {
   cvt_bf16_kernel<<<t->sm_count * 4, 256, 0, st>>>(src, dst, n);     // n is a multiple of 4 (k and H are)
   DES_LAUNCH_CHECK(t, "cvt_bf16_kernel");
@@ -167,8 +181,13 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
                                 const float* part_pooled, cudaStream_t st) {
   if (!part_dense && t->use_tc) {
     const int FK = t->F * t->k;
-    des_status_t e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
-    if (e != DES_OK) return e;
+    // the pooling kernel of the same forward has usually left the bfloat16 copy already
+    const bool have = t->pooled_b_src == pooled;
+    t->pooled_b_src = nullptr;                         // good for one product only
+    if (!have) {
+      des_status_t e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
+      if (e != DES_OK) return e;
+    }
     const int rc = des_tc_gemm_fwd(B, t->H, FK, 1, t->pooled_b, t->W1b, Z, Z, 0.f, t->gemm_ws, t->gemm_ws_bytes, st);
     if (rc == 0) { DES_LAUNCH_CHECK(t, "tc_gemm_fwd"); return DES_OK; }
     if (rc != 1) return DES_ERR_CUDA;
@@ -192,9 +211,9 @@ des_status_t des_dense1_backward(des_table* t, const float* pooled, const float*
                                  float* gE_work, int B, cudaStream_t st) {
   const int FK = t->F * t->k;
   if (t->use_tc) {
-    des_status_t e = to_bf16(t, gZ, t->gZ_b, (size_t)B * t->H, st);
-    if (e == DES_OK) e = to_bf16(t, pooled, t->pooled_b, (size_t)B * FK, st);
-    if (e != DES_OK) return e;
+    t->pooled_b_src = nullptr;
+    cvt_bf16_pair_kernel<<<t->sm_count * 4, 256, 0, st>>>(gZ, t->gZ_b, (size_t)B * t->H, pooled, t->pooled_b, (size_t)B * FK);
+    DES_LAUNCH_CHECK(t, "cvt_bf16_kernel");
     const int rc1 = des_tc_gemm_dgrad(B, FK, t->H, 1, t->gZ_b, t->W1b, gE ? gE : gE_work, gE_work, gE ? 1.f : 0.f,
                                       t->gemm_ws, t->gemm_ws_bytes, st);
     if (rc1 == 0) {

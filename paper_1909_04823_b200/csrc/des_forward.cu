@@ -140,16 +140,22 @@ __global__ void __launch_bounds__(256) route_kernel(
   }
 }
 
-// U rows per lane in flight: occurrences i, i + P, ... of a (sample, shard) segment.
+// One round of a (sample, shard) segment: U rows per lane in flight, occurrences i, i + P, ... below `hi`;
+// positions past the segment's end read the all-zero row behind the table, so a round has no branch.
 template <int U, int P, bool HAS_VALS>
-__device__ __forceinline__ void sp_step(const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted,
-                                        int i, const char* __restrict__ Wc, const char* __restrict__ Wt, unsigned rowB,
-                                        float4& acc, float& m1lr, float& m2) {
-  float4 v[U]; float2 tl[U]; float x[U];
+__device__ __forceinline__ void sp_round(const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted,
+                                         int i, int hi, uint32_t null_row, const char* __restrict__ Wc,
+                                         const char* __restrict__ Wt, unsigned rowB, float4& acc, float& m1lr, float& m2) {
+  float4 v[U]; float2 tl[U]; float x[U]; uint32_t g[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
-    const size_t off = (size_t)DES_DBG_ROW(__ldg(grow_sorted + i + u * P)) * rowB;
-    if (HAS_VALS) x[u] = __ldg(x_sorted + i + u * P);
+    const bool in = i + u * P < hi;
+    g[u] = in ? __ldg(grow_sorted + i + u * P) : null_row;
+    if (HAS_VALS) x[u] = in ? __ldg(x_sorted + i + u * P) : 0.f;
+  }
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const size_t off = (size_t)DES_DBG_ROW(g[u]) * rowB;
     v[u] = __ldg(reinterpret_cast<const float4*>(Wc + off));
     tl[u] = __ldg(reinterpret_cast<const float2*>(Wt + off));
   }
@@ -191,27 +197,30 @@ __device__ __forceinline__ void pool_step(const uint32_t* __restrict__ grow_csr,
 
 // One WARP per sample walks the sample's S segments in shard order.  The warp is
 // split into P = 32 / G sub-groups of G lanes (one 16-byte column per lane);
-// sub-group p takes occurrences p, p + P, ... of a segment, two of them in
-// flight, and the sub-groups' sums are combined by a butterfly when the segment
-// ends — so both halves of a warp always run the same trip counts, whatever the
-// skew between shards, and every warp has the same amount of work (a sample's
-// occurrences).  The loop body is kept to the loads and adds: whole iterations
-// carry no bound checks, row addresses are one multiply-add from a per-lane base,
-// and lanes without a column of their own (k not a multiple of 4 G) re-read
-// column 0 instead of branching.  In a long segment a lane's float32 sums move on
-// into a second set of accumulators every SP_FLUSH iterations; the sum over shards
-// runs in double.  part_small
+// sub-group p takes occurrences p, p + P, ... of a segment, SP_U of them in
+// flight per round, and the sub-groups' sums are combined by a butterfly when the
+// segment ends — so both halves of a warp always run the same trip counts, whatever
+// the skew between shards, and every warp has the same amount of work (a sample's
+// occurrences).  What a warp waits for is memory latency, one dependent chain per
+// sample, so the chain is kept short: the sample's S + 1 segment bounds are read
+// once (two per lane) and handed round by shuffles, and a round's row numbers are
+// all fetched before its rows (positions past the segment's end name the all-zero
+// row: no branch).  Lanes without a column of their own (k not a multiple of 4 G)
+// re-read column 0 instead of branching.  A lane's float32 sums move on into a
+// second set of accumulators every SP_FLUSH rounds, so that no accumulator takes more
+// than a few dozen additions; the sum over shards runs in double.  part_small
 // (optional) receives each segment's partial sums, rounded to float32, as soon as
 // the segment ends; with FUSED the aggregation (+) over shards and the substitution
 // operator F are applied on chip, in the same shard order and with the same
 // arithmetic as aggregate_small_kernel (the sum of the float32-rounded partials in
 // double), and out_small is written directly — the per-shard partials then never
 // touch memory.
-#define SP_FLUSH 8
+#define SP_U 4
+#define SP_FLUSH 4
 template <int G, bool HAS_VALS, bool FUSED>
-__global__ void __launch_bounds__(256, FUSED ? 4 : 8) shard_partials_kernel(
+__global__ void __launch_bounds__(256) shard_partials_kernel(
     const uint32_t* __restrict__ grow_sorted, const float* __restrict__ x_sorted, const int32_t* __restrict__ seg_off,
-    int B, int S, int k, uint32_t ops, const float* __restrict__ W, float* __restrict__ part_small,
+    int B, int S, int k, uint32_t ops, const float* __restrict__ W, uint32_t null_row, float* __restrict__ part_small,
     float* __restrict__ out_small) {
   constexpr int P = 32 / G;
   const int K4 = k >> 2, stride = k + 4;
@@ -226,32 +235,27 @@ __global__ void __launch_bounds__(256, FUSED ? 4 : 8) shard_partials_kernel(
   const char* Wc = reinterpret_cast<const char*>(W) + (col ? c4 : 0) * 16;
   const char* Wt = reinterpret_cast<const char*>(W + k);                       // (w, |v|^2)
   double Ax = 0.0, Ay = 0.0, Az = 0.0, Aw = 0.0, R = 0.0, Q = 0.0;   // FUSED: (+)M_1, (+)M_1^lr, (+)M_2
+  // the sample's segment bounds: lane l holds bounds l and l + 32, lane 0 also bound 64 (S <= 64)
   const int32_t* so = seg_off + (size_t)b * (S + 1);
-  int hi = __ldg(so);
+  static_assert(DES_MAX_SHARDS <= 64, "three bounds per lane");
+  const int o0 = lane <= S ? __ldg(so + lane) : 0, o1 = lane + 32 <= S ? __ldg(so + lane + 32) : 0;
+  const int o2 = (lane == 0 && S == 64) ? __ldg(so + 64) : 0;
+  auto bound = [&](int s) { return s < 32 ? __shfl_sync(0xFFFFFFFFu, o0, s) : s < 64 ? __shfl_sync(0xFFFFFFFFu, o1, s - 32)
+                                                                                     : __shfl_sync(0xFFFFFFFFu, o2, 0); };
+  int hi = bound(0);
   for (int s = 0; s < S; ++s) {
     const int lo = hi;
-    hi = __ldg(so + s + 1);
-    float4 acc = zero4;
-    float m1lr = 0.f, m2 = 0.f;
-    int i0 = lo;
-    // a long segment (one hot id occurring hundreds of times in the sample): the sums move on into a second
-    // set of accumulators every SP_FLUSH iterations, so that no float32 accumulator takes more than a few
-    // dozen additions (a single chain of hundreds of equal terms would lose the 1e-5 the sum must keep)
-    float4 up = zero4;
-    float up_l = 0.f, up_q = 0.f;
-    while (hi - i0 > 4 * P * SP_FLUSH) {
-#pragma unroll 1
-      for (int it = 0; it < SP_FLUSH; ++it, i0 += 2 * P)
-        sp_step<2, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
-      up.x += acc.x; up.y += acc.y; up.z += acc.z; up.w += acc.w; up_l += m1lr; up_q += m2;
-      acc = zero4; m1lr = 0.f; m2 = 0.f;
+    hi = bound(s + 1);
+    float4 acc = zero4, up = zero4;
+    float m1lr = 0.f, m2 = 0.f, up_l = 0.f, up_q = 0.f;
+    int round = 0;
+    for (int i0 = lo; i0 < hi; i0 += SP_U * P) {
+      sp_round<SP_U, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, hi, null_row, Wc, Wt, rowB, acc, m1lr, m2);
+      if ((++round & (SP_FLUSH - 1)) == 0) {           // (a long segment: one hot id, hundreds of times in the sample)
+        up.x += acc.x; up.y += acc.y; up.z += acc.z; up.w += acc.w; up_l += m1lr; up_q += m2;
+        acc = zero4; m1lr = 0.f; m2 = 0.f;
+      }
     }
-    // whole blocks of 2 and 1 occurrences per lane (no bound checks), then one checked step; segments are
-    // short (a sample's occurrences spread over S shards), so deeper unrolling only adds ragged steps
-    for (; i0 + 2 * P <= hi; i0 += 2 * P)
-      sp_step<2, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
-    if (i0 + P <= hi) { sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2); i0 += P; }
-    if (i0 + p < hi) sp_step<1, P, HAS_VALS>(grow_sorted, x_sorted, i0 + p, Wc, Wt, rowB, acc, m1lr, m2);
     acc.x += up.x; acc.y += up.y; acc.z += up.z; acc.w += up.w; m1lr += up_l; m2 += up_q;
 #pragma unroll
     for (int d = G; d < 32; d <<= 1) {                 // combine the sub-groups (same result in every lane)
@@ -281,11 +285,17 @@ __global__ void __launch_bounds__(256, FUSED ? 4 : 8) shard_partials_kernel(
   }
 }
 
-template <int G, int P, bool HAS_VALS, bool MATERIALISE>
+// four floats rounded to bfloat16 (RNE), one 8-byte store
+__device__ __forceinline__ void store_bf16x4(__nv_bfloat16* dst, const float4& v) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+}
+
+template <int G, int P, bool HAS_VALS, bool MATERIALISE, bool BF16OUT>
 __global__ void __launch_bounds__(256) pool_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ grow_csr,
     const uint8_t* __restrict__ shards, long long nbags, int B, int F, int k, const float* __restrict__ W,
-    uint32_t null_row, float* __restrict__ pooled, float* __restrict__ part_pooled) {
+    uint32_t null_row, float* __restrict__ pooled, float* __restrict__ part_pooled, __nv_bfloat16* __restrict__ pooled_b) {
   constexpr int LB = G * P;                            // lanes per bag
   const int K4 = k >> 2, stride = k + 4;
   const int sub = threadIdx.x % LB, c4 = sub % G, p = sub / G;
@@ -322,7 +332,10 @@ __global__ void __launch_bounds__(256) pool_kernel(
       acc.x += __shfl_xor_sync(0xFFFFFFFFu, acc.x, d); acc.y += __shfl_xor_sync(0xFFFFFFFFu, acc.y, d);
       acc.z += __shfl_xor_sync(0xFFFFFFFFu, acc.z, d); acc.w += __shfl_xor_sync(0xFFFFFFFFu, acc.w, d);
     }
-    if (live && p == 0 && col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+    if (live && p == 0 && col) {
+      reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+      if (BF16OUT) store_bf16x4(pooled_b + bag * k + c4 * 4, acc);    // operand of the first-layer product
+    }
   }
 }
 
@@ -394,7 +407,8 @@ template <int G, int P, bool HAS_VALS>
 __global__ void __launch_bounds__(256) single_gather_kernel(
     const int32_t* __restrict__ offsets, const float* __restrict__ vals, const uint32_t* __restrict__ rows,
     const uint8_t* __restrict__ shards, long long nbags, int S, int k, const float* __restrict__ W,
-    const DevMeta* __restrict__ meta, uint32_t null_row, float* __restrict__ pooled, float2* __restrict__ bag_tail) {
+    const DevMeta* __restrict__ meta, uint32_t null_row, float* __restrict__ pooled, float2* __restrict__ bag_tail,
+    __nv_bfloat16* __restrict__ pooled_b) {
   constexpr int LB = G * P;                            // lanes per bag
   __shared__ uint32_t s_base[DES_MAX_SHARDS];
   if (threadIdx.x < S) s_base[threadIdx.x] = (uint32_t)meta->row_base[threadIdx.x];
@@ -431,7 +445,10 @@ __global__ void __launch_bounds__(256) single_gather_kernel(
       bl += __shfl_xor_sync(0xFFFFFFFFu, bl, d); bq += __shfl_xor_sync(0xFFFFFFFFu, bq, d);
     }
     if (live && p == 0) {
-      if (col) reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+      if (col) {
+        reinterpret_cast<float4*>(pooled + bag * k)[c4] = acc;
+        if (pooled_b) store_bf16x4(pooled_b + bag * k + c4 * 4, acc);
+      }
       if (c4 == 0) bag_tail[bag] = make_float2(bl, bq);
     }
   }
@@ -525,7 +542,7 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   if (ps || fused_out) {
     const unsigned grid = (unsigned)((B + 7) / 8);      // one warp per sample
 #define SP3(GG, HV, FU) shard_partials_kernel<GG, HV, FU><<<grid, 256, 0, cs>>>(grow_sorted, x_sorted, t->seg_off, B, t->S, \
-                                                                              t->k, ops, t->W, ps, fused_out)
+                                                                              t->k, ops, t->W, (uint32_t)t->total_rows, ps, fused_out)
 #define SP(GG) do { if (fused_out) { if (b->vals) SP3(GG, true, true); else SP3(GG, false, true); } \
                     else { if (b->vals) SP3(GG, true, false); else SP3(GG, false, false); } } while (0)
     switch (G) { case 1: SP(1); break; case 2: SP(2); break; case 4: SP(4); break; case 8: SP(8); break; default: SP(16); }
@@ -541,16 +558,21 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
     long long blocks = (threads + 255) / 256;
     if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
     const unsigned grid = (unsigned)blocks;
-#define PK4(GG, PP, HV, MT) pool_kernel<GG, PP, HV, MT><<<grid, 256, 0, cs>>>(b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, \
-                                                                             t->k, t->W, (uint32_t)t->total_rows, pl, pp)
-#define PK3(GG, HV, MT) do { if (wide) PK4(GG, 32 / GG, HV, MT); else PK4(GG, 1, HV, MT); } while (0)
-#define PK(GG) do { if (pp) { if (b->vals) PK3(GG, true, true); else PK3(GG, false, true); } \
-                    else { if (b->vals) PK3(GG, true, false); else PK3(GG, false, false); } } while (0)
+    // with the first layer among the operators the pooled vectors are also left as bfloat16, the operand
+    // format of the tensor-core product that follows (one conversion pass less)
+    __nv_bfloat16* pb = ((ops & DES_OP_DENSE1) && t->use_tc && !pp) ? t->pooled_b : nullptr;
+#define PK5(GG, PP, HV, MT, BO) pool_kernel<GG, PP, HV, MT, BO><<<grid, 256, 0, cs>>>(                                 \
+        b->offsets, b->vals, grow_csr, b->shards, nbags, B, t->F, t->k, t->W, (uint32_t)t->total_rows, pl, pp, pb)
+#define PK3(GG, HV, MT, BO) do { if (wide) PK5(GG, 32 / GG, HV, MT, BO); else PK5(GG, 1, HV, MT, BO); } while (0)
+#define PK2(GG, HV) do { if (pp) PK3(GG, HV, true, false); else if (pb) PK3(GG, HV, false, true); else PK3(GG, HV, false, false); } while (0)
+#define PK(GG) do { if (b->vals) PK2(GG, true); else PK2(GG, false); } while (0)
     switch (G) { case 1: PK(1); break; case 2: PK(2); break; case 4: PK(4); break; case 8: PK(8); break; default: PK(16); }
 #undef PK
+#undef PK2
 #undef PK3
-#undef PK4
+#undef PK5
     DES_LAUNCH_CHECK(t, "pool_kernel");
+    t->pooled_b_src = pb ? pl : nullptr;
   }
   return DES_OK;
 }
@@ -570,9 +592,10 @@ static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const de
     long long blocks = (threads + 255) / 256;
     if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
     const unsigned grid = (unsigned)blocks;
+    __nv_bfloat16* pb = ((ops & DES_OP_DENSE1) && t->use_tc) ? t->pooled_b : nullptr;
 #define SG3(GG, PP, HV) single_gather_kernel<GG, PP, HV><<<grid, 256, 0, cs>>>(b->offsets, b->vals, b->rows, b->shards, nbags,   \
                                                                               (int)t->S, t->k, t->W, t->meta,                 \
-                                                                              (uint32_t)t->total_rows, pooled, t->bag_tail)
+                                                                              (uint32_t)t->total_rows, pooled, t->bag_tail, pb)
 #define SG2(GG, HV) do { if (wide) SG3(GG, 32 / GG, HV); else SG3(GG, 1, HV); } while (0)
 #define SG(GG) do { if (b->vals) SG2(GG, true); else SG2(GG, false); } while (0)
     switch (G) { case 1: SG(1); break; case 2: SG(2); break; case 4: SG(4); break; case 8: SG(8); break; default: SG(16); }
@@ -580,6 +603,7 @@ static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const de
 #undef SG2
 #undef SG3
     DES_LAUNCH_CHECK(t, "single_gather_kernel");
+    t->pooled_b_src = pb ? pooled : nullptr;
   }
   {
     const int grid = (int)(((long long)B * G + 255) / 256);
@@ -642,6 +666,7 @@ extern "C" des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_ba
       // materialised per-shard pooled partials: aggregate them in shard order
       reduce_shards_kernel<<<t->sm_count * 4, 256, 0, cs>>>(part->part_pooled, n, t->S, out->pooled);
       DES_LAUNCH_CHECK(t, "reduce_shards_kernel");
+      t->pooled_b_src = nullptr;
     } else if (out->pooled != part->pooled) {
       DES_CUDA(cudaMemcpyAsync(out->pooled, part->pooled, n * 4, cudaMemcpyDeviceToDevice, cs));
     }

@@ -109,6 +109,8 @@ struct des_table {
   float* gW1_part; int gw1_splits;   // [splits][F*k][H]
   int use_tc;                        // tensor-core GEMM path usable for this table's shapes
   __nv_bfloat16 *pooled_b, *gZ_b;    // bf16 copies of V [max_batch][F*k] and gZ [max_batch][H]
+  const float* pooled_b_src;         // the pooled array whose bf16 copy the pooling kernel has just left in pooled_b
+                                     // (consumed, once, by the first-layer product that follows); NULL otherwise
   void* gemm_ws; size_t gemm_ws_bytes;
   // host-step staging
   int32_t* st_offsets[2]; unsigned long long* st_ids[2]; float* st_vals[2];   // two input slots (pipelined submit)
