@@ -210,13 +210,18 @@ class ClockSampler:
 # own batch on a 4e6-key table (the 2e8-key table cannot be captured under multi-pass replay).  The scatter's traffic does not depend on
 # the table; kernels that touch table rows move fewer DRAM bytes there (U = 1.06 M instead of 1.81 M).
 NCU_DRAM_TRAFFIC = {
-    ("cfg5", "grad_scatter_kernel"): 1806e6,
+    ("cfg5", "grad_scatter_kernel"): 1807e6,
     ("cfg5", "super_dense_kernel"): 533e6,
-    ("cfg5", "shard_partials_kernel"): 939e6,
-    ("cfg5", "pool_kernel"): 1211e6,
-    ("cfg5", "update_rows_kernel"): 1937e6,
+    ("cfg5", "shard_partials_kernel"): 962e6,
+    ("cfg5", "pool_kernel"): 1213e6,
+    ("cfg5", "update_rows_kernel"): 1933e6,
     ("cfg5", "probe_claim_kernel"): 596e6,
-    ("cfg5", "route_kernel"): 454e6,
+    ("cfg5", "flag_count_kernel"): 566e6,
+    ("cfg5", "resolve_kernel"): 421e6,
+    ("cfg5", "make_dest_kernel"): 225e6,
+    ("cfg5", "route_kernel"): 456e6,
+    ("cfg5", "single_gather_kernel"): 1290e6,
+    ("cfg5", "fused_finish_kernel"): 440e6,
 }
 
 
@@ -242,6 +247,10 @@ def kernel_bytes(name, st):
         return 4 * B * (S + 1) + 4 * nnz + row * U + 4 * S * B * (k + 4)
     if name == "pool_kernel":
         return 4 * (B * F + 1) + 4 * nnz + 4 * k * U + 4 * B * F * k
+    if name == "single_gather_kernel":   # rows + shards in, every unique row once, pooled + bag tails out
+        return 4 * (B * F + 1) + 5 * nnz + row * U + 4 * B * F * k + 8 * B * F
+    if name == "fused_finish_kernel":
+        return 4 * B * F * k + 8 * B * F + 4 * B * (k + 4)
     if name == "aggregate_small_kernel":
         return 4 * S * B * (k + 4) + 4 * B * (k + 4)
     if name == "make_dest_kernel":

@@ -89,10 +89,7 @@ __global__ void __launch_bounds__(256) hot_select_kernel(uint32_t* hinfo, const 
                                                          uint32_t h_max, uint32_t rep_max, DevMeta* meta,
                                                          uint32_t* hot_work, uint32_t work_max, uint32_t super_min) {
   long long U = *n_uniq;
-  if (U > max_uniq) {           // the gradient buffer cannot hold this batch: report, update what fits
-    if (blockIdx.x == 0 && threadIdx.x == 0) des_raise(meta, DES_ERR_CAPACITY);
-    U = max_uniq;
-  }
+  if (U > max_uniq) U = max_uniq;   // more unique keys than the gradient buffer holds: the backward reports it
   for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (long long)gridDim.x * blockDim.x) {
     const uint32_t est = hinfo[u] << shift;
     uint32_t h = DES_ROW_NONE;
@@ -485,13 +482,16 @@ __global__ void adam_tick_kernel(DevMeta* meta, float beta1, float beta2) {
 template <int G, bool ADAM>
 __global__ void __launch_bounds__(256, UP_MINB) update_rows_kernel(
     const uint32_t* __restrict__ uniq_rows, const uint32_t* __restrict__ n_uniq, long long max_uniq, int k,
-    uint32_t ops, const OptParams opt_in, const DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
+    uint32_t ops, const OptParams opt_in, DevMeta* __restrict__ meta, float* __restrict__ Gbuf,
     float* __restrict__ W, float* __restrict__ A, float* __restrict__ A2) {
   const int K4 = k >> 2, stride = k + 4;
   const OptParams opt = des_opt_load(opt_in, meta);
   const float stamp = des_stamp_bits(meta->clock);     // "updated in the step of the current batch" (eviction by age)
   long long U = *n_uniq;
-  if (U > max_uniq) U = max_uniq;
+  if (U > max_uniq) {           // the gradient buffer cannot hold this batch: report, update what fits
+    if (blockIdx.x == 0 && threadIdx.x == 0) des_raise(meta, DES_ERR_CAPACITY);
+    U = max_uniq;
+  }
   const int c4 = (int)(threadIdx.x % G);
   const bool col = c4 < K4, lead = c4 == 0;
   const bool upd_v = ops & (DES_OP_FM | DES_OP_POOL | DES_OP_DENSE1), upd_w = ops & DES_OP_LR;

@@ -190,6 +190,30 @@ def test_capacity_and_reserved_key_are_reported_not_faulted():
         t.close()
 
 
+def test_gradient_buffer_capacity_is_reported_by_the_backward_only():
+    # max_uniq sizes the gradient buffer: a batch with more distinct keys than that inserts and forwards fine
+    # (pre-population, inference); only a backward over it raises DES_ERR_CAPACITY — and faults nothing
+    from paper_1909_04823_b200.binding import DeviceBatch, Table
+    w = _mk(S=3)
+    ids = synth.fmix64(np.arange(600, dtype=np.uint64))
+    b = synth.prepopulation_batch(ids, w.fields)
+    t = Table.for_workload(w, max_rows=2000, max_nnz=1024, max_batch=b.batch, max_uniq=100)
+    try:
+        db = DeviceBatch.from_synth(b)
+        t.find_or_insert(db, True)
+        S, B, k, F = w.shards, b.batch, w.emb_dim, w.fields
+        ps = torch.zeros((S, B, k + 4), device="cuda"); pooled = torch.zeros((B, F * k), device="cuda")
+        out = torch.zeros((B, k + 4), device="cuda")
+        t.forward_partials(w.ops, db, ps, pooled)
+        t.aggregate(w.ops, db, ps, pooled, out_small=out)
+        assert t.status() == 0 and sum(t.size()) == 600
+        g = {n: torch.from_numpy(v).cuda() for n, v in synth.upstream_grads(w, B, 0).items()}
+        t.backward_update(w.ops, db, out, pooled, None, g["gL"], g["gF"], g["gE"], None, None)
+        assert t.status() == 3
+    finally:
+        t.close()
+
+
 def test_invalid_arguments_are_rejected_on_the_host():
     from paper_1909_04823_b200.binding import DesError, DeviceBatch, Table
     w = _mk()
