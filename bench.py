@@ -255,9 +255,11 @@ def kernel_bytes(name, st):
         return 4 * S * B * (k + 4) + 4 * B * (k + 4)
     if name == "make_dest_kernel":
         return 8 * nnz + 4 * U
-    if name == "grad_scatter_kernel":   # + the per-bag counts of the register-summed keys on skewed batches
-        return (4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + 2 * row * (U + R)
-                + (64 * B * F if st["super"] else 0))
+    if name == "grad_scatter_kernel":
+        # offsets, one index word per occurrence, gE once, A, gL / gF, and every key's summed gradient landing once
+        # (the read-modify-write of the gradient rows by the atomics and the per-bag counts of the counted keys are
+        # implementation traffic, not algorithmic bytes)
+        return 4 * (B * F + 1) + 4 * nnz + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B + row * (U + R)
     if name == "super_dense_kernel":
         return 64 * B * F + (4 * B * F * k if pool else 0) + 4 * B * (k + 4) + 8 * B
     if name == "sample_count_kernel":
@@ -268,6 +270,17 @@ def kernel_bytes(name, st):
         return U * (2 * row + 2 * row * (1 + state) + 8)
     if name == "cvt_bf16_kernel":          # one launch per step: gZ and pooled of the backward (the forward's copy of
         return 6 * (B * F * k + B * st["H"])   # pooled comes out of the pooling kernel)
+    return None
+
+
+# Bytes the load / store units move per launch when every occurrence reads (or adds to) its own row: the figure
+# the L1 data path sees.  L1 peak = 128 bytes per clock and SM (148 SMs at the sampled SM clock).
+def occurrence_bytes(name, st):
+    nnz, k = st["nnz"], st["k"]
+    if name == "pool_kernel":
+        return 4 * k * nnz
+    if name in ("shard_partials_kernel", "single_gather_kernel"):
+        return (4 * k + 32) * nnz          # the vector and the 32-byte sector that holds the row's tail
     return None
 
 
@@ -286,6 +299,16 @@ def kernel_flops(name, st):
     return None
 
 
+# What ncu shows to be the busiest unit of each occurrence-level kernel (captures summarised under profiles/): none of
+# them is near the HBM bound of its algorithmic bytes, because every occurrence moves a row through the L1 data path
+# while only the unique rows come from HBM.
+BOUND_NOTES = {
+    "grad_scatter_kernel": "busiest unit per ncu: L1TEX 87 % / L2 67 % (one 16-byte vector atomic per lane and occurrence); DRAM 26 %",
+    "shard_partials_kernel": "busiest unit per ncu: L1TEX 73 % (a 272-byte row per occurrence through L1); DRAM 15 %",
+    "pool_kernel": "busiest unit per ncu: L1TEX 77 % (a 256-byte vector per occurrence through L1); DRAM 27 %",
+    "single_gather_kernel": "busiest unit per ncu: L1TEX 65 % (a 272-byte row per occurrence through L1); DRAM 16 %",
+    "update_rows_kernel": "random 272-byte rows of weights and state: DRAM-bound (56 % on a small table under ncu)",
+}
 TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch on the benchmark's own batch with a "
                   "4e6-key table (the 2e8-key table cannot be captured under multi-pass replay); constant, not measured "
                   "in this run")
@@ -415,9 +438,13 @@ def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want
             by = kernel_bytes(name, stats)
             fl = kernel_flops(name, stats)
             avg = ms / n_
+            ob = occurrence_bytes(name, stats)
             kernels.append({"kernel": name, "launches": n_, "ms_per_launch": round(avg, 4), "share": round(ms / tot_k, 4),
                             "alg_gbs": None if by is None else round(by / avg / 1e6, 1),
-                            "tflops": None if fl is None else round(fl / avg / 1e9, 1)})
+                            "tflops": None if fl is None else round(fl / avg / 1e9, 1),
+                            # occurrence-level bytes through L1 against 128 B / clock / SM x 148 SMs x 1.965 GHz
+                            "l1_gbs": None if ob is None else round(ob / avg / 1e6, 1),
+                            "l1_frac_of_nominal": None if ob is None else round(ob / avg / 1e6 / (128 * 148 * 1.965), 3)})
         roofline = None
         for top in kernels:      # the kernel with the largest share of the timed region that has a byte / flop model
             if top["alg_gbs"] is not None:
@@ -425,7 +452,8 @@ def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want
                 roofline = {"bound": "hbm", "kernel": top["kernel"], "achieved": top["alg_gbs"], "peak": hbm_peak,
                             "unit": "GB/s", "frac": round(top["alg_gbs"] / hbm_peak, 4), "traffic": tr,
                             "traffic_source": TRAFFIC_SOURCE if tr is not None else None,
-                            "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"]}
+                            "peak_kind": f"of {peak_kind}", "ms_per_launch": top["ms_per_launch"], "share": top["share"],
+                            "note": BOUND_NOTES.get(top["kernel"])}
                 break
             if top["tflops"] is not None:
                 roofline = {"bound": "tensor", "kernel": top["kernel"], "achieved": top["tflops"], "peak": tc_peak,
