@@ -104,10 +104,12 @@ def rows_per_shard_for(w, cap_total):
 class Pair:
     """Oracle table + CUDA table for one workload."""
 
-    def __init__(self, w, max_rows, max_nnz, max_batch=None, max_uniq=0, resync=True):
+    def __init__(self, w, max_rows, max_nnz, max_batch=None, max_uniq=0, resync=True, omp=False):
+        """omp: use the all-cores build of the oracle (the same source compiled with -fopenmp, pinned equal to the
+        sequential build by tests/test_oracle_pins.py) — only for runs the sequential build would take minutes for."""
         from paper_1909_04823_b200.binding import Table
         self.w = w
-        self.o = Oracle.for_workload(w)
+        self.o = Oracle.for_workload(w, omp=omp)
         self.t = Table.for_workload(w, max_rows=max_rows, max_nnz=max_nnz, max_batch=max_batch or w.batch,
                                     rows_per_shard=rows_per_shard_for(w, max_rows), max_uniq=max_uniq)
         self.row_base = np.array(self.t.row_base(), dtype=np.int64)

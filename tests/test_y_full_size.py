@@ -236,6 +236,25 @@ def test_cfg3_deepfm_full_size():
     _assert_tolerance_counts(w.name + " B=16384", 1e-3)
 
 
+def test_cfg3_deepfm_full_size_twenty_steps():
+    """The same workload for all of its 20 steps.  One step of the sequential oracle's dense backward takes 45 s
+    here, so this run uses the oracle's all-cores build (the same source compiled with -fopenmp; a CPU test pins
+    it equal to the sequential build, which the two-step test above uses)."""
+    from harness import Pair
+    w = synth.config(3)
+    st = synth.Stream(w)
+    b = st.next_batch()
+    p = Pair(w, max_rows=6_000_000, max_nnz=int(b.nnz * 1.2) + 1024, omp=True)
+    try:
+        sel = np.sort(np.random.default_rng(6).choice(w.batch, 64, replace=False))
+        for s in range(w.steps):
+            p.step(b, synth.upstream_grads(w, b.batch, s), check_init=(s == 0), dense_samples=sel)
+            b = st.next_batch()
+    finally:
+        p.close()
+    _assert_tolerance_counts(w.name + " B=16384", 1e-3)
+
+
 def test_cfg4_streaming_scaled_hundred_steps():
     """The streaming workload scaled to batch 4096 from a 1e5-key table for all of its 100 steps against
     the oracle (row numbers, new rows, every stage of every step)."""
