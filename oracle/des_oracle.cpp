@@ -36,8 +36,11 @@
 // FM pair form == linear form; DES form == original for any S and both
 // partitions; S = 1 == any S; gradients == central finite differences;
 // dedup/Adagrad special cases; row-split GEMM == one dense matmul; canonical
-// row numbering vs a dictionary walk.  The hash/shard rule itself is fixed by
-// no passage: "parity unpinned" beyond bijectivity and balance.
+// row numbering vs a dictionary walk; Adagrad / Adam / FTRL vs library optimizers
+// and closed forms; eviction vs a brute-force model of its rule; the read-out head
+// vs the library's log loss and autograd.  Fixed by no passage of the paper, hence
+// "parity unpinned" by it: the hash / shard rule (pinned only by bijectivity and
+// balance), the eviction rule, the read-out head.
 #ifdef _OPENMP
 #include <omp.h>
 #endif
