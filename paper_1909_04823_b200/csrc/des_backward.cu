@@ -640,8 +640,8 @@ extern "C" des_status_t des_backward_update(des_table_t* t, uint32_t ops, const 
   const int G = group_for(t->k);
   const int nnz = (int)b->nnz;
   const long long nbags = (long long)B * t->F;
-  // hot-key detection on a sample, replica assignment, per-occurrence destination row: normally done when
-  // find_or_insert closed (the forward uses the same tags); rebuilt here if another batch came in between
+  // hot-key detection on a sample, replica assignment, per-occurrence destination row (kept if this very batch
+  // has been through it since its find_or_insert)
   if ((st = des_tags_ensure(t, b, cs)) != DES_OK) return st;
   const bool use_super = t->tag_super;
   {

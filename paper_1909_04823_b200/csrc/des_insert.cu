@@ -469,7 +469,7 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   cudaStream_t cs = (cudaStream_t)stream;
   des_api_begin(t, cs);
   DES_DBG_ARM(t, cs);
-  t->tag_valid = 0;                                    // dest[] is scratch of this call; its tags are rebuilt at the end
+  t->tag_valid = 0;                                    // dest[] is scratch of this call: the backward rebuilds its tags
   const int nnz = (int)b->nnz;
   const int nbags = b->batch * (int)t->F;
   if (nnz == 0) {
@@ -517,7 +517,5 @@ extern "C" des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* b,
   DES_LAUNCH_CHECK(t, "resolve_kernel");
   finish_kernel<<<1, DES_MAX_SHARDS, 0, cs>>>(t->S, nnz, (uint32_t)t->max_nnz, t->meta, b->n_uniq);
   DES_LAUNCH_CHECK(t, "finish_kernel");
-  // the batch's unique index is complete: mark the keys that own the batch and give every occurrence its
-  // gradient row, for the forward (which counts the marked keys instead of gathering them) and the backward
-  return des_tags_ensure(t, b, cs);
+  return DES_OK;
 }

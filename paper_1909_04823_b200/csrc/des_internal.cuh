@@ -90,9 +90,8 @@ struct des_table {
   float* Gbuf;                       // [max_uniq + rep_max][stride]: per-unique gradient rows, then
                                      // hot-key replica rows; all zero between calls
   uint32_t* hinfo;                   // [max_uniq] sampled count, then hot index; zero between calls
-  uint32_t* dest;                    // [max_nnz] gradient row of each occurrence (or SUPER_TAG | slot); made by the
-                                     // hot-key pass that closes find_or_insert; the forward reads "hot or not" from
-                                     // it, the backward scatters by it
+  uint32_t* dest;                    // [max_nnz] gradient row of each occurrence (or SUPER_TAG | slot), made by the
+                                     // hot-key pass that opens the backward; scratch of find_or_insert before that
   float* x_sorted;                   // [max_nnz] forward routing: feature values in shard-major order
   float2* bag_tail;                  // [max_batch * F] single-gather forward: per-bag sums of (w x, |v|^2 x^2)
   // which batch the tags in dest[] / the hot lists belong to (they are rebuilt when another batch comes)
@@ -293,5 +292,5 @@ des_status_t des_dense1_forward(des_table* t, const float* pooled, int B, float*
 des_status_t des_dense1_backward(des_table* t, const float* pooled, const float* gE, const float* gZ,
                                  float* gE_work, int B, cudaStream_t st);
 // Hot-key pass over a batch's unique indices (sampled counts, hot list, replica assignment, dest[] with
-// the super-key tags); a no-op when dest[] already belongs to this batch.
+// the super-key tags); a no-op when dest[] already belongs to this batch (a second backward over it).
 des_status_t des_tags_ensure(des_table* t, const des_batch_t* b, cudaStream_t st);

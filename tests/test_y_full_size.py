@@ -185,15 +185,21 @@ def test_streaming_full_size_growth_invariants():
 
 # ------------------------------------------------------------------ first-layer workloads at full size
 def _assert_tolerance_counts(prefix, cap):
-    """At most `cap` of the compared elements of any output of the workloads whose label starts with
-    `prefix` may need more than the stated 1e-5 relative / 1e-6 absolute bound."""
+    """Of the workloads whose label starts with `prefix`: NO element of a forward output (partials, aggregates)
+    may need more than the stated 1e-5 relative / 1e-6 absolute bound, and at most `cap` of the compared
+    elements of the updated rows (keys whose gradient terms cancel: Adagrad turns a rounding-sized gradient
+    into a step of the size of the learning rate)."""
     from harness import TOL_STATS
     seen = False
     for name, st in TOL_STATS.items():
-        if not name.startswith(prefix) or name.split(": ", 1)[1].startswith("[gemm]"):
+        what = name.split(": ", 1)[1]
+        if not name.startswith(prefix) or what.startswith("[gemm]"):
             continue
         seen = True
-        assert st["outside_stated"] <= cap * st["total"], (name, st)
+        if what.startswith("updated rows"):
+            assert st["outside_stated"] <= cap * st["total"], (name, st)
+        else:
+            assert st["outside_stated"] == 0, (name, st)
     assert seen, prefix
 
 
