@@ -412,8 +412,8 @@ def run_workload(args, cfg_index, w, ctx, *, steps, warmup, repeats, modes, want
     def step(i):
         db = dbs[i % len(dbs)]
         t.find_or_insert(db, True)
-        if args.fused:
-            t.forward_fused(w.ops, db, None, pooled, out_small, Z)
+        if args.fused or args.fused_partials:
+            t.forward_fused(w.ops | (16 if args.fused_partials else 0), db, None, pooled, out_small, Z)
         else:
             t.forward_partials(w.ops, db, part_small, pooled)
             t.aggregate(w.ops, db, part_small, pooled, out_small=out_small, Z=Z)
@@ -629,6 +629,9 @@ def main():
                          "come from a separate, untimed eager pass")
     ap.add_argument("--fused", action="store_true",
                     help="use des_forward_fused (per-shard partials kept on chip) instead of partials + aggregate")
+    ap.add_argument("--fused-partials", action="store_true",
+                    help="des_forward_fused in its shard-by-shard form: per-shard partials formed on chip in shard order, "
+                         "aggregated and passed through F without being written (bit-identical to the default path)")
     ap.add_argument("--closed-loop", action="store_true",
                     help="gradients from the fixed read-out (des_head) on the step's own forward instead of seeded "
                          "upstream gradients: the whole Criteo-shaped Wide&Deep / DeepFM step with --config 2 / 3 "
@@ -725,7 +728,8 @@ def main():
                            "ops": w.ops, "optimizer": "adagrad" if w.optimizer else "sgd",
                            "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
                            "launch": "CUDA graph replay" if args.graph else "eager",
-                           "forward": "fused (per-shard partials on chip)" if args.fused else
+                           "forward": "fused, single gather (per-shard partials never formed)" if args.fused else
+                                      "fused, per-shard partials formed on chip in shard order" if args.fused_partials else
                                       "per-shard partials materialised, then aggregated",
                            "tensor_core_gemm": bool(binding.uses_tensor_cores()),
                            "gradients": "closed loop: fixed read-out + log loss on the step's own forward (synthetic labels; "

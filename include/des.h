@@ -85,6 +85,8 @@ typedef enum {
 
 /* operator kind bitmask */
 enum { DES_OP_LR = 1, DES_OP_FM = 2, DES_OP_POOL = 4, DES_OP_DENSE1 = 8 };
+/* modifier, des_forward_fused only: keep the shard-by-shard form (see there) */
+enum { DES_FUSED_SHARD_ORDER = 16 };
 /* weight placement: HASH = mix64(id) mod S (Section 4.2 allows any partition
  * that keeps the shards balanced); FIELD = field mod S (the rule of Section 5,
  * paragraph on large-scale sparse features; required for a weight-disjoint row
@@ -236,8 +238,9 @@ des_status_t des_aggregate(des_table_t* t, uint32_t ops, const des_batch_t* batc
  *    partials as well): every sample's partials are formed shard by shard in
  *    registers, aggregated in the same fixed shard order and passed through F
  *    without being written; results are bit-identical to the two-call path.
- *  - `ops` holds LR / FM together with POOL / DENSE1 and part->part_small is
- *    NULL: every occurrence's row is gathered once; the pass that pools a bag
+ *  - `ops` holds LR / FM together with POOL / DENSE1, part->part_small is
+ *    NULL and DES_FUSED_SHARD_ORDER is not set in `ops`: every occurrence's row
+ *    is gathered once; the pass that pools a bag
  *    also sums its linear weights and squared norms, and (+)M_1, (+)M_1^lr,
  *    (+)M_2 are the sums over a sample's bags, taken in double in field order.
  *    The per-shard partials are never formed — Eq. 1's sum over a sample's

@@ -14,6 +14,7 @@ import torch
 from . import build as _build
 
 OP_LR, OP_FM, OP_POOL, OP_DENSE1 = 1, 2, 4, 8
+FUSED_SHARD_ORDER = 16        # des_forward_fused: keep the shard-by-shard form
 PART_HASH, PART_FIELD = 0, 1
 OPT_SGD, OPT_ADAGRAD, OPT_ADAM = 0, 1, 2
 LIN_SAME, LIN_FTRL = 0, 1

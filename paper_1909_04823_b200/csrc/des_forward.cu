@@ -617,12 +617,14 @@ static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const de
 
 extern "C" des_status_t des_forward_fused(des_table_t* t, uint32_t ops, const des_batch_t* b,
                                           const des_partials_t* part, const des_outputs_t* out, void* stream) {
-  if (!t || !part || !out || (ops & ~15u) || ops == 0) return DES_ERR_INVALID_ARG;
+  if (!t || !part || !out || (ops & ~31u) || (ops & 15u) == 0) return DES_ERR_INVALID_ARG;
+  const bool shard_order = ops & DES_FUSED_SHARD_ORDER;   // the shard-by-shard form even where one gather pass would do
+  ops &= 15u;
   if ((ops & (DES_OP_LR | DES_OP_FM)) && !out->out_small) return DES_ERR_INVALID_ARG;
   if (part->part_pooled || part->part_dense) return DES_ERR_INVALID_ARG;      // materialised partials: use the two-call path
   const uint32_t rest = ops & ~(uint32_t)(DES_OP_LR | DES_OP_FM);
   des_status_t st;
-  if ((ops & (DES_OP_LR | DES_OP_FM)) && rest && !part->part_small) {
+  if ((ops & (DES_OP_LR | DES_OP_FM)) && rest && !part->part_small && !shard_order) {
     // LR / FM together with pooling and no request for the per-shard partials: one gather pass
     st = des_check_batch(t, b, 0);
     if (st != DES_OK) return st;

@@ -281,6 +281,15 @@ class Pair:
             assert self.t.status() == 0
             if (ops & (OP_LR | OP_FM)) and (ops & (OP_POOL | OP_DENSE1)):
                 fused_osm = f_small.cpu().numpy()
+                # ... and its shard-by-shard form (partials formed on chip in shard order) is bit-identical
+                s_small = torch.full((B, k + 4), float("nan"), device=dev)
+                s_pooled = torch.full((B, F * k), float("nan"), device=dev)
+                s_Z = torch.full((B, max(H, 1)), float("nan"), device=dev)
+                self.t.forward_fused(ops | 16, db, None, s_pooled, s_small, s_Z)
+                torch.cuda.synchronize()
+                assert self.t.status() == 0
+                assert torch.equal(s_small.view(torch.int32), out_small.view(torch.int32)), "fused (shard order) out_small"
+                assert torch.equal(s_pooled.view(torch.int32), pooled.view(torch.int32)), "fused (shard order) pooled"
             elif ops & (OP_LR | OP_FM):
                 assert torch.equal(f_small.view(torch.int32), out_small.view(torch.int32)), "fused out_small"
             if ops & (OP_POOL | OP_DENSE1):
