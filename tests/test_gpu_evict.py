@@ -76,9 +76,11 @@ def test_evict_keys_matches_oracle(partition):
         p.close()
 
 
-def test_evict_stale_matches_oracle():
+@pytest.mark.parametrize("optimizer", [OPT_ADAGRAD, synth.OPT_ADAM])
+def test_evict_stale_matches_oracle(optimizer):
+    # (Adam: a second state array moves with the rows; the steps after the eviction would not match otherwise)
     from harness import Pair
-    w = synth.config(4).scaled(batch=384, prepopulate=0, init_scale=0.05, shards=7)
+    w = synth.config(4).scaled(batch=384, prepopulate=0, init_scale=0.05, shards=7, optimizer=optimizer)
     st = synth.Stream(w)
     b = st.next_batch()
     p = Pair(w, max_rows=200000, max_nnz=int(b.nnz * 1.3) + 1024)
@@ -93,7 +95,9 @@ def test_evict_stale_matches_oracle():
         assert n_g == n_o and 0 < n_g < n0
         assert _export_by_key(p.t, n0 - n_g) == _oracle_by_key(p.o)
         assert p.t.evict_stale(4) == 0
-        p.step(b, synth.upstream_grads(w, b.batch, 9))
+        for s in range(2):
+            p.step(b, synth.upstream_grads(w, b.batch, 9 + s))
+            b = st.next_batch()
     finally:
         p.close()
 
