@@ -249,6 +249,8 @@ def kernel_bytes(name, st):
         return 4 * (B * F + 1) + 4 * nnz + 4 * k * U + 4 * B * F * k
     if name == "single_gather_kernel":   # rows + shards in, every unique row once, pooled + bag tails out
         return 4 * (B * F + 1) + 5 * nnz + row * U + 4 * B * F * k + 8 * B * F
+    if name == "field_partials_kernel":   # pooled vectors and bag tails in, per-shard partials out
+        return 4 * B * F * k + 8 * B * F + 4 * S * B * (k + 4)
     if name == "fused_finish_kernel":
         return 4 * B * F * k + 8 * B * F + 4 * B * (k + 4)
     if name == "aggregate_small_kernel":

@@ -217,7 +217,10 @@ des_status_t des_table_destroy(des_table_t* t);
 des_status_t des_find_or_insert(des_table_t* t, const des_batch_t* batch, int insert, void* stream);
 
 /* Sub-operators M_j of every shard (Eq. of Sections 4.1-4.3), see
- * des_partials_t.  `batch` must have been through des_find_or_insert. */
+ * des_partials_t.  `batch` must have been through des_find_or_insert.  (Under
+ * DES_PART_FIELD with pooling among the operators a shard's sub-operators are formed
+ * as the sums over the bags of its own fields, from the same pass that pools them;
+ * otherwise shard by shard from the shard's own occurrences.) */
 des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const des_batch_t* batch,
                                   const des_partials_t* part, void* stream);
 

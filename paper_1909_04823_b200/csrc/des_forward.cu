@@ -24,6 +24,11 @@
 //                 registers.  The per-shard pooled partial [S][B][F*k] is only
 //                 materialised (with atomics) when the caller asks for it.
 //
+// FIELD partition (field f on shard f mod S): a bag belongs to one shard, so when pooling is among the
+// operators one gather pass (single_gather_kernel: pooled vectors and per-bag sums of the linear weights and
+// squared norms) feeds everything, and field_partials_kernel forms shard s's sub-operators as the sums over
+// the bags of its own fields — no routing pass, no second gather.
+//
 // Accuracy.  A lane never adds more than a few dozen terms into one float32 accumulator (long
 // segments are summed in two levels), and the sum over shards is taken in double and rounded once, so
 // every per-sample sum keeps the stated float32 tolerance even when one key contributes
@@ -498,6 +503,55 @@ __global__ void __launch_bounds__(256) fused_finish_kernel(const float* __restri
   if (c4 == 0) o[K4] = make_float4((float)tr, fm ? (float)(0.5 * aa - 0.5 * tq) : 0.f, (float)tq, 0.f);
 }
 
+// FIELD partition: a bag belongs to one shard (field f lives on shard f mod S), so the sub-operators of shard s
+// are sums over the bags of its own fields — which the pooling pass has already formed (pooled vectors, bag
+// tails).  G lanes per sample walk the shards in order; shard s adds its fields f = s, s + S, ... in field order
+// (float32, a handful of terms), part_small receives the partial, and with FUSED the partials are added in
+// double in shard order and passed through F exactly as aggregate_small_kernel does.
+template <int G, bool FUSED>
+__global__ void __launch_bounds__(256) field_partials_kernel(const float* __restrict__ pooled, const float2* __restrict__ bag_tail,
+                                                             int B, int F, int S, int k, uint32_t ops,
+                                                             float* __restrict__ part_small, float* __restrict__ out_small) {
+  const int K4 = k >> 2, stride = k + 4;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = t / G, c4 = t % G;
+  const bool live = b < B, col = c4 < K4;
+  const bool lr = ops & DES_OP_LR, fm = ops & DES_OP_FM;
+  double Ax = 0.0, Ay = 0.0, Az = 0.0, Aw = 0.0, R = 0.0, Q = 0.0;
+  if (live) {
+    const float4* pb = reinterpret_cast<const float4*>(pooled + (size_t)b * F * k) + c4;
+    const float2* tb = bag_tail + (size_t)b * F;
+    for (int s = 0; s < S; ++s) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float m1lr = 0.f, m2 = 0.f;
+      for (int f = s; f < F; f += S) {
+        if (col && fm) { const float4 v = __ldg(pb + (size_t)f * K4); acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w; }
+        if (c4 == 0) { const float2 tl = __ldg(tb + f); m1lr += tl.x; m2 += tl.y; }
+      }
+      if (!fm) m2 = 0.f;
+      if (!lr) m1lr = 0.f;
+      if (part_small) {
+        float4* dst = reinterpret_cast<float4*>(part_small + ((size_t)s * B + b) * stride);
+        if (col) dst[c4] = acc;
+        if (c4 == 0) dst[K4] = make_float4(m1lr, m2, 0.f, 0.f);
+      }
+      if (FUSED) {
+        Ax += (double)acc.x; Ay += (double)acc.y; Az += (double)acc.z; Aw += (double)acc.w;
+        R += (double)m1lr; Q += (double)m2;
+      }
+    }
+  }
+  if (FUSED) {
+    double aa = col ? Ax * Ax + Ay * Ay + Az * Az + Aw * Aw : 0.0;
+#pragma unroll
+    for (int d = 1; d < G; d <<= 1) aa += __shfl_xor_sync(0xFFFFFFFFu, aa, d);
+    if (!live) return;
+    float4* o = reinterpret_cast<float4*>(out_small + (size_t)b * stride);
+    if (col) o[c4] = make_float4((float)Ax, (float)Ay, (float)Az, (float)Aw);
+    if (c4 == 0) o[K4] = make_float4((float)R, fm ? (float)(0.5 * aa - 0.5 * Q) : 0.f, (float)Q, 0.f);
+  }
+}
+
 // sum over shards of a dense [S][B][n] tensor (materialised pooled / dense partials)
 __global__ void reduce_shards_kernel(const float* __restrict__ part, size_t per_shard, int S, float* __restrict__ out) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x, st = (size_t)gridDim.x * blockDim.x;
@@ -509,6 +563,8 @@ __global__ void reduce_shards_kernel(const float* __restrict__ part, size_t per_
 }
 
 static int group_for(int k) { int K4 = k / 4, G = 1; while (G < K4) G <<= 1; return G; }
+
+static des_status_t launch_single_gather(des_table_t* t, uint32_t ops, const des_batch_t* b, float* pooled, cudaStream_t cs);
 
 // shared by des_forward_partials (fused_out == NULL) and des_forward_fused
 static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t* b, const des_partials_t* part,
@@ -530,6 +586,19 @@ static des_status_t forward_impl(des_table_t* t, uint32_t ops, const des_batch_t
   float* pp = pool ? part->part_pooled : nullptr;
   if (pp) DES_CUDA(cudaMemsetAsync(pp, 0, (size_t)t->S * B * t->F * t->k * 4, cs));
   const int G = group_for(t->k);
+  if (t->cfg.partition == DES_PART_FIELD && pl && !pp && (ps || fused_out)) {
+    // FIELD partition with pooling among the operators: one gather pass (pooled vectors + bag tails), then the
+    // per-shard sub-operators as sums over each shard's own fields — no routing pass, no second gather
+    if ((st = launch_single_gather(t, ops, b, pl, cs)) != DES_OK) return st;
+    const int grid = (int)(((long long)B * G + 255) / 256);
+#define FP2(GG, FU) field_partials_kernel<GG, FU><<<grid, 256, 0, cs>>>(pl, t->bag_tail, B, (int)t->F, (int)t->S, t->k, ops, ps, fused_out)
+#define FP(GG) do { if (fused_out) FP2(GG, true); else FP2(GG, false); } while (0)
+    switch (G) { case 1: FP(1); break; case 2: FP(2); break; case 4: FP(4); break; case 8: FP(8); break; default: FP(16); }
+#undef FP
+#undef FP2
+    DES_LAUNCH_CHECK(t, "field_partials_kernel");
+    return DES_OK;
+  }
   // routing: rows of every occurrence in shard-major order per sample (workspace shared with find_or_insert,
   // which has finished with it by the time a forward can run on the same stream)
   uint32_t* grow_csr = t->uslot;
@@ -581,37 +650,42 @@ extern "C" des_status_t des_forward_partials(des_table_t* t, uint32_t ops, const
   return forward_impl(t, ops, b, part, nullptr, stream);
 }
 
-// des_forward_fused with pooling among the operators: one gather pass for everything.
-static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const des_batch_t* b, float* pooled,
-                                          float* out_small, cudaStream_t cs) {
+// the gather pass of the single-gather forms: pooled vectors (and their bfloat16 copy when the first layer
+// follows) and per-bag sums of the linear weights and squared norms
+static des_status_t launch_single_gather(des_table_t* t, uint32_t ops, const des_batch_t* b, float* pooled, cudaStream_t cs) {
   const int B = b->batch, G = group_for(t->k);
   const long long nbags = (long long)B * t->F;
-  {
-    const bool wide = b->nnz >= 8 * nbags;
-    const long long threads = nbags * (wide ? 32 : G);
-    long long blocks = (threads + 255) / 256;
-    if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
-    const unsigned grid = (unsigned)blocks;
-    __nv_bfloat16* pb = ((ops & DES_OP_DENSE1) && t->use_tc) ? t->pooled_b : nullptr;
+  const bool wide = b->nnz >= 8 * nbags;
+  const long long threads = nbags * (wide ? 32 : G);
+  long long blocks = (threads + 255) / 256;
+  if (blocks > (long long)t->sm_count * POOL_BLOCKS_PER_SM) blocks = (long long)t->sm_count * POOL_BLOCKS_PER_SM;
+  const unsigned grid = (unsigned)blocks;
+  __nv_bfloat16* pb = ((ops & DES_OP_DENSE1) && t->use_tc) ? t->pooled_b : nullptr;
 #define SG3(GG, PP, HV) single_gather_kernel<GG, PP, HV><<<grid, 256, 0, cs>>>(b->offsets, b->vals, b->rows, b->shards, nbags,   \
                                                                               (int)t->S, t->k, t->W, t->meta,                 \
                                                                               (uint32_t)t->total_rows, pooled, t->bag_tail, pb)
 #define SG2(GG, HV) do { if (wide) SG3(GG, 32 / GG, HV); else SG3(GG, 1, HV); } while (0)
 #define SG(GG) do { if (b->vals) SG2(GG, true); else SG2(GG, false); } while (0)
-    switch (G) { case 1: SG(1); break; case 2: SG(2); break; case 4: SG(4); break; case 8: SG(8); break; default: SG(16); }
+  switch (G) { case 1: SG(1); break; case 2: SG(2); break; case 4: SG(4); break; case 8: SG(8); break; default: SG(16); }
 #undef SG
 #undef SG2
 #undef SG3
-    DES_LAUNCH_CHECK(t, "single_gather_kernel");
-    t->pooled_b_src = pb ? pooled : nullptr;
-  }
-  {
-    const int grid = (int)(((long long)B * G + 255) / 256);
+  DES_LAUNCH_CHECK(t, "single_gather_kernel");
+  t->pooled_b_src = pb ? pooled : nullptr;
+  return DES_OK;
+}
+
+// des_forward_fused with pooling among the operators: one gather pass for everything.
+static des_status_t forward_single_gather(des_table_t* t, uint32_t ops, const des_batch_t* b, float* pooled,
+                                          float* out_small, cudaStream_t cs) {
+  des_status_t st = launch_single_gather(t, ops, b, pooled, cs);
+  if (st != DES_OK) return st;
+  const int B = b->batch, G = group_for(t->k);
+  const int grid = (int)(((long long)B * G + 255) / 256);
 #define FF(GG) fused_finish_kernel<GG><<<grid, 256, 0, cs>>>(pooled, t->bag_tail, B, (int)t->F, t->k, ops, out_small)
-    switch (G) { case 1: FF(1); break; case 2: FF(2); break; case 4: FF(4); break; case 8: FF(8); break; default: FF(16); }
+  switch (G) { case 1: FF(1); break; case 2: FF(2); break; case 4: FF(4); break; case 8: FF(8); break; default: FF(16); }
 #undef FF
-    DES_LAUNCH_CHECK(t, "fused_finish_kernel");
-  }
+  DES_LAUNCH_CHECK(t, "fused_finish_kernel");
   return DES_OK;
 }
 
