@@ -91,6 +91,19 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     if not force and not needs_build(debug):
         return lib
     os.makedirs(OBJ, exist_ok=True)
+    # several processes of one job (one per GPU) may get here together: one builds, the others wait and find it done
+    import fcntl
+    with open(os.path.join(OBJ, ".lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if not force and not needs_build(debug):
+                return lib
+            return _build_locked(lib, force, verbose, debug)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
+
+
+def _build_locked(lib, force, verbose, debug):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     base = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
             "--fmad=true", "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC",
