@@ -708,7 +708,9 @@ def main():
                 side.append({"workload": f"config {ci}", "error": repr(ex)})
 
     mode = "graph" if args.graph else "eager"
-    r = run_workload(args, args.config, w, ctx, steps=args.steps, warmup=args.warmup, repeats=args.repeats, modes=[mode],
+    # (the default run also replays the same step from a CUDA graph, reported beside the eager headline)
+    modes = [mode] if (args.graph or world > 1) else ["eager", "graph"]
+    r = run_workload(args, args.config, w, ctx, steps=args.steps, warmup=args.warmup, repeats=args.repeats, modes=modes,
                      want_e2e=not (args.no_e2e or args.closed_loop), want_cpu=(rank == 0 and world == 1 and not args.no_cpu_baseline),
                      profile_in_timed=True)
     clocks = sampler.stop(r["windows"]) if sampler else None
@@ -750,6 +752,11 @@ def main():
                         # mostly L1 / L2 hits in a skewed batch, so this is not an HBM figure
                         "occ_bytes_per_step": int(occ_bytes), "occ_gbs": round(occ_bytes / ms_step / 1e6, 1)},
                 "kernels": m["kernels"], "cpu_baseline": r["cpu"], "configs": side}
+        if "graph" in r["results"] and mode != "graph":
+            gm = r["results"]["graph"]
+            line["graph_replay"] = {"ms_per_step": gm["ms_per_step"], "value": gm["value"], "unit": UNIT,
+                                    "repeats_ms": gm["repeats"]["ms_per_step"],
+                                    "note": "the same step replayed from a CUDA graph (one graph per resident batch)"}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
